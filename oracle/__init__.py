@@ -1,0 +1,148 @@
+"""ctypes access to the CPU oracle (``vl_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library and its Python binding never do.  The C file is built
+with gcc on first use (``build()``), next to the source.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "vl_oracle.c")
+_LIB = os.path.join(_HERE, "libvl_oracle.so")
+# The mutation test points these at a deliberately broken copy in a temp directory.
+if os.environ.get("VL_ORACLE_MUTANT_SRC"):
+    _SRC = os.environ["VL_ORACLE_MUTANT_SRC"]
+    _LIB = os.path.splitext(_SRC)[0] + ".so"
+
+PASS, INCONSISTENT, OUT_OF_RANGE, INTERFERENCE = 1, 2, 4, 8
+
+VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
+                          ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-Wall", "-Wextra", "-fPIC", "-shared", _SRC, "-o", _LIB])
+    return _LIB
+
+
+class _Prog(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("n_blocks", "n_instrs", "n_vregs", "n_operands", "n_edges", "P", "B")] + [
+        ("block_instr_off", C.c_void_p), ("succ_off", C.c_void_p), ("succ", C.c_void_p),
+        ("instr_op_off", C.c_void_p), ("instr_n_defs", C.c_void_p), ("op_vreg", C.c_void_p),
+        ("vreg_width", C.c_void_p)]
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = C.CDLL(build())
+        lib.vlo_block_liveness.restype = C.c_uint32
+        lib.vlo_block_liveness.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int]
+        lib.vlo_instr_liveness.restype = C.c_uint64
+        lib.vlo_instr_liveness.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        lib.vlo_verify_rows.restype = None
+        lib.vlo_verify_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
+        lib.vlo_violations.restype = None
+        lib.vlo_violations.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.vlo_conflicts.restype = C.c_uint64
+        lib.vlo_conflicts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+@dataclass
+class Liveness:
+    blk_live_in: np.ndarray    # uint8 [n_blocks, n_vregs]
+    blk_live_out: np.ndarray   # uint8 [n_blocks, n_vregs]
+    lo_off: np.ndarray         # uint64 [n_instrs+1]
+    lo: np.ndarray             # uint32 [lo_off[-1]], ascending inside each instruction
+    sweeps: int
+
+    def live_after(self, i: int) -> np.ndarray:
+        return self.lo[int(self.lo_off[i]): int(self.lo_off[i + 1])]
+
+    def packed(self, which: str) -> np.ndarray:
+        """Block sets as little-endian 32-bit words, [n_blocks, ceil(V/32)]."""
+        a = self.blk_live_in if which == "in" else self.blk_live_out
+        nB, V = a.shape
+        words = (V + 31) // 32
+        pad = np.zeros((nB, words * 32), dtype=np.uint8)
+        pad[:, :V] = a
+        return np.packbits(pad, axis=1, bitorder="little").view("<u4").reshape(nB, words)
+
+
+class OracleProgram:
+    """Keeps the numpy arrays alive and exposes the C struct."""
+
+    def __init__(self, prog):
+        self.src = prog
+        self.arrays = dict(
+            block_instr_off=np.ascontiguousarray(prog.block_instr_off, dtype=np.uint32),
+            succ_off=np.ascontiguousarray(prog.succ_off, dtype=np.uint32),
+            succ=np.ascontiguousarray(np.concatenate([prog.succ, [0]]), dtype=np.uint32),
+            instr_op_off=np.ascontiguousarray(prog.instr_op_off, dtype=np.uint32),
+            instr_n_defs=np.ascontiguousarray(np.concatenate([prog.instr_n_defs, [0]]), dtype=np.uint8),
+            op_vreg=np.ascontiguousarray(np.concatenate([prog.op_vreg, [0]]), dtype=np.uint32),
+            vreg_width=np.ascontiguousarray(np.concatenate([prog.vreg_width, [1]]), dtype=np.uint8),
+        )
+        self.c = _Prog(prog.n_blocks, prog.n_instrs, prog.n_vregs, prog.n_operands, prog.n_edges, prog.P, prog.B,
+                       *[self.arrays[k].ctypes.data for k in
+                         ("block_instr_off", "succ_off", "succ", "instr_op_off", "instr_n_defs", "op_vreg", "vreg_width")])
+        self.n_blocks, self.n_instrs, self.n_vregs = prog.n_blocks, prog.n_instrs, prog.n_vregs
+
+    def liveness(self, order: int = 0) -> Liveness:
+        lib = _load()
+        nB, V, nI = self.n_blocks, self.n_vregs, self.n_instrs
+        lin = np.zeros((nB, V), dtype=np.uint8)
+        lout = lin.copy()
+        sweeps = lib.vlo_block_liveness(C.byref(self.c), _ptr(lin), _ptr(lout), order)
+        lo_off = np.zeros(nI + 1, dtype=np.uint64)
+        total = lib.vlo_instr_liveness(C.byref(self.c), _ptr(lout), _ptr(lo_off), None, 0)
+        lo = np.zeros(max(int(total), 1), dtype=np.uint32)
+        lib.vlo_instr_liveness(C.byref(self.c), _ptr(lout), _ptr(lo_off), _ptr(lo), total)
+        return Liveness(lin, lout, lo_off, lo[: int(total)], int(sweeps))
+
+    def verify(self, live: Liveness, rows: np.ndarray) -> np.ndarray:
+        """Verdict record for every row of a uint16 [K, pitch] matrix."""
+        lib = _load()
+        rows = np.ascontiguousarray(rows, dtype=np.uint16)
+        if rows.ndim == 1:
+            rows = rows[None, :]
+        K, pitch = rows.shape
+        out = np.zeros(K, dtype=VERDICT_DTYPE)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        lib.vlo_verify_rows(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(rows), K, pitch, _ptr(out))
+        return out
+
+    def violations(self, live: Liveness, row: np.ndarray) -> np.ndarray:
+        lib = _load()
+        row = np.ascontiguousarray(row, dtype=np.uint16)
+        kinds = np.zeros(max(self.n_instrs, 1), dtype=np.uint8)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        lib.vlo_violations(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(kinds))
+        return kinds[: self.n_instrs]
+
+    def conflicts(self, live: Liveness, row: np.ndarray) -> np.ndarray:
+        """All (instruction, defined vreg, other vreg) overlap records of one row."""
+        lib = _load()
+        row = np.ascontiguousarray(row, dtype=np.uint16)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        n = lib.vlo_conflicts(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), None, 0)
+        tr = np.zeros((max(int(n), 1), 3), dtype=np.uint32)
+        lib.vlo_conflicts(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(tr), n)
+        return tr[: int(n)]

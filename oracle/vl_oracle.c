@@ -1,0 +1,293 @@
+/*
+ * CPU oracle for the candidate-allocation check.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the plain, slow, single-threaded statement of what the CUDA
+ * library must compute.  It shares no code, header, table or helper with the
+ * CUDA path; only tests, the smoke check and the benchmark's CPU-baseline leg
+ * may call it.  Nothing here is tuned.
+ *
+ * What is checked (paper, Section 1, correctness conditions (1) and (2);
+ * Section 3.4, "Consistency", "Safety", "Realizability"; Section 2, register
+ * tuples and the 4-bank register file; Section 4.5, a dataflow violation is a
+ * write that clobbers a value still live later):
+ *
+ *   liveness   backward dataflow over the control-flow graph to the least
+ *              fixed point, then a backward walk of every block giving the
+ *              set of virtual registers live after each instruction;
+ *   C          every occurrence of a virtual register carries the physical
+ *              register of its first occurrence (the table T);
+ *   R          at every definition of v: [T[v], T[v]+width(v)) lies in [0,P);
+ *   I          at every definition of v at instruction i: that range is
+ *              disjoint from the range of every other virtual register that
+ *              is live after i or also defined by i;
+ *   bank tally per instruction, distinct source base registers that share a
+ *              bank (T mod B) cost one extra cycle each beyond the first.
+ *
+ * The paper states the properties, not an encoding; equivalence with the
+ * authors' SMT verifier is therefore: parity unpinned.  Every function below
+ * is pinned by the tests under tests/ against brute-force path enumeration,
+ * closed forms and hand-worked programs.
+ *
+ * Conventions: an instruction's operands are its definitions followed by its
+ * reads; operand index == column of the candidate row; reads happen before
+ * writes inside one instruction.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+    uint32_t n_blocks, n_instrs, n_vregs, n_operands, n_edges, P, B;
+    const uint32_t *block_instr_off; /* [n_blocks+1] */
+    const uint32_t *succ_off;        /* [n_blocks+1] */
+    const uint32_t *succ;            /* [n_edges]    */
+    const uint32_t *instr_op_off;    /* [n_instrs+1] */
+    const uint8_t *instr_n_defs;     /* [n_instrs]   */
+    const uint32_t *op_vreg;         /* [n_operands] */
+    const uint8_t *vreg_width;       /* [n_vregs]    */
+} vlo_program;
+
+typedef struct {
+    uint32_t flags;                /* bit0 pass, bit1 inconsistent, bit2 out of range, bit3 interference */
+    int32_t first_violation_instr; /* lowest instruction index with any violation, -1 if none */
+    uint32_t conflict_pairs;       /* number of (instruction, definition, other vreg) overlaps */
+    uint32_t bank_conflicts;       /* extra read cycles summed over instructions */
+} vlo_verdict;
+
+enum { VLO_PASS = 1, VLO_INCONSISTENT = 2, VLO_OUT_OF_RANGE = 4, VLO_INTERFERENCE = 8 };
+
+/* ---------------------------------------------------------------- liveness */
+
+/*
+ * Block-level sets and fixed point (one byte per (block, vreg)).
+ *   use[b] = vregs read in b before any write to them in b
+ *   def[b] = vregs written in b
+ *   out[b] = union of in[s] over successors s;  in[b] = use[b] | (out[b] - def[b])
+ * starting from empty sets, sweeping until a sweep changes nothing.
+ * order = 0 sweeps blocks last to first, order = 1 first to last; the least
+ * fixed point does not depend on it.  Returns the number of sweeps.
+ */
+uint32_t vlo_block_liveness(const vlo_program *p, uint8_t *live_in, uint8_t *live_out, int order)
+{
+    const uint32_t nB = p->n_blocks, V = p->n_vregs;
+    uint8_t *use = calloc((size_t)nB * V + 1, 1);
+    uint8_t *def = calloc((size_t)nB * V + 1, 1);
+    for (uint32_t b = 0; b < nB; ++b) {
+        for (uint32_t i = p->block_instr_off[b]; i < p->block_instr_off[b + 1]; ++i) {
+            uint32_t o0 = p->instr_op_off[i], o1 = p->instr_op_off[i + 1], nd = p->instr_n_defs[i];
+            for (uint32_t o = o0 + nd; o < o1; ++o) { /* reads first */
+                uint32_t v = p->op_vreg[o];
+                if (!def[(size_t)b * V + v]) use[(size_t)b * V + v] = 1;
+            }
+            for (uint32_t o = o0; o < o0 + nd; ++o) def[(size_t)b * V + p->op_vreg[o]] = 1;
+        }
+    }
+    memset(live_in, 0, (size_t)nB * V);
+    memset(live_out, 0, (size_t)nB * V);
+    uint32_t sweeps = 0;
+    int changed = 1;
+    while (changed) {
+        changed = 0;
+        ++sweeps;
+        for (uint32_t n = 0; n < nB; ++n) {
+            uint32_t b = order ? n : nB - 1 - n;
+            for (uint32_t v = 0; v < V; ++v) {
+                uint8_t o = 0;
+                for (uint32_t e = p->succ_off[b]; e < p->succ_off[b + 1]; ++e)
+                    o |= live_in[(size_t)p->succ[e] * V + v];
+                uint8_t in = use[(size_t)b * V + v] | (o & !def[(size_t)b * V + v]);
+                if (o != live_out[(size_t)b * V + v] || in != live_in[(size_t)b * V + v]) changed = 1;
+                live_out[(size_t)b * V + v] = o;
+                live_in[(size_t)b * V + v] = in;
+            }
+        }
+    }
+    free(use);
+    free(def);
+    return sweeps;
+}
+
+/*
+ * Per-instruction live-after sets in CSR form, ascending vreg id.
+ * Walk each block backwards from out[b]:  live_after(i) = live;
+ * live = (live - defs(i)) | reads(i).
+ * lo_off has n_instrs+1 entries.  At most cap ids are stored in lo; the total
+ * count is returned (call once with cap = 0 to size the buffer).
+ */
+uint64_t vlo_instr_liveness(const vlo_program *p, const uint8_t *blk_live_out,
+                            uint64_t *lo_off, uint32_t *lo, uint64_t cap)
+{
+    const uint32_t V = p->n_vregs, nI = p->n_instrs;
+    uint8_t *live = malloc((size_t)V + 1);
+    uint64_t *cnt = calloc((size_t)nI + 1, sizeof(uint64_t));
+    /* pass 1: sizes */
+    for (uint32_t b = 0; b < p->n_blocks; ++b) {
+        memcpy(live, blk_live_out + (size_t)b * V, V);
+        for (uint32_t i = p->block_instr_off[b + 1]; i-- > p->block_instr_off[b];) {
+            uint64_t c = 0;
+            for (uint32_t v = 0; v < V; ++v) c += live[v];
+            cnt[i] = c;
+            uint32_t o0 = p->instr_op_off[i], o1 = p->instr_op_off[i + 1], nd = p->instr_n_defs[i];
+            for (uint32_t o = o0; o < o0 + nd; ++o) live[p->op_vreg[o]] = 0;
+            for (uint32_t o = o0 + nd; o < o1; ++o) live[p->op_vreg[o]] = 1;
+        }
+    }
+    uint64_t total = 0;
+    for (uint32_t i = 0; i < nI; ++i) { lo_off[i] = total; total += cnt[i]; }
+    lo_off[nI] = total;
+    /* pass 2: ids */
+    for (uint32_t b = 0; b < p->n_blocks; ++b) {
+        memcpy(live, blk_live_out + (size_t)b * V, V);
+        for (uint32_t i = p->block_instr_off[b + 1]; i-- > p->block_instr_off[b];) {
+            uint64_t at = lo_off[i];
+            for (uint32_t v = 0; v < V; ++v)
+                if (live[v]) { if (at < cap) lo[at] = v; ++at; }
+            uint32_t o0 = p->instr_op_off[i], o1 = p->instr_op_off[i + 1], nd = p->instr_n_defs[i];
+            for (uint32_t o = o0; o < o0 + nd; ++o) live[p->op_vreg[o]] = 0;
+            for (uint32_t o = o0 + nd; o < o1; ++o) live[p->op_vreg[o]] = 1;
+        }
+    }
+    free(live);
+    free(cnt);
+    return total;
+}
+
+/* ------------------------------------------------------------------ verify */
+
+static int ranges_overlap(uint32_t a, uint32_t wa, uint32_t b, uint32_t wb)
+{
+    return a < b + wb && b < a + wa; /* plain integers, no wrap: a,b <= 65535, w <= 255 */
+}
+
+/*
+ * Core walk shared by the three reporting functions below (they differ only in
+ * what they write down).  kinds, if given, receives per instruction the OR of
+ * the violation bits raised there; triples, if given, receives up to cap
+ * (instruction, defined vreg, other vreg) overlap records; *n_triples counts all.
+ */
+static void walk(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                 const uint16_t *row, vlo_verdict *out, uint8_t *kinds,
+                 uint32_t *triples, uint64_t cap, uint64_t *n_triples)
+{
+    const uint32_t V = p->n_vregs, nI = p->n_instrs;
+    int32_t *T = malloc(((size_t)V + 1) * sizeof(int32_t));
+    for (uint32_t v = 0; v < V; ++v) T[v] = -1;
+    uint32_t *Q = malloc(((size_t)p->n_operands + 1) * sizeof(uint32_t));
+    uint32_t flags = 0, pairs = 0, bank = 0;
+    int64_t first = -1;
+    uint64_t nt = 0;
+    if (kinds) memset(kinds, 0, nI);
+
+    /* table and consistency: operands in program order, first occurrence wins */
+    for (uint32_t i = 0; i < nI; ++i) {
+        for (uint32_t o = p->instr_op_off[i]; o < p->instr_op_off[i + 1]; ++o) {
+            uint32_t v = p->op_vreg[o];
+            if (T[v] < 0) T[v] = row[o];
+            else if ((uint32_t)T[v] != row[o]) {
+                flags |= VLO_INCONSISTENT;
+                if (kinds) kinds[i] |= VLO_INCONSISTENT;
+                if (first < 0 || (int64_t)i < first) first = i;
+            }
+        }
+    }
+
+    for (uint32_t i = 0; i < nI; ++i) {
+        uint32_t o0 = p->instr_op_off[i], o1 = p->instr_op_off[i + 1], nd = p->instr_n_defs[i];
+        for (uint32_t d = o0; d < o0 + nd; ++d) {
+            uint32_t v = p->op_vreg[d];
+            uint32_t s = (uint32_t)T[v], w = p->vreg_width[v];
+            int bad = 0;
+            /* realizability: the tuple fits in the register file */
+            if (s + w > p->P) {
+                flags |= VLO_OUT_OF_RANGE;
+                if (kinds) kinds[i] |= VLO_OUT_OF_RANGE;
+                bad = 1;
+            }
+            /* safety: every other vreg live after i ... */
+            for (uint64_t e = lo_off[i]; e < lo_off[i + 1]; ++e) {
+                uint32_t u = lo[e];
+                if (u == v) continue;
+                if (ranges_overlap(s, w, (uint32_t)T[u], p->vreg_width[u])) {
+                    ++pairs;
+                    if (triples && nt < cap) { triples[3 * nt] = i; triples[3 * nt + 1] = v; triples[3 * nt + 2] = u; }
+                    ++nt;
+                    flags |= VLO_INTERFERENCE;
+                    if (kinds) kinds[i] |= VLO_INTERFERENCE;
+                    bad = 1;
+                }
+            }
+            /* ... and every other vreg written by the same instruction that is not live after it */
+            for (uint32_t d2 = o0; d2 < o0 + nd; ++d2) {
+                uint32_t u = p->op_vreg[d2];
+                if (u == v) continue;
+                int in_live = 0;
+                for (uint64_t e = lo_off[i]; e < lo_off[i + 1]; ++e) if (lo[e] == u) in_live = 1;
+                if (in_live) continue;
+                if (ranges_overlap(s, w, (uint32_t)T[u], p->vreg_width[u])) {
+                    ++pairs;
+                    if (triples && nt < cap) { triples[3 * nt] = i; triples[3 * nt + 1] = v; triples[3 * nt + 2] = u; }
+                    ++nt;
+                    flags |= VLO_INTERFERENCE;
+                    if (kinds) kinds[i] |= VLO_INTERFERENCE;
+                    bad = 1;
+                }
+            }
+            if (bad && (first < 0 || (int64_t)i < first)) first = i;
+        }
+        /* bank tally: Q = distinct source base registers of this instruction; every
+         * bank holding n of them costs n-1 extra cycles */
+        uint32_t nq = 0;
+        for (uint32_t a = o0 + nd; a < o1; ++a) {
+            uint32_t ta = (uint32_t)T[p->op_vreg[a]];
+            int dup = 0;
+            for (uint32_t q = 0; q < nq; ++q) if (Q[q] == ta) dup = 1;
+            if (!dup) Q[nq++] = ta;
+        }
+        for (uint32_t q = 0; q < nq; ++q) {
+            int first_of_bank = 1;
+            for (uint32_t r = 0; r < q; ++r) if (Q[r] % p->B == Q[q] % p->B) first_of_bank = 0;
+            if (!first_of_bank) continue;
+            uint32_t n = 0;
+            for (uint32_t r = 0; r < nq; ++r) if (Q[r] % p->B == Q[q] % p->B) ++n;
+            bank += n - 1;
+        }
+    }
+    free(Q);
+    if (!flags) flags = VLO_PASS;
+    out->flags = flags;
+    out->first_violation_instr = (int32_t)first;
+    out->conflict_pairs = pairs;
+    out->bank_conflicts = bank;
+    if (n_triples) *n_triples = nt;
+    free(T);
+}
+
+void vlo_verify(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                const uint16_t *row, vlo_verdict *out)
+{
+    walk(p, lo_off, lo, row, out, NULL, NULL, 0, NULL);
+}
+
+void vlo_verify_rows(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                     const uint16_t *rows, uint64_t K, uint64_t pitch, vlo_verdict *out)
+{
+    for (uint64_t k = 0; k < K; ++k) walk(p, lo_off, lo, rows + k * pitch, out + k, NULL, NULL, 0, NULL);
+}
+
+/* per-instruction violation kinds for one row */
+void vlo_violations(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                    const uint16_t *row, uint8_t *kinds)
+{
+    vlo_verdict v;
+    walk(p, lo_off, lo, row, &v, kinds, NULL, 0, NULL);
+}
+
+/* every (instruction, defined vreg, other vreg) overlap of one row; returns the total */
+uint64_t vlo_conflicts(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                       const uint16_t *row, uint32_t *triples, uint64_t cap)
+{
+    vlo_verdict v;
+    uint64_t n = 0;
+    walk(p, lo_off, lo, row, &v, NULL, triples, cap, &n);
+    return n;
+}

@@ -1,0 +1,40 @@
+"""The pins must be able to fail: plant one plausible mistake at a time in a copy of the
+oracle (CPU only), rerun the pin tests against the copy and expect a failure."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "vl_oracle.c")
+
+MUTANTS = [
+    ("overlap uses <= (touching ranges collide)", "return a < b + wb && b < a + wa;", "return a <= b + wb && b < a + wa;"),
+    ("range check off by one", "if (s + w > p->P)", "if (s + w >= p->P)"),
+    ("definition compared with itself", "if (u == v) continue;", ""),
+    ("kill dropped from the block transfer function",
+     "uint8_t in = use[(size_t)b * V + v] | (o & !def[(size_t)b * V + v]);", "uint8_t in = use[(size_t)b * V + v] | o;"),
+    ("reads after writes count as upward exposed", "if (!def[(size_t)b * V + v]) use[(size_t)b * V + v] = 1;",
+     "use[(size_t)b * V + v] = 1;"),
+    ("writes before reads in the backward walk",
+     "for (uint32_t o = o0; o < o0 + nd; ++o) live[p->op_vreg[o]] = 0;\n            for (uint32_t o = o0 + nd; o < o1; ++o) live[p->op_vreg[o]] = 1;",
+     "for (uint32_t o = o0 + nd; o < o1; ++o) live[p->op_vreg[o]] = 1;\n            for (uint32_t o = o0; o < o0 + nd; ++o) live[p->op_vreg[o]] = 0;"),
+    ("duplicate source registers counted twice", "if (!dup) Q[nq++] = ta;", "Q[nq++] = ta;"),
+    ("bank cost n instead of n-1", "bank += n - 1;", "bank += n;"),
+    ("last occurrence wins", "if (T[v] < 0) T[v] = row[o];", "if (T[v] < 0 || 1) T[v] = row[o];"),
+    ("co-defined vregs ignored", "if (in_live) continue;", "continue;"),
+]
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_pins_catch_planted_mistake(tmp_path, name, old, new):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, "mutation site vanished: " + name
+    mutant = tmp_path / "vl_oracle_mutant.c"
+    mutant.write_text(text.replace(old, new))        # every occurrence
+    env = dict(os.environ, VL_ORACLE_MUTANT_SRC=str(mutant))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+                       cwd=ROOT, env=env, capture_output=True, text=True)
+    assert r.returncode == 1, f"pins did not notice: {name}\n{r.stdout[-400:]}"

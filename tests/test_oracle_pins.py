@@ -1,0 +1,324 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked against
+brute force, closed forms and hand-worked programs (no GPU)."""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2506_17506_b200 import synth
+from tests import helpers as H
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+PASS, INCONS, RANGE, INTERF = 1, 2, 4, 8
+
+
+def _oracle(oracle_mod, p):
+    op = oracle_mod.OracleProgram(p)
+    return op, op.liveness()
+
+
+# ------------------------------------------------------------------ liveness pins
+@pytest.mark.parametrize("seed", range(60))
+def test_liveness_equals_path_definition(oracle_mod, seed):
+    """Liveness is *defined* by paths; the fixed point must reproduce it exactly,
+    on strict and non-strict programs, with loops and unreachable blocks."""
+    p = H.random_program(seed, strict=(seed % 2 == 0), reachable=(seed % 3 != 0))
+    op, lv = _oracle(oracle_mod, p)
+    live_after, blk_in, blk_out = H.path_liveness(p)
+    for i in range(p.n_instrs):
+        assert list(lv.live_after(i)) == live_after[i], f"instr {i}"
+    assert np.array_equal(lv.blk_live_in, blk_in)
+    assert np.array_equal(lv.blk_live_out, blk_out)
+
+
+def test_liveness_closed_form_single_block(oracle_mod):
+    """One block: v is live after i iff the next event on v after i is a read."""
+    p = synth.build_program(synth.shape_tiny(), 0)
+    op, lv = _oracle(oracle_mod, p)
+    ins, _, _ = H.instr_lists(p)
+    for i in range(p.n_instrs):
+        expect = []
+        for v in range(p.n_vregs):
+            for j in range(i + 1, p.n_instrs):
+                d, u = ins[j]
+                if v in u:
+                    expect.append(v)
+                    break
+                if v in d:
+                    break
+        assert list(lv.live_after(i)) == expect
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_liveness_fixed_point_equations_and_sweep_order(oracle_mod, idx):
+    wl = synth.workload(idx)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    op = oracle_mod.OracleProgram(p)
+    a, b = op.liveness(order=0), op.liveness(order=1)
+    assert np.array_equal(a.blk_live_in, b.blk_live_in) and np.array_equal(a.blk_live_out, b.blk_live_out)
+    assert np.array_equal(a.lo_off, b.lo_off) and np.array_equal(a.lo, b.lo)
+    ins, blk, succ = H.instr_lists(p)
+    for bb in range(p.n_blocks):
+        out = np.zeros(p.n_vregs, dtype=np.uint8)
+        for s in succ[bb]:
+            out |= a.blk_live_in[s]
+        assert np.array_equal(out, a.blk_live_out[bb])
+    assert a.blk_live_in[0].sum() == 0          # the generator's programs are strict
+    # lists ascending, no duplicates
+    for i in range(0, p.n_instrs, max(1, p.n_instrs // 50)):
+        l = a.live_after(i)
+        assert np.all(np.diff(l.astype(np.int64)) > 0)
+
+
+# -------------------------------------------------------------- interference pins
+@pytest.mark.parametrize("seed", range(80))
+def test_def_point_rule_equals_all_pairs_definition(oracle_mod, seed):
+    """Strict programs with every block reachable: the set of vreg pairs that overlap
+    at a definition point equals the set of pairs that are ever live together with
+    intersecting ranges; so the interference flag is the all-pairs decision."""
+    p = H.random_program(1000 + seed, strict=True, reachable=True, P=12)
+    op, lv = _oracle(oracle_mod, p)
+    live_after, _, _ = H.path_liveness(p)
+    rng = np.random.default_rng(seed)
+    for trial in range(6):
+        T = rng.integers(0, p.P, size=p.n_vregs)
+        if trial == 0:
+            T[:] = 0
+        row = H.row_from_table(p, T)
+        tr = op.conflicts(lv, row)
+        dedup = {(min(int(v), int(u)), max(int(v), int(u))) for _, v, u in tr}
+        brute = H.copointed_overlapping_pairs(p, live_after, row)
+        assert dedup == brute
+        vd = op.verify(lv, row)[0]
+        assert bool(vd["flags"] & INTERF) == bool(brute)
+        assert vd["conflict_pairs"] == len(tr)
+        # each triple is a real overlap at a definition of v with u live after or co-defined
+        ins, _, _ = H.instr_lists(p)
+        w = p.vreg_width
+        for i, v, u in tr:
+            assert v in ins[i][0] and v != u
+            assert (u in live_after[i]) or (u in ins[i][0])
+            assert H.overlap(int(T[v]), int(w[v]), int(T[u]), int(w[u]))
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_conflict_count_closed_form_all_zero_candidate(oracle_mod, seed):
+    """All widths 1 and every vreg on register 0: every pair overlaps, so the count is
+    sum over definitions of |(live_after(i) | defs(i)) - {v}|, a function of liveness only."""
+    p = H.random_program(2000 + seed, strict=True, reachable=(seed % 2 == 0), widths=(1,))
+    op, lv = _oracle(oracle_mod, p)
+    live_after, _, _ = H.path_liveness(p)
+    ins, _, _ = H.instr_lists(p)
+    expect = sum(len((set(live_after[i]) | set(d)) - {v}) for i, (d, _) in enumerate(ins) for v in d)
+    vd = op.verify(lv, np.zeros(p.pitch, dtype=np.uint16))[0]
+    assert vd["conflict_pairs"] == expect
+    assert bool(vd["flags"] & INTERF) == (expect > 0)
+    assert not vd["flags"] & (INCONS | RANGE)
+
+
+def test_sequential_no_reuse_assignment(oracle_mod):
+    """Appendix B's pattern (a fresh register for every vreg, no reuse) can never
+    interfere; it is valid iff it fits in the register file, otherwise the first
+    violation is the lowest-index definition of a vreg that sticks out."""
+    shape = synth.shape_gemm()
+    p = synth.build_program(shape, 1)
+    w = p.vreg_width.astype(np.int64)
+    T = np.concatenate([[0], np.cumsum(w)[:-1]])
+    total = int(w.sum())
+    row = H.row_from_table(p, T)
+    for P in (total, total - 1, 256):
+        q = synth.Program(**{**p.__dict__, "P": P})
+        op, lv = _oracle(oracle_mod, q)
+        vd = op.verify(lv, row)[0]
+        assert vd["conflict_pairs"] == 0 and not vd["flags"] & (INTERF | INCONS)
+        if total <= P:
+            assert vd["flags"] == PASS and vd["first_violation_instr"] == -1
+        else:
+            assert vd["flags"] == RANGE
+            sticking = np.nonzero(T + w > P)[0]
+            assert vd["first_violation_instr"] == int(p.gen["first_def_instr"][sticking].min())
+
+
+# ------------------------------------------------------------------ bank pins
+def _bank_case(oracle_mod, regs, B=4, P=16):
+    n = len(regs)
+    blocks = [[([v], []) for v in range(n)] + [([n], list(range(n)))]]
+    p = synth.program_from_lists(blocks, [], n + 1, [1] * (n + 1), P, B)
+    # sources sit on `regs`; the result goes to a register none of them uses
+    free = [r for r in range(P) if r not in regs][0]
+    tab = list(regs) + [free]
+    # repeated registers among the sources would interfere at their definitions; the bank
+    # tally is defined regardless, which is what is checked here
+    op, lv = _oracle(oracle_mod, p)
+    return op.verify(lv, H.row_from_table(p, tab))[0]
+
+
+def test_bank_tally_paper_example_and_hand_cases(oracle_mod):
+    # Section 2: 4 banks; the FFMA of Figure 1 reads R4, R6, R9, which sit in separate banks.
+    with open(os.path.join(GOLDEN, "ffma_banks.txt")) as f:
+        lines = [l.split("#")[0].split() for l in f if l.strip() and not l.startswith("#")]
+    for toks in lines:
+        B, expect, regs = int(toks[0]), int(toks[1]), [int(t) for t in toks[2:]]
+        assert _bank_case(oracle_mod, regs, B=B)["bank_conflicts"] == expect, toks
+    assert _bank_case(oracle_mod, [4, 8])["bank_conflicts"] == 1
+    assert _bank_case(oracle_mod, [4, 8, 12])["bank_conflicts"] == 2
+    assert _bank_case(oracle_mod, [4, 4, 8])["bank_conflicts"] == 1     # same register read twice counts once
+    assert _bank_case(oracle_mod, [5])["bank_conflicts"] == 0
+    assert _bank_case(oracle_mod, [0, 1, 2, 3])["bank_conflicts"] == 0
+    assert _bank_case(oracle_mod, [0, 4, 1, 5])["bank_conflicts"] == 2
+    assert _bank_case(oracle_mod, [0, 4, 1, 5], B=1)["bank_conflicts"] == 3
+    assert _bank_case(oracle_mod, [1, 4, 7, 10], B=3)["bank_conflicts"] == 3
+
+
+# ------------------------------------------------------------ hand-built programs
+def test_hand_straight_line_with_reuse(oracle_mod):
+    #  i0: v0=       i1: v1=      i2: v2=f(v0,v1)     i3: v3=f(v2)     i4: =f(v3) (no def)
+    p = synth.program_from_lists([[([0], []), ([1], []), ([2], [0, 1]), ([3], [2]), ([], [3])]], [], 4, [1, 1, 1, 1], 2)
+    op, lv = _oracle(oracle_mod, p)
+    assert [list(lv.live_after(i)) for i in range(5)] == [[0], [0, 1], [2], [3], []]
+    ok = op.verify(lv, H.row_from_table(p, [0, 1, 0, 0]))[0]      # v2 reuses v0's register at its last use
+    assert tuple(ok) == (PASS, -1, 0, 0)
+    bad = op.verify(lv, H.row_from_table(p, [0, 0, 1, 0]))[0]     # v1 clobbers v0 while v0 is live
+    assert bad["flags"] == INTERF and bad["first_violation_instr"] == 1 and bad["conflict_pairs"] == 1
+    # bank tally of the bad row: i2 reads v0 and v1, same register -> one distinct source
+    assert bad["bank_conflicts"] == 0
+
+
+def test_hand_diamond_and_dead_def(oracle_mod):
+    # b0: v0= ; v1=       b1: v2=f(v0)      b2: v2=f(v1) ; v3= (dead)     b3: =f(v2)
+    blocks = [[([0], []), ([1], [])], [([2], [0])], [([2], [1]), ([3], [])], [([], [2])]]
+    p = synth.program_from_lists(blocks, [(0, 1), (0, 2), (1, 3), (2, 3)], 4, [1, 1, 1, 1], 3)
+    op, lv = _oracle(oracle_mod, p)
+    assert [list(lv.live_after(i)) for i in range(6)] == [[0], [0, 1], [2], [2], [2], []]
+    assert tuple(op.verify(lv, H.row_from_table(p, [0, 1, 0, 1]))[0]) == (PASS, -1, 0, 0)
+    # the dead def of v3 at instr 4 clobbers v2 (live after it): interference at its own instruction
+    vd = op.verify(lv, H.row_from_table(p, [0, 1, 2, 2]))[0]
+    assert vd["flags"] == INTERF and vd["first_violation_instr"] == 4 and vd["conflict_pairs"] == 1
+    # v2 on v1's register: b1 defines v2 while v1 is dead there, b2 reads v1 at the same instruction -> legal
+    assert op.verify(lv, H.row_from_table(p, [0, 1, 1, 0]))[0]["flags"] == PASS
+    # v2 on v0's register: in b2 v0 is dead as well -> legal
+    assert op.verify(lv, H.row_from_table(p, [0, 1, 0, 2]))[0]["flags"] == PASS
+
+
+def test_hand_loop_carried_and_self_update(oracle_mod):
+    # b0: acc= ; x=      b1 (self loop): t=f(x) ; acc=f(acc,t)       b2: =f(acc)
+    blocks = [[([0], []), ([1], [])], [([2], [1]), ([0], [0, 2])], [([], [0])]]
+    p = synth.program_from_lists(blocks, [(0, 1), (1, 1), (1, 2)], 3, [2, 1, 1], 4)
+    op, lv = _oracle(oracle_mod, p)
+    assert [list(lv.live_after(i)) for i in range(5)] == [[0], [0, 1], [0, 1, 2], [0, 1], []]
+    assert lv.blk_live_in.tolist() == [[0, 0, 0], [1, 1, 0], [1, 0, 0]]
+    assert lv.blk_live_out.tolist() == [[1, 1, 0], [1, 1, 0], [0, 0, 0]]
+    assert op.verify(lv, H.row_from_table(p, [0, 2, 3]))[0]["flags"] == PASS       # acc = {0,1}
+    # t on x's register: x is loop-invariant and live around the back edge
+    vd = op.verify(lv, H.row_from_table(p, [0, 2, 2]))[0]
+    assert vd["flags"] == INTERF and vd["first_violation_instr"] == 2 and vd["conflict_pairs"] == 1
+    # x inside the accumulator pair (register 1): seen at x's def (acc live) and at every def of acc
+    vd = op.verify(lv, H.row_from_table(p, [0, 1, 3]))[0]
+    assert vd["flags"] == INTERF and vd["first_violation_instr"] == 1 and vd["conflict_pairs"] == 2
+    # pair sticking out of a 4-register file
+    vd = op.verify(lv, H.row_from_table(p, [3, 0, 1]))[0]
+    assert vd["flags"] == RANGE and vd["first_violation_instr"] == 0 and vd["conflict_pairs"] == 0
+
+
+def test_hand_nested_loops(oracle_mod):
+    # b0: a= ; b=   b1(outer head): c=f(a)   b2(inner, self): d=f(c,b)   b3(latch -> b1): a=f(a,c)   b4: =f(a)
+    blocks = [[([0], []), ([1], [])], [([2], [0])], [([3], [2, 1])], [([0], [0, 2])], [([], [0])]]
+    edges = [(0, 1), (1, 2), (2, 2), (2, 3), (3, 1), (3, 4)]
+    p = synth.program_from_lists(blocks, edges, 4, [1, 1, 1, 1], 4)
+    op, lv = _oracle(oracle_mod, p)
+    assert [list(lv.live_after(i)) for i in range(6)] == [[0], [0, 1], [0, 1, 2], [0, 1, 2], [0, 1], []]
+    assert op.verify(lv, H.row_from_table(p, [0, 1, 2, 3]))[0]["flags"] == PASS
+    # d is dead (never read) but is written while a, b, c are live
+    vd = op.verify(lv, H.row_from_table(p, [0, 1, 2, 1]))[0]
+    assert vd["flags"] == INTERF and vd["first_violation_instr"] == 3
+
+
+def test_hand_wide_tuples_contiguity(oracle_mod):
+    """Section 2 / Section 4.5: a 64-bit value takes two consecutive registers
+    (vgpr0_vgpr1); anything placed on either of them while it is live collides."""
+    blocks = [[([0], []), ([1], []), ([], [0, 1])]]
+    p = synth.program_from_lists(blocks, [], 2, [2, 1], 8)
+    op, lv = _oracle(oracle_mod, p)
+    assert op.verify(lv, H.row_from_table(p, [0, 2]))[0]["flags"] == PASS
+    for clash in (0, 1):
+        vd = op.verify(lv, H.row_from_table(p, [0, clash]))[0]
+        assert vd["flags"] == INTERF and vd["first_violation_instr"] == 1
+    assert op.verify(lv, H.row_from_table(p, [7, 0]))[0]["flags"] == RANGE     # {7,8} leaves an 8-register file
+    assert op.verify(lv, H.row_from_table(p, [6, 0]))[0]["flags"] == PASS
+
+
+def test_hand_multi_def_instruction_and_inconsistency(oracle_mod):
+    # i0: (v0,v1)=     i1: v2=f(v0)     i2: =f(v1,v2)
+    p = synth.program_from_lists([[([0, 1], []), ([2], [0]), ([], [1, 2])]], [], 3, [1, 1, 1], 4)
+    op, lv = _oracle(oracle_mod, p)
+    assert [list(lv.live_after(i)) for i in range(3)] == [[0, 1], [1, 2], []]
+    # both results of i0 on one register: counted once from each side
+    vd = op.verify(lv, H.row_from_table(p, [0, 0, 1]))[0]
+    assert vd["flags"] == INTERF and vd["first_violation_instr"] == 0 and vd["conflict_pairs"] == 2
+    # inconsistent occurrence: v0 is R0 at its definition and R3 at its read; the table keeps R0
+    row = H.row_from_table(p, [0, 1, 2])
+    row[3] = 3
+    vd = op.verify(lv, row)[0]
+    assert vd["flags"] == INCONS and vd["first_violation_instr"] == 1 and vd["conflict_pairs"] == 0
+    # values beyond the file are compared as plain integers (no wrap)
+    vd = op.verify(lv, H.row_from_table(p, [65535, 65535, 0]))[0]
+    assert vd["flags"] == (RANGE | INTERF) and vd["conflict_pairs"] == 2
+
+
+def test_hand_unreachable_block_and_dead_code(oracle_mod):
+    # b0: v0= ; =f(v0)      b1 (unreachable): v1=f(v0)   -- v0 is not live into b0 (defined first)
+    blocks = [[([0], []), ([], [0])], [([1], [0])]]
+    p = synth.program_from_lists(blocks, [], 2, [1, 1], 2)
+    op, lv = _oracle(oracle_mod, p)
+    assert lv.blk_live_in.tolist() == [[0, 0], [1, 0]]
+    assert [list(lv.live_after(i)) for i in range(3)] == [[0], [], []]
+    assert op.verify(lv, H.row_from_table(p, [0, 0]))[0]["flags"] == PASS   # v1 may take v0's register: v0 dies at its read
+
+
+# ----------------------------------------------------------- generator-based pins
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_generator_valid_rows_pass_and_faults_fail_where_injected(oracle_mod, idx):
+    wl = synth.workload(idx)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    K = min(wl.K, 150)
+    rows, faults = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[0], 0, K)
+    clean, _ = synth.candidate_rows(p, wl.K, 0.0, wl.seeds[0], 0, K)
+    op, lv = _oracle(oracle_mod, p)
+    vd = op.verify(lv, rows)
+    vc = op.verify(lv, clean)
+    assert np.all(vc["flags"] == PASS) and np.all(vc["first_violation_instr"] == -1) and np.all(vc["conflict_pairs"] == 0)
+    kinds = faults[:, 0]
+    assert (kinds != 0).sum() > 0
+    for k in range(K):
+        kind, instr, v, u, o = [int(x) for x in faults[k]]
+        if kind == synth.FAULT_NONE:
+            assert tuple(vd[k]) == tuple(vc[k])
+        elif kind == synth.FAULT_INCONSISTENT:
+            # only the consistency bit; everything derived from the table is unchanged
+            assert vd[k]["flags"] == INCONS and vd[k]["first_violation_instr"] == instr
+            assert vd[k]["conflict_pairs"] == 0 and vd[k]["bank_conflicts"] == vc[k]["bank_conflicts"]
+        elif kind == synth.FAULT_RANGE:
+            assert vd[k]["flags"] == RANGE and vd[k]["first_violation_instr"] == instr
+            assert vd[k]["conflict_pairs"] == 0
+        else:
+            assert vd[k]["flags"] & INTERF and not vd[k]["flags"] & INCONS
+            assert 0 <= vd[k]["first_violation_instr"] <= instr
+            assert op.violations(lv, rows[k])[instr] & INTERF
+            tr = op.conflicts(lv, rows[k])
+            assert any((int(a), int(b), int(c)) == (instr, v, u) for a, b, c in tr)
+
+
+def test_generator_batch_members_and_stress_sample(oracle_mod):
+    wl = synth.workload(3)
+    for j in (0, 17, 255):
+        p = synth.build_program(wl.shapes[j], wl.seeds[j])
+        rows, faults = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[j], 0, 40)
+        op, lv = _oracle(oracle_mod, p)
+        vd = op.verify(lv, rows)
+        assert np.array_equal(vd["flags"] == PASS, faults[:, 0] == 0)
+    wl = synth.workload(4)
+    p = synth.build_program(synth.shape_stress(8000, 2500), 4)
+    rows, faults = synth.candidate_rows(p, 64, 0.25, 4)
+    op, lv = _oracle(oracle_mod, p)
+    vd = op.verify(lv, rows)
+    assert np.array_equal(vd["flags"] == PASS, faults[:, 0] == 0)
