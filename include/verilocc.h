@@ -1,0 +1,170 @@
+/*
+ * verilocc.h -- C ABI of the batch verifier for register-allocation candidates.
+ *
+ * The library checks K candidate allocations of one program (a GPU kernel in
+ * machine-IR form: basic blocks, CFG edges, per-instruction definitions and
+ * reads of virtual registers, register-tuple widths) against the correctness
+ * conditions of the paper:
+ *   Section 1, conditions (1) and (2); Section 3.4 "Consistency", "Safety",
+ *   "Realizability"; Section 2 (a wide value takes consecutive registers; the
+ *   register file has 4 banks and reads from one bank stall).
+ * The check is the polynomial-time one the paper names in Section 4.6 (following
+ * control and data dependence), not an SMT query.
+ *
+ * All functions return VL_OK (0) or a negative VL_ERR_* code; none throws,
+ * aborts or prints.  An invalid candidate is never an error, it is a verdict.
+ * The library is not thread-safe per program handle; distinct handles may be
+ * used from distinct threads.  There is no CPU fallback: every entry point that
+ * computes needs a CUDA device of compute capability 10.0.
+ */
+#ifndef VERILOCC_H
+#define VERILOCC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    VL_OK = 0,
+    VL_ERR_INVALID_ARG = -1,       /* null pointer, bad size, misaligned buffer */
+    VL_ERR_MALFORMED_PROGRAM = -2, /* CSR offsets not monotone, ids out of range, zero width, duplicate def */
+    VL_ERR_NOT_STRICT = -3,        /* some vreg is live into the entry block (read before any write) */
+    VL_ERR_LIVENESS_NOT_RUN = -4,  /* vl_verify* before a successful vl_liveness */
+    VL_ERR_UNSUPPORTED = -5,       /* program exceeds the shared-memory plan or a 32-bit size */
+    VL_ERR_NO_CONVERGE = -6,       /* liveness did not reach its fixed point within n_blocks + 2 sweeps */
+    VL_ERR_CUDA = -7,              /* a CUDA call failed; vl_last_cuda_error() has the code */
+    VL_ERR_DEVICE_WAIT = -8        /* a bounded wait inside a kernel gave up (copy engine never signalled) */
+};
+
+/* Verdict flag bits.  VL_PASS is set iff none of the others is. */
+enum { VL_PASS = 1u, VL_INCONSISTENT = 2u, VL_OUT_OF_RANGE = 4u, VL_INTERFERENCE = 8u };
+
+/* Tunables for vl_program_set_option (set before vl_liveness). */
+enum {
+    VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 128) */
+    VL_OPT_GROUP = 2         /* candidates per thread block: 0 = choose, else 1, 2 or 4 */
+};
+
+/*
+ * Program descriptor.  All pointers are HOST memory, read during
+ * vl_program_create only (borrowed, never freed, may be released afterwards).
+ *
+ * Instructions are numbered in layout order; block b owns instructions
+ * [block_instr_off[b], block_instr_off[b+1]); block 0 is the entry.  The
+ * operands of instruction i are [instr_op_off[i], instr_op_off[i+1]): first its
+ * instr_n_defs[i] definitions, then its reads.  An operand's index is its
+ * column in a candidate row.  Reads of an instruction happen before its writes.
+ * A vreg of width w mapped to physical register p occupies [p, p+w).
+ */
+typedef struct {
+    uint32_t n_blocks, n_instrs, n_vregs, n_operands, n_edges;
+    uint32_t P;                      /* physical registers, 1..65535 */
+    uint32_t B;                      /* register banks, >= 1 (bank = register mod B) */
+    const uint32_t *block_instr_off; /* [n_blocks+1] */
+    const uint32_t *succ_off;        /* [n_blocks+1] */
+    const uint32_t *succ;            /* [n_edges] successor block ids */
+    const uint32_t *instr_op_off;    /* [n_instrs+1] */
+    const uint8_t *instr_n_defs;     /* [n_instrs] */
+    const uint32_t *op_vreg;         /* [n_operands], each < n_vregs (n_vregs <= 65535) */
+    const uint8_t *vreg_width;       /* [n_vregs], 1..255 */
+} vl_program_desc;
+
+/* One record per candidate (16 bytes). */
+typedef struct {
+    uint32_t flags;                /* VL_PASS or an OR of the violation bits */
+    int32_t first_violation_instr; /* lowest instruction index carrying any violation; -1 if none */
+    uint32_t conflict_pairs;       /* (instruction, definition, other vreg) range overlaps, summed */
+    uint32_t bank_conflicts;       /* extra read cycles: per instruction, per bank, distinct source
+                                      base registers beyond the first (bank model of Section 2) */
+} vl_verdict;
+
+typedef struct vl_program vl_program; /* opaque; owns device copies of the program and of its liveness */
+
+/*
+ * Validates the descriptor on the host and uploads it to `device`.
+ * Errors: INVALID_ARG, MALFORMED_PROGRAM, UNSUPPORTED, CUDA.  *out is set only on VL_OK.
+ */
+int vl_program_create(const vl_program_desc *desc, int device, vl_program **out);
+
+/* Frees every device and host resource of the handle.  NULL is accepted. */
+void vl_program_destroy(vl_program *prog);
+
+/* Sets a tunable; must precede vl_liveness.  Errors: INVALID_ARG. */
+int vl_program_set_option(vl_program *prog, int option, uint32_t value);
+
+/*
+ * Liveness (what "overlapping life cycles" in Section 2 and "Safety" in Section 3.4
+ * rest on): per-block read/write bitsets, backward dataflow to the least fixed point,
+ * then the set of vregs live after every instruction as CSR lists (ascending ids),
+ * plus the per-program tables vl_verify consumes.  Runs on `cuda_stream`
+ * (a cudaStream_t, may be NULL) and synchronises it before returning, because list
+ * lengths and the status word are read back.
+ * Errors: NOT_STRICT, NO_CONVERGE, UNSUPPORTED, CUDA.
+ */
+int vl_liveness(vl_program *prog, void *cuda_stream);
+
+/*
+ * Device pointers to the liveness results; owned by the handle, valid until
+ * vl_program_destroy or the next vl_liveness.  Any out pointer may be NULL.
+ *   blk_live_in / blk_live_out : [n_blocks][ceil(n_vregs/32)] little-endian bitsets
+ *   lo_off [n_instrs+1], lo [lo_len] : vregs live after each instruction, ascending
+ */
+int vl_liveness_result(const vl_program *prog, const uint32_t **blk_live_in, const uint32_t **blk_live_out,
+                       const uint32_t **lo_off, const uint32_t **lo, uint64_t *lo_len);
+
+/*
+ * Checks K candidates.  d_cand is DEVICE memory, uint16, candidate-major:
+ * d_cand[k * pitch_elems + o] is the physical register candidate k gives operand o.
+ * Requirements: base 16-byte aligned, pitch_elems >= n_operands rounded up to 8,
+ * pitch_elems % 8 == 0.  d_out is DEVICE memory for K records (4-byte aligned).
+ * Buffers are borrowed for the call; the work is enqueued on `cuda_stream` and the
+ * function returns without synchronising.  K == 0 is a no-op.
+ *
+ * Per candidate (Section 3.4): T[v] = register at the first occurrence of v;
+ * Consistency: every occurrence equals T[v]; Realizability: at every definition
+ * [T[v], T[v]+width) lies inside [0, P); Safety: at every definition of v the range of
+ * v is disjoint from the range of every other vreg live after that instruction or
+ * defined by it.  Bank tally per Section 2 with B banks.
+ * Errors: INVALID_ARG, LIVENESS_NOT_RUN, UNSUPPORTED, CUDA.
+ */
+int vl_verify(const vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pitch_elems,
+              vl_verdict *d_out, void *cuda_stream);
+
+/*
+ * The same check for n independent programs in one call (all on the device of the
+ * first program): program j checks K[j] rows of d_cand[j] into d_out[j].  The arrays of
+ * pointers and sizes are HOST memory.  Stream-ordered, no synchronisation.
+ */
+int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
+                    const uint64_t *K, const uint64_t *pitch_elems, vl_verdict *const *d_out,
+                    void *cuda_stream);
+
+/*
+ * End-to-end form with HOST buffers: h_cand (K rows, same layout rules, ideally
+ * pinned) is copied to the device in slabs through two staging buffers owned by the
+ * handle, each slab is checked, and the verdicts are copied back to h_out.  Copies and
+ * kernels of successive slabs overlap on two internal streams; the call returns after
+ * everything has finished (it synchronises).  `cuda_stream` orders the start of the work.
+ * Errors: as vl_verify.
+ */
+int vl_verify_host(vl_program *prog, const uint16_t *h_cand, uint64_t K, uint64_t pitch_elems,
+                   vl_verdict *h_out, void *cuda_stream);
+
+/* Reads and clears the device-side status word of the handle's verify calls
+ * (VL_OK or VL_ERR_DEVICE_WAIT).  Synchronises `cuda_stream`. */
+int vl_verify_status(vl_program *prog, void *cuda_stream);
+
+/* Number of kernels this library has launched in this process (all handles). */
+uint64_t vl_kernel_launches(void);
+
+/* Last CUDA error code seen by the handle (0 if none). */
+int vl_last_cuda_error(const vl_program *prog);
+
+const char *vl_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VERILOCC_H */

@@ -1,0 +1,276 @@
+// C ABI entry points: program handle, validation, host-buffer verify, error strings.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "vl_internal.cuh"
+
+std::atomic<uint64_t> g_vl_launches{0};
+
+static int validate(const vl_program_desc *d)
+{
+    if (!d) return VL_ERR_INVALID_ARG;
+    if (!d->block_instr_off || !d->succ_off || !d->instr_op_off) return VL_ERR_INVALID_ARG;
+    if (d->n_edges && !d->succ) return VL_ERR_INVALID_ARG;
+    if (d->n_instrs && !d->instr_n_defs) return VL_ERR_INVALID_ARG;
+    if (d->n_operands && !d->op_vreg) return VL_ERR_INVALID_ARG;
+    if (d->n_vregs && !d->vreg_width) return VL_ERR_INVALID_ARG;
+    if (d->n_blocks == 0 || d->P == 0 || d->P > 65535 || d->B == 0) return VL_ERR_INVALID_ARG;
+    if (d->n_vregs > 65535) return VL_ERR_UNSUPPORTED;
+    if (d->n_operands > 0xFFFFFFF0u - 64 || d->n_instrs > 0x7FFFFFF0u) return VL_ERR_UNSUPPORTED;
+
+    if (d->block_instr_off[0] != 0 || d->block_instr_off[d->n_blocks] != d->n_instrs) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t b = 0; b < d->n_blocks; ++b)
+        if (d->block_instr_off[b] > d->block_instr_off[b + 1]) return VL_ERR_MALFORMED_PROGRAM;
+    if (d->succ_off[0] != 0 || d->succ_off[d->n_blocks] != d->n_edges) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t b = 0; b < d->n_blocks; ++b)
+        if (d->succ_off[b] > d->succ_off[b + 1]) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t e = 0; e < d->n_edges; ++e)
+        if (d->succ[e] >= d->n_blocks) return VL_ERR_MALFORMED_PROGRAM;
+    if (d->instr_op_off[0] != 0 || d->instr_op_off[d->n_instrs] != d->n_operands) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t i = 0; i < d->n_instrs; ++i) {
+        uint32_t o0 = d->instr_op_off[i], o1 = d->instr_op_off[i + 1];
+        if (o0 > o1 || o1 > d->n_operands) return VL_ERR_MALFORMED_PROGRAM;
+        if (d->instr_n_defs[i] > o1 - o0) return VL_ERR_MALFORMED_PROGRAM;
+    }
+    for (uint32_t o = 0; o < d->n_operands; ++o)
+        if (d->op_vreg[o] >= d->n_vregs) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t v = 0; v < d->n_vregs; ++v)
+        if (d->vreg_width[v] == 0) return VL_ERR_MALFORMED_PROGRAM;
+    for (uint32_t i = 0; i < d->n_instrs; ++i) {  // one instruction must not define a vreg twice
+        uint32_t o0 = d->instr_op_off[i], nd = d->instr_n_defs[i];
+        for (uint32_t a = 0; a < nd; ++a)
+            for (uint32_t b = a + 1; b < nd; ++b)
+                if (d->op_vreg[o0 + a] == d->op_vreg[o0 + b]) return VL_ERR_MALFORMED_PROGRAM;
+    }
+    return VL_OK;
+}
+
+template <typename T>
+static cudaError_t upload(T **dst, const T *src, size_t n)
+{
+    cudaError_t e = cudaMalloc((void **)dst, std::max<size_t>(n, 1) * sizeof(T) + 64);
+    if (e != cudaSuccess) return e;
+    if (n) e = cudaMemcpy(*dst, src, n * sizeof(T), cudaMemcpyHostToDevice);
+    return e;
+}
+
+extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_program **out)
+{
+    if (!out) return VL_ERR_INVALID_ARG;
+    int rc = validate(d);
+    if (rc != VL_OK) return rc;
+    vl_program *p = new (std::nothrow) vl_program();
+    if (!p) return VL_ERR_CUDA;
+    p->device = device;
+    p->nB = d->n_blocks; p->nI = d->n_instrs; p->V = d->n_vregs; p->nO = d->n_operands; p->nE = d->n_edges;
+    p->P = d->P; p->B = d->B;
+    p->Wv = std::max(1u, (p->V + 31) / 32);
+    p->nOp8 = std::max(8u, (p->nO + 7) / 8 * 8);
+    p->wmax = 1;
+    for (uint32_t v = 0; v < p->V; ++v) p->wmax = std::max<uint32_t>(p->wmax, d->vreg_width[v]);
+    p->h_blk_off.assign(d->block_instr_off, d->block_instr_off + p->nB + 1);
+    p->h_op_off.assign(d->instr_op_off, d->instr_op_off + p->nI + 1);
+
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = upload(&p->d_blk_off, d->block_instr_off, (size_t)p->nB + 1);
+    if (e == cudaSuccess) e = upload(&p->d_succ_off, d->succ_off, (size_t)p->nB + 1);
+    if (e == cudaSuccess) e = upload(&p->d_succ, d->succ, (size_t)p->nE);
+    if (e == cudaSuccess) e = upload(&p->d_op_off, d->instr_op_off, (size_t)p->nI + 1);
+    if (e == cudaSuccess) e = upload(&p->d_ndefs, d->instr_n_defs, (size_t)p->nI);
+    if (e == cudaSuccess) e = upload(&p->d_op_vreg, d->op_vreg, (size_t)p->nO);
+    if (e == cudaSuccess) e = upload(&p->d_width, d->vreg_width, (size_t)p->V);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_status, 64);
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 64);
+    if (e != cudaSuccess) {
+        p->last_cuda_error = (int)e;
+        vl_program_destroy(p);
+        return VL_ERR_CUDA;
+    }
+    *out = p;
+    return VL_OK;
+}
+
+void vl_free_liveness(vl_program *p)
+{
+    cudaFree(p->d_chunk_i0); cudaFree(p->d_chunk_i1); cudaFree(p->d_chunk_blk); cudaFree(p->d_blk_chunk_off);
+    cudaFree(p->d_blk_in); cudaFree(p->d_blk_out); cudaFree(p->d_lo_off); cudaFree(p->d_lo);
+    cudaFree(p->d_vreg16); cudaFree(p->d_slotmeta); cudaFree(p->d_opflags); cudaFree(p->d_first_def_instr);
+    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_grp_off); cudaFree(p->d_ev);
+    p->d_chunk_i0 = p->d_chunk_i1 = p->d_chunk_blk = p->d_blk_chunk_off = nullptr;
+    p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
+    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_first_def_instr = nullptr;
+    p->d_th_off = p->d_th = p->d_grp_off = p->d_ev = nullptr;
+    p->live_ok = false;
+    p->lo_len = 0;
+}
+
+extern "C" void vl_program_destroy(vl_program *p)
+{
+    if (!p) return;
+    cudaSetDevice(p->device);
+    vl_free_liveness(p);
+    cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
+    cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
+    for (int j = 0; j < 2; ++j) {
+        cudaFree(p->d_stage[j]);
+        cudaFree(p->d_stage_out[j]);
+        if (p->h_streams[j]) cudaStreamDestroy(p->h_streams[j]);
+        if (p->h_events[j]) cudaEventDestroy(p->h_events[j]);
+    }
+    delete p;
+}
+
+extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    switch (option) {
+    case VL_OPT_CHUNK_INSTRS:
+        if (value < 8 || value > 65536) return VL_ERR_INVALID_ARG;
+        p->chunk_instrs = value;
+        p->live_ok = false;
+        return VL_OK;
+    case VL_OPT_GROUP:
+        if (value != 0 && value != 1 && value != 2 && value != 4) return VL_ERR_INVALID_ARG;
+        p->group_opt = value;
+        return VL_OK;
+    default:
+        return VL_ERR_INVALID_ARG;
+    }
+}
+
+extern "C" int vl_liveness(vl_program *p, void *stream)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    VL_CUDA(p, cudaSetDevice(p->device));
+    return vl_liveness_impl(p, (cudaStream_t)stream);
+}
+
+extern "C" int vl_liveness_result(const vl_program *p, const uint32_t **blk_live_in, const uint32_t **blk_live_out,
+                                  const uint32_t **lo_off, const uint32_t **lo, uint64_t *lo_len)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    if (!p->live_ok) return VL_ERR_LIVENESS_NOT_RUN;
+    if (blk_live_in) *blk_live_in = p->d_blk_in;
+    if (blk_live_out) *blk_live_out = p->d_blk_out;
+    if (lo_off) *lo_off = p->d_lo_off;
+    if (lo) *lo = p->d_lo;
+    if (lo_len) *lo_len = p->lo_len;
+    return VL_OK;
+}
+
+static int check_verify_args(const vl_program *p, const void *cand, uint64_t K, uint64_t pitch, const void *out)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    if (!p->live_ok) return VL_ERR_LIVENESS_NOT_RUN;
+    if (K == 0) return VL_OK;
+    if (!cand || !out) return VL_ERR_INVALID_ARG;
+    if (((uintptr_t)cand & 15) || ((uintptr_t)out & 3)) return VL_ERR_INVALID_ARG;
+    if (pitch % 8 != 0 || pitch < p->nOp8) return VL_ERR_INVALID_ARG;
+    if (K > 0x7FFFFFFFull) return VL_ERR_INVALID_ARG;
+    return VL_OK;
+}
+
+extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+                         void *stream)
+{
+    int rc = check_verify_args(p, d_cand, K, pitch, d_out);
+    if (rc != VL_OK || K == 0) return rc;
+    cudaError_t e = cudaSetDevice(p->device);
+    if (e != cudaSuccess) return VL_ERR_CUDA;
+    return vl_verify_impl(p, d_cand, K, pitch, d_out, (cudaStream_t)stream);
+}
+
+extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
+                               const uint64_t *K, const uint64_t *pitch, vl_verdict *const *d_out, void *stream)
+{
+    if (n == 0) return VL_OK;
+    if (!progs || !d_cand || !K || !pitch || !d_out) return VL_ERR_INVALID_ARG;
+    for (uint32_t j = 0; j < n; ++j) {
+        int rc = check_verify_args(progs[j], d_cand[j], K[j], pitch[j], d_out[j]);
+        if (rc != VL_OK) return rc;
+        if (progs[j]->device != progs[0]->device) return VL_ERR_INVALID_ARG;
+    }
+    if (cudaSetDevice(progs[0]->device) != cudaSuccess) return VL_ERR_CUDA;
+    for (uint32_t j = 0; j < n; ++j) {
+        if (K[j] == 0) continue;
+        int rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], (cudaStream_t)stream);
+        if (rc != VL_OK) return rc;
+    }
+    return VL_OK;
+}
+
+extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K, uint64_t pitch, vl_verdict *h_out,
+                              void *stream)
+{
+    int rc = check_verify_args(p, h_cand, K, pitch, h_out);
+    if (rc != VL_OK || K == 0) return rc;
+    VL_CUDA(p, cudaSetDevice(p->device));
+    // slabs of about 64 MiB, a multiple of 4 rows
+    uint64_t rows = std::max<uint64_t>(4, ((64ull << 20) / (pitch * 2)) / 4 * 4);
+    rows = std::min<uint64_t>(rows, (K + 3) / 4 * 4);
+    if (p->stage_rows < rows || p->stage_pitch != pitch) {
+        for (int j = 0; j < 2; ++j) {
+            cudaFree(p->d_stage[j]); cudaFree(p->d_stage_out[j]);
+            p->d_stage[j] = nullptr; p->d_stage_out[j] = nullptr;
+        }
+        p->stage_rows = 0;
+        for (int j = 0; j < 2; ++j) {
+            VL_CUDA(p, cudaMalloc((void **)&p->d_stage[j], rows * pitch * 2));
+            VL_CUDA(p, cudaMalloc((void **)&p->d_stage_out[j], rows * sizeof(vl_verdict)));
+        }
+        p->stage_rows = rows;
+        p->stage_pitch = pitch;
+    }
+    rows = p->stage_rows;
+    for (int j = 0; j < 2; ++j) {
+        if (!p->h_streams[j]) VL_CUDA(p, cudaStreamCreateWithFlags(&p->h_streams[j], cudaStreamNonBlocking));
+        if (!p->h_events[j]) VL_CUDA(p, cudaEventCreateWithFlags(&p->h_events[j], cudaEventDisableTiming));
+    }
+    VL_CUDA(p, cudaEventRecord(p->h_events[0], (cudaStream_t)stream));
+    for (int j = 0; j < 2; ++j) VL_CUDA(p, cudaStreamWaitEvent(p->h_streams[j], p->h_events[0], 0));
+    uint64_t slab = 0;
+    for (uint64_t k0 = 0; k0 < K; k0 += rows, ++slab) {
+        int j = (int)(slab & 1);
+        uint64_t n = std::min(rows, K - k0);
+        VL_CUDA(p, cudaMemcpyAsync(p->d_stage[j], h_cand + k0 * pitch, n * pitch * 2, cudaMemcpyHostToDevice,
+                                   p->h_streams[j]));
+        rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j]);
+        if (rc != VL_OK) return rc;
+        VL_CUDA(p, cudaMemcpyAsync(h_out + k0, p->d_stage_out[j], n * sizeof(vl_verdict), cudaMemcpyDeviceToHost,
+                                   p->h_streams[j]));
+    }
+    for (int j = 0; j < 2; ++j) VL_CUDA(p, cudaStreamSynchronize(p->h_streams[j]));
+    return VL_OK;
+}
+
+extern "C" int vl_verify_status(vl_program *p, void *stream)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    VL_CUDA(p, cudaSetDevice(p->device));
+    uint32_t st = 0;
+    VL_CUDA(p, cudaMemcpyAsync(&st, p->d_status + 1, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    VL_CUDA(p, cudaMemsetAsync(p->d_status + 1, 0, 4, (cudaStream_t)stream));
+    VL_CUDA(p, cudaStreamSynchronize((cudaStream_t)stream));
+    return (st & ST_DEVICE_WAIT) ? VL_ERR_DEVICE_WAIT : VL_OK;
+}
+
+extern "C" uint64_t vl_kernel_launches(void) { return g_vl_launches.load(); }
+
+extern "C" int vl_last_cuda_error(const vl_program *p) { return p ? p->last_cuda_error : 0; }
+
+extern "C" const char *vl_strerror(int code)
+{
+    switch (code) {
+    case VL_OK: return "ok";
+    case VL_ERR_INVALID_ARG: return "invalid argument";
+    case VL_ERR_MALFORMED_PROGRAM: return "malformed program";
+    case VL_ERR_NOT_STRICT: return "program is not strict: a virtual register is live into the entry block";
+    case VL_ERR_LIVENESS_NOT_RUN: return "vl_liveness has not been run on this program";
+    case VL_ERR_UNSUPPORTED: return "program exceeds what the kernels support";
+    case VL_ERR_NO_CONVERGE: return "liveness did not converge";
+    case VL_ERR_CUDA: return "CUDA call failed";
+    case VL_ERR_DEVICE_WAIT: return "a bounded wait inside a kernel ran out";
+    default: return "unknown error";
+    }
+}

@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libverilocc.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "verilocc.h"
+
+// ---- per-operand flag byte written by the liveness walk (device array opflags[n_operands])
+enum : uint8_t {
+    OPF_DEF = 1,    // operand is a definition
+    OPF_KILL = 2,   // read: the value dies here (first read of the vreg in the instruction)
+    OPF_DUP = 4,    // read: same vreg read earlier by this instruction
+    OPF_ELIDE = 8,  // definition of a vreg the instruction also reads and that stays live:
+                    //   occupancy unchanged, no walk event
+    OPF_SET = 16,   // definition: becomes occupied (live after, or several defs in the instruction)
+    OPF_POST = 32,  // definition: dead, released again after the instruction's definitions
+    OPF_DEAD = 64   // definition: vreg not live after the instruction
+};
+
+// ---- walk events (one 32-bit word): vreg | width << 16 | type bits
+enum : uint32_t { EV_TEST = 1u << 24, EV_SET = 1u << 25, EV_CLEAR = 1u << 26 };
+
+// ---- device status word bits (prog->d_status[0] liveness, d_status[1] verify)
+enum : uint32_t {
+    ST_NO_CONVERGE = 1u,
+    ST_NOT_STRICT = 2u,
+    ST_MANY_USES = 4u,      // some instruction reads more than 4 operands (bank tally takes the general path)
+    ST_SIZE_OVERFLOW = 8u,  // a list length does not fit 32 bits
+    ST_DEVICE_WAIT = 16u    // a bounded wait in a verify kernel ran out
+};
+
+#define VL_MAX_GROUP 4
+
+struct vl_program {
+    int device = 0;
+    uint32_t nB = 0, nI = 0, V = 0, nO = 0, nE = 0, P = 0, B = 0;
+    uint32_t Wv = 0;    // 32-bit words per vreg bitset
+    uint32_t nOp8 = 0;  // n_operands rounded up to 8 (at least 8)
+    uint32_t wmax = 1;  // widest vreg
+    uint32_t chunk_instrs = 128;
+    uint32_t group_opt = 0;
+
+    // chunks: every chunk lies inside one block
+    uint32_t nC = 0;
+    std::vector<uint32_t> h_chunk_i0, h_chunk_i1, h_chunk_blk, h_blk_chunk_off;
+    std::vector<uint32_t> h_blk_off, h_op_off;
+
+    // device copies of the program
+    uint32_t *d_blk_off = nullptr, *d_succ_off = nullptr, *d_succ = nullptr, *d_op_off = nullptr, *d_op_vreg = nullptr;
+    uint8_t *d_ndefs = nullptr, *d_width = nullptr;
+    uint32_t *d_chunk_i0 = nullptr, *d_chunk_i1 = nullptr, *d_chunk_blk = nullptr, *d_blk_chunk_off = nullptr;
+
+    // liveness results
+    uint32_t *d_blk_in = nullptr, *d_blk_out = nullptr, *d_lo_off = nullptr, *d_lo = nullptr;
+    uint64_t lo_len = 0;
+
+    // tables consumed by the verify kernels
+    uint16_t *d_vreg16 = nullptr;           // [nOp8 + 8] vreg id per operand (padding operands: id V)
+    uint64_t *d_slotmeta = nullptr;         // [nOp8 / 8] per 8 operands: first-occurrence bits, bank compare masks
+    uint8_t *d_opflags = nullptr;           // [nO]
+    uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
+    uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
+    uint32_t th_len = 0;
+    uint32_t nGroups = 0;           // groups of 32 chunks
+    uint32_t *d_grp_off = nullptr;  // [nGroups+1] first step of each group
+    uint32_t *d_ev = nullptr;       // [steps][32] walk events, lane = chunk within its group
+    uint32_t ev_steps = 0;
+    int bank_fast = 0;  // B in {1,2,4} and every instruction reads <= 4 operands
+    int use_th = 0;
+
+    uint32_t *d_status = nullptr;  // [16] device status words
+    int last_cuda_error = 0;
+    bool live_ok = false;
+
+    // staging for vl_verify_host
+    uint16_t *d_stage[2] = {nullptr, nullptr};
+    vl_verdict *d_stage_out[2] = {nullptr, nullptr};
+    uint64_t stage_rows = 0, stage_pitch = 0;
+    cudaStream_t h_streams[2] = {nullptr, nullptr};
+    cudaEvent_t h_events[2] = {nullptr, nullptr};
+};
+
+extern std::atomic<uint64_t> g_vl_launches;
+
+#define VL_CUDA(prog, call)                     \
+    do {                                        \
+        cudaError_t e__ = (call);               \
+        if (e__ != cudaSuccess) {               \
+            (prog)->last_cuda_error = (int)e__; \
+            return VL_ERR_CUDA;                 \
+        }                                       \
+    } while (0)
+
+int vl_liveness_impl(vl_program *p, cudaStream_t st);
+int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+                   cudaStream_t st);
+void vl_free_liveness(vl_program *p);
