@@ -1,0 +1,237 @@
+"""Thin ctypes binding onto ``libverilocc.so``: argument marshalling only.
+
+Same names as the C ABI (``include/verilocc.h``).  torch is used for device memory and
+streams, nothing else; every step of the check runs in the library's CUDA kernels.
+Importing this module fails loudly when the library has not been built
+(``python -m paper_2506_17506_b200.build``); there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libverilocc.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_17506_b200.build` "
+                      "(needs nvcc); this package has no CPU fallback")
+_lib = C.CDLL(LIB_PATH)
+
+VL_OK = 0
+VL_ERR_INVALID_ARG, VL_ERR_MALFORMED_PROGRAM, VL_ERR_NOT_STRICT, VL_ERR_LIVENESS_NOT_RUN = -1, -2, -3, -4
+VL_ERR_UNSUPPORTED, VL_ERR_NO_CONVERGE, VL_ERR_CUDA, VL_ERR_DEVICE_WAIT = -5, -6, -7, -8
+VL_PASS, VL_INCONSISTENT, VL_OUT_OF_RANGE, VL_INTERFERENCE = 1, 2, 4, 8
+VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP = 1, 2
+
+EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness",
+           "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
+           "vl_kernel_launches", "vl_last_cuda_error", "vl_strerror"]
+
+VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
+                          ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
+
+
+class vl_program_desc(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("n_blocks", "n_instrs", "n_vregs", "n_operands", "n_edges", "P", "B")] + [
+        ("block_instr_off", C.c_void_p), ("succ_off", C.c_void_p), ("succ", C.c_void_p),
+        ("instr_op_off", C.c_void_p), ("instr_n_defs", C.c_void_p), ("op_vreg", C.c_void_p),
+        ("vreg_width", C.c_void_p)]
+
+
+_lib.vl_program_create.restype = C.c_int
+_lib.vl_program_create.argtypes = [C.POINTER(vl_program_desc), C.c_int, C.POINTER(C.c_void_p)]
+_lib.vl_program_destroy.restype = None
+_lib.vl_program_destroy.argtypes = [C.c_void_p]
+_lib.vl_program_set_option.restype = C.c_int
+_lib.vl_program_set_option.argtypes = [C.c_void_p, C.c_int, C.c_uint32]
+_lib.vl_liveness.restype = C.c_int
+_lib.vl_liveness.argtypes = [C.c_void_p, C.c_void_p]
+_lib.vl_liveness_result.restype = C.c_int
+_lib.vl_liveness_result.argtypes = [C.c_void_p] + [C.POINTER(C.c_void_p)] * 4 + [C.POINTER(C.c_uint64)]
+_lib.vl_verify.restype = C.c_int
+_lib.vl_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+_lib.vl_verify_batch.restype = C.c_int
+_lib.vl_verify_batch.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.vl_verify_host.restype = C.c_int
+_lib.vl_verify_host.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+_lib.vl_verify_status.restype = C.c_int
+_lib.vl_verify_status.argtypes = [C.c_void_p, C.c_void_p]
+_lib.vl_kernel_launches.restype = C.c_uint64
+_lib.vl_kernel_launches.argtypes = []
+_lib.vl_last_cuda_error.restype = C.c_int
+_lib.vl_last_cuda_error.argtypes = [C.c_void_p]
+_lib.vl_strerror.restype = C.c_char_p
+_lib.vl_strerror.argtypes = [C.c_int]
+
+
+class VlError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        self.code = code
+        msg = f"{where}: {vl_strerror(code)} ({code})"
+        if cuda:
+            msg += f" [cuda error {cuda}]"
+        super().__init__(msg)
+
+
+def vl_strerror(code: int) -> str:
+    return _lib.vl_strerror(code).decode()
+
+
+def vl_kernel_launches() -> int:
+    return int(_lib.vl_kernel_launches())
+
+
+def _stream_ptr(stream) -> C.c_void_p:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(int(getattr(stream, "cuda_stream", stream)))
+
+
+def make_desc(prog):
+    """(descriptor, keep-alive arrays) from any object with the descriptor's fields as numpy arrays."""
+    keep = dict(
+        block_instr_off=np.ascontiguousarray(prog.block_instr_off, dtype=np.uint32),
+        succ_off=np.ascontiguousarray(prog.succ_off, dtype=np.uint32),
+        succ=np.ascontiguousarray(prog.succ, dtype=np.uint32),
+        instr_op_off=np.ascontiguousarray(prog.instr_op_off, dtype=np.uint32),
+        instr_n_defs=np.ascontiguousarray(prog.instr_n_defs, dtype=np.uint8),
+        op_vreg=np.ascontiguousarray(prog.op_vreg, dtype=np.uint32),
+        vreg_width=np.ascontiguousarray(prog.vreg_width, dtype=np.uint8),
+    )
+    def ptr(a):
+        return a.ctypes.data if a.size else None
+    d = vl_program_desc(prog.n_blocks, prog.n_instrs, prog.n_vregs, prog.n_operands, prog.n_edges, prog.P, prog.B,
+                        ptr(keep["block_instr_off"]), ptr(keep["succ_off"]), ptr(keep["succ"]),
+                        ptr(keep["instr_op_off"]), ptr(keep["instr_n_defs"]), ptr(keep["op_vreg"]),
+                        ptr(keep["vreg_width"]))
+    return d, keep
+
+
+def vl_program_create_raw(desc: vl_program_desc, device: int = 0):
+    """Returns (code, handle) without raising; for error-path tests."""
+    h = C.c_void_p()
+    rc = _lib.vl_program_create(C.byref(desc) if desc is not None else None, device, C.byref(h))
+    return rc, h
+
+
+class _DevView:
+    """Borrowed view of library-owned device memory (int32 elements) for torch.as_tensor."""
+
+    def __init__(self, ptr: int, count: int):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<i4", "data": (ptr, True), "version": 2}
+
+
+class Program:
+    """Owns a ``vl_program`` handle."""
+
+    def __init__(self, prog, device: int = 0):
+        self.n_blocks, self.n_instrs, self.n_vregs = prog.n_blocks, prog.n_instrs, prog.n_vregs
+        self.n_operands = prog.n_operands
+        self.pitch = max(8, (prog.n_operands + 7) // 8 * 8)
+        self.device = device
+        desc, keep = make_desc(prog)
+        self._h = C.c_void_p()
+        rc = _lib.vl_program_create(C.byref(desc), device, C.byref(self._h))
+        if rc != VL_OK:
+            self._h = C.c_void_p()
+            raise VlError(rc, "vl_program_create")
+
+    def _check(self, rc: int, where: str):
+        if rc != VL_OK:
+            raise VlError(rc, where, _lib.vl_last_cuda_error(self._h))
+
+    def set_option(self, option: int, value: int):
+        self._check(_lib.vl_program_set_option(self._h, option, value), "vl_program_set_option")
+
+    def vl_liveness(self, stream=None):
+        self._check(_lib.vl_liveness(self._h, _stream_ptr(stream)), "vl_liveness")
+
+    def vl_liveness_result(self):
+        """Copies of the liveness results as numpy arrays:
+        (blk_live_in [nB, W] u32, blk_live_out [nB, W] u32, lo_off [nI+1] u32, lo [len] u32)."""
+        import torch
+        p = [C.c_void_p() for _ in range(4)]
+        n = C.c_uint64()
+        self._check(_lib.vl_liveness_result(self._h, *[C.byref(x) for x in p], C.byref(n)), "vl_liveness_result")
+        W = max(1, (self.n_vregs + 31) // 32)
+        sizes = [self.n_blocks * W, self.n_blocks * W, self.n_instrs + 1, int(n.value)]
+        out = []
+        torch.cuda.synchronize(self.device)
+        for ptr, cnt in zip(p, sizes):
+            if cnt:
+                view = _DevView(ptr.value, cnt)
+                out.append(torch.as_tensor(view, device=f"cuda:{self.device}").cpu().numpy().view(np.uint32).copy())
+            else:
+                out.append(np.zeros(0, dtype=np.uint32))
+        return out[0].reshape(self.n_blocks, W), out[1].reshape(self.n_blocks, W), out[2], out[3]
+
+    def vl_verify(self, cand, out=None, stream=None):
+        """cand: CUDA uint16 tensor [K, pitch]; returns a CUDA int32 tensor [K, 4]
+        (flags, first_violation_instr, conflict_pairs, bank_conflicts)."""
+        import torch
+        assert cand.is_cuda and cand.dtype in (torch.uint16, torch.int16) and cand.dim() == 2 and cand.is_contiguous()
+        K, pitch = cand.shape
+        if out is None:
+            out = torch.empty((K, 4), dtype=torch.int32, device=cand.device)
+        self._check(_lib.vl_verify(self._h, cand.data_ptr(), K, pitch, out.data_ptr(), _stream_ptr(stream)), "vl_verify")
+        return out
+
+    def vl_verify_host(self, cand: "np.ndarray | object", out: np.ndarray | None = None, stream=None):
+        """cand: host uint16 [K, pitch] (numpy array or pinned CPU tensor); returns a numpy verdict array."""
+        if hasattr(cand, "data_ptr"):
+            K, pitch = cand.shape
+            ptr = cand.data_ptr()
+        else:
+            assert cand.dtype == np.uint16 and cand.ndim == 2 and cand.flags.c_contiguous
+            K, pitch = cand.shape
+            ptr = cand.ctypes.data
+        if out is None:
+            out = np.zeros(K, dtype=VERDICT_DTYPE)
+        optr = out.data_ptr() if hasattr(out, "data_ptr") else out.ctypes.data
+        self._check(_lib.vl_verify_host(self._h, ptr, K, pitch, optr, _stream_ptr(stream)), "vl_verify_host")
+        return out
+
+    def vl_verify_status(self, stream=None):
+        self._check(_lib.vl_verify_status(self._h, _stream_ptr(stream)), "vl_verify_status")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def close(self):
+        if self._h:
+            _lib.vl_program_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def vl_verify_batch(programs, cands, outs=None, stream=None):
+    """One call over n programs; cands[j] is the CUDA uint16 [K_j, pitch_j] tensor of program j."""
+    import torch
+    n = len(programs)
+    if outs is None:
+        outs = [torch.empty((c.shape[0], 4), dtype=torch.int32, device=c.device) for c in cands]
+    hp = (C.c_void_p * n)(*[p.handle for p in programs])
+    cp = (C.c_void_p * n)(*[c.data_ptr() for c in cands])
+    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+    Ks = (C.c_uint64 * n)(*[c.shape[0] for c in cands])
+    Ps = (C.c_uint64 * n)(*[c.shape[1] for c in cands])
+    rc = _lib.vl_verify_batch(n, hp, cp, Ks, Ps, op, _stream_ptr(stream))
+    if rc != VL_OK:
+        raise VlError(rc, "vl_verify_batch")
+    return outs
+
+
+def verdicts_to_numpy(t) -> np.ndarray:
+    """CUDA/CPU int32 [K, 4] tensor -> structured numpy array."""
+    a = t.detach().cpu().numpy().astype(np.int32, copy=False)
+    return np.ascontiguousarray(a).view(VERDICT_DTYPE).reshape(-1)

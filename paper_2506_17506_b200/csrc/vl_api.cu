@@ -96,7 +96,8 @@ void vl_free_liveness(vl_program *p)
     cudaFree(p->d_chunk_i0); cudaFree(p->d_chunk_i1); cudaFree(p->d_chunk_blk); cudaFree(p->d_blk_chunk_off);
     cudaFree(p->d_blk_in); cudaFree(p->d_blk_out); cudaFree(p->d_lo_off); cudaFree(p->d_lo);
     cudaFree(p->d_vreg16); cudaFree(p->d_slotmeta); cudaFree(p->d_opflags); cudaFree(p->d_first_def_instr);
-    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_grp_off); cudaFree(p->d_ev);
+    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_grp_off); cudaFree(p->d_ev); cudaFree(p->d_vinfo);
+    p->d_vinfo = nullptr;
     p->d_chunk_i0 = p->d_chunk_i1 = p->d_chunk_blk = p->d_blk_chunk_off = nullptr;
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
     p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_first_def_instr = nullptr;

@@ -20,8 +20,10 @@ enum : uint8_t {
     OPF_DEAD = 64   // definition: vreg not live after the instruction
 };
 
-// ---- walk events (one 32-bit word): vreg | width << 16 | type bits
+// ---- walk events (one 32-bit word): vreg | width << 16 | type bits.  A no-op event names the
+// spare table entry V with width 1 and no type bit.
 enum : uint32_t { EV_TEST = 1u << 24, EV_SET = 1u << 25, EV_CLEAR = 1u << 26 };
+enum : uint32_t { VINFO_OCCURS = 1u << 8, VINFO_DEFINED = 1u << 9 };
 
 // ---- device status word bits (prog->d_status[0] liveness, d_status[1] verify)
 enum : uint32_t {
@@ -62,6 +64,7 @@ struct vl_program {
     uint64_t *d_slotmeta = nullptr;         // [nOp8 / 8] per 8 operands: first-occurrence bits, bank compare masks
     uint8_t *d_opflags = nullptr;           // [nO]
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
+    uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
     uint32_t th_len = 0;
     uint32_t nGroups = 0;           // groups of 32 chunks

@@ -1,0 +1,595 @@
+// Liveness on the GPU and the per-program tables the verify kernels consume.
+//
+// Pipeline (all kernels on the caller's stream):
+//   chunk read/write sets -> block sets -> fixed point over blocks (one thread per
+//   bitset word) -> live set at every chunk boundary -> backward walk of every chunk
+//   (count, then fill) giving the per-instruction live-after lists in CSR form and the
+//   per-operand flags -> operand metadata, walk events, through-sets.
+#include <algorithm>
+#include <vector>
+
+#include "vl_internal.cuh"
+
+#define NT 128  // threads per block in every kernel of this file
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ bool bit_get(const uint32_t *s, uint32_t v) { return (s[v >> 5] >> (v & 31)) & 1u; }
+__device__ __forceinline__ void bit_set(uint32_t *s, uint32_t v) { s[v >> 5] |= 1u << (v & 31); }
+__device__ __forceinline__ void bit_clr(uint32_t *s, uint32_t v) { s[v >> 5] &= ~(1u << (v & 31)); }
+
+// Exclusive scan over the NT threads of a block; *total gets the block sum.
+// s_scan needs 34 words.  Contains barriers: every thread of the block must call it.
+__device__ uint32_t block_excl_scan(uint32_t x, uint32_t *s_scan, uint32_t *total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += y;
+    }
+    __syncthreads();  // protects s_scan against readers of a previous call
+    if (lane == 31) s_scan[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        uint32_t t = lane < NT / 32 ? s_scan[lane] : 0u;
+        uint32_t ti = t;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t y = __shfl_up_sync(0xffffffffu, ti, d);
+            if (lane >= d) ti += y;
+        }
+        if (lane < NT / 32) s_scan[lane] = ti - t;
+        if (lane == 31) s_scan[33] = ti;
+    }
+    __syncthreads();
+    *total = s_scan[33];
+    return s_scan[w] + inc - x;
+}
+
+// Calls emit(rank, bit index) for every set bit of words[0..nwords), ranks ascending with
+// the bit index.  Contains barriers.
+template <class F>
+__device__ void compact_bits(const uint32_t *words, uint32_t nwords, uint32_t *s_scan, uint32_t *total, F emit)
+{
+    const uint32_t per = (nwords + NT - 1) / NT;
+    const uint32_t w0 = min(nwords, threadIdx.x * per), w1 = min(nwords, w0 + per);
+    uint32_t cnt = 0;
+    for (uint32_t w = w0; w < w1; ++w) cnt += __popc(words[w]);
+    uint32_t off = block_excl_scan(cnt, s_scan, total);
+    for (uint32_t w = w0; w < w1; ++w) {
+        uint32_t x = words[w];
+        while (x) {
+            uint32_t b = __ffs(x) - 1;
+            x &= x - 1;
+            emit(off++, w * 32 + b);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------- kernels
+// Per chunk: use = vregs read before any write inside the chunk, def = vregs written.
+__global__ void k_chunk_sets(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
+                             const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                             const uint32_t *__restrict__ op_vreg, uint32_t Wv, uint32_t *chunk_use,
+                             uint32_t *chunk_def)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t *s_use = sm, *s_def = sm + Wv;
+    const uint32_t c = blockIdx.x;
+    for (uint32_t w = threadIdx.x; w < 2 * Wv; w += NT) sm[w] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (uint32_t i = chunk_i0[c]; i < chunk_i1[c]; ++i) {
+            const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+            for (uint32_t o = o0 + nd; o < o1; ++o) {  // reads first
+                uint32_t v = op_vreg[o];
+                if (!bit_get(s_def, v)) bit_set(s_use, v);
+            }
+            for (uint32_t o = o0; o < o0 + nd; ++o) bit_set(s_def, op_vreg[o]);
+        }
+    }
+    __syncthreads();
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        chunk_use[(size_t)c * Wv + w] = s_use[w];
+        chunk_def[(size_t)c * Wv + w] = s_def[w];
+    }
+}
+
+// Per block: compose the chunk sets in order.
+__global__ void k_block_sets(const uint32_t *__restrict__ blk_chunk_off, uint32_t Wv,
+                             const uint32_t *__restrict__ chunk_use, const uint32_t *__restrict__ chunk_def,
+                             uint32_t *blk_use, uint32_t *blk_def)
+{
+    const uint32_t b = blockIdx.x;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        uint32_t u = 0, d = 0;
+        for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) {
+            u |= chunk_use[(size_t)c * Wv + w] & ~d;
+            d |= chunk_def[(size_t)c * Wv + w];
+        }
+        blk_use[(size_t)b * Wv + w] = u;
+        blk_def[(size_t)b * Wv + w] = d;
+    }
+}
+
+// Backward dataflow to the least fixed point.  Bitset words are independent of each other,
+// so one thread iterates one word column over all blocks until nothing changes; no barrier.
+__global__ void k_fixed_point(uint32_t nB, uint32_t Wv, const uint32_t *__restrict__ succ_off,
+                              const uint32_t *__restrict__ succ, const uint32_t *__restrict__ blk_use,
+                              const uint32_t *__restrict__ blk_def, uint32_t *live_in, uint32_t *live_out,
+                              uint32_t *status)
+{
+    const uint32_t w = blockIdx.x * NT + threadIdx.x;
+    if (w >= Wv) return;
+    bool changed = true;
+    for (uint32_t sweep = 0; sweep < nB + 2 && changed; ++sweep) {
+        changed = false;
+        for (uint32_t n = 0; n < nB; ++n) {
+            const uint32_t b = nB - 1 - n;
+            uint32_t o = 0;
+            for (uint32_t e = succ_off[b]; e < succ_off[b + 1]; ++e) o |= live_in[(size_t)succ[e] * Wv + w];
+            const uint32_t in = blk_use[(size_t)b * Wv + w] | (o & ~blk_def[(size_t)b * Wv + w]);
+            if (o != live_out[(size_t)b * Wv + w] || in != live_in[(size_t)b * Wv + w]) changed = true;
+            live_out[(size_t)b * Wv + w] = o;
+            live_in[(size_t)b * Wv + w] = in;
+        }
+    }
+    if (changed) atomicOr(status, ST_NO_CONVERGE);
+    if (live_in[w] != 0) atomicOr(status, ST_NOT_STRICT);  // block 0 is the entry
+}
+
+// Live set after the last instruction of every chunk (chunk_end) and before its first (chunk_entry).
+__global__ void k_chunk_boundaries(const uint32_t *__restrict__ blk_chunk_off, uint32_t Wv,
+                                   const uint32_t *__restrict__ live_out, const uint32_t *__restrict__ chunk_use,
+                                   const uint32_t *__restrict__ chunk_def, uint32_t *chunk_end, uint32_t *chunk_entry)
+{
+    const uint32_t b = blockIdx.x;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        uint32_t live = live_out[(size_t)b * Wv + w];
+        for (uint32_t c = blk_chunk_off[b + 1]; c-- > blk_chunk_off[b];) {
+            chunk_end[(size_t)c * Wv + w] = live;
+            live = chunk_use[(size_t)c * Wv + w] | (live & ~chunk_def[(size_t)c * Wv + w]);
+            chunk_entry[(size_t)c * Wv + w] = live;
+        }
+    }
+}
+
+// Backward walk of one chunk.  FILL = false: list sizes, per-operand flags, walk-event counts,
+// and the set of vregs whose occupancy changes inside the chunk.  FILL = true: the lists.
+template <bool FILL>
+__global__ void k_instr_walk(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
+                             const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                             const uint32_t *__restrict__ op_vreg, uint32_t Wv,
+                             const uint32_t *__restrict__ chunk_end, uint32_t *lo_cnt, uint32_t *ev_cnt,
+                             uint8_t *opflags, uint32_t *chunk_touch, const uint32_t *__restrict__ lo_off,
+                             uint32_t *lo)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t *s_live = sm, *s_touch = sm + Wv;
+    __shared__ uint32_t s_scan[34];
+    const uint32_t c = blockIdx.x;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        s_live[w] = chunk_end[(size_t)c * Wv + w];
+        if (!FILL) s_touch[w] = 0;
+    }
+    __syncthreads();
+    for (uint32_t i = chunk_i1[c]; i-- > chunk_i0[c];) {
+        uint32_t total;
+        if (FILL) {
+            const uint32_t base = lo_off[i];
+            compact_bits(s_live, Wv, s_scan, &total, [&](uint32_t rank, uint32_t v) { lo[base + rank] = v; });
+        } else {
+            uint32_t cnt = 0;
+            for (uint32_t w = threadIdx.x; w < Wv; w += NT) cnt += __popc(s_live[w]);
+            block_excl_scan(cnt, s_scan, &total);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+            if (!FILL) {
+                lo_cnt[i] = total;
+                uint32_t evs = 0;
+                for (uint32_t o = o0 + nd; o < o1; ++o) {
+                    const uint32_t v = op_vreg[o];
+                    bool dup = false, isdef = false;
+                    for (uint32_t q = o0 + nd; q < o; ++q) dup |= (op_vreg[q] == v);
+                    for (uint32_t q = o0; q < o0 + nd; ++q) isdef |= (op_vreg[q] == v);
+                    const bool lv = bit_get(s_live, v);
+                    const bool kill = !dup && !lv;  // a read of a vreg that stays live releases nothing
+                    opflags[o] = (uint8_t)((kill ? OPF_KILL : 0) | (dup ? OPF_DUP : 0));
+                    if (kill) { ++evs; bit_set(s_touch, v); }
+                }
+                for (uint32_t o = o0; o < o0 + nd; ++o) {
+                    const uint32_t v = op_vreg[o];
+                    bool selfuse = false;
+                    for (uint32_t q = o0 + nd; q < o1; ++q) selfuse |= (op_vreg[q] == v);
+                    const bool lv = bit_get(s_live, v);
+                    const bool elide = selfuse && lv;
+                    const bool set = lv || nd > 1;
+                    const bool post = !lv && nd > 1;
+                    opflags[o] = (uint8_t)(OPF_DEF | (elide ? OPF_ELIDE : 0) | (set ? OPF_SET : 0) |
+                                           (post ? OPF_POST : 0) | (lv ? 0 : OPF_DEAD));
+                    if (!elide) { evs += 1 + (post ? 1 : 0); bit_set(s_touch, v); }
+                }
+                ev_cnt[i] = evs;
+            }
+            for (uint32_t o = o0; o < o0 + nd; ++o) bit_clr(s_live, op_vreg[o]);
+            for (uint32_t o = o0 + nd; o < o1; ++o) bit_set(s_live, op_vreg[o]);
+        }
+        __syncthreads();
+    }
+    if (!FILL)
+        for (uint32_t w = threadIdx.x; w < Wv; w += NT) chunk_touch[(size_t)c * Wv + w] = s_touch[w];
+}
+
+// Exclusive scan of a u32 array by one block; out[n] = total (saturated), total64 exact.
+__global__ void k_scan(const uint32_t *__restrict__ in, uint32_t *out, uint32_t n, unsigned long long *total64,
+                       uint32_t *status)
+{
+    __shared__ uint32_t s_scan[34];
+    unsigned long long carry = 0;
+    for (uint32_t base = 0; base < n; base += NT) {
+        const uint32_t idx = base + threadIdx.x;
+        const uint32_t x = idx < n ? in[idx] : 0u;
+        uint32_t total;
+        const uint32_t ex = block_excl_scan(x, s_scan, &total);
+        if (idx < n) out[idx] = (uint32_t)(carry + ex);
+        carry += total;
+    }
+    if (threadIdx.x == 0) {
+        out[n] = carry > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)carry;
+        *total64 = carry;
+        if (carry > 0xFFFFFFF0ull) atomicOr(status, ST_SIZE_OVERFLOW);
+    }
+}
+
+// Through-set of a block: live on entry and never touched by a walk event inside it.
+__global__ void k_block_through(const uint32_t *__restrict__ blk_chunk_off, uint32_t Wv, int use_th,
+                                const uint32_t *__restrict__ live_in, const uint32_t *__restrict__ chunk_touch,
+                                uint32_t *blk_th)
+{
+    const uint32_t b = blockIdx.x;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        uint32_t t = 0;
+        for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) t |= chunk_touch[(size_t)c * Wv + w];
+        blk_th[(size_t)b * Wv + w] = use_th ? (live_in[(size_t)b * Wv + w] & ~t) : 0u;
+    }
+}
+
+// chunk_entry &= ~through(block); entry count; events of the chunk = entries + instruction events.
+__global__ void k_chunk_entry(const uint32_t *__restrict__ chunk_blk, const uint32_t *__restrict__ chunk_i0,
+                              const uint32_t *__restrict__ chunk_i1, uint32_t Wv,
+                              const uint32_t *__restrict__ blk_th, uint32_t *chunk_entry,
+                              const uint32_t *__restrict__ ev_off, uint32_t *centry_cnt, uint32_t *cev)
+{
+    __shared__ uint32_t s_scan[34];
+    const uint32_t c = blockIdx.x, b = chunk_blk[c];
+    uint32_t cnt = 0;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+        const uint32_t x = chunk_entry[(size_t)c * Wv + w] & ~blk_th[(size_t)b * Wv + w];
+        chunk_entry[(size_t)c * Wv + w] = x;
+        cnt += __popc(x);
+    }
+    uint32_t total;
+    block_excl_scan(cnt, s_scan, &total);
+    if (threadIdx.x == 0) {
+        centry_cnt[c] = total;
+        cev[c] = total + (ev_off[chunk_i1[c]] - ev_off[chunk_i0[c]]);
+    }
+}
+
+__global__ void k_row_popc(uint32_t Wv, const uint32_t *__restrict__ rows, uint32_t *cnt)
+{
+    __shared__ uint32_t s_scan[34];
+    const uint32_t r = blockIdx.x;
+    uint32_t c = 0;
+    for (uint32_t w = threadIdx.x; w < Wv; w += NT) c += __popc(rows[(size_t)r * Wv + w]);
+    uint32_t total;
+    block_excl_scan(c, s_scan, &total);
+    if (threadIdx.x == 0) cnt[r] = total;
+}
+
+// Per instruction: vreg id per operand (16 bit), first occurrence / first definition of every
+// vreg, and the bank-compare distances of every read.
+__global__ void k_first_occ(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                            const uint32_t *__restrict__ op_vreg, uint32_t *first_occ, uint32_t *first_def_instr)
+{
+    const uint32_t i = blockIdx.x * NT + threadIdx.x;
+    if (i >= nI) return;
+    const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+    for (uint32_t o = o0; o < o1; ++o) {
+        atomicMin(&first_occ[op_vreg[o]], o);
+        if (o < o0 + nd) atomicMin(&first_def_instr[op_vreg[o]], i);
+    }
+}
+
+__global__ void k_vreg_info(uint32_t V, const uint8_t *__restrict__ width, const uint32_t *__restrict__ first_occ,
+                            const uint32_t *__restrict__ first_def_instr, uint32_t *vinfo)
+{
+    const uint32_t v = blockIdx.x * NT + threadIdx.x;
+    if (v >= V) return;
+    vinfo[v] = width[v] | (first_occ[v] != 0xFFFFFFFFu ? VINFO_OCCURS : 0u) |
+               (first_def_instr[v] != 0xFFFFFFFFu ? VINFO_DEFINED : 0u);
+}
+
+__global__ void k_fill_u32(uint32_t *dst, size_t n, uint32_t value)
+{
+    for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT) dst[i] = value;
+}
+
+__global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                               const uint32_t *__restrict__ op_vreg, const uint32_t *__restrict__ first_occ,
+                               const uint8_t *__restrict__ opflags, uint16_t *vreg16, uint8_t *opmeta,
+                               uint32_t *status)
+{
+    const uint32_t i = blockIdx.x * NT + threadIdx.x;
+    if (i >= nI) return;
+    const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+    if (o1 - o0 - nd > 4) atomicOr(status, ST_MANY_USES);
+    for (uint32_t o = o0; o < o1; ++o) {
+        const uint32_t v = op_vreg[o];
+        uint8_t m = (first_occ[v] == o) ? 1 : 0;
+        if (o >= o0 + nd && !(opflags[o] & OPF_DUP)) {
+            const uint32_t u = o - (o0 + nd);  // reads of this instruction before this one
+            if (u >= 1) m |= 2;
+            if (u >= 2) m |= 4;
+            if (u >= 3) m |= 8;
+        }
+        vreg16[o] = (uint16_t)v;
+        opmeta[o] = m;
+    }
+}
+
+// Per 8 operands: bits 0..7 first occurrence; for d = 1..3 a 16-bit field at 8 + 16 (d-1) with
+// bit 2 j set when operand j compares its bank with the operand d places before it.
+__global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8_t *__restrict__ opmeta,
+                             uint16_t *vreg16, uint64_t *slotmeta)
+{
+    const uint32_t s = blockIdx.x * NT + threadIdx.x;
+    if (s >= nOp8 / 8) return;
+    uint64_t m = 0;
+    for (uint32_t j = 0; j < 8; ++j) {
+        const uint32_t o = s * 8 + j;
+        if (o >= nO) {
+            vreg16[o] = (uint16_t)V;  // padding operand: writes the spare table entry, never compared
+            m |= 1ull << j;
+            continue;
+        }
+        const uint8_t x = opmeta[o];
+        if (x & 1) m |= 1ull << j;
+        if (x & 2) m |= 1ull << (8 + 2 * j);
+        if (x & 4) m |= 1ull << (24 + 2 * j);
+        if (x & 8) m |= 1ull << (40 + 2 * j);
+    }
+    slotmeta[s] = m;
+}
+
+// Walk events of one chunk: entry occupancy (ascending vreg id), then per instruction the
+// releases of dying reads, the definitions, and the releases of dead co-definitions.
+__global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
+                              const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                              const uint32_t *__restrict__ op_vreg, const uint8_t *__restrict__ width,
+                              const uint8_t *__restrict__ opflags, uint32_t Wv,
+                              const uint32_t *__restrict__ chunk_entry, const uint32_t *__restrict__ centry_cnt,
+                              const uint32_t *__restrict__ ev_off, const uint32_t *__restrict__ grp_off,
+                              uint32_t *ev)
+{
+    __shared__ uint32_t s_scan[34];
+    const uint32_t c = blockIdx.x;
+    const size_t base = (size_t)grp_off[c >> 5] * 32 + (c & 31);
+    uint32_t total;
+    compact_bits(chunk_entry + (size_t)c * Wv, Wv, s_scan, &total, [&](uint32_t rank, uint32_t v) {
+        ev[base + (size_t)rank * 32] = v | ((uint32_t)width[v] << 16) | EV_TEST | EV_SET;
+    });
+    const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
+    const uint32_t e_base = centry_cnt[c];
+    for (uint32_t i = i0 + threadIdx.x; i < i1; i += NT) {
+        uint32_t e = e_base + (ev_off[i] - ev_off[i0]);
+        const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+        for (uint32_t o = o0 + nd; o < o1; ++o)
+            if (opflags[o] & OPF_KILL) {
+                const uint32_t v = op_vreg[o];
+                ev[base + (size_t)(e++) * 32] = v | ((uint32_t)width[v] << 16) | EV_CLEAR;
+            }
+        for (uint32_t o = o0; o < o0 + nd; ++o)
+            if (!(opflags[o] & OPF_ELIDE)) {
+                const uint32_t v = op_vreg[o];
+                ev[base + (size_t)(e++) * 32] =
+                    v | ((uint32_t)width[v] << 16) | EV_TEST | ((opflags[o] & OPF_SET) ? EV_SET : 0u);
+            }
+        for (uint32_t o = o0; o < o0 + nd; ++o)
+            if ((opflags[o] & OPF_POST) && !(opflags[o] & OPF_ELIDE)) {
+                const uint32_t v = op_vreg[o];
+                ev[base + (size_t)(e++) * 32] = v | ((uint32_t)width[v] << 16) | EV_CLEAR;
+            }
+    }
+}
+
+__global__ void k_fill_through(uint32_t Wv, const uint32_t *__restrict__ blk_th, const uint8_t *__restrict__ width,
+                               const uint32_t *__restrict__ th_off, uint32_t *th)
+{
+    __shared__ uint32_t s_scan[34];
+    const uint32_t b = blockIdx.x;
+    const uint32_t base = th_off[b];
+    uint32_t total;
+    compact_bits(blk_th + (size_t)b * Wv, Wv, s_scan, &total,
+                 [&](uint32_t rank, uint32_t v) { th[base + rank] = v | ((uint32_t)width[v] << 16); });
+}
+
+// --------------------------------------------------------------------------- host
+namespace {
+struct Scratch {
+    std::vector<void *> ptrs;
+    ~Scratch() { for (void *q : ptrs) cudaFree(q); }
+    template <typename T>
+    cudaError_t get(T **out, size_t n, bool zero, cudaStream_t st)
+    {
+        cudaError_t e = cudaMalloc((void **)out, std::max<size_t>(n, 1) * sizeof(T) + 64);
+        if (e != cudaSuccess) return e;
+        ptrs.push_back(*out);
+        if (zero) e = cudaMemsetAsync(*out, 0, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
+        return e;
+    }
+};
+template <typename T>
+cudaError_t keep(T **out, size_t n, int fill, cudaStream_t st)
+{
+    cudaError_t e = cudaMalloc((void **)out, std::max<size_t>(n, 1) * sizeof(T) + 64);
+    if (e != cudaSuccess) return e;
+    return cudaMemsetAsync(*out, fill, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
+}
+}  // namespace
+
+#define LAUNCH(kernel, grid, smem, st, ...)                          \
+    do {                                                             \
+        if ((grid) > 0) {                                            \
+            kernel<<<(grid), NT, (smem), (st)>>>(__VA_ARGS__);       \
+            g_vl_launches.fetch_add(1);                              \
+        }                                                            \
+    } while (0)
+
+int vl_liveness_impl(vl_program *p, cudaStream_t st)
+{
+    vl_free_liveness(p);
+    const uint32_t nB = p->nB, nI = p->nI, V = p->V, nO = p->nO, Wv = p->Wv;
+
+    // ---- chunks: split every block into pieces of about chunk_instrs instructions
+    p->h_chunk_i0.clear(); p->h_chunk_i1.clear(); p->h_chunk_blk.clear();
+    p->h_blk_chunk_off.assign(nB + 1, 0);
+    for (uint32_t b = 0; b < nB; ++b) {
+        const uint64_t s = p->h_blk_off[b], n = p->h_blk_off[b + 1] - s;
+        const uint64_t nc = (n + p->chunk_instrs - 1) / p->chunk_instrs;
+        for (uint64_t j = 0; j < nc; ++j) {
+            p->h_chunk_i0.push_back((uint32_t)(s + j * n / nc));
+            p->h_chunk_i1.push_back((uint32_t)(s + (j + 1) * n / nc));
+            p->h_chunk_blk.push_back(b);
+        }
+        p->h_blk_chunk_off[b + 1] = (uint32_t)p->h_chunk_i0.size();
+    }
+    const uint32_t nC = p->nC = (uint32_t)p->h_chunk_i0.size();
+    p->nGroups = (nC + 31) / 32;
+
+    const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
+    p->use_th = ((uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
+    const size_t smem2 = (size_t)2 * Wv * 4;
+
+    VL_CUDA(p, keep(&p->d_chunk_i0, nC, 0, st));
+    VL_CUDA(p, keep(&p->d_chunk_i1, nC, 0, st));
+    VL_CUDA(p, keep(&p->d_chunk_blk, nC, 0, st));
+    VL_CUDA(p, keep(&p->d_blk_chunk_off, (size_t)nB + 1, 0, st));
+    if (nC) {
+        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_i0, p->h_chunk_i0.data(), nC * 4, cudaMemcpyHostToDevice, st));
+        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_i1, p->h_chunk_i1.data(), nC * 4, cudaMemcpyHostToDevice, st));
+        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_blk, p->h_chunk_blk.data(), nC * 4, cudaMemcpyHostToDevice, st));
+    }
+    VL_CUDA(p, cudaMemcpyAsync(p->d_blk_chunk_off, p->h_blk_chunk_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
+    VL_CUDA(p, keep(&p->d_blk_in, (size_t)nB * Wv, 0, st));
+    VL_CUDA(p, keep(&p->d_blk_out, (size_t)nB * Wv, 0, st));
+    VL_CUDA(p, keep(&p->d_lo_off, (size_t)nI + 1, 0, st));
+    VL_CUDA(p, keep(&p->d_opflags, (size_t)nO, 0, st));
+    VL_CUDA(p, keep(&p->d_first_def_instr, (size_t)V, 0xFF, st));
+    VL_CUDA(p, keep(&p->d_vreg16, (size_t)p->nOp8 + 8, 0, st));
+    VL_CUDA(p, keep(&p->d_slotmeta, (size_t)p->nOp8 / 8, 0, st));
+    VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
+
+    Scratch sc;
+    uint32_t *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry, *blk_use, *blk_def, *blk_th;
+    uint32_t *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
+    uint8_t *opmeta;
+    unsigned long long *totals;
+    VL_CUDA(p, sc.get(&chunk_use, (size_t)nC * Wv, false, st));
+    VL_CUDA(p, sc.get(&chunk_def, (size_t)nC * Wv, false, st));
+    VL_CUDA(p, sc.get(&chunk_touch, (size_t)nC * Wv, false, st));
+    VL_CUDA(p, sc.get(&chunk_end, (size_t)nC * Wv, false, st));
+    VL_CUDA(p, sc.get(&chunk_entry, (size_t)nC * Wv, false, st));
+    VL_CUDA(p, sc.get(&blk_use, (size_t)nB * Wv, false, st));
+    VL_CUDA(p, sc.get(&blk_def, (size_t)nB * Wv, false, st));
+    VL_CUDA(p, sc.get(&blk_th, (size_t)nB * Wv, false, st));
+    VL_CUDA(p, sc.get(&lo_cnt, (size_t)nI + 1, true, st));
+    VL_CUDA(p, sc.get(&ev_cnt, (size_t)nI + 1, true, st));
+    VL_CUDA(p, sc.get(&ev_off, (size_t)nI + 1, true, st));
+    VL_CUDA(p, sc.get(&centry_cnt, (size_t)nC, true, st));
+    VL_CUDA(p, sc.get(&cev, (size_t)nC, true, st));
+    VL_CUDA(p, sc.get(&th_cnt, (size_t)nB, true, st));
+    VL_CUDA(p, sc.get(&first_occ, (size_t)V, false, st));
+    VL_CUDA(p, cudaMemsetAsync(first_occ, 0xFF, std::max<size_t>(V, 1) * 4, st));
+    VL_CUDA(p, sc.get(&opmeta, (size_t)nO, true, st));
+    VL_CUDA(p, sc.get(&totals, 4, true, st));
+
+    LAUNCH(k_chunk_sets, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, Wv,
+           chunk_use, chunk_def);
+    LAUNCH(k_block_sets, nB, 0, st, p->d_blk_chunk_off, Wv, chunk_use, chunk_def, blk_use, blk_def);
+    LAUNCH(k_fixed_point, (Wv + NT - 1) / NT, 0, st, nB, Wv, p->d_succ_off, p->d_succ, blk_use, blk_def, p->d_blk_in,
+           p->d_blk_out, p->d_status);
+    LAUNCH(k_chunk_boundaries, nB, 0, st, p->d_blk_chunk_off, Wv, p->d_blk_out, chunk_use, chunk_def, chunk_end,
+           chunk_entry);
+    LAUNCH(k_instr_walk<false>, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
+           Wv, chunk_end, lo_cnt, ev_cnt, p->d_opflags, chunk_touch, (const uint32_t *)nullptr, (uint32_t *)nullptr);
+    LAUNCH(k_scan, 1, 0, st, lo_cnt, p->d_lo_off, nI, totals + 0, p->d_status);
+    LAUNCH(k_scan, 1, 0, st, ev_cnt, ev_off, nI, totals + 1, p->d_status);
+    LAUNCH(k_block_through, nB, 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
+    LAUNCH(k_chunk_entry, nC, 0, st, p->d_chunk_blk, p->d_chunk_i0, p->d_chunk_i1, Wv, blk_th, chunk_entry, ev_off,
+           centry_cnt, cev);
+    LAUNCH(k_row_popc, nB, 0, st, Wv, blk_th, th_cnt);
+
+    // ---- read back sizes and status
+    uint32_t status = 0;
+    unsigned long long h_tot[2] = {0, 0};
+    std::vector<uint32_t> h_cev(nC), h_thc(nB);
+    VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 16, cudaMemcpyDeviceToHost, st));
+    if (nC) VL_CUDA(p, cudaMemcpyAsync(h_cev.data(), cev, nC * 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaMemcpyAsync(h_thc.data(), th_cnt, nB * 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaStreamSynchronize(st));
+    if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
+    if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
+    if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
+    p->lo_len = h_tot[0];
+
+    std::vector<uint32_t> h_grp_off(p->nGroups + 1, 0), h_th_off(nB + 1, 0);
+    uint64_t steps = 0;
+    for (uint32_t g = 0; g < p->nGroups; ++g) {
+        uint32_t mx = 0;
+        for (uint32_t c = g * 32; c < std::min(nC, g * 32 + 32); ++c) mx = std::max(mx, h_cev[c]);
+        h_grp_off[g] = (uint32_t)steps;
+        steps += mx;
+    }
+    h_grp_off[p->nGroups] = (uint32_t)steps;
+    uint64_t thn = 0;
+    for (uint32_t b = 0; b < nB; ++b) { h_th_off[b] = (uint32_t)thn; thn += h_thc[b]; }
+    h_th_off[nB] = (uint32_t)thn;
+    if (steps * 32 > 0xFFFFFFF0ull) return VL_ERR_UNSUPPORTED;
+    p->ev_steps = (uint32_t)steps;
+    p->th_len = (uint32_t)thn;
+
+    VL_CUDA(p, keep(&p->d_lo, (size_t)p->lo_len, 0, st));
+    VL_CUDA(p, keep(&p->d_ev, (size_t)steps * 32, 0, st));
+    VL_CUDA(p, keep(&p->d_vinfo, (size_t)V, 0, st));
+    LAUNCH(k_fill_u32, (uint32_t)std::min<uint64_t>(1024, (steps * 32 + NT - 1) / NT), 0, st, p->d_ev,
+           (size_t)steps * 32, V | (1u << 16));  // every slot starts as a no-op event
+    VL_CUDA(p, keep(&p->d_th, (size_t)thn, 0, st));
+    VL_CUDA(p, keep(&p->d_grp_off, (size_t)p->nGroups + 1, 0, st));
+    VL_CUDA(p, keep(&p->d_th_off, (size_t)nB + 1, 0, st));
+    VL_CUDA(p, cudaMemcpyAsync(p->d_grp_off, h_grp_off.data(), (p->nGroups + 1) * 4, cudaMemcpyHostToDevice, st));
+    VL_CUDA(p, cudaMemcpyAsync(p->d_th_off, h_th_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
+
+    LAUNCH(k_instr_walk<true>, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
+           Wv, chunk_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr, (uint32_t *)nullptr,
+           (const uint32_t *)p->d_lo_off, p->d_lo);
+    LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+           p->d_first_def_instr);
+    LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, st, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
+    LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+           p->d_opflags, p->d_vreg16, opmeta, p->d_status);
+    LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, st, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
+    LAUNCH(k_fill_events, nC, 0, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
+           p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_grp_off, p->d_ev);
+    LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
+    VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaStreamSynchronize(st));
+    VL_CUDA(p, cudaGetLastError());
+    p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !(status & ST_MANY_USES)) ? 1 : 0;
+    p->live_ok = true;
+    return VL_OK;
+}

@@ -1,0 +1,211 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI, field by field and bit-exact."""
+import numpy as np
+import pytest
+
+from paper_2506_17506_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2506_17506_b200 import binding
+    return binding
+
+
+def _to_dev(rows):
+    import torch
+    return torch.from_numpy(rows.view(np.int16)).cuda().view(torch.uint16)
+
+
+def _gpu_verify(B, gp, rows):
+    import torch
+    out = gp.vl_verify(_to_dev(rows))
+    torch.cuda.synchronize()
+    gp.vl_verify_status()
+    return B.verdicts_to_numpy(out)
+
+
+def _assert_same(got, want, what=""):
+    for f in ("flags", "first_violation_instr", "conflict_pairs", "bank_conflicts"):
+        bad = np.nonzero(got[f] != want[f])[0]
+        assert len(bad) == 0, f"{what} field {f}: rows {bad[:8]} got {got[f][bad[:8]]} want {want[f][bad[:8]]}"
+
+
+def _check_liveness(B, oracle_mod, p, gp=None):
+    gp = gp or B.Program(p)
+    gp.vl_liveness()
+    bin_, bout, lo_off, lo = gp.vl_liveness_result()
+    lv = oracle_mod.OracleProgram(p).liveness()
+    assert np.array_equal(bin_, lv.packed("in"))
+    assert np.array_equal(bout, lv.packed("out"))
+    assert np.array_equal(lo_off.astype(np.uint64), lv.lo_off)
+    assert np.array_equal(lo, lv.lo)
+    return gp, lv
+
+
+def _garbage_rows(p, n, seed):
+    rng = np.random.default_rng(seed)
+    rows = np.zeros((n, p.pitch), dtype=np.uint16)
+    for k in range(n):
+        mode = k % 6
+        if mode == 0:
+            rows[k, :] = 0
+        elif mode == 1:
+            rows[k, :] = 0xFFFF
+        elif mode == 2:                                   # consistent random table inside the file
+            rows[k] = H.row_from_table(p, rng.integers(0, p.P, size=p.n_vregs))
+        elif mode == 3:                                   # consistent random table, partly outside
+            rows[k] = H.row_from_table(p, rng.integers(0, p.P + 40, size=p.n_vregs))
+        elif mode == 4:                                   # per-operand noise (inconsistent)
+            rows[k, : p.n_operands] = rng.integers(0, p.P, size=p.n_operands)
+        else:                                             # full 16-bit noise
+            rows[k, : p.n_operands] = rng.integers(0, 65536, size=p.n_operands)
+    return rows
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_small_programs(B, oracle_mod, seed):
+    """Random CFGs with multi-definition instructions, wide tuples and >4 reads per instruction;
+    valid-ish and garbage rows; every verdict field must match."""
+    p = H.random_program(5000 + seed, strict=True, reachable=(seed % 4 != 0), max_instrs=60, max_vregs=20,
+                         P=[8, 16, 33, 64][seed % 4], widths=(1, 1, 2, 2, 4, 8) if seed % 2 else (1, 2, 3, 5),
+                         B=[4, 4, 2, 1, 3, 8][seed % 6])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    rows = _garbage_rows(p, 48, seed)
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    for G in (0, 1, 2, 4):
+        gp.set_option(B.VL_OPT_GROUP, G)
+        _assert_same(_gpu_verify(B, gp, rows), want, f"seed {seed} G {G}")
+    gp.close()
+
+
+def test_hand_programs(B, oracle_mod):
+    cases = []
+    cases.append((synth.program_from_lists([[([0], []), ([1], []), ([2], [0, 1]), ([3], [2]), ([], [3])]], [], 4, [1] * 4, 2),
+                  [[0, 1, 0, 0], [0, 0, 1, 0]]))
+    cases.append((synth.program_from_lists([[([0], []), ([1], [])], [([2], [1]), ([0], [0, 2])], [([], [0])]],
+                                           [(0, 1), (1, 1), (1, 2)], 3, [2, 1, 1], 4),
+                  [[0, 2, 3], [0, 2, 2], [0, 1, 3], [3, 0, 1]]))
+    cases.append((synth.program_from_lists([[([0, 1], []), ([2], [0]), ([], [1, 2])]], [], 3, [1, 1, 1], 4),
+                  [[0, 0, 1], [0, 1, 2], [65535, 65535, 0]]))
+    cases.append((synth.program_from_lists([[([0], []), ([], [0])], [([1], [0])]], [], 2, [1, 1], 2), [[0, 0], [1, 1]]))
+    for p, tables in cases:
+        gp, lv = _check_liveness(B, oracle_mod, p)
+        rows = np.stack([H.row_from_table(p, t) for t in tables])
+        rows[-1, min(3, p.n_operands - 1)] ^= 1           # one inconsistent row as well
+        _assert_same(_gpu_verify(B, gp, rows), oracle_mod.OracleProgram(p).verify(lv, rows))
+        gp.close()
+
+
+def test_not_strict_and_order_errors(B):
+    p = synth.program_from_lists([[([], [0]), ([0], [])]], [], 1, [1], 4)      # reads v0 before writing it
+    gp = B.Program(p)
+    with pytest.raises(B.VlError) as e:
+        gp.vl_liveness()
+    assert e.value.code == B.VL_ERR_NOT_STRICT
+    import torch
+    cand = torch.zeros((1, 8), dtype=torch.int16, device="cuda").view(torch.uint16)
+    with pytest.raises(B.VlError) as e:
+        gp.vl_verify(cand)
+    assert e.value.code == B.VL_ERR_LIVENESS_NOT_RUN
+    gp.close()
+    ok = synth.program_from_lists([[([0], []), ([], [0])]], [], 1, [1], 4)
+    gp = B.Program(ok)
+    gp.vl_liveness()
+    bad_pitch = torch.zeros((1, 12), dtype=torch.int16, device="cuda").view(torch.uint16)
+    with pytest.raises(B.VlError) as e:
+        gp.vl_verify(bad_pitch)
+    assert e.value.code == B.VL_ERR_INVALID_ARG
+    empty = torch.zeros((0, 8), dtype=torch.int16, device="cuda").view(torch.uint16)
+    assert gp.vl_verify(empty).shape[0] == 0
+    gp.close()
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_workloads_full(B, oracle_mod, idx):
+    """Workloads 1-3 in full: every row of the seeded candidate matrix."""
+    wl = synth.workload(idx)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    rows, faults = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[0])
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    got = _gpu_verify(B, gp, rows)
+    _assert_same(got, want, wl.name)
+    assert np.array_equal(got["flags"] == B.VL_PASS, faults[:, 0] == 0)
+    # host-buffer entry point gives the same records
+    host = gp.vl_verify_host(rows)
+    _assert_same(host, want, wl.name + " host")
+    # extra rows: garbage of every kind
+    rows2 = _garbage_rows(p, 24, idx)
+    _assert_same(_gpu_verify(B, gp, rows2), oracle_mod.OracleProgram(p).verify(lv, rows2), wl.name + " garbage")
+    gp.close()
+
+
+@pytest.mark.parametrize("chunk,G", [(16, 4), (64, 2), (512, 1), (4096, 0)])
+def test_options_do_not_change_results(B, oracle_mod, chunk, G):
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp = B.Program(p)
+    gp.set_option(B.VL_OPT_CHUNK_INSTRS, chunk)
+    gp.set_option(B.VL_OPT_GROUP, G)
+    gp, lv = _check_liveness(B, oracle_mod, p, gp)
+    rows, _ = synth.candidate_rows(p, wl.K, 0.5, 77)
+    rows = np.concatenate([rows[:61], _garbage_rows(p, 12, 3)])     # ragged: 73 rows
+    _assert_same(_gpu_verify(B, gp, rows), oracle_mod.OracleProgram(p).verify(lv, rows), f"chunk {chunk} G {G}")
+    gp.close()
+
+
+def test_batch_call(B, oracle_mod):
+    """Workload 4 (256 independent programs): a sample of members through vl_verify_batch."""
+    import torch
+    wl = synth.workload(3)
+    members = [0, 1, 2, 3, 100, 255]
+    progs, gps, cands, wants = [], [], [], []
+    for j in members:
+        p = synth.build_program(wl.shapes[j], wl.seeds[j])
+        gp, lv = _check_liveness(B, oracle_mod, p)
+        rows, _ = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[j])
+        progs.append(p); gps.append(gp); cands.append(_to_dev(rows))
+        wants.append(oracle_mod.OracleProgram(p).verify(lv, rows))
+    outs = B.vl_verify_batch(gps, cands)
+    torch.cuda.synchronize()
+    for j, o, w in zip(members, outs, wants):
+        _assert_same(B.verdicts_to_numpy(o), w, f"batch member {j}")
+    for gp in gps:
+        gp.close()
+
+
+def test_stress_workload_sampled(B, oracle_mod):
+    """Workload 5 at full program size: liveness in full; a slab of rows through the kernel in the
+    launch configuration the benchmark uses, verdicts compared on sampled rows (each oracle row
+    costs ~10 ms) and on every faulted row of the slab."""
+    wl = synth.workload(4)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    K = 600
+    rows, faults = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[0], 0, K)
+    got = _gpu_verify(B, gp, rows)
+    assert np.array_equal(got["flags"] == B.VL_PASS, faults[:, 0] == 0)     # valid by construction / injected
+    sample = sorted(set(np.nonzero(faults[:, 0] != 0)[0].tolist()) | set(range(0, K, 9)))
+    want = oracle_mod.OracleProgram(p).verify(lv, rows[sample])
+    _assert_same(got[sample], want, "stress")
+    garbage = _garbage_rows(p, 6, 9)
+    _assert_same(_gpu_verify(B, gp, garbage), oracle_mod.OracleProgram(p).verify(lv, garbage), "stress garbage")
+    gp.close()
+
+
+def test_determinism(B):
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp = B.Program(p)
+    gp.vl_liveness()
+    rows, _ = synth.candidate_rows(p, wl.K, 0.5, 5)
+    a = _gpu_verify(B, gp, rows)
+    b = _gpu_verify(B, gp, rows)
+    assert a.tobytes() == b.tobytes()
+    gp.close()

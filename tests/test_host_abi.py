@@ -1,0 +1,93 @@
+"""Host-side checks that need no GPU: the library loads, exports every declared symbol,
+and rejects malformed descriptors before touching the device."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2506_17506_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2506_17506_b200 import build
+    build.build()
+    from paper_2506_17506_b200 import binding
+    return binding
+
+
+def test_every_declared_symbol_is_exported(B):
+    header = open(os.path.join(ROOT, "include", "verilocc.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(vl_[a-z_0-9]+)\s*\(", header))
+    assert {"vl_liveness", "vl_verify"} <= declared
+    lib = C.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTS)
+
+
+def test_strerror_and_counters(B):
+    assert B.vl_strerror(0) == "ok"
+    for code in range(-8, 0):
+        assert B.vl_strerror(code) not in ("ok", "unknown error")
+    assert B.vl_strerror(-99) == "unknown error"
+    assert B.vl_kernel_launches() == 0
+
+
+def _good():
+    return synth.program_from_lists([[([0], []), ([1], [0]), ([], [1, 0])], [([0], [1])]], [(0, 1), (1, 1)], 2, [1, 2], 8)
+
+
+def _create(B, p):
+    desc, keep = B.make_desc(p)
+    rc, h = B.vl_program_create_raw(desc)
+    assert not h.value or rc == 0
+    return rc
+
+
+@pytest.mark.parametrize("name", ["blk_off_end", "blk_off_order", "succ_range", "op_off_order", "ndefs", "vreg_range",
+                                  "zero_width", "dup_def", "zero_P", "big_P", "zero_B", "no_blocks"])
+def test_malformed_descriptors_are_rejected(B, name):
+    p = _good()
+    expect = B.VL_ERR_MALFORMED_PROGRAM
+    if name == "blk_off_end":
+        p.block_instr_off[-1] += 1
+    elif name == "blk_off_order":
+        p.block_instr_off[1] = 9
+    elif name == "succ_range":
+        p.succ[0] = 7
+    elif name == "op_off_order":
+        p.instr_op_off[1], p.instr_op_off[2] = p.instr_op_off[2], p.instr_op_off[1]
+    elif name == "ndefs":
+        p.instr_n_defs[0] = 3
+    elif name == "vreg_range":
+        p.op_vreg[0] = 2
+    elif name == "zero_width":
+        p.vreg_width[1] = 0
+    elif name == "dup_def":
+        p = synth.program_from_lists([[([0, 0], [])]], [], 1, [1], 4)
+    elif name == "zero_P":
+        p.P, expect = 0, B.VL_ERR_INVALID_ARG
+    elif name == "big_P":
+        p.P, expect = 65536, B.VL_ERR_INVALID_ARG
+    elif name == "zero_B":
+        p.B, expect = 0, B.VL_ERR_INVALID_ARG
+    elif name == "no_blocks":
+        p.n_blocks, expect = 0, B.VL_ERR_INVALID_ARG
+    assert _create(B, p) == expect
+
+
+def test_null_arguments(B):
+    assert B.vl_program_create_raw(None)[0] == B.VL_ERR_INVALID_ARG
+    lib = C.CDLL(B.LIB_PATH)
+    lib.vl_program_destroy(None)
+    lib.vl_liveness.restype = C.c_int
+    assert lib.vl_liveness(None, None) == B.VL_ERR_INVALID_ARG
+    lib.vl_verify.restype = C.c_int
+    lib.vl_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+    assert lib.vl_verify(None, None, 1, 8, None, None) == B.VL_ERR_INVALID_ARG
