@@ -1,0 +1,302 @@
+#!/usr/bin/env python
+"""Benchmark: candidate verifications per second on the stress workload (one program of 32,000
+instructions / 10,000 vregs, K = 10,000 per-operand uint16 candidate rows, about 2 GB).
+
+A step is the whole path for one batch: vl_liveness on the program, then vl_verify over the
+K rows.  `value` is measured with the rows resident in HBM; `e2e` goes through vl_verify_host
+with pinned host buffers, copies inside the timed region.  Prints one JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--rows R]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2506_17506_b200 import synth  # noqa: E402
+
+METRIC = "candidate_verifications_per_sec"
+UNIT = "verifications/s"
+WORKLOAD_INDEX = 4
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-i", str(self.index),
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            parts = [x.strip() for x in s.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                mhz.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+def build_inputs(rank: int, rows: int, pinned: bool):
+    wl = synth.workload(WORKLOAD_INDEX)
+    prog = synth.build_program(wl.shapes[0], wl.seeds[0])
+    K = rows or wl.K
+    pitch = prog.pitch
+    if pinned:
+        import torch
+        host = torch.empty((K, pitch), dtype=torch.int16, pin_memory=True)
+        arr = host.numpy().view(np.uint16)
+    else:
+        host = None
+        arr = np.empty((K, pitch), dtype=np.uint16)
+    t0 = time.time()
+    # rank r checks rows [r*K, (r+1)*K) of the same seeded candidate stream
+    synth.candidate_rows(prog, (rank + 1) * K, wl.fault_rate, wl.seeds[0], rank * K, (rank + 1) * K, out=arr, chunk=256)
+    log(f"[bench] rank {rank}: generated {K} rows x {pitch} operands in {time.time() - t0:.1f}s")
+    return wl, prog, K, host, arr
+
+
+def oracle_rate(prog, arr, n_rows: int, threads: int):
+    """Oracle verdicts for the first n_rows rows, split over `threads` host threads."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    op = oracle.OracleProgram(prog)
+    t0 = time.perf_counter()
+    lv = op.liveness()
+    t_live = time.perf_counter() - t0
+    n_rows = min(n_rows, arr.shape[0])
+    bounds = np.linspace(0, n_rows, threads + 1).astype(int)
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        outs = list(ex.map(lambda j: op.verify(lv, arr[bounds[j]:bounds[j + 1]]), range(threads)))
+    dt = time.perf_counter() - t0
+    return n_rows / dt, dt, t_live, np.concatenate(outs), lv
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    threads = os.cpu_count() or 1
+    sample = max(threads, threads * 8)
+    wl, prog, K, _, arr = build_inputs(0, sample, pinned=False)
+    rates = []
+    for s in range(args.warmup + args.steps):
+        rate, dt, t_live, _, _ = oracle_rate(prog, arr, sample, threads)
+        if s >= args.warmup:
+            rates.append(rate)
+    value = float(np.mean(rates))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sample / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+        "config": {"workload": "stress", "n_instrs": prog.n_instrs, "n_vregs": prog.n_vregs,
+                   "n_operands": prog.n_operands, "P": prog.P, "K": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"{sample} rows of the stress workload per step, {threads} host threads"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--rows", type=int, default=0, help="candidate rows per GPU (default: the workload's 10,000)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--group", type=int, default=0)
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2506_17506_b200 import binding as vl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl, prog, K, host, arr = build_inputs(rank, args.rows, pinned=True)
+    gp = vl.Program(prog, device=local)
+    if args.group:
+        gp.set_option(vl.VL_OPT_GROUP, args.group)
+    if args.chunk:
+        gp.set_option(vl.VL_OPT_CHUNK_INSTRS, args.chunk)
+    dev_rows = host.cuda().view(torch.uint16)
+    out = torch.empty((K, 4), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        gp.vl_liveness(stream)
+        gp.vl_verify(dev_rows, out, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+
+    # ---- timed region: K rows per step, rows (2 GB) far larger than L2, no flush needed
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = vl.vl_kernel_launches()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    ev[0].record(stream)
+    for s in range(args.steps):
+        lev[s][0].record(stream)
+        gp.vl_liveness(stream)
+        lev[s][1].record(stream)
+        kev[s][0].record(stream)
+        gp.vl_verify(dev_rows, out, stream)
+        kev[s][1].record(stream)
+    ev[1].record(stream)
+    barrier()
+    launches = vl.vl_kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    gp.vl_verify_status(stream)
+    total_ms = ev[0].elapsed_time(ev[1])
+    verify_ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+    live_ms = float(np.mean([a.elapsed_time(b) for a, b in lev]))
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    value = world * K * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point
+    e2e_steps = max(1, args.e2e_steps)
+    out_host = np.zeros(K, dtype=vl.VERDICT_DTYPE)
+    gp.vl_liveness(stream)
+    gp.vl_verify_host(host, out_host, stream)      # warm: allocates the staging buffers
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        gp.vl_liveness(stream)
+        gp.vl_verify_host(host, out_host, stream)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * K * e2e_steps / float(t.item())
+
+    # sanity: device-resident and host-buffer results agree
+    dev_v = vl.verdicts_to_numpy(out)
+    same = bool(np.array_equal(dev_v.view(np.int32), out_host.view(np.int32)))
+    n_pass = int((dev_v["flags"] == 1).sum())
+
+    if rank == 0:
+        peak, peak_kind = measured_peak_gbs()
+        bytes_per_launch = 2.0 * prog.pitch * K + 16.0 * K
+        achieved = bytes_per_launch / (verify_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u16", "data": "synthetic",
+            "config": {"workload": "stress", "n_blocks": prog.n_blocks, "n_instrs": prog.n_instrs,
+                       "n_vregs": prog.n_vregs, "n_operands": prog.n_operands, "P": prog.P, "B": prog.B,
+                       "K_per_gpu": K, "fault_rate": wl.fault_rate, "parallelism": f"rows sharded over {world} GPU(s)",
+                       "l2": "inputs (2 GB per step) larger than L2, no flush"},
+            "operand_checks_per_sec": value * prog.n_operands,
+            "verify_ms": verify_ms, "liveness_ms": live_ms,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "kernel": "k_verify", "of": peak_kind,
+                         "frac_of_8TBs_nominal": achieved / 8000.0},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(2 * prog.pitch * K),
+                    "d2h_bytes_per_step": int(16 * K)},
+            "gpu_launches": int(launches),
+            "checks": {"host_equals_device": same, "rows_passing": n_pass},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            threads = os.cpu_count() or 1
+            sample = min(K, max(threads * 16, 256))
+            rate, dt, t_live, ov, _ = oracle_rate(prog, arr, sample, threads)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": f"first {sample} rows of the same workload, {dt:.1f}s on {threads} threads "
+                                              f"(+{t_live:.1f}s liveness, 1 thread)"}
+            line["checks"]["oracle_sample_equal"] = bool(np.array_equal(ov.view(np.int32), dev_v[:sample].view(np.int32)))
+        print(json.dumps(line), flush=True)
+    gp.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

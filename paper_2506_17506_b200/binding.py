@@ -122,7 +122,7 @@ class _DevView:
     """Borrowed view of library-owned device memory (int32 elements) for torch.as_tensor."""
 
     def __init__(self, ptr: int, count: int):
-        self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<i4", "data": (ptr, True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<i4", "data": (ptr, False), "version": 2}
 
 
 class Program:
