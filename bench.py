@@ -93,8 +93,10 @@ class ClockSampler:
                 "samples": len(mhz)}
 
 
-def build_inputs(rank: int, rows: int, pinned: bool):
+def build_inputs(rank: int, rows: int, pinned: bool, fault_rate: float = -1.0):
     wl = synth.workload(WORKLOAD_INDEX)
+    if fault_rate >= 0:
+        wl.fault_rate = fault_rate
     prog = synth.build_program(wl.shapes[0], wl.seeds[0])
     K = rows or wl.K
     pitch = prog.pitch
@@ -168,6 +170,7 @@ def main():
     ap.add_argument("--group", type=int, default=0)
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fault-rate", type=float, default=-1.0, help="override the workload's faulted fraction")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -183,7 +186,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    wl, prog, K, host, arr = build_inputs(rank, args.rows, pinned=True)
+    wl, prog, K, host, arr = build_inputs(rank, args.rows, pinned=True, fault_rate=args.fault_rate)
     gp = vl.Program(prog, device=local)
     if args.group:
         gp.set_option(vl.VL_OPT_GROUP, args.group)

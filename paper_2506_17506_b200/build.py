@@ -23,7 +23,7 @@ def stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, extra=()) -> str:
     if not force and not stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(HERE, "csrc")]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", LIB] + sources()
+    cmd += list(extra) + ["-o", LIB] + sources()
     subprocess.check_call(cmd)
     return LIB
 

@@ -256,6 +256,19 @@ extern "C" int vl_verify_status(vl_program *p, void *stream)
     return (st & ST_DEVICE_WAIT) ? VL_ERR_DEVICE_WAIT : VL_OK;
 }
 
+#ifdef VL_PHASE_TIMERS
+// Profiling builds only: copies the 16 device status words (phase cycle counters from word 2 of the
+// verify status on) to the host and clears them.
+extern "C" int vl_debug_read_status(vl_program *p, uint32_t *out16)
+{
+    if (!p || !out16) return VL_ERR_INVALID_ARG;
+    VL_CUDA(p, cudaDeviceSynchronize());
+    VL_CUDA(p, cudaMemcpy(out16, p->d_status, 64, cudaMemcpyDeviceToHost));
+    VL_CUDA(p, cudaMemset(p->d_status + 1, 0, 60));
+    return VL_OK;
+}
+#endif
+
 extern "C" uint64_t vl_kernel_launches(void) { return g_vl_launches.load(); }
 
 extern "C" int vl_last_cuda_error(const vl_program *p) { return p ? p->last_cuda_error : 0; }

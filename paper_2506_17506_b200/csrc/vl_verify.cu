@@ -17,6 +17,7 @@
 #define TILE (NTV * 8)              // operands per tile and candidate
 #define STAGE_BYTES ((TILE + 8) * 2)  // 8 operands of halo in front of every tile
 #define MAX_STAGES 4
+#define WU 8  // walk events fetched per batch
 
 struct VParams {
     uint32_t nI, V, nO, nOp8, P, B, Bmask, nB, nC, nGroups, Wp, ntiles;
@@ -41,6 +42,23 @@ struct Misc {
     uint32_t out_raw[VL_MAX_GROUP], full[VL_MAX_GROUP], ganom[VL_MAX_GROUP], thcol[VL_MAX_GROUP];
     uint32_t abort_flag, any_anom;
 };
+
+// Optional per-phase cycle counters (thread 0 of every block adds its elapsed clocks to
+// status[2 + phase]); compiled in only with -DVL_PHASE_TIMERS, for profiling builds.
+#ifdef VL_PHASE_TIMERS
+#define PT_INIT() long long pt_last = clock64()
+#define PT(idx)                                                                           \
+    do {                                                                                  \
+        if (threadIdx.x == 0) {                                                           \
+            long long now = clock64();                                                    \
+            atomicAdd(q.status + 2 + (idx), (uint32_t)((now - pt_last) >> 6));            \
+            pt_last = now;                                                                \
+        }                                                                                 \
+    } while (0)
+#else
+#define PT_INIT()
+#define PT(idx)
+#endif
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -174,6 +192,7 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
     }
     for (uint32_t i = tid; i < G * q.AW; i += NTV) s_anom[i] = 0;
     __syncthreads();
+    PT_INIT();
 
     // ---------------------------------------------------------------- pass 1
     auto issue_tile = [&](uint32_t t) {
@@ -193,8 +212,24 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
 #pragma unroll
     for (int g = 0; g < G; ++g) tally[g] = 0;
 
+    // operand metadata of the next tile is fetched one iteration ahead (global memory, L2 latency)
+    uint4 nx_v4 = make_uint4(0, 0, 0, 0);
+    uint64_t nx_meta = 0;
+    if (tid * 8 < q.nOp8) {
+        nx_v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + tid * 8);
+        nx_meta = q.slotmeta[tid];
+    }
     for (uint32_t t = 0; t < q.ntiles; ++t) {
         const uint32_t stage = t % q.NS, parity = (t / q.NS) & 1;
+        const uint4 v4 = nx_v4;
+        const uint64_t smeta_cur = nx_meta;
+        {
+            const uint32_t o_next = (t + 1) * TILE + tid * 8;
+            if (t + 1 < q.ntiles && o_next < q.nOp8) {
+                nx_v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + o_next);
+                nx_meta = q.slotmeta[o_next >> 3];
+            }
+        }
         {   // bounded wait for the tile
             uint32_t spins = 0;
             const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 22);
@@ -214,9 +249,8 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
         uint32_t hb[G];  // registers of the 3 operands in front of this thread's 8 (two words)
         uint32_t hb2[G];
         if (act) {
-            const uint4 v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + o_base);
             vr[0] = v4.x; vr[1] = v4.y; vr[2] = v4.z; vr[3] = v4.w;
-            smeta = q.slotmeta[o_base >> 3];
+            smeta = smeta_cur;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const unsigned char *buf = region + (size_t)(stage * G + g) * STAGE_BYTES + 16 + tid * 16;
@@ -304,22 +338,33 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
         if (lane == 0 && x) atomicAdd(&M->bank[g], x);
     }
     __syncthreads();
+    PT(0);
 
     // ------------------------------------------------- realizability, one sweep over the vregs
-    for (uint32_t v = tid; v < q.V; v += NTV) {
-        const uint32_t vi = q.vinfo[v];
-        if (!(vi & VINFO_OCCURS)) continue;
-        const uint32_t w = vi & 0xFFu;
-        const uint64_t tt = t_load<G>(Tt, v);
+    for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NTV) {
+        uint32_t vis[4], fds[4];
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const uint32_t tv = pk_get(tt, g);
-            if (tv + w > q.P) {
-                if (vi & VINFO_DEFINED) {
-                    atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
-                    atomicMin(&M->minR[g], q.first_def_instr[v]);
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t v = v0 + u * NTV;
+            vis[u] = v < q.V ? q.vinfo[v] : 0u;
+            fds[u] = v < q.V ? q.first_def_instr[v] : 0xFFFFFFFFu;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t v = v0 + u * NTV, vi = vis[u];
+            if (!(vi & VINFO_OCCURS)) continue;
+            const uint32_t w = vi & 0xFFu;
+            const uint64_t tt = t_load<G>(Tt, v);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const uint32_t tv = pk_get(tt, g);
+                if (tv + w > q.P) {
+                    if (vi & VINFO_DEFINED) {
+                        atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
+                        atomicMin(&M->minR[g], fds[u]);
+                    }
+                    if (atomicAdd(&M->nout[g], 1u) == 0) { M->out_v[g] = v; M->out_raw[g] = tv; }
                 }
-                if (atomicAdd(&M->nout[g], 1u) == 0) { M->out_v[g] = v; M->out_raw[g] = tv; }
             }
         }
     }
@@ -338,6 +383,7 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
     if (q.use_th)
         for (uint32_t i = tid; i < q.nB * G * q.Wp; i += NTV) s_th[i] = 0;
     __syncthreads();
+    PT(1);
 
     // ---------------------------------------------------------------- pass 2
     // masks of the vregs that stay occupied through a whole block, per (block, candidate)
@@ -367,6 +413,7 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
     uint32_t fullmask = 0;
 #pragma unroll
     for (int g = 0; g < G; ++g) fullmask |= M->full[g] ? (1u << g) : 0u;
+    PT(2);
 
     if (tid < q.S) {
         const uint32_t stride = G * q.S;  // words between consecutive mask words of one (slot, candidate)
@@ -383,16 +430,32 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
 #pragma unroll
             for (int g = 0; g < G; ++g) viol[g] = 0;
             const uint32_t s0 = q.grp_off[gi], s1 = q.grp_off[gi + 1];
-            for (uint32_t s = s0; s < s1; ++s) {
-                const uint32_t e = q.ev[(size_t)s * 32 + lane];
-                const uint32_t v = e & 0xFFFFu, w = (e >> 16) & 0xFFu;
-                const uint32_t tmask = (e & EV_TEST) ? 0xFFFFFFFFu : 0u, smask = (e & EV_SET) ? 0xFFFFFFFFu : 0u,
-                               cmask = (e & EV_CLEAR) ? 0xFFFFFFFFu : 0u;
-                const uint64_t tt = t_load<G>(Tt, v);
+            const uint32_t nop = q.V | (1u << 16);
+            uint32_t nxt[WU];
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    if (fullmask & (1u << g)) continue;
-                    viol[g] |= occ_event(s_occ + (size_t)g * q.S + tid, stride, pk_get(tt, g), w, tmask, smask, cmask);
+            for (int u = 0; u < WU; ++u) nxt[u] = (s0 + u < s1) ? q.ev[(size_t)(s0 + u) * 32 + lane] : nop;
+            for (uint32_t s = s0; s < s1; s += WU) {
+                uint32_t cur[WU];
+                uint64_t tts[WU];
+#pragma unroll
+                for (int u = 0; u < WU; ++u) cur[u] = nxt[u];
+#pragma unroll
+                for (int u = 0; u < WU; ++u)
+                    nxt[u] = (s + WU + u < s1) ? q.ev[(size_t)(s + WU + u) * 32 + lane] : nop;
+#pragma unroll
+                for (int u = 0; u < WU; ++u) tts[u] = t_load<G>(Tt, cur[u] & 0xFFFFu);
+#pragma unroll
+                for (int u = 0; u < WU; ++u) {
+                    const uint32_t e = cur[u];
+                    const uint32_t w = (e >> 16) & 0xFFu;
+                    const uint32_t tmask = (e & EV_TEST) ? 0xFFFFFFFFu : 0u, smask = (e & EV_SET) ? 0xFFFFFFFFu : 0u,
+                                   cmask = (e & EV_CLEAR) ? 0xFFFFFFFFu : 0u;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        if (fullmask & (1u << g)) continue;
+                        viol[g] |= occ_event(s_occ + (size_t)g * q.S + tid, stride, pk_get(tts[u], g), w, tmask, smask,
+                                             cmask);
+                    }
                 }
             }
             if (have) {
@@ -407,6 +470,7 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
         }
     }
     __syncthreads();
+    PT(3);
 
     // ------------------------------------------- exact recount of the chunks that collided
     if (tid < G) {
@@ -415,20 +479,30 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
     }
     __syncthreads();
     if (M->any_anom) {
-        for (uint32_t item = warp; item < G * q.nC; item += NTV / 32) {
+        for (uint32_t item = 0; item < G * q.nC; ++item) {
             const uint32_t g = item / q.nC, c = item % q.nC;
             if (!M->full[g] && !((s_anom[g * q.AW + (c >> 5)] >> (c & 31)) & 1u)) continue;
             uint32_t pairs = 0, mind = 0xFFFFFFFFu;
-            for (uint32_t i = q.chunk_i0[c]; i < q.chunk_i1[c]; ++i) {
+            for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += NTV / 32) {
                 const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
                 const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
                 for (uint32_t d = o0; d < o0 + nd; ++d) {
                     const uint32_t v = q.op_vreg[d];
                     const uint32_t s = Tt[(size_t)v * G + g], w = q.width[v];
                     uint32_t cnt = 0;
-                    for (uint32_t e = l0 + lane; e < l1; e += 32) {
-                        const uint32_t u = q.lo[e];
-                        if (u != v && ranges_overlap(s, w, Tt[(size_t)u * G + g], q.width[u])) ++cnt;
+                    for (uint32_t e0 = l0; e0 < l1; e0 += 128) {   // 4 list entries per lane in flight
+                        uint32_t us[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint32_t e = e0 + u * 32 + lane;
+                            us[u] = e < l1 ? q.lo[e] : v;
+                        }
+                        uint32_t ws[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (us[u] != v && ranges_overlap(s, w, Tt[(size_t)us[u] * G + g], ws[u])) ++cnt;
                     }
                     // co-defined vregs that are not live after the instruction
                     for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
@@ -447,6 +521,8 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
             }
         }
     }
+    __syncthreads();
+    PT(4);
     // ------------------- exact bank tally from the table where the row-based one cannot be trusted
     uint32_t need_bank = 0;
 #pragma unroll
@@ -487,6 +563,7 @@ __global__ void __launch_bounds__(NTV) k_verify(const VParams q)
         }
     }
     __syncthreads();
+    PT(5);
 
     // ----------------------------------------------------------------- verdicts
     if (tid < G && k0 + tid < q.K) {
