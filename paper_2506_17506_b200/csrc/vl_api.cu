@@ -80,6 +80,32 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
     if (e == cudaSuccess) e = upload(&p->d_ndefs, d->instr_n_defs, (size_t)p->nI);
     if (e == cudaSuccess) e = upload(&p->d_op_vreg, d->op_vreg, (size_t)p->nO);
     if (e == cudaSuccess) e = upload(&p->d_width, d->vreg_width, (size_t)p->V);
+    {   // instructions grouped by their number of distinct sources (2, 3, 4), for the bank tally
+        std::vector<uint2> cls[3];
+        for (uint32_t i = 0; i < p->nI; ++i) {
+            uint32_t ids[4], n = 0;
+            bool many = false;
+            for (uint32_t o = d->instr_op_off[i] + d->instr_n_defs[i]; o < d->instr_op_off[i + 1]; ++o) {
+                const uint32_t v = d->op_vreg[o];
+                bool dup = false;
+                for (uint32_t k = 0; k < n; ++k) dup |= (ids[k] == v);
+                if (dup) continue;
+                if (n == 4) { many = true; break; }
+                ids[n++] = v;
+            }
+            if (many) { p->bank_many = 1; continue; }
+            if (n < 2) continue;
+            for (uint32_t k = n; k < 4; ++k) ids[k] = 0;
+            cls[n - 2].push_back(make_uint2(ids[0] | (ids[1] << 16), ids[2] | (ids[3] << 16)));
+        }
+        std::vector<uint2> all;
+        p->bank_seg[0] = 0;
+        for (int c = 0; c < 3; ++c) {
+            all.insert(all.end(), cls[c].begin(), cls[c].end());
+            p->bank_seg[c + 1] = (uint32_t)all.size();
+        }
+        if (e == cudaSuccess) e = upload(&p->d_bank_list, all.data(), all.size());
+    }
     if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_status, 64);
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 64);
     if (e != cudaSuccess) {
@@ -113,6 +139,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     vl_free_liveness(p);
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
+    cudaFree(p->d_bank_list);
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
         cudaFree(p->d_stage_out[j]);
@@ -134,6 +161,10 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     case VL_OPT_GROUP:
         if (value != 0 && value != 1 && value != 2 && value != 4) return VL_ERR_INVALID_ARG;
         p->group_opt = value;
+        return VL_OK;
+    case VL_OPT_THREADS:
+        if (value != 0 && value != 256 && value != 512) return VL_ERR_INVALID_ARG;
+        p->threads_opt = value;
         return VL_OK;
     default:
         return VL_ERR_INVALID_ARG;

@@ -71,7 +71,11 @@ struct vl_program {
     uint32_t *d_grp_off = nullptr;  // [nGroups+1] first step of each group
     uint32_t *d_ev = nullptr;       // [steps][32] walk events, lane = chunk within its group
     uint32_t ev_steps = 0;
-    int bank_fast = 0;  // B in {1,2,4} and every instruction reads <= 4 operands
+    int bank_fast = 0;  // B in {1,2,4} and every instruction reads <= 4 distinct vregs
+    int bank_many = 0;  // some instruction reads more than 4 distinct vregs
+    uint2 *d_bank_list = nullptr;   // instructions with 2, 3, 4 distinct sources: their vreg ids, 16 bits each
+    uint32_t bank_seg[4] = {0, 0, 0, 0};
+    uint32_t threads_opt = 0;
     int use_th = 0;
 
     uint32_t *d_status = nullptr;  // [16] device status words

@@ -326,7 +326,6 @@ __global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off,
     const uint32_t i = blockIdx.x * NT + threadIdx.x;
     if (i >= nI) return;
     const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
-    if (o1 - o0 - nd > 4) atomicOr(status, ST_MANY_USES);
     for (uint32_t o = o0; o < o1; ++o) {
         const uint32_t v = op_vreg[o];
         uint8_t m = (first_occ[v] == o) ? 1 : 0;
@@ -471,7 +470,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     p->nGroups = (nC + 31) / 32;
 
     const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
-    p->use_th = ((uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
+    p->use_th = (nB <= 32 && (uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
     const size_t smem2 = (size_t)2 * Wv * 4;
 
     VL_CUDA(p, keep(&p->d_chunk_i0, nC, 0, st));
@@ -589,7 +588,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaStreamSynchronize(st));
     VL_CUDA(p, cudaGetLastError());
-    p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !(status & ST_MANY_USES)) ? 1 : 0;
+    p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     p->live_ok = true;
     return VL_OK;
 }

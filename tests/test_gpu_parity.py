@@ -146,13 +146,14 @@ def test_workloads_full(B, oracle_mod, idx):
     gp.close()
 
 
-@pytest.mark.parametrize("chunk,G", [(16, 4), (64, 2), (512, 1), (4096, 0)])
-def test_options_do_not_change_results(B, oracle_mod, chunk, G):
+@pytest.mark.parametrize("chunk,G,threads", [(16, 4, 256), (64, 2, 512), (512, 1, 0), (4096, 0, 512), (128, 4, 512)])
+def test_options_do_not_change_results(B, oracle_mod, chunk, G, threads):
     wl = synth.workload(1)
     p = synth.build_program(wl.shapes[0], wl.seeds[0])
     gp = B.Program(p)
     gp.set_option(B.VL_OPT_CHUNK_INSTRS, chunk)
     gp.set_option(B.VL_OPT_GROUP, G)
+    gp.set_option(B.VL_OPT_THREADS, threads)
     gp, lv = _check_liveness(B, oracle_mod, p, gp)
     rows, _ = synth.candidate_rows(p, wl.K, 0.5, 77)
     rows = np.concatenate([rows[:61], _garbage_rows(p, 12, 3)])     # ragged: 73 rows
