@@ -153,6 +153,37 @@ int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *
 int vl_verify_host(vl_program *prog, const uint16_t *h_cand, uint64_t K, uint64_t pitch_elems,
                    vl_verdict *h_out, void *cuda_stream);
 
+/*
+ * Block-level liveness without any allocation.  (The paper has no counterpart; this exists for
+ * hosts that cannot allocate device memory when they call in: a process that handed all of HBM to
+ * its own pools at start-up, a plugin under a memory budget it does not control, or a loop that
+ * cannot afford the device-wide synchronisation an allocation brings.)
+ *
+ * Computes the same live-in / live-out block bitsets as vl_liveness + vl_liveness_result, from a
+ * program whose CSR arrays are already in DEVICE memory (same meaning and layout as the fields of
+ * vl_program_desc; the program is not validated), into the caller's DEVICE buffers d_live_in and
+ * d_live_out, each [n_blocks][max(1, ceil(n_vregs/32))] 32-bit words.  Nothing is checked for
+ * strictness here.
+ *
+ * The per-block read and write sets are kept in one fixed array inside the library,
+ * VL_STATIC_SCRATCH_WORDS words (1 MiB) on every GPU that loads it, for the life of the process.
+ * A program needs 2 * n_blocks * max(1, ceil(n_vregs/32)) of those words; a larger one is refused
+ * with VL_ERR_UNSUPPORTED.  All calls on a device share the array and it keeps what the last call
+ * left (each call rewrites every word it reads), so two calls whose kernels may overlap on the GPU
+ * (different streams, different threads) race: serialise them.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that
+ * first call outside any stream capture.  The call launches on `cuda_stream`, then waits for it,
+ * because the convergence status is read back.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine.
+ * Errors: INVALID_ARG, UNSUPPORTED, NO_CONVERGE, CUDA.
+ */
+#define VL_STATIC_SCRATCH_WORDS (1u << 18)
+int vl_block_liveness_static(int device, uint32_t n_blocks, uint32_t n_vregs, const uint32_t *d_block_instr_off,
+                             const uint32_t *d_succ_off, const uint32_t *d_succ, const uint32_t *d_instr_op_off,
+                             const uint8_t *d_instr_n_defs, const uint32_t *d_op_vreg, uint32_t *d_live_in,
+                             uint32_t *d_live_out, void *cuda_stream);
+
 /* Reads and clears the device-side status word of the handle's verify calls
  * (VL_OK or VL_ERR_DEVICE_WAIT).  Synchronises `cuda_stream`. */
 int vl_verify_status(vl_program *prog, void *cuda_stream);

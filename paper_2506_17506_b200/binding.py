@@ -28,7 +28,7 @@ VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS = 1, 2, 3
 
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
-           "vl_kernel_launches", "vl_last_cuda_error", "vl_strerror"]
+           "vl_kernel_launches", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -65,6 +65,11 @@ _lib.vl_last_cuda_error.restype = C.c_int
 _lib.vl_last_cuda_error.argtypes = [C.c_void_p]
 _lib.vl_strerror.restype = C.c_char_p
 _lib.vl_strerror.argtypes = [C.c_int]
+
+
+_lib.vl_block_liveness_static.restype = C.c_int
+_lib.vl_block_liveness_static.argtypes = [C.c_int, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9
+VL_STATIC_SCRATCH_WORDS = 1 << 18
 
 
 class VlError(RuntimeError):
@@ -212,6 +217,18 @@ class Program:
             self.close()
         except Exception:
             pass
+
+
+def vl_block_liveness_static(n_blocks, n_vregs, block_instr_off, succ_off, succ, instr_op_off, instr_n_defs, op_vreg,
+                             live_in, live_out, device: int = 0, stream=None) -> int:
+    """Block liveness with no allocation inside the library: every argument after the two counts is
+    a CUDA tensor the caller owns (CSR arrays in, the two bitset buffers out).  Returns the C
+    return code without raising, so callers can test the refusal of oversized programs."""
+    def ptr(t):
+        return t.data_ptr() if t is not None and t.numel() else None
+    return int(_lib.vl_block_liveness_static(device, n_blocks, n_vregs, ptr(block_instr_off), ptr(succ_off), ptr(succ),
+                                             ptr(instr_op_off), ptr(instr_n_defs), ptr(op_vreg), ptr(live_in),
+                                             ptr(live_out), _stream_ptr(stream)))
 
 
 def vl_verify_batch(programs, cands, outs=None, stream=None):
