@@ -122,12 +122,15 @@ void vl_free_liveness(vl_program *p)
     cudaFree(p->d_chunk_i0); cudaFree(p->d_chunk_i1); cudaFree(p->d_chunk_blk); cudaFree(p->d_blk_chunk_off);
     cudaFree(p->d_blk_in); cudaFree(p->d_blk_out); cudaFree(p->d_lo_off); cudaFree(p->d_lo);
     cudaFree(p->d_vreg16); cudaFree(p->d_slotmeta); cudaFree(p->d_opflags); cudaFree(p->d_first_def_instr);
-    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_grp_off); cudaFree(p->d_ev); cudaFree(p->d_vinfo);
+    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_cev_off); cudaFree(p->d_ev); cudaFree(p->d_vinfo);
+    cudaFree(p->d_item_blk); cudaFree(p->d_item_c0); cudaFree(p->d_item_c1);
+    p->d_item_blk = p->d_item_c0 = p->d_item_c1 = nullptr;
     p->d_vinfo = nullptr;
     p->d_chunk_i0 = p->d_chunk_i1 = p->d_chunk_blk = p->d_blk_chunk_off = nullptr;
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
     p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_first_def_instr = nullptr;
-    p->d_th_off = p->d_th = p->d_grp_off = p->d_ev = nullptr;
+    p->d_th_off = p->d_th = p->d_cev_off = nullptr;
+    p->d_ev = nullptr;
     p->live_ok = false;
     p->lo_len = 0;
 }
@@ -140,6 +143,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
+    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); }
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
         cudaFree(p->d_stage_out[j]);
@@ -161,6 +165,10 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     case VL_OPT_GROUP:
         if (value != 0 && value != 1 && value != 2 && value != 4) return VL_ERR_INVALID_ARG;
         p->group_opt = value;
+        return VL_OK;
+    case VL_OPT_SUB_BATCH:
+        if (value < 32 || value % 32) return VL_ERR_INVALID_ARG;
+        p->sub_batch = value;
         return VL_OK;
     case VL_OPT_THREADS:
         if (value != 0 && value != 256 && value != 512) return VL_ERR_INVALID_ARG;
@@ -210,7 +218,7 @@ extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K
     if (rc != VL_OK || K == 0) return rc;
     cudaError_t e = cudaSetDevice(p->device);
     if (e != cudaSuccess) return VL_ERR_CUDA;
-    return vl_verify_impl(p, d_cand, K, pitch, d_out, (cudaStream_t)stream);
+    return vl_verify_impl(p, d_cand, K, pitch, d_out, (cudaStream_t)stream, 2);
 }
 
 extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
@@ -226,7 +234,7 @@ extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const
     if (cudaSetDevice(progs[0]->device) != cudaSuccess) return VL_ERR_CUDA;
     for (uint32_t j = 0; j < n; ++j) {
         if (K[j] == 0) continue;
-        int rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], (cudaStream_t)stream);
+        int rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], (cudaStream_t)stream, 2);
         if (rc != VL_OK) return rc;
     }
     return VL_OK;
@@ -267,7 +275,7 @@ extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K,
         uint64_t n = std::min(rows, K - k0);
         VL_CUDA(p, cudaMemcpyAsync(p->d_stage[j], h_cand + k0 * pitch, n * pitch * 2, cudaMemcpyHostToDevice,
                                    p->h_streams[j]));
-        rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j]);
+        rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j], j);
         if (rc != VL_OK) return rc;
         VL_CUDA(p, cudaMemcpyAsync(h_out + k0, p->d_stage_out[j], n * sizeof(vl_verdict), cudaMemcpyDeviceToHost,
                                    p->h_streams[j]));

@@ -20,9 +20,6 @@ enum : uint8_t {
     OPF_DEAD = 64   // definition: vreg not live after the instruction
 };
 
-// ---- walk events (one 32-bit word): vreg | width << 16 | type bits.  A no-op event names the
-// spare table entry V with width 1 and no type bit.
-enum : uint32_t { EV_TEST = 1u << 24, EV_SET = 1u << 25, EV_CLEAR = 1u << 26 };
 enum : uint32_t { VINFO_OCCURS = 1u << 8, VINFO_DEFINED = 1u << 9 };
 
 // ---- device status word bits (prog->d_status[0] liveness, d_status[1] verify)
@@ -67,10 +64,12 @@ struct vl_program {
     uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
     uint32_t th_len = 0;
-    uint32_t nGroups = 0;           // groups of 32 chunks
-    uint32_t *d_grp_off = nullptr;  // [nGroups+1] first step of each group
-    uint32_t *d_ev = nullptr;       // [steps][32] walk events, lane = chunk within its group
-    uint32_t ev_steps = 0;
+    uint32_t *d_cev_off = nullptr;  // [nC+1] first walk event of each chunk (every chunk padded to 8 events)
+    uint4 *d_ev = nullptr;          // walk events (16 bytes each), chunk after chunk
+    uint32_t ev_total = 0;
+    // walk work items: a run of chunks of one block
+    uint32_t nItems = 0;
+    uint32_t *d_item_blk = nullptr, *d_item_c0 = nullptr, *d_item_c1 = nullptr;
     int bank_fast = 0;  // B in {1,2,4} and every instruction reads <= 4 distinct vregs
     int bank_many = 0;  // some instruction reads more than 4 distinct vregs
     uint2 *d_bank_list = nullptr;   // instructions with 2, 3, 4 distinct sources: their vreg ids, 16 bits each
@@ -81,6 +80,16 @@ struct vl_program {
     uint32_t *d_status = nullptr;  // [16] device status words
     int last_cuda_error = 0;
     bool live_ok = false;
+
+    // per-call working memory of vl_verify (one set per internal stream slot), grown on demand
+    struct VScratch {
+        uint16_t *tg = nullptr;      // [groups][V+1][32] tables, 32 candidates side by side
+        uint32_t *cstate = nullptr;  // [rows][8]
+        uint32_t *anom = nullptr;    // [rows][AW] chunks whose walk collided
+        uint32_t *work = nullptr;    // [1 + rows] count, then candidates that need the exact recount
+        uint64_t rows = 0, aw = 0, vregs = 0;
+    } vs[3];
+    uint32_t sub_batch = 4096;       // candidates per pass of the three verify kernels
 
     // staging for vl_verify_host
     uint16_t *d_stage[2] = {nullptr, nullptr};
@@ -103,5 +112,5 @@ extern std::atomic<uint64_t> g_vl_launches;
 
 int vl_liveness_impl(vl_program *p, cudaStream_t st);
 int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
-                   cudaStream_t st);
+                   cudaStream_t st, int slot);
 void vl_free_liveness(vl_program *p);

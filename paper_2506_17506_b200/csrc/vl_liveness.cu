@@ -313,9 +313,10 @@ __global__ void k_vreg_info(uint32_t V, const uint8_t *__restrict__ width, const
                (first_def_instr[v] != 0xFFFFFFFFu ? VINFO_DEFINED : 0u);
 }
 
-__global__ void k_fill_u32(uint32_t *dst, size_t n, uint32_t value)
+__global__ void k_fill_noop(uint4 *dst, size_t n, uint32_t spare_vreg)
 {
-    for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT) dst[i] = value;
+    for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT)
+        dst[i] = make_uint4(spare_vreg, 0u, 0u, 0u);
 }
 
 __global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
@@ -364,6 +365,16 @@ __global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8
     slotmeta[s] = m;
 }
 
+// A walk event is 16 bytes: x = vreg, y = bits to test, z = bits to toggle (the width-w mask
+// (1<<w)-1, or 0), w = 1 if the range may straddle a 32-bit word (w > 1).  Ranges wider than 32
+// registers carry w = 2 | width << 8 and y, z as 0/1 flags.  A no-op names the spare vreg V.
+__device__ __forceinline__ uint4 make_event(uint32_t v, uint32_t w, bool test, bool toggle)
+{
+    if (w > 32) return make_uint4(v, test ? 1u : 0u, toggle ? 1u : 0u, 2u | (w << 8));
+    const uint32_t wm = w == 32 ? 0xFFFFFFFFu : ((1u << w) - 1u);
+    return make_uint4(v, test ? wm : 0u, toggle ? wm : 0u, w > 1 ? 1u : 0u);
+}
+
 // Walk events of one chunk: entry occupancy (ascending vreg id), then per instruction the
 // releases of dying reads, the definitions, and the releases of dead co-definitions.
 __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
@@ -371,15 +382,15 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
                               const uint32_t *__restrict__ op_vreg, const uint8_t *__restrict__ width,
                               const uint8_t *__restrict__ opflags, uint32_t Wv,
                               const uint32_t *__restrict__ chunk_entry, const uint32_t *__restrict__ centry_cnt,
-                              const uint32_t *__restrict__ ev_off, const uint32_t *__restrict__ grp_off,
-                              uint32_t *ev)
+                              const uint32_t *__restrict__ ev_off, const uint32_t *__restrict__ cev_off,
+                              uint4 *ev)
 {
     __shared__ uint32_t s_scan[34];
     const uint32_t c = blockIdx.x;
-    const size_t base = (size_t)grp_off[c >> 5] * 32 + (c & 31);
+    const size_t base = cev_off[c];
     uint32_t total;
     compact_bits(chunk_entry + (size_t)c * Wv, Wv, s_scan, &total, [&](uint32_t rank, uint32_t v) {
-        ev[base + (size_t)rank * 32] = v | ((uint32_t)width[v] << 16) | EV_TEST | EV_SET;
+        ev[base + rank] = make_event(v, width[v], true, true);
     });
     const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
     const uint32_t e_base = centry_cnt[c];
@@ -389,18 +400,17 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
         for (uint32_t o = o0 + nd; o < o1; ++o)
             if (opflags[o] & OPF_KILL) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (size_t)(e++) * 32] = v | ((uint32_t)width[v] << 16) | EV_CLEAR;
+                ev[base + (e++)] = make_event(v, width[v], false, true);
             }
         for (uint32_t o = o0; o < o0 + nd; ++o)
             if (!(opflags[o] & OPF_ELIDE)) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (size_t)(e++) * 32] =
-                    v | ((uint32_t)width[v] << 16) | EV_TEST | ((opflags[o] & OPF_SET) ? EV_SET : 0u);
+                ev[base + (e++)] = make_event(v, width[v], true, (opflags[o] & OPF_SET) != 0);
             }
         for (uint32_t o = o0; o < o0 + nd; ++o)
             if ((opflags[o] & OPF_POST) && !(opflags[o] & OPF_ELIDE)) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (size_t)(e++) * 32] = v | ((uint32_t)width[v] << 16) | EV_CLEAR;
+                ev[base + (e++)] = make_event(v, width[v], false, true);
             }
     }
 }
@@ -467,7 +477,6 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
         p->h_blk_chunk_off[b + 1] = (uint32_t)p->h_chunk_i0.size();
     }
     const uint32_t nC = p->nC = (uint32_t)p->h_chunk_i0.size();
-    p->nGroups = (nC + 31) / 32;
 
     const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
     p->use_th = (nB <= 32 && (uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
@@ -546,31 +555,46 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
     p->lo_len = h_tot[0];
 
-    std::vector<uint32_t> h_grp_off(p->nGroups + 1, 0), h_th_off(nB + 1, 0);
-    uint64_t steps = 0;
-    for (uint32_t g = 0; g < p->nGroups; ++g) {
-        uint32_t mx = 0;
-        for (uint32_t c = g * 32; c < std::min(nC, g * 32 + 32); ++c) mx = std::max(mx, h_cev[c]);
-        h_grp_off[g] = (uint32_t)steps;
-        steps += mx;
+    std::vector<uint32_t> h_cev_off(nC + 1, 0), h_th_off(nB + 1, 0);
+    uint64_t steps = 0;  // walk events in total, every chunk padded to a multiple of 8 with no-ops
+    for (uint32_t c = 0; c < nC; ++c) {
+        h_cev_off[c] = (uint32_t)steps;
+        steps += (h_cev[c] + 7) / 8 * 8;
     }
-    h_grp_off[p->nGroups] = (uint32_t)steps;
+    h_cev_off[nC] = (uint32_t)steps;
+    // walk work items: runs of at most 16 chunks of one block
+    std::vector<uint32_t> it_blk, it_c0, it_c1;
+    for (uint32_t b = 0; b < nB; ++b)
+        for (uint32_t c = p->h_blk_chunk_off[b]; c < p->h_blk_chunk_off[b + 1]; c += 16) {
+            it_blk.push_back(b);
+            it_c0.push_back(c);
+            it_c1.push_back(std::min(c + 16, p->h_blk_chunk_off[b + 1]));
+        }
+    p->nItems = (uint32_t)it_blk.size();
     uint64_t thn = 0;
     for (uint32_t b = 0; b < nB; ++b) { h_th_off[b] = (uint32_t)thn; thn += h_thc[b]; }
     h_th_off[nB] = (uint32_t)thn;
-    if (steps * 32 > 0xFFFFFFF0ull) return VL_ERR_UNSUPPORTED;
-    p->ev_steps = (uint32_t)steps;
+    if (steps > 0xFFFFFFF0ull) return VL_ERR_UNSUPPORTED;
+    p->ev_total = (uint32_t)steps;
     p->th_len = (uint32_t)thn;
 
     VL_CUDA(p, keep(&p->d_lo, (size_t)p->lo_len, 0, st));
-    VL_CUDA(p, keep(&p->d_ev, (size_t)steps * 32, 0, st));
+    VL_CUDA(p, keep(&p->d_ev, (size_t)steps, 0, st));
     VL_CUDA(p, keep(&p->d_vinfo, (size_t)V, 0, st));
-    LAUNCH(k_fill_u32, (uint32_t)std::min<uint64_t>(1024, (steps * 32 + NT - 1) / NT), 0, st, p->d_ev,
-           (size_t)steps * 32, V | (1u << 16));  // every slot starts as a no-op event
+    LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)steps,
+           V);  // every slot starts as a no-op event
     VL_CUDA(p, keep(&p->d_th, (size_t)thn, 0, st));
-    VL_CUDA(p, keep(&p->d_grp_off, (size_t)p->nGroups + 1, 0, st));
+    VL_CUDA(p, keep(&p->d_cev_off, (size_t)nC + 1, 0, st));
+    VL_CUDA(p, keep(&p->d_item_blk, (size_t)p->nItems, 0, st));
+    VL_CUDA(p, keep(&p->d_item_c0, (size_t)p->nItems, 0, st));
+    VL_CUDA(p, keep(&p->d_item_c1, (size_t)p->nItems, 0, st));
+    if (p->nItems) {
+        VL_CUDA(p, cudaMemcpyAsync(p->d_item_blk, it_blk.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
+        VL_CUDA(p, cudaMemcpyAsync(p->d_item_c0, it_c0.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
+        VL_CUDA(p, cudaMemcpyAsync(p->d_item_c1, it_c1.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
+    }
     VL_CUDA(p, keep(&p->d_th_off, (size_t)nB + 1, 0, st));
-    VL_CUDA(p, cudaMemcpyAsync(p->d_grp_off, h_grp_off.data(), (p->nGroups + 1) * 4, cudaMemcpyHostToDevice, st));
+    VL_CUDA(p, cudaMemcpyAsync(p->d_cev_off, h_cev_off.data(), (nC + 1) * 4, cudaMemcpyHostToDevice, st));
     VL_CUDA(p, cudaMemcpyAsync(p->d_th_off, h_th_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
 
     LAUNCH(k_instr_walk<true>, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
@@ -583,7 +607,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
            p->d_opflags, p->d_vreg16, opmeta, p->d_status);
     LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, st, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
     LAUNCH(k_fill_events, nC, 0, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
-           p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_grp_off, p->d_ev);
+           p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev);
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
     VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaStreamSynchronize(st));

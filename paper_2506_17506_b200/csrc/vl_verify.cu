@@ -1,63 +1,76 @@
-// The verify kernel: G candidates per thread block, packed side by side.
+// The verify path: three kernels per pass over at most `sub_batch` candidates.
 //
-// Pass 1 streams the G candidate rows (bulk async copies into a shared-memory ring, completion
-// on mbarriers), builds the vreg -> preg tables T (G 16-bit entries per vreg, shared memory)
-// from first occurrences and compares every other occurrence with T (Consistency).
-// One sweep over the vregs checks [T, T+width) against the register file (Realizability).
-// A sweep over the instructions with two or more distinct sources tallies bank conflicts from T.
-// Pass 2 walks the program's precompiled event stream, one thread per chunk of instructions,
-// keeping a bitmask of occupied registers per (chunk, candidate) in shared memory (Safety).
-// A chunk whose walk sees no collision provably has no overlap; chunks that do are recounted
-// exactly from the per-instruction live-after lists by whole warps.
+// k_tables   one thread block per G candidates, packed side by side.  Streams the G rows (bulk
+//            async copies into a shared-memory ring, completion on mbarriers), builds the
+//            vreg -> preg tables T (G 16-bit entries per vreg, shared memory) from first
+//            occurrences, compares every other occurrence with T (Consistency), sweeps the vregs for
+//            [T, T+width) inside the register file (Realizability), tallies bank conflicts from T
+//            over the instructions with 2..4 distinct sources, and writes T to global memory with 32
+//            candidates side by side per vreg.
+// k_walk     one lane per candidate, one warp per chunk of instructions: the program's precompiled
+//            event stream is the same for all 32 lanes, the occupancy bitmask of each lane sits in
+//            shared memory at [word][lane] (Safety).  A chunk whose walk sees no collision provably
+//            has no overlap.
+// k_finish / k_recount   verdicts for clean candidates; candidates with a collision are recounted
+//            exactly from the per-instruction live-after lists, one thread block per candidate.
 #include <algorithm>
 
 #include "vl_internal.cuh"
 
 #define MAX_STAGES 4
-#define WU 8  // walk events fetched per batch
+#define WALK_WARPS 8
+#define RC_THREADS 256
 
-struct VParams {
-    uint32_t nI, V, nO, nOp8, P, B, Bmask, nB, nC, nGroups, Wp, ntiles;
-    int bank_fast, use_th;
+// per-candidate state between the kernels (8 words)
+enum { CS_FLAGS = 0, CS_FIRST = 1, CS_BANK = 2, CS_NOUT = 3, CS_OUTV = 4, CS_OUTRAW = 5, CS_WALK = 6, CS_THCOL = 7 };
+enum : uint32_t { WALK_ANOM = 1u, WALK_FULL = 2u };
+
+struct TParams {
+    uint32_t nI, V, nO, nOp8, P, Bmask, ntiles;
+    int bank_fast;
     const uint16_t *vreg16;
     const uint64_t *slotmeta;
-    const uint32_t *vinfo, *first_def_instr, *th_off, *th, *grp_off, *ev;
-    const uint32_t *chunk_i0, *chunk_i1, *chunk_blk, *op_off, *op_vreg, *lo_off, *lo;
-    const uint8_t *ndefs, *width, *opflags;
+    const uint32_t *vinfo, *first_def_instr, *op_off;
     const uint2 *bank_list;
     uint32_t bank_seg[4];  // entries with n = 2, 3, 4 distinct sources: [seg[n-2], seg[n-1])
     const uint16_t *cand;
     uint64_t K, pitch;
-    vl_verdict *out;
+    uint16_t *tg;
+    uint32_t *cstate;
     uint32_t *status;
-    uint32_t S, NS, AW;
-    uint32_t off_T, off_region, off_occ, off_anom, off_misc;
+    uint32_t NS, off_region, off_misc;
 };
 
-struct Misc {
+struct TMisc {
     unsigned long long bar[MAX_STAGES];
-    uint32_t flags[VL_MAX_GROUP], minop[VL_MAX_GROUP], minR[VL_MAX_GROUP], minD[VL_MAX_GROUP];
-    uint32_t pairs[VL_MAX_GROUP], bank[VL_MAX_GROUP], nout[VL_MAX_GROUP], out_v[VL_MAX_GROUP];
-    uint32_t out_raw[VL_MAX_GROUP], full[VL_MAX_GROUP], ganom[VL_MAX_GROUP], thcol[VL_MAX_GROUP];
-    uint32_t abort_flag, any_anom;
+    uint32_t flags[VL_MAX_GROUP], minop[VL_MAX_GROUP], minR[VL_MAX_GROUP], bank[VL_MAX_GROUP];
+    uint32_t nout[VL_MAX_GROUP], out_v[VL_MAX_GROUP], out_raw[VL_MAX_GROUP];
+    uint32_t abort_flag;
 };
 
-// Optional per-phase cycle counters (thread 0 of every block adds its elapsed clocks to
-// status[2 + phase]); compiled in only with -DVL_PHASE_TIMERS, for profiling builds.
-#ifdef VL_PHASE_TIMERS
-#define PT_INIT() long long pt_last = clock64()
-#define PT(idx)                                                                \
-    do {                                                                       \
-        if (threadIdx.x == 0) {                                                \
-            long long now = clock64();                                         \
-            atomicAdd(q.status + 2 + (idx), (uint32_t)((now - pt_last) >> 6)); \
-            pt_last = now;                                                     \
-        }                                                                      \
-    } while (0)
-#else
-#define PT_INIT()
-#define PT(idx)
-#endif
+struct WParams {
+    uint32_t V, P, nB, nC, Wp, AW, use_th;
+    uint64_t K;
+    const uint32_t *th_off, *th, *cev_off, *item_blk, *item_c0, *item_c1;
+    const uint4 *ev;
+    const uint16_t *tg, *tg_zero;
+    uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
+    uint32_t *cstate, *anom;
+};
+
+struct RParams {
+    uint32_t nI, V, B, nB, nC, AW;
+    int bank_fast;
+    uint64_t K;
+    const uint32_t *vinfo, *chunk_i0, *chunk_i1, *chunk_blk, *op_off, *op_vreg, *lo_off, *lo;
+    const uint8_t *ndefs, *width, *opflags;
+    const uint16_t *tg;
+    const uint32_t *cstate, *anom;
+    const uint2 *bank_list;
+    uint32_t bank_seg[4];
+    uint32_t *work;
+    vl_verdict *out;
+};
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -91,7 +104,7 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
 }
 
 // ------------------------------------------------------------- packed table access
-// T holds, per vreg, the G candidates' registers side by side (16 bits each).
+// In shared memory T holds, per vreg, the G candidates' registers side by side (16 bits each).
 template <int G>
 __device__ __forceinline__ uint64_t t_load(const uint16_t *Tt, uint32_t v)
 {
@@ -122,63 +135,34 @@ __device__ __forceinline__ bool ranges_overlap(uint32_t a, uint32_t wa, uint32_t
     return a < b + wb && b < a + wa;
 }
 
-// One walk event of one candidate, any width, on a mask whose consecutive 32-bit words are `stride`
-// words apart.  tm: all ones if the event tests, xm: all ones if it toggles occupancy (becoming
-// occupied and being released are both a toggle as long as no collision has been seen; after a
-// collision the chunk is recounted exactly anyway).  [t, t+w) lies inside the mask.
-__device__ __forceinline__ uint32_t occ_event_wide(uint32_t *mask, uint32_t stride, uint32_t t, uint32_t w, uint32_t tm,
-                                                   uint32_t xm)
-{
-    uint32_t viol = 0, left = w, pos = t;
-    while (left) {
-        const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
-        const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
-        uint32_t *a = mask + (pos >> 5) * stride;
-        const uint32_t o = *a;
-        viol |= o & m & tm;
-        *a = o ^ (m & xm);
-        pos += n;
-        left -= n;
-    }
-    return viol;
-}
-
-// ------------------------------------------------------------------------- kernel
-template <int G, int NT, bool WIDE>
-__global__ void __launch_bounds__(NT) k_verify(const VParams q)
+// =========================================================================== k_tables
+template <int G, int NT>
+__global__ void __launch_bounds__(NT) k_tables(const TParams q)
 {
     constexpr uint32_t TILE = NT * 8;  // operands per tile and candidate
     constexpr uint32_t STAGE_BYTES = TILE * 2;
     extern __shared__ __align__(16) unsigned char smem[];
-    uint16_t *Tt = reinterpret_cast<uint16_t *>(smem + q.off_T);
+    uint16_t *Tt = reinterpret_cast<uint16_t *>(smem);
     unsigned char *region = smem + q.off_region;
-    uint32_t *s_th = reinterpret_cast<uint32_t *>(region);             // [nB][G][Wp], pass 2 only
-    uint32_t *s_occ = reinterpret_cast<uint32_t *>(smem + q.off_occ);  // [Wp][G][S], pass 2 only
-    uint32_t *s_anom = reinterpret_cast<uint32_t *>(smem + q.off_anom);
-    Misc *M = reinterpret_cast<Misc *>(smem + q.off_misc);
+    TMisc *M = reinterpret_cast<TMisc *>(smem + q.off_misc);
 
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
     const uint64_t k0 = (uint64_t)blockIdx.x * G;
     const uint16_t *rows[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) rows[g] = q.cand + min(k0 + g, q.K - 1) * q.pitch;
 
     if (tid < G) {
-        M->flags[tid] = 0; M->minop[tid] = 0xFFFFFFFFu; M->minR[tid] = 0xFFFFFFFFu; M->minD[tid] = 0xFFFFFFFFu;
-        M->pairs[tid] = 0; M->bank[tid] = 0; M->nout[tid] = 0; M->out_v[tid] = 0; M->out_raw[tid] = 0;
-        M->full[tid] = 0; M->ganom[tid] = 0; M->thcol[tid] = 0;
+        M->flags[tid] = 0; M->minop[tid] = 0xFFFFFFFFu; M->minR[tid] = 0xFFFFFFFFu; M->bank[tid] = 0;
+        M->nout[tid] = 0; M->out_v[tid] = 0; M->out_raw[tid] = 0;
     }
     if (tid == 0) {
         M->abort_flag = 0;
-        M->any_anom = 0;
         for (uint32_t s = 0; s < q.NS; ++s) mbar_init(&M->bar[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (uint32_t i = tid; i < G * q.AW; i += NT) s_anom[i] = 0;
     __syncthreads();
-    PT_INIT();
 
-    // ---------------------------------------------------------------- pass 1
     auto issue_tile = [&](uint32_t t) {
         const uint32_t stage = t % q.NS;
         const uint32_t bytes = min(TILE, q.nOp8 - t * TILE) * 2;
@@ -287,7 +271,6 @@ __global__ void __launch_bounds__(NT) k_verify(const VParams q)
         }
     }
     __syncthreads();
-    PT(0);
 
     // ------------------------------------------------- realizability, one sweep over the vregs
     for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NT) {
@@ -317,12 +300,11 @@ __global__ void __launch_bounds__(NT) k_verify(const VParams q)
             }
         }
     }
-    PT(1);
 
     // ------------------------------- bank tally from T: instructions with 2..4 distinct sources.
     // Distinct vregs read by one instruction are live together, so a candidate whose walk sees no
     // collision has them on distinct registers and only the banks need comparing; candidates with
-    // a collision get the general tally further down.
+    // a collision get the general tally in k_recount.
     if (q.bank_fast) {
         constexpr uint64_t L1 = 0x0001000100010001ull;
         const uint64_t BM = L1 * q.Bmask;
@@ -330,20 +312,21 @@ __global__ void __launch_bounds__(NT) k_verify(const VParams q)
         auto same = [&](uint64_t x) -> uint64_t { return ((x | (x >> 1)) & L1) ^ L1; };  // per lane: x == 0
         for (uint32_t e = q.bank_seg[0] + tid; e < q.bank_seg[1]; e += NT) {
             const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu) & BM, b = t_load<G>(Tt, ids.x >> 16) & BM;
-            acc += same(a ^ b);
+            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16);
+            acc += same((a ^ b) & BM);
         }
         for (uint32_t e = q.bank_seg[1] + tid; e < q.bank_seg[2]; e += NT) {
             const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu) & BM, b = t_load<G>(Tt, ids.x >> 16) & BM,
-                           c = t_load<G>(Tt, ids.y & 0xFFFFu) & BM;
-            acc += same(a ^ b) + (same(c ^ a) | same(c ^ b));
+            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16),
+                           c = t_load<G>(Tt, ids.y & 0xFFFFu);
+            acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM));
         }
         for (uint32_t e = q.bank_seg[2] + tid; e < q.bank_seg[3]; e += NT) {
             const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu) & BM, b = t_load<G>(Tt, ids.x >> 16) & BM,
-                           c = t_load<G>(Tt, ids.y & 0xFFFFu) & BM, d = t_load<G>(Tt, ids.y >> 16) & BM;
-            acc += same(a ^ b) + (same(c ^ a) | same(c ^ b)) + (same(d ^ a) | same(d ^ b) | same(d ^ c));
+            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16),
+                           c = t_load<G>(Tt, ids.y & 0xFFFFu), d = t_load<G>(Tt, ids.y >> 16);
+            acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM)) +
+                   (same((d ^ a) & BM) | same((d ^ b) & BM) | same((d ^ c) & BM));
         }
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -354,241 +337,31 @@ __global__ void __launch_bounds__(NT) k_verify(const VParams q)
         }
     }
     __syncthreads();
-    PT(2);
-    // One vreg sticking out of the file cannot overlap another one out there: park it at P (bits
-    // beyond P are padding) and walk as usual.  Two or more: that candidate is recounted in full.
+
+    // ------------------------------------------------- hand-over to the walk
+    // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
+    // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
     if (tid < G) {
         const uint32_t g = tid;
-        if (M->nout[g] == 1) {
-            if (M->out_raw[g] >= q.P) Tt[(size_t)M->out_v[g] * G + g] = (uint16_t)q.P;
-        } else if (M->nout[g] >= 2) {
-            M->full[g] = 1;
-        }
+        if (M->nout[g] == 1 && M->out_raw[g] >= q.P) Tt[(size_t)M->out_v[g] * G + g] = (uint16_t)q.P;
         Tt[(size_t)q.V * G + g] = 0;  // the spare entry that no-op events look up
     }
-    if (q.use_th)
-        for (uint32_t i = tid; i < q.nB * G * q.Wp; i += NT) s_th[i] = 0;
     __syncthreads();
-
-    // ---------------------------------------------------------------- pass 2
-    // masks of the vregs that stay occupied through a whole block, per (block, candidate)
-    if (q.use_th) {
-        for (uint32_t b = 0; b < q.nB; ++b)
-            for (uint32_t e = q.th_off[b] + tid; e < q.th_off[b + 1]; e += NT) {
-                const uint32_t x = q.th[e], v = x & 0xFFFFu, w = x >> 16;
-                const uint64_t tt = t_load<G>(Tt, v);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    if (M->full[g]) continue;
-                    uint32_t pos = pk_get(tt, g), left = w;
-                    while (left) {
-                        const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
-                        const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
-                        const uint32_t old = atomicOr(&s_th[(size_t)(b * G + g) * q.Wp + (pos >> 5)], m);
-                        if (old & m) atomicOr(&M->thcol[g], 1u << b);  // through-sets are used only if nB <= 32
-                        pos += n;
-                        left -= n;
-                    }
-                }
-            }
-        __syncthreads();
-    }
-    uint32_t fullmask = 0;
-#pragma unroll
-    for (int g = 0; g < G; ++g) fullmask |= M->full[g] ? (1u << g) : 0u;
-    PT(3);
-
-    if (tid < q.S) {
-        const uint32_t stride = G * q.S;  // words between consecutive mask words of one (slot, candidate)
-        const uint32_t nop = q.V | (1u << 16);
-        uint32_t tsel[G];  // a candidate that is recounted in full is walked on register 0 (its table may hold anything)
-#pragma unroll
-        for (int g = 0; g < G; ++g) tsel[g] = (fullmask & (1u << g)) ? 0u : 0xFFFFu;
-        for (uint32_t gi = warp; gi < q.nGroups; gi += q.S / 32) {
-            const uint32_t c = gi * 32 + lane;
-            const bool have = c < q.nC;
-            const uint32_t b = have ? q.chunk_blk[c] : 0;
-            for (uint32_t wd = 0; wd < q.Wp; ++wd)
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-                    s_occ[(size_t)(wd * G + g) * q.S + tid] =
-                        (q.use_th && have) ? s_th[(size_t)(b * G + g) * q.Wp + wd] : 0u;
-            uint32_t viol[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) viol[g] = 0;
-            const uint32_t s0 = q.grp_off[gi], s1 = q.grp_off[gi + 1];
-            uint32_t nxt[WU];
-#pragma unroll
-            for (int u = 0; u < WU; ++u) nxt[u] = (s0 + u < s1) ? q.ev[(size_t)(s0 + u) * 32 + lane] : nop;
-            for (uint32_t s = s0; s < s1; s += WU) {
-                uint32_t cur[WU];
-                uint64_t tts[WU];
-#pragma unroll
-                for (int u = 0; u < WU; ++u) cur[u] = nxt[u];
-#pragma unroll
-                for (int u = 0; u < WU; ++u)
-                    nxt[u] = (s + WU + u < s1) ? q.ev[(size_t)(s + WU + u) * 32 + lane] : nop;
-#pragma unroll
-                for (int u = 0; u < WU; ++u) tts[u] = t_load<G>(Tt, cur[u] & 0xFFFFu);
-#pragma unroll
-                for (int u = 0; u < WU; ++u) {
-                    const uint32_t e = cur[u];
-                    const uint32_t w = (e >> 16) & 0xFFu;
-                    const uint32_t wm = (!WIDE || w < 32) ? ((1u << (w & 31)) - 1u) : 0xFFFFFFFFu;
-                    const uint32_t tm = 0u - ((e >> 24) & 1u);
-                    const uint32_t xm = (e & (EV_SET | EV_CLEAR)) ? 0xFFFFFFFFu : 0u;
-                    if (!WIDE || w <= 32) {
-                        // the G candidates' words are independent: all loads first, then all stores
-                        uint32_t *a[G];
-                        uint32_t o[G], m0[G], m1[G];
-#pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            const uint32_t t = (uint32_t)(tts[u] >> (16 * g)) & tsel[g];
-                            m0[g] = wm << (t & 31);
-                            m1[g] = __funnelshift_l(wm, 0u, t);  // bits that spill into the next word
-                            a[g] = s_occ + (size_t)g * q.S + tid + (t >> 5) * stride;
-                            o[g] = *a[g];
-                        }
-                        uint32_t spill = 0;
-#pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            if (fullmask & (1u << g)) continue;
-                            viol[g] |= o[g] & m0[g] & tm;
-                            *a[g] = o[g] ^ (m0[g] & xm);
-                            spill |= m1[g];
-                        }
-                        if (spill) {
-#pragma unroll
-                            for (int g = 0; g < G; ++g) {
-                                if (!m1[g] || (fullmask & (1u << g))) continue;
-                                uint32_t *a2 = a[g] + stride;
-                                const uint32_t o2 = *a2;
-                                viol[g] |= o2 & m1[g] & tm;
-                                *a2 = o2 ^ (m1[g] & xm);
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            if (fullmask & (1u << g)) continue;
-                            viol[g] |= occ_event_wide(s_occ + (size_t)g * q.S + tid, stride, pk_get(tts[u], g), w, tm, xm);
-                        }
-                    }
-                }
-            }
-            if (have) {
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-                    if (viol[g]) {
-                        atomicOr(&s_anom[g * q.AW + (c >> 5)], 1u << (c & 31));
-                        M->ganom[g] = 1;
-                        M->any_anom = 1;
-                    }
+    {   // tables to global memory, 32 candidates side by side per vreg
+        const uint64_t grp = k0 >> 5;
+        const uint32_t l0 = (uint32_t)(k0 & 31);
+        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        for (uint32_t v = tid; v <= q.V; v += NT) {
+            const uint64_t x = t_load<G>(Tt, v);
+            if constexpr (G == 4) {
+                *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2((uint32_t)x, (uint32_t)(x >> 32));
+            } else if constexpr (G == 2) {
+                *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = (uint32_t)x;
+            } else {
+                dst[(size_t)v * 32] = (uint16_t)x;
             }
         }
     }
-    __syncthreads();
-    PT(4);
-
-    // ------------------------------------------- exact recount where the walk cannot vouch
-    if (tid < G) {
-        if (M->nout[tid] == 1) Tt[(size_t)M->out_v[tid] * G + tid] = (uint16_t)M->out_raw[tid];  // true value back
-        if (M->full[tid] || M->thcol[tid]) { M->ganom[tid] = 1; M->any_anom = 1; }
-    }
-    __syncthreads();
-    if (M->any_anom) {
-        for (uint32_t item = 0; item < G * q.nC; ++item) {
-            const uint32_t g = item / q.nC, c = item % q.nC;
-            // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
-            // a block whose through-set collided: the definitions the walk skipped (a vreg redefined
-            // from itself while it stays occupied), since everything else in it was walked exactly
-            const bool all_defs = M->full[g] || ((s_anom[g * q.AW + (c >> 5)] >> (c & 31)) & 1u);
-            const bool elided_only = !all_defs && ((M->thcol[g] >> (q.chunk_blk[c] & 31)) & 1u);
-            if (!all_defs && !elided_only) continue;
-            uint32_t pairs = 0, mind = 0xFFFFFFFFu;
-            for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += NT / 32) {
-                const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
-                const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
-                for (uint32_t d = o0; d < o0 + nd; ++d) {
-                    if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
-                    const uint32_t v = q.op_vreg[d];
-                    const uint32_t s = Tt[(size_t)v * G + g], w = q.width[v];
-                    uint32_t cnt = 0;
-                    for (uint32_t e0 = l0; e0 < l1; e0 += 128) {  // 4 list entries per lane in flight
-                        uint32_t us[4], ws[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const uint32_t e = e0 + u * 32 + lane;
-                            us[u] = e < l1 ? q.lo[e] : v;
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (us[u] != v && ranges_overlap(s, w, Tt[(size_t)us[u] * G + g], ws[u])) ++cnt;
-                    }
-                    // co-defined vregs that are not live after the instruction
-                    for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
-                        if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
-                        const uint32_t u = q.op_vreg[d2];
-                        if (ranges_overlap(s, w, Tt[(size_t)u * G + g], q.width[u])) ++cnt;
-                    }
-#pragma unroll
-                    for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
-                    if (cnt) { pairs += cnt; mind = min(mind, i); }
-                }
-            }
-            if (lane == 0 && pairs) {
-                atomicAdd(&M->pairs[g], pairs);
-                atomicMin(&M->minD[g], mind);
-            }
-        }
-    }
-    __syncthreads();
-    PT(5);
-    // ------------------- general bank tally (distinct registers, not distinct vregs) where needed
-    uint32_t need_bank = 0;
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-        if (!q.bank_fast || M->ganom[g]) need_bank |= 1u << g;
-    __syncthreads();
-    if (need_bank) {
-        if (tid < G && (need_bank >> tid) & 1u) M->bank[tid] = 0;
-        __syncthreads();
-        uint32_t bt[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) bt[g] = 0;
-        for (uint32_t i = tid; i < q.nI; i += NT) {
-            const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
-            for (uint32_t a = u0 + 1; a < u1; ++a) {
-                const uint64_t ta = t_load<G>(Tt, q.op_vreg[a]);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    if (!((need_bank >> g) & 1u)) continue;
-                    const uint32_t xa = pk_get(ta, g);
-                    bool seen_value = false, seen_bank = false;
-                    for (uint32_t bb = u0; bb < a; ++bb) {
-                        const uint32_t xb = Tt[(size_t)q.op_vreg[bb] * G + g];
-                        seen_value |= (xb == xa);
-                        seen_bank |= (xb % q.B == xa % q.B);
-                    }
-                    // a new distinct register landing in a bank already in use costs one cycle
-                    if (!seen_value && seen_bank) ++bt[g];
-                }
-            }
-        }
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            uint32_t x = bt[g];
-#pragma unroll
-            for (int d = 16; d; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
-            if (lane == 0 && x) atomicAdd(&M->bank[g], x);
-        }
-    }
-    __syncthreads();
-    PT(6);
-
-    // ----------------------------------------------------------------- verdicts
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
@@ -601,77 +374,353 @@ __global__ void __launch_bounds__(NT) k_verify(const VParams q)
             }
             first = lo_i;
         }
-        first = min(first, min(M->minR[g], M->minD[g]));
-        uint32_t flags = M->flags[g] | (M->pairs[g] ? (uint32_t)VL_INTERFERENCE : 0u);
-        if (!flags) flags = VL_PASS;
-        vl_verdict vd;
-        vd.flags = flags;
-        vd.first_violation_instr = first == 0xFFFFFFFFu ? -1 : (int32_t)first;
-        vd.conflict_pairs = M->pairs[g];
-        vd.bank_conflicts = M->bank[g];
-        q.out[k0 + g] = vd;
+        uint32_t *cs = q.cstate + (k0 + g) * 8;
+        cs[CS_FLAGS] = M->flags[g];
+        cs[CS_FIRST] = min(first, M->minR[g]);
+        cs[CS_BANK] = M->bank[g];
+        cs[CS_NOUT] = M->nout[g];
+        cs[CS_OUTV] = M->out_v[g];
+        cs[CS_OUTRAW] = M->out_raw[g];
+        cs[CS_WALK] = M->nout[g] >= 2 ? WALK_FULL : 0u;
+        cs[CS_THCOL] = 0;
+    }
+}
+
+// =========================================================================== k_walk
+// grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
+// Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
+__global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
+{
+    extern __shared__ __align__(16) uint32_t wsm[];
+    uint32_t *s_th = wsm;  // [Wp][32]
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t per_warp = q.Wp * 32 + q.ev_cap * 4;  // words
+    uint32_t *s_occ = wsm + q.Wp * 32 + (size_t)warp * per_warp;  // [Wp][32]
+    uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap]
+    const uint32_t item = blockIdx.x, grp = blockIdx.y;
+    const uint32_t b = q.item_blk[item], c0 = q.item_c0[item], c1 = q.item_c1[item];
+    const uint64_t k = (uint64_t)grp * 32 + lane;
+    uint32_t *cs = q.cstate + k * 8;  // rows beyond K exist in the working buffers (whole groups)
+    // lanes without a candidate, and candidates that are recounted in full anyway (their table may
+    // hold anything), read an all-zero table instead
+    const bool walked = k < q.K && !(cs[CS_WALK] & WALK_FULL);
+    const uint16_t *tg = walked ? q.tg + (uint64_t)grp * (q.V + 1) * 32 + lane : q.tg_zero + lane;
+
+    for (uint32_t i = threadIdx.x; i < q.Wp * 32; i += WALK_WARPS * 32) s_th[i] = 0;
+    __syncthreads();
+    // mask of the vregs that stay occupied through the whole block
+    if (q.use_th) {
+        bool thcol = false;
+        const uint32_t e1 = q.th_off[b + 1];
+        for (uint32_t e0 = q.th_off[b] + warp * 8; e0 < e1; e0 += WALK_WARPS * 8) {
+            uint32_t x[8], t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) x[u] = e0 + u < e1 ? q.th[e0 + u] : (q.V | (0u << 16));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) t[u] = tg[(size_t)(x[u] & 0xFFFFu) * 32];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                uint32_t pos = t[u], left = x[u] >> 16;
+                while (left) {
+                    const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
+                    const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
+                    const uint32_t old = atomicOr(&s_th[(pos >> 5) * 32 + lane], m);
+                    thcol |= (old & m) != 0;
+                    pos += n;
+                    left -= n;
+                }
+            }
+        }
+        if (thcol && walked) atomicOr(&cs[CS_THCOL], 1u << b);  // through-sets are used only if nB <= 32
+        __syncthreads();
+    }
+
+    for (uint32_t c = c0 + warp; c < c1; c += WALK_WARPS) {
+        for (uint32_t wd = 0; wd < q.Wp; ++wd) s_occ[wd * 32 + lane] = s_th[wd * 32 + lane];
+        uint32_t viol = 0;
+        const uint32_t s0 = q.cev_off[c], n_ev = q.cev_off[c + 1] - s0;  // a multiple of 8 events
+        for (uint32_t done = 0; done < n_ev; done += q.ev_cap) {
+            const uint32_t n = min(q.ev_cap, n_ev - done);
+            __syncwarp();
+            for (uint32_t i = lane; i < n; i += 32) s_ev[i] = q.ev[s0 + done + i];  // events of this piece, once
+            __syncwarp();
+            // table entries of the next 8 events are fetched while the current 8 are applied
+            uint32_t tn[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) tn[u] = tg[(size_t)s_ev[u].x * 32];
+            for (uint32_t s = 0; s < n; s += 8) {
+                uint32_t t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t[u] = tn[u];
+                if (s + 8 < n) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) tn[u] = tg[(size_t)s_ev[s + 8 + u].x * 32];
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint4 e = s_ev[s + u];
+                    const uint32_t tv = t[u];
+                    if (!(e.w & 2u)) {
+                        uint32_t *a = s_occ + (tv >> 5) * 32 + lane;
+                        const uint32_t o = *a;
+                        viol |= o & __funnelshift_l(0u, e.y, tv);
+                        *a = o ^ __funnelshift_l(0u, e.z, tv);
+                        if (e.w) {  // wider than one register: bits that spill into the next word
+                            const uint32_t m1t = __funnelshift_l(e.y, 0u, tv), m1x = __funnelshift_l(e.z, 0u, tv);
+                            if (m1t | m1x) {
+                                const uint32_t o2 = a[32];
+                                viol |= o2 & m1t;
+                                a[32] = o2 ^ m1x;
+                            }
+                        }
+                    } else {
+                        uint32_t left = e.w >> 8, pos = tv;
+                        while (left) {
+                            const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
+                            const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
+                            uint32_t *a = s_occ + (pos >> 5) * 32 + lane;
+                            const uint32_t o = *a;
+                            if (e.y) viol |= o & m;
+                            if (e.z) *a = o ^ m;
+                            pos += nn;
+                            left -= nn;
+                        }
+                    }
+                }
+            }
+        }
+        if (viol && walked) {
+            atomicOr(&q.anom[k * q.AW + (c >> 5)], 1u << (c & 31));
+            atomicOr(&cs[CS_WALK], WALK_ANOM);
+        }
+    }
+}
+
+// =========================================================================== k_finish
+// Verdicts of the candidates the walk vouches for; the others go on the work list.
+__global__ void k_finish(uint64_t K, const uint32_t *__restrict__ cstate, uint32_t *work, vl_verdict *out)
+{
+    const uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const uint32_t *cs = cstate + k * 8;
+    if (cs[CS_WALK] | cs[CS_THCOL]) {
+        work[1 + atomicAdd(work, 1u)] = (uint32_t)k;
+        return;
+    }
+    vl_verdict vd;
+    vd.flags = cs[CS_FLAGS] ? cs[CS_FLAGS] : (uint32_t)VL_PASS;
+    vd.first_violation_instr = cs[CS_FIRST] == 0xFFFFFFFFu ? -1 : (int32_t)cs[CS_FIRST];
+    vd.conflict_pairs = 0;
+    vd.bank_conflicts = cs[CS_BANK];
+    out[k] = vd;
+}
+
+// Programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction with
+// more than 4 distinct sources): every candidate goes through k_recount.
+__global__ void k_list_all(uint64_t K, uint32_t *work)
+{
+    const uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < K) work[1 + k] = (uint32_t)k;
+    if (k == 0) work[0] = (uint32_t)K;
+}
+
+// =========================================================================== k_recount
+// One thread block per listed candidate (blocks loop over the list): its table column in shared
+// memory, exact overlap counts from the live-after lists where the walk could not vouch, and the
+// general bank tally (distinct registers rather than distinct vregs).
+// Shared memory: [T (V+1) x u16][chunks needing every definition, AW words][chunks needing only the
+// definitions the walk skipped, AW words].
+__global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
+{
+    extern __shared__ __align__(16) uint16_t T[];
+    __shared__ uint32_t s_pairs, s_mind, s_bank;
+    uint32_t *s_all = reinterpret_cast<uint32_t *>(T + ((q.V + 1 + 7) & ~7u));
+    uint32_t *s_eli = s_all + q.AW;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t nwork = q.work[0];
+    for (uint32_t wi = blockIdx.x; wi < nwork; wi += gridDim.x) {
+        const uint64_t k = q.work[1 + wi];
+        const uint32_t *cs = q.cstate + k * 8;
+        const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
+        __syncthreads();
+        for (uint32_t v = tid; v < q.V; v += RC_THREADS) T[v] = tg[(size_t)v * 32];
+        for (uint32_t i = tid; i < 2 * q.AW; i += RC_THREADS) s_all[i] = 0;
+        if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
+        __syncthreads();
+        if (tid == 0 && cs[CS_NOUT] == 1) T[cs[CS_OUTV]] = (uint16_t)cs[CS_OUTRAW];  // the true value, not the parked one
+        const bool full = cs[CS_WALK] & WALK_FULL;
+        const uint32_t thcol = cs[CS_THCOL];
+        const uint32_t *anom = q.anom + k * q.AW;
+        // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
+        // a block whose through-set collided: the definitions the walk skipped (a vreg redefined
+        // from itself while it stays occupied), since everything else in it was walked exactly
+        for (uint32_t c = tid; c < q.nC; c += RC_THREADS) {
+            const bool all_defs = full || ((anom[c >> 5] >> (c & 31)) & 1u);
+            const bool elided_only = !all_defs && ((thcol >> (q.chunk_blk[c] & 31)) & 1u);
+            if (all_defs) atomicOr(&s_all[c >> 5], 1u << (c & 31));
+            if (elided_only) atomicOr(&s_eli[c >> 5], 1u << (c & 31));
+        }
+        __syncthreads();
+        for (uint32_t cw = 0; cw < q.AW; ++cw) {
+            uint32_t bits = s_all[cw] | s_eli[cw];
+            while (bits) {
+                const uint32_t cb = __ffs(bits) - 1;
+                bits &= bits - 1;
+                const uint32_t c = cw * 32 + cb;
+                const bool elided_only = !((s_all[cw] >> cb) & 1u);
+                uint32_t pairs = 0, mind = 0xFFFFFFFFu;
+                for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += RC_THREADS / 32) {
+                    const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
+                    const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
+                    for (uint32_t d = o0; d < o0 + nd; ++d) {
+                        if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
+                        const uint32_t v = q.op_vreg[d];
+                        const uint32_t s = T[v], w = q.width[v];
+                        uint32_t cnt = 0;
+                        for (uint32_t e0 = l0; e0 < l1; e0 += 128) {  // 4 list entries per lane in flight
+                            uint32_t us[4], ws[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const uint32_t e = e0 + u * 32 + lane;
+                                us[u] = e < l1 ? q.lo[e] : v;
+                            }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (us[u] != v && ranges_overlap(s, w, T[us[u]], ws[u])) ++cnt;
+                        }
+                        // co-defined vregs that are not live after the instruction
+                        for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
+                            if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
+                            const uint32_t u = q.op_vreg[d2];
+                            if (ranges_overlap(s, w, T[u], q.width[u])) ++cnt;
+                        }
+#pragma unroll
+                        for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
+                        if (cnt) { pairs += cnt; mind = min(mind, i); }
+                    }
+                }
+                if (lane == 0 && pairs) {
+                    atomicAdd(&s_pairs, pairs);
+                    atomicMin(&s_mind, mind);
+                }
+            }
+        }
+        // general bank tally: a source counts when its register is new among the instruction's sources
+        // and its bank is not
+        uint32_t bt = 0;
+        if (q.bank_fast) {
+            for (uint32_t e = tid; e < q.bank_seg[3]; e += RC_THREADS) {
+                const uint2 ids = q.bank_list[e];
+                const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
+                uint32_t x[4];
+                x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
+#pragma unroll
+                for (uint32_t a = 1; a < 4; ++a) {
+                    if (a >= n) break;
+                    bool seen_value = false, seen_bank = false;
+#pragma unroll
+                    for (uint32_t bb = 0; bb < a; ++bb) {
+                        seen_value |= (x[bb] == x[a]);
+                        seen_bank |= ((x[bb] ^ x[a]) & (q.B - 1)) == 0;
+                    }
+                    if (!seen_value && seen_bank) ++bt;
+                }
+            }
+        } else {
+            for (uint32_t i = tid; i < q.nI; i += RC_THREADS) {
+                const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
+                for (uint32_t a = u0 + 1; a < u1; ++a) {
+                    const uint32_t xa = T[q.op_vreg[a]];
+                    bool seen_value = false, seen_bank = false;
+                    for (uint32_t bb = u0; bb < a; ++bb) {
+                        const uint32_t xb = T[q.op_vreg[bb]];
+                        seen_value |= (xb == xa);
+                        seen_bank |= (xb % q.B == xa % q.B);
+                    }
+                    if (!seen_value && seen_bank) ++bt;
+                }
+            }
+        }
+#pragma unroll
+        for (int d = 16; d; d >>= 1) bt += __shfl_xor_sync(0xffffffffu, bt, d);
+        if (lane == 0 && bt) atomicAdd(&s_bank, bt);
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t flags = cs[CS_FLAGS] | (s_pairs ? (uint32_t)VL_INTERFERENCE : 0u);
+            if (!flags) flags = VL_PASS;
+            const uint32_t first = min(cs[CS_FIRST], s_mind);
+            vl_verdict vd;
+            vd.flags = flags;
+            vd.first_violation_instr = first == 0xFFFFFFFFu ? -1 : (int32_t)first;
+            vd.conflict_pairs = s_pairs;
+            vd.bank_conflicts = s_bank;
+            q.out[k] = vd;
+        }
     }
 }
 
 // --------------------------------------------------------------------------- host
 namespace {
-struct Plan { uint32_t G, NT, S, NS, smem, off_T, off_region, off_occ, off_anom, off_misc, AW, Wp; bool ok; };
+struct Plan { uint32_t G, NT, NS, smem, off_region, off_misc; bool ok; };
 
 inline uint64_t align16(uint64_t x) { return (x + 15u) & ~15ull; }
 
-// Shared memory of one block: [T][region][anomaly bitmap][misc]; the region holds the copy ring in
-// pass 1 and the through-set masks followed by the walkers' masks in pass 2.
-Plan make_plan(const vl_program *p, uint32_t G, uint32_t NT, uint32_t budget, uint32_t min_slots)
+// Shared memory of one k_tables block: [T][copy ring][misc].
+Plan make_plan(const vl_program *p, uint32_t G, uint32_t NT, uint32_t budget)
 {
     Plan pl{};
     pl.G = G; pl.NT = NT;
-    pl.Wp = (p->P + p->wmax + 31) / 32;
-    pl.AW = std::max(1u, (p->nC + 31) / 32);
     const uint64_t stage = (uint64_t)NT * 8 * 2 * G;
     const uint64_t tbytes = align16((uint64_t)(p->V + 1) * G * 2);
-    const uint64_t thbytes = p->use_th ? align16((uint64_t)p->nB * G * pl.Wp * 4) : 0;
-    const uint64_t anom = align16((uint64_t)G * pl.AW * 4);
-    const uint64_t misc = align16(sizeof(Misc));
-    const uint64_t fixed = tbytes + anom + misc;
-    const uint64_t slot = (uint64_t)G * pl.Wp * 4;
+    const uint64_t misc = align16(sizeof(TMisc));
     pl.ok = false;
-    if (fixed + 2 * stage > budget || fixed + thbytes + 32 * slot > budget) return pl;
-    const uint64_t room = budget - fixed;
-    uint32_t S = (uint32_t)std::min<uint64_t>(NT, (room - thbytes) / slot) / 32 * 32;
-    const uint32_t want = std::min<uint32_t>(NT, std::max(1u, p->nGroups) * 32);
-    S = std::min(S, want);
-    if (S < std::min(min_slots, want)) return pl;
-    const uint32_t NS = (uint32_t)std::min<uint64_t>(MAX_STAGES, room / stage);
-    const uint64_t region = std::max<uint64_t>((uint64_t)NS * stage, thbytes + (uint64_t)S * slot);
-    pl.S = S; pl.NS = NS;
-    pl.off_T = 0;
+    if (tbytes + misc + 2 * stage > budget) return pl;
+    pl.NS = (uint32_t)std::min<uint64_t>(MAX_STAGES, (budget - tbytes - misc) / stage);
     pl.off_region = (uint32_t)tbytes;
-    pl.off_occ = (uint32_t)(tbytes + thbytes);
-    pl.off_anom = (uint32_t)(tbytes + align16(region));
-    pl.off_misc = pl.off_anom + (uint32_t)anom;
+    pl.off_misc = (uint32_t)(tbytes + pl.NS * stage);
     pl.smem = pl.off_misc + (uint32_t)misc;
-    pl.ok = pl.smem <= budget;
+    pl.ok = true;
     return pl;
 }
 
-template <int G, int NT, bool WIDE>
-cudaError_t launch(const VParams &q, uint32_t grid, uint32_t smem, cudaStream_t st)
+template <int G, int NT>
+cudaError_t launch_tables(const TParams &q, uint32_t grid, uint32_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(k_verify<G, NT, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_tables<G, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_verify<G, NT, WIDE><<<grid, NT, smem, st>>>(q);
+    k_tables<G, NT><<<grid, NT, smem, st>>>(q);
     return cudaGetLastError();
 }
-template <int G, int NT>
-cudaError_t launch_w(bool wide, const VParams &q, uint32_t grid, uint32_t smem, cudaStream_t st)
+
+int ensure_scratch(vl_program *p, int slot, uint64_t rows)
 {
-    return wide ? launch<G, NT, true>(q, grid, smem, st) : launch<G, NT, false>(q, grid, smem, st);
+    vl_program::VScratch &v = p->vs[slot];
+    const uint64_t aw = std::max(1u, (p->nC + 31) / 32);
+    const uint64_t groups = (rows + 31) / 32;
+    if (v.rows >= rows && v.aw == aw && v.vregs == p->V) return VL_OK;
+    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work);
+    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr;
+    v.rows = 0;
+    // one more group than needed: it stays all zero, for lanes that have nothing to walk
+    VL_CUDA(p, cudaMalloc((void **)&v.tg, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
+    VL_CUDA(p, cudaMemset(v.tg, 0, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * 32 * 8 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work, (1 + groups * 32) * sizeof(uint32_t)));
+    v.rows = groups * 32;
+    v.aw = aw;
+    v.vregs = p->V;
+    return VL_OK;
 }
 }  // namespace
 
-int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
-                   cudaStream_t st)
+int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+                   cudaStream_t st, int slot)
 {
+    vl_program *p = const_cast<vl_program *>(cp);  // the handle owns the working memory of its calls
     const uint32_t SM_BYTES = 227 * 1024;
     // preference: the largest group that still lets two blocks share an SM, then anything that fits
     Plan pl{};
@@ -680,45 +729,87 @@ int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint
     for (int pass = 0; pass < 2 && !pl.ok; ++pass)
         for (uint32_t G : groups) {
             if (p->group_opt && G != p->group_opt) continue;
-            const uint32_t budget = pass == 0 ? (SM_BYTES / 2 - 1024) : SM_BYTES;
-            pl = make_plan(p, G, NT, budget, pass == 0 ? 64 : 32);
+            pl = make_plan(p, G, NT, pass == 0 ? (SM_BYTES / 2 - 1024) : SM_BYTES);
             if (pl.ok) break;
         }
     if (!pl.ok) return VL_ERR_UNSUPPORTED;
+    const uint32_t Wp = (p->P + p->wmax + 31) / 32;
+    const uint32_t ev_cap = 256;
+    const uint32_t walk_smem = (Wp * 32 + WALK_WARPS * (Wp * 32 + ev_cap * 4)) * 4;
+    const uint32_t rc_smem = (uint32_t)align16((uint64_t)((p->V + 1 + 7) & ~7u) * 2 + 2ull * std::max(1u, (p->nC + 31) / 32) * 4);
+    if (walk_smem > SM_BYTES || rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
 
-    VParams q{};
-    q.nI = p->nI; q.V = p->V; q.nO = p->nO; q.nOp8 = p->nOp8; q.P = p->P; q.B = p->B; q.Bmask = p->B - 1;
-    q.nB = p->nB; q.nC = p->nC; q.nGroups = p->nGroups; q.Wp = pl.Wp;
-    q.ntiles = (p->nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
-    q.bank_fast = p->bank_fast; q.use_th = p->use_th;
-    q.vreg16 = p->d_vreg16; q.slotmeta = p->d_slotmeta; q.vinfo = p->d_vinfo; q.first_def_instr = p->d_first_def_instr;
-    q.th_off = p->d_th_off; q.th = p->d_th; q.grp_off = p->d_grp_off; q.ev = p->d_ev;
-    q.chunk_i0 = p->d_chunk_i0; q.chunk_i1 = p->d_chunk_i1; q.chunk_blk = p->d_chunk_blk;
-    q.op_off = p->d_op_off; q.op_vreg = p->d_op_vreg; q.lo_off = p->d_lo_off; q.lo = p->d_lo;
-    q.ndefs = p->d_ndefs; q.width = p->d_width; q.opflags = p->d_opflags;
-    q.bank_list = p->d_bank_list;
-    for (int j = 0; j < 4; ++j) q.bank_seg[j] = p->bank_seg[j];
-    q.cand = d_cand; q.K = K; q.pitch = pitch; q.out = d_out; q.status = p->d_status + 1;
-    q.S = pl.S; q.NS = pl.NS; q.AW = pl.AW;
-    q.off_T = pl.off_T; q.off_region = pl.off_region; q.off_occ = pl.off_occ; q.off_anom = pl.off_anom;
-    q.off_misc = pl.off_misc;
+    const uint64_t sub = std::min<uint64_t>(K, p->sub_batch);
+    int rc = ensure_scratch(p, slot, sub);
+    if (rc != VL_OK) return rc;
+    vl_program::VScratch &vs = p->vs[slot];
+    cudaError_t e = cudaSuccess;
+    if (walk_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
+    if (e == cudaSuccess && rc_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rc_smem);
+    if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
 
-    const uint32_t grid = (uint32_t)((K + pl.G - 1) / pl.G);
-    const bool wide = p->wmax > 31;
-    cudaError_t e = cudaErrorInvalidValue;
-    if (pl.NT == 256) {
-        if (pl.G == 4) e = launch_w<4, 256>(wide, q, grid, pl.smem, st);
-        else if (pl.G == 2) e = launch_w<2, 256>(wide, q, grid, pl.smem, st);
-        else e = launch_w<1, 256>(wide, q, grid, pl.smem, st);
-    } else {
-        if (pl.G == 4) e = launch_w<4, 512>(wide, q, grid, pl.smem, st);
-        else if (pl.G == 2) e = launch_w<2, 512>(wide, q, grid, pl.smem, st);
-        else e = launch_w<1, 512>(wide, q, grid, pl.smem, st);
+    for (uint64_t kb = 0; kb < K; kb += sub) {
+        const uint64_t n = std::min(sub, K - kb);
+        const uint32_t ngrp = (uint32_t)((n + 31) / 32);
+        VL_CUDA(p, cudaMemsetAsync(vs.anom, 0, (size_t)ngrp * 32 * vs.aw * 4, st));
+        VL_CUDA(p, cudaMemsetAsync(vs.work, 0, 4, st));
+
+        TParams tq{};
+        tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
+        tq.ntiles = (p->nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
+        tq.bank_fast = p->bank_fast;
+        tq.vreg16 = p->d_vreg16; tq.slotmeta = p->d_slotmeta; tq.vinfo = p->d_vinfo;
+        tq.first_def_instr = p->d_first_def_instr; tq.op_off = p->d_op_off;
+        tq.bank_list = p->d_bank_list;
+        for (int j = 0; j < 4; ++j) tq.bank_seg[j] = p->bank_seg[j];
+        tq.cand = d_cand + kb * pitch; tq.K = n; tq.pitch = pitch;
+        tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
+        tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
+        const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
+        if (pl.NT == 256) {
+            if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
+            else if (pl.G == 2) e = launch_tables<2, 256>(tq, tgrid, pl.smem, st);
+            else e = launch_tables<1, 256>(tq, tgrid, pl.smem, st);
+        } else {
+            if (pl.G == 4) e = launch_tables<4, 512>(tq, tgrid, pl.smem, st);
+            else if (pl.G == 2) e = launch_tables<2, 512>(tq, tgrid, pl.smem, st);
+            else e = launch_tables<1, 512>(tq, tgrid, pl.smem, st);
+        }
+        if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+        g_vl_launches.fetch_add(1);
+
+        if (p->nItems) {
+            WParams wq{};
+            wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = Wp; wq.AW = (uint32_t)vs.aw;
+            wq.use_th = (uint32_t)p->use_th; wq.K = n;
+            wq.th_off = p->d_th_off; wq.th = p->d_th; wq.cev_off = p->d_cev_off; wq.ev = p->d_ev;
+            wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
+            wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = ev_cap;
+            wq.cstate = vs.cstate; wq.anom = vs.anom;
+            k_walk<<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+            g_vl_launches.fetch_add(1);
+        }
+
+        if (p->bank_fast) k_finish<<<(uint32_t)((n + 255) / 256), 256, 0, st>>>(n, vs.cstate, vs.work, d_out + kb);
+        else k_list_all<<<(uint32_t)((n + 255) / 256), 256, 0, st>>>(n, vs.work);
+        RParams rq{};
+        rq.nI = p->nI; rq.V = p->V; rq.B = p->B; rq.nB = p->nB; rq.nC = p->nC; rq.AW = (uint32_t)vs.aw;
+        rq.bank_fast = p->bank_fast; rq.K = n;
+        rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
+        rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
+        rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags;
+        rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out + kb;
+        rq.bank_list = p->d_bank_list;
+        for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
+        const uint32_t rgrid = (uint32_t)std::min<uint64_t>(n, 148 * 4);
+        k_recount<<<rgrid, RC_THREADS, rc_smem, st>>>(rq);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+        g_vl_launches.fetch_add(2);
     }
-    if (e != cudaSuccess) {
-        const_cast<vl_program *>(p)->last_cuda_error = (int)e;
-        return VL_ERR_CUDA;
-    }
-    g_vl_launches.fetch_add(1);
     return VL_OK;
 }
