@@ -123,6 +123,8 @@ void vl_free_liveness(vl_program *p)
     cudaFree(p->d_blk_in); cudaFree(p->d_blk_out); cudaFree(p->d_lo_off); cudaFree(p->d_lo);
     cudaFree(p->d_vreg16); cudaFree(p->d_slotmeta); cudaFree(p->d_opflags); cudaFree(p->d_first_def_instr);
     cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_cev_off); cudaFree(p->d_ev); cudaFree(p->d_vinfo);
+    cudaFree(p->d_iflags);
+    p->d_iflags = nullptr;
     cudaFree(p->d_item_blk); cudaFree(p->d_item_c0); cudaFree(p->d_item_c1);
     p->d_item_blk = p->d_item_c0 = p->d_item_c1 = nullptr;
     p->d_vinfo = nullptr;
@@ -143,7 +145,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
-    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); }
+    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); }
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
         cudaFree(p->d_stage_out[j]);

@@ -60,6 +60,7 @@ struct vl_program {
     uint16_t *d_vreg16 = nullptr;           // [nOp8 + 8] vreg id per operand (padding operands: id V)
     uint64_t *d_slotmeta = nullptr;         // [nOp8 / 8] per 8 operands: first-occurrence bits, bank compare masks
     uint8_t *d_opflags = nullptr;           // [nO]
+    uint8_t *d_iflags = nullptr;            // [nI] 1 if the instruction has a definition the walk skips
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
     uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
@@ -87,6 +88,7 @@ struct vl_program {
         uint32_t *cstate = nullptr;  // [rows][8]
         uint32_t *anom = nullptr;    // [rows][AW] chunks whose walk collided
         uint32_t *work = nullptr;    // [1 + rows] count, then candidates that need the exact recount
+        uint32_t *racc = nullptr;    // [rows][4] recount accumulators: pairs, lowest instruction, bank tally, slices done
         uint64_t rows = 0, aw = 0, vregs = 0;
     } vs[3];
     uint32_t sub_batch = 4096;       // candidates per pass of the three verify kernels

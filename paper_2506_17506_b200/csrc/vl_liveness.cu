@@ -313,6 +313,19 @@ __global__ void k_vreg_info(uint32_t V, const uint8_t *__restrict__ width, const
                (first_def_instr[v] != 0xFFFFFFFFu ? VINFO_DEFINED : 0u);
 }
 
+// Per instruction: 1 if it has a definition the walk skips (a vreg redefined from itself while it
+// stays occupied); the recount visits only those when a block's through-set collided.
+__global__ void k_instr_flags(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                              const uint8_t *__restrict__ opflags, uint8_t *iflags)
+{
+    const uint32_t i = blockIdx.x * NT + threadIdx.x;
+    if (i >= nI) return;
+    uint8_t f = 0;
+    for (uint32_t o = op_off[i]; o < op_off[i] + ndefs[i]; ++o)
+        if (opflags[o] & OPF_ELIDE) f = 1;
+    iflags[i] = f;
+}
+
 __global__ void k_fill_noop(uint4 *dst, size_t n, uint32_t spare_vreg)
 {
     for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT)
@@ -581,6 +594,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     VL_CUDA(p, keep(&p->d_lo, (size_t)p->lo_len, 0, st));
     VL_CUDA(p, keep(&p->d_ev, (size_t)steps, 0, st));
     VL_CUDA(p, keep(&p->d_vinfo, (size_t)V, 0, st));
+    VL_CUDA(p, keep(&p->d_iflags, (size_t)nI, 0, st));
     LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)steps,
            V);  // every slot starts as a no-op event
     VL_CUDA(p, keep(&p->d_th, (size_t)thn, 0, st));
@@ -609,6 +623,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     LAUNCH(k_fill_events, nC, 0, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
            p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev);
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
+    LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaStreamSynchronize(st));
     VL_CUDA(p, cudaGetLastError());

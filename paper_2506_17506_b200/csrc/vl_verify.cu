@@ -20,6 +20,7 @@
 #define MAX_STAGES 4
 #define WALK_WARPS 8
 #define RC_THREADS 256
+#define RC_SLICES 8
 
 // per-candidate state between the kernels (8 words)
 enum { CS_FLAGS = 0, CS_FIRST = 1, CS_BANK = 2, CS_NOUT = 3, CS_OUTV = 4, CS_OUTRAW = 5, CS_WALK = 6, CS_THCOL = 7 };
@@ -63,9 +64,10 @@ struct RParams {
     int bank_fast;
     uint64_t K;
     const uint32_t *vinfo, *chunk_i0, *chunk_i1, *chunk_blk, *op_off, *op_vreg, *lo_off, *lo;
-    const uint8_t *ndefs, *width, *opflags;
+    const uint8_t *ndefs, *width, *opflags, *iflags;
     const uint16_t *tg;
     const uint32_t *cstate, *anom;
+    uint32_t *racc;
     const uint2 *bank_list;
     uint32_t bank_seg[4];
     uint32_t *work;
@@ -386,6 +388,39 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
 }
 
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// A range wider than 32 registers (rare): word by word.
+__device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, uint32_t tv, uint4 e)
+{
+    uint32_t viol = 0, left = e.w >> 8, pos = tv;
+    while (left) {
+        const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
+        const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
+        uint32_t *a = s_occ + (pos >> 5) * 32 + lane;
+        const uint32_t o = *a;
+        if (e.y) viol |= o & m;
+        if (e.z) *a = o ^ m;
+        pos += nn;
+        left -= nn;
+    }
+    return viol;
+}
+
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
@@ -438,6 +473,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
     for (uint32_t c = c0 + warp; c < c1; c += WALK_WARPS) {
         for (uint32_t wd = 0; wd < q.Wp; ++wd) s_occ[wd * 32 + lane] = s_th[wd * 32 + lane];
         uint32_t viol = 0;
+        const uint32_t occ_addr = smem_u32(s_occ) + lane * 4, ev_addr = smem_u32(s_ev);
         const uint32_t s0 = q.cev_off[c], n_ev = q.cev_off[c + 1] - s0;  // a multiple of 8 events
         for (uint32_t done = 0; done < n_ev; done += q.ev_cap) {
             const uint32_t n = min(q.ev_cap, n_ev - done);
@@ -458,33 +494,23 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const uint4 e = s_ev[s + u];
+                    const uint4 e = lds128(ev_addr + (s + u) * 16);
                     const uint32_t tv = t[u];
                     if (!(e.w & 2u)) {
-                        uint32_t *a = s_occ + (tv >> 5) * 32 + lane;
-                        const uint32_t o = *a;
+                        const uint32_t a = occ_addr + ((tv >> 5) << 7);  // word (tv / 32) of this lane's mask
+                        const uint32_t o = lds32(a);
                         viol |= o & __funnelshift_l(0u, e.y, tv);
-                        *a = o ^ __funnelshift_l(0u, e.z, tv);
+                        sts32(a, o ^ __funnelshift_l(0u, e.z, tv));
                         if (e.w) {  // wider than one register: bits that spill into the next word
                             const uint32_t m1t = __funnelshift_l(e.y, 0u, tv), m1x = __funnelshift_l(e.z, 0u, tv);
                             if (m1t | m1x) {
-                                const uint32_t o2 = a[32];
+                                const uint32_t o2 = lds32(a + 128);
                                 viol |= o2 & m1t;
-                                a[32] = o2 ^ m1x;
+                                sts32(a + 128, o2 ^ m1x);
                             }
                         }
                     } else {
-                        uint32_t left = e.w >> 8, pos = tv;
-                        while (left) {
-                            const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
-                            const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
-                            uint32_t *a = s_occ + (pos >> 5) * 32 + lane;
-                            const uint32_t o = *a;
-                            if (e.y) viol |= o & m;
-                            if (e.z) *a = o ^ m;
-                            pos += nn;
-                            left -= nn;
-                        }
+                        viol |= walk_very_wide(s_occ, lane, tv, e);
                     }
                 }
             }
@@ -525,21 +551,27 @@ __global__ void k_list_all(uint64_t K, uint32_t *work)
 }
 
 // =========================================================================== k_recount
-// One thread block per listed candidate (blocks loop over the list): its table column in shared
-// memory, exact overlap counts from the live-after lists where the walk could not vouch, and the
-// general bank tally (distinct registers rather than distinct vregs).
+// Exact answers for the listed candidates.  A candidate is cut into RC_SLICES slices of the chunk
+// range; one thread block handles one (candidate, slice): it copies the candidate's table column to
+// shared memory, recounts overlaps from the live-after lists in the chunks of its slice where the
+// walk could not vouch, adds its part to the candidate's accumulators, and the slice that finishes
+// last writes the verdict.  Slice 0 also does the general bank tally (distinct registers rather than
+// distinct vregs).
 // Shared memory: [T (V+1) x u16][chunks needing every definition, AW words][chunks needing only the
 // definitions the walk skipped, AW words].
 __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 {
     extern __shared__ __align__(16) uint16_t T[];
-    __shared__ uint32_t s_pairs, s_mind, s_bank;
+    __shared__ uint32_t s_pairs, s_mind, s_bank, s_last;
     uint32_t *s_all = reinterpret_cast<uint32_t *>(T + ((q.V + 1 + 7) & ~7u));
     uint32_t *s_eli = s_all + q.AW;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t nwork = q.work[0];
-    for (uint32_t wi = blockIdx.x; wi < nwork; wi += gridDim.x) {
-        const uint64_t k = q.work[1 + wi];
+    const uint32_t per = (q.nC + RC_SLICES - 1) / RC_SLICES;
+    for (uint32_t vi = blockIdx.x; vi < nwork * RC_SLICES; vi += gridDim.x) {
+        const uint64_t k = q.work[1 + vi / RC_SLICES];
+        const uint32_t slice = vi % RC_SLICES;
+        const uint32_t cbeg = min(q.nC, slice * per), cend = min(q.nC, cbeg + per);
         const uint32_t *cs = q.cstate + k * 8;
         const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
         __syncthreads();
@@ -554,14 +586,14 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
         // a block whose through-set collided: the definitions the walk skipped (a vreg redefined
         // from itself while it stays occupied), since everything else in it was walked exactly
-        for (uint32_t c = tid; c < q.nC; c += RC_THREADS) {
+        for (uint32_t c = cbeg + tid; c < cend; c += RC_THREADS) {
             const bool all_defs = full || ((anom[c >> 5] >> (c & 31)) & 1u);
             const bool elided_only = !all_defs && ((thcol >> (q.chunk_blk[c] & 31)) & 1u);
             if (all_defs) atomicOr(&s_all[c >> 5], 1u << (c & 31));
             if (elided_only) atomicOr(&s_eli[c >> 5], 1u << (c & 31));
         }
         __syncthreads();
-        for (uint32_t cw = 0; cw < q.AW; ++cw) {
+        for (uint32_t cw = cbeg >> 5; cw < (cend + 31) >> 5; ++cw) {
             uint32_t bits = s_all[cw] | s_eli[cw];
             while (bits) {
                 const uint32_t cb = __ffs(bits) - 1;
@@ -570,6 +602,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 const bool elided_only = !((s_all[cw] >> cb) & 1u);
                 uint32_t pairs = 0, mind = 0xFFFFFFFFu;
                 for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += RC_THREADS / 32) {
+                    if (elided_only && !q.iflags[i]) continue;
                     const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
                     const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
                     for (uint32_t d = o0; d < o0 + nd; ++d) {
@@ -609,54 +642,67 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         }
         // general bank tally: a source counts when its register is new among the instruction's sources
         // and its bank is not
-        uint32_t bt = 0;
-        if (q.bank_fast) {
-            for (uint32_t e = tid; e < q.bank_seg[3]; e += RC_THREADS) {
-                const uint2 ids = q.bank_list[e];
-                const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
-                uint32_t x[4];
-                x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
+        if (slice == 0) {
+            uint32_t bt = 0;
+            if (q.bank_fast) {
+                for (uint32_t e = tid; e < q.bank_seg[3]; e += RC_THREADS) {
+                    const uint2 ids = q.bank_list[e];
+                    const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
+                    uint32_t x[4];
+                    x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
 #pragma unroll
-                for (uint32_t a = 1; a < 4; ++a) {
-                    if (a >= n) break;
-                    bool seen_value = false, seen_bank = false;
+                    for (uint32_t a = 1; a < 4; ++a) {
+                        if (a >= n) break;
+                        bool seen_value = false, seen_bank = false;
 #pragma unroll
-                    for (uint32_t bb = 0; bb < a; ++bb) {
-                        seen_value |= (x[bb] == x[a]);
-                        seen_bank |= ((x[bb] ^ x[a]) & (q.B - 1)) == 0;
+                        for (uint32_t bb = 0; bb < a; ++bb) {
+                            seen_value |= (x[bb] == x[a]);
+                            seen_bank |= ((x[bb] ^ x[a]) & (q.B - 1)) == 0;
+                        }
+                        if (!seen_value && seen_bank) ++bt;
                     }
-                    if (!seen_value && seen_bank) ++bt;
+                }
+            } else {
+                for (uint32_t i = tid; i < q.nI; i += RC_THREADS) {
+                    const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
+                    for (uint32_t a = u0 + 1; a < u1; ++a) {
+                        const uint32_t xa = T[q.op_vreg[a]];
+                        bool seen_value = false, seen_bank = false;
+                        for (uint32_t bb = u0; bb < a; ++bb) {
+                            const uint32_t xb = T[q.op_vreg[bb]];
+                            seen_value |= (xb == xa);
+                            seen_bank |= (xb % q.B == xa % q.B);
+                        }
+                        if (!seen_value && seen_bank) ++bt;
+                    }
                 }
             }
-        } else {
-            for (uint32_t i = tid; i < q.nI; i += RC_THREADS) {
-                const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
-                for (uint32_t a = u0 + 1; a < u1; ++a) {
-                    const uint32_t xa = T[q.op_vreg[a]];
-                    bool seen_value = false, seen_bank = false;
-                    for (uint32_t bb = u0; bb < a; ++bb) {
-                        const uint32_t xb = T[q.op_vreg[bb]];
-                        seen_value |= (xb == xa);
-                        seen_bank |= (xb % q.B == xa % q.B);
-                    }
-                    if (!seen_value && seen_bank) ++bt;
-                }
-            }
+#pragma unroll
+            for (int d = 16; d; d >>= 1) bt += __shfl_xor_sync(0xffffffffu, bt, d);
+            if (lane == 0 && bt) atomicAdd(&s_bank, bt);
         }
-#pragma unroll
-        for (int d = 16; d; d >>= 1) bt += __shfl_xor_sync(0xffffffffu, bt, d);
-        if (lane == 0 && bt) atomicAdd(&s_bank, bt);
         __syncthreads();
         if (tid == 0) {
-            uint32_t flags = cs[CS_FLAGS] | (s_pairs ? (uint32_t)VL_INTERFERENCE : 0u);
-            if (!flags) flags = VL_PASS;
-            const uint32_t first = min(cs[CS_FIRST], s_mind);
-            vl_verdict vd;
-            vd.flags = flags;
-            vd.first_violation_instr = first == 0xFFFFFFFFu ? -1 : (int32_t)first;
-            vd.conflict_pairs = s_pairs;
-            vd.bank_conflicts = s_bank;
-            q.out[k] = vd;
+            uint32_t *acc = q.racc + k * 4;
+            if (s_pairs) atomicAdd(&acc[0], s_pairs);
+            if (s_mind != 0xFFFFFFFFu) atomicMax(&acc[1], ~s_mind);  // accumulators start at 0: keep the complement
+            if (s_bank) atomicAdd(&acc[2], s_bank);
+            __threadfence();
+            s_last = atomicAdd(&acc[3], 1u) == RC_SLICES - 1;
+            if (s_last) {
+                __threadfence();
+                const uint32_t pairs = atomicAdd(&acc[0], 0u), mind = ~atomicMax(&acc[1], 0u),
+                               bank = atomicAdd(&acc[2], 0u);
+                uint32_t flags = cs[CS_FLAGS] | (pairs ? (uint32_t)VL_INTERFERENCE : 0u);
+                if (!flags) flags = VL_PASS;
+                const uint32_t first = min(cs[CS_FIRST], mind);
+                vl_verdict vd;
+                vd.flags = flags;
+                vd.first_violation_instr = first == 0xFFFFFFFFu ? -1 : (int32_t)first;
+                vd.conflict_pairs = pairs;
+                vd.bank_conflicts = bank;
+                q.out[k] = vd;
+            }
         }
     }
 }
@@ -700,8 +746,8 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     const uint64_t aw = std::max(1u, (p->nC + 31) / 32);
     const uint64_t groups = (rows + 31) / 32;
     if (v.rows >= rows && v.aw == aw && v.vregs == p->V) return VL_OK;
-    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work);
-    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr;
+    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc);
+    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr;
     v.rows = 0;
     // one more group than needed: it stays all zero, for lanes that have nothing to walk
     VL_CUDA(p, cudaMalloc((void **)&v.tg, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
@@ -710,6 +756,7 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.work, (1 + groups * 32) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
     v.rows = groups * 32;
     v.aw = aw;
     v.vregs = p->V;
@@ -755,6 +802,7 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         const uint32_t ngrp = (uint32_t)((n + 31) / 32);
         VL_CUDA(p, cudaMemsetAsync(vs.anom, 0, (size_t)ngrp * 32 * vs.aw * 4, st));
         VL_CUDA(p, cudaMemsetAsync(vs.work, 0, 4, st));
+        VL_CUDA(p, cudaMemsetAsync(vs.racc, 0, (size_t)ngrp * 32 * 16, st));
 
         TParams tq{};
         tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
@@ -801,7 +849,8 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         rq.bank_fast = p->bank_fast; rq.K = n;
         rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
         rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
-        rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags;
+        rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
+        rq.racc = vs.racc;
         rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out + kb;
         rq.bank_list = p->d_bank_list;
         for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
