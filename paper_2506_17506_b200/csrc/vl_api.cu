@@ -119,20 +119,16 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
 
 void vl_free_liveness(vl_program *p)
 {
-    cudaFree(p->d_chunk_i0); cudaFree(p->d_chunk_i1); cudaFree(p->d_chunk_blk); cudaFree(p->d_blk_chunk_off);
-    cudaFree(p->d_blk_in); cudaFree(p->d_blk_out); cudaFree(p->d_lo_off); cudaFree(p->d_lo);
-    cudaFree(p->d_vreg16); cudaFree(p->d_slotmeta); cudaFree(p->d_opflags); cudaFree(p->d_first_def_instr);
-    cudaFree(p->d_th_off); cudaFree(p->d_th); cudaFree(p->d_cev_off); cudaFree(p->d_ev); cudaFree(p->d_vinfo);
-    cudaFree(p->d_iflags);
-    p->d_iflags = nullptr;
-    cudaFree(p->d_item_blk); cudaFree(p->d_item_c0); cudaFree(p->d_item_c1);
-    p->d_item_blk = p->d_item_c0 = p->d_item_c1 = nullptr;
-    p->d_vinfo = nullptr;
+    // everything below lives in the handle's pools, which are rewound, not freed
+    p->live_arena.reset();
+    p->tmp_arena.reset();
     p->d_chunk_i0 = p->d_chunk_i1 = p->d_chunk_blk = p->d_blk_chunk_off = nullptr;
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
-    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_first_def_instr = nullptr;
+    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_iflags = nullptr;
+    p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
+    p->d_item_blk = p->d_item_c0 = p->d_item_c1 = nullptr;
     p->live_ok = false;
     p->lo_len = 0;
 }
@@ -142,6 +138,8 @@ extern "C" void vl_program_destroy(vl_program *p)
     if (!p) return;
     cudaSetDevice(p->device);
     vl_free_liveness(p);
+    p->live_arena.release();
+    p->tmp_arena.release();
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);

@@ -33,6 +33,39 @@ enum : uint32_t {
 
 #define VL_MAX_GROUP 4
 
+// Device memory pool of a program handle: slabs are kept across calls, so that a repeated
+// vl_liveness on the same handle allocates nothing.
+struct VlArena {
+    struct Slab { char *ptr; size_t size; };
+    std::vector<Slab> slabs;
+    size_t cur = 0, off = 0;
+    cudaError_t alloc(void **out, size_t bytes)
+    {
+        bytes = (bytes + 64 + 255) & ~(size_t)255;
+        for (; cur < slabs.size(); ++cur, off = 0)
+            if (off + bytes <= slabs[cur].size) {
+                *out = slabs[cur].ptr + off;
+                off += bytes;
+                return cudaSuccess;
+            }
+        Slab s{nullptr, bytes > ((size_t)4 << 20) ? bytes : ((size_t)4 << 20)};
+        cudaError_t e = cudaMalloc((void **)&s.ptr, s.size);
+        if (e != cudaSuccess) return e;
+        slabs.push_back(s);
+        cur = slabs.size() - 1;
+        *out = s.ptr;
+        off = bytes;
+        return cudaSuccess;
+    }
+    void reset() { cur = 0; off = 0; }
+    void release()
+    {
+        for (auto &s : slabs) cudaFree(s.ptr);
+        slabs.clear();
+        reset();
+    }
+};
+
 struct vl_program {
     int device = 0;
     uint32_t nB = 0, nI = 0, V = 0, nO = 0, nE = 0, P = 0, B = 0;
@@ -78,6 +111,7 @@ struct vl_program {
     uint32_t threads_opt = 0;
     int use_th = 0;
 
+    VlArena live_arena, tmp_arena;  // liveness results and tables / liveness working sets
     uint32_t *d_status = nullptr;  // [16] device status words
     int last_cuda_error = 0;
     bool live_ok = false;

@@ -155,55 +155,90 @@ __global__ void k_chunk_boundaries(const uint32_t *__restrict__ blk_chunk_off, u
     }
 }
 
-// Backward walk of one chunk.  FILL = false: list sizes, per-operand flags, walk-event counts,
-// and the set of vregs whose occupancy changes inside the chunk.  FILL = true: the lists.
+// Backward walk of one chunk by one warp.  FILL = false: list sizes, per-operand flags, walk-event
+// counts, and the set of vregs whose occupancy changes inside the chunk.  FILL = true: the lists.
+// The chunk's slice of the operand arrays is staged in shared memory when it fits (WALK_CAP_I
+// instructions, WALK_CAP_O operands); lane 0 does the per-instruction bookkeeping, all lanes the
+// population count / compaction of the live bitset.
+#define WALK_CAP_I 256
+#define WALK_CAP_O 2048
 template <bool FILL>
-__global__ void k_instr_walk(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
-                             const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
-                             const uint32_t *__restrict__ op_vreg, uint32_t Wv,
-                             const uint32_t *__restrict__ chunk_end, uint32_t *lo_cnt, uint32_t *ev_cnt,
-                             uint8_t *opflags, uint32_t *chunk_touch, const uint32_t *__restrict__ lo_off,
-                             uint32_t *lo)
+__global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ chunk_i0,
+                                                   const uint32_t *__restrict__ chunk_i1,
+                                                   const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
+                                                   const uint32_t *__restrict__ op_vreg, uint32_t Wv,
+                                                   const uint32_t *__restrict__ chunk_end, uint32_t *lo_cnt,
+                                                   uint32_t *ev_cnt, uint8_t *opflags, uint32_t *chunk_touch,
+                                                   const uint32_t *__restrict__ lo_off, uint32_t *lo)
 {
     extern __shared__ uint32_t sm[];
     uint32_t *s_live = sm, *s_touch = sm + Wv;
-    __shared__ uint32_t s_scan[34];
-    const uint32_t c = blockIdx.x;
-    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
+    uint32_t *s_off = sm + 2 * Wv;                 // [WALK_CAP_I + 1]
+    uint32_t *s_lo = s_off + WALK_CAP_I + 1;       // [WALK_CAP_I] list offsets (FILL)
+    uint32_t *s_ops = s_lo + WALK_CAP_I;           // [WALK_CAP_O]
+    uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_ops + WALK_CAP_O);  // [WALK_CAP_I]
+    const uint32_t c = blockIdx.x, lane = threadIdx.x;
+    const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
+    for (uint32_t w = lane; w < Wv; w += 32) {
         s_live[w] = chunk_end[(size_t)c * Wv + w];
         if (!FILL) s_touch[w] = 0;
     }
-    __syncthreads();
-    for (uint32_t i = chunk_i1[c]; i-- > chunk_i0[c];) {
-        uint32_t total;
-        if (FILL) {
-            const uint32_t base = lo_off[i];
-            compact_bits(s_live, Wv, s_scan, &total, [&](uint32_t rank, uint32_t v) { lo[base + rank] = v; });
-        } else {
-            uint32_t cnt = 0;
-            for (uint32_t w = threadIdx.x; w < Wv; w += NT) cnt += __popc(s_live[w]);
-            block_excl_scan(cnt, s_scan, &total);
+    const uint32_t ob = i1 > i0 ? op_off[i0] : 0, oe = i1 > i0 ? op_off[i1] : 0;
+    const bool staged = (i1 - i0) <= WALK_CAP_I && (oe - ob) <= WALK_CAP_O;
+    if (staged) {
+        for (uint32_t i = i0 + lane; i <= i1; i += 32) s_off[i - i0] = op_off[i];
+        for (uint32_t i = i0 + lane; i < i1; i += 32) {
+            s_nd[i - i0] = ndefs[i];
+            if (FILL) s_lo[i - i0] = lo_off[i];
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+        for (uint32_t o = ob + lane; o < oe; o += 32) s_ops[o - ob] = op_vreg[o];
+    }
+    __syncwarp();
+    auto OFF = [&](uint32_t i) { return staged ? s_off[i - i0] : op_off[i]; };
+    auto ND = [&](uint32_t i) -> uint32_t { return staged ? s_nd[i - i0] : ndefs[i]; };
+    auto OP = [&](uint32_t o) { return staged ? s_ops[o - ob] : op_vreg[o]; };
+    const uint32_t per = (Wv + 31) / 32;
+    const uint32_t w0 = min(Wv, lane * per), w1 = min(Wv, w0 + per);
+    for (uint32_t i = i1; i-- > i0;) {
+        uint32_t cnt = 0;
+        for (uint32_t w = w0; w < w1; ++w) cnt += __popc(s_live[w]);
+        uint32_t inc = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += y;
+        }
+        const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+        if (FILL) {
+            uint32_t at = (staged ? s_lo[i - i0] : lo_off[i]) + inc - cnt;
+            for (uint32_t w = w0; w < w1; ++w) {
+                uint32_t x = s_live[w];
+                while (x) {
+                    const uint32_t bpos = __ffs(x) - 1;
+                    x &= x - 1;
+                    lo[at++] = w * 32 + bpos;
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            const uint32_t o0 = OFF(i), o1 = OFF(i + 1), nd = ND(i);
             if (!FILL) {
                 lo_cnt[i] = total;
                 uint32_t evs = 0;
                 for (uint32_t o = o0 + nd; o < o1; ++o) {
-                    const uint32_t v = op_vreg[o];
-                    bool dup = false, isdef = false;
-                    for (uint32_t q = o0 + nd; q < o; ++q) dup |= (op_vreg[q] == v);
-                    for (uint32_t q = o0; q < o0 + nd; ++q) isdef |= (op_vreg[q] == v);
+                    const uint32_t v = OP(o);
+                    bool dup = false;
+                    for (uint32_t q = o0 + nd; q < o; ++q) dup |= (OP(q) == v);
                     const bool lv = bit_get(s_live, v);
                     const bool kill = !dup && !lv;  // a read of a vreg that stays live releases nothing
                     opflags[o] = (uint8_t)((kill ? OPF_KILL : 0) | (dup ? OPF_DUP : 0));
                     if (kill) { ++evs; bit_set(s_touch, v); }
                 }
                 for (uint32_t o = o0; o < o0 + nd; ++o) {
-                    const uint32_t v = op_vreg[o];
+                    const uint32_t v = OP(o);
                     bool selfuse = false;
-                    for (uint32_t q = o0 + nd; q < o1; ++q) selfuse |= (op_vreg[q] == v);
+                    for (uint32_t q = o0 + nd; q < o1; ++q) selfuse |= (OP(q) == v);
                     const bool lv = bit_get(s_live, v);
                     const bool elide = selfuse && lv;
                     const bool set = lv || nd > 1;
@@ -214,30 +249,59 @@ __global__ void k_instr_walk(const uint32_t *__restrict__ chunk_i0, const uint32
                 }
                 ev_cnt[i] = evs;
             }
-            for (uint32_t o = o0; o < o0 + nd; ++o) bit_clr(s_live, op_vreg[o]);
-            for (uint32_t o = o0 + nd; o < o1; ++o) bit_set(s_live, op_vreg[o]);
+            for (uint32_t o = o0; o < o0 + nd; ++o) bit_clr(s_live, OP(o));
+            for (uint32_t o = o0 + nd; o < o1; ++o) bit_set(s_live, OP(o));
         }
-        __syncthreads();
+        __syncwarp();
     }
     if (!FILL)
-        for (uint32_t w = threadIdx.x; w < Wv; w += NT) chunk_touch[(size_t)c * Wv + w] = s_touch[w];
+        for (uint32_t w = lane; w < Wv; w += 32) chunk_touch[(size_t)c * Wv + w] = s_touch[w];
 }
 
-// Exclusive scan of a u32 array by one block; out[n] = total (saturated), total64 exact.
-__global__ void k_scan(const uint32_t *__restrict__ in, uint32_t *out, uint32_t n, unsigned long long *total64,
-                       uint32_t *status)
+// Exclusive scan of a u32 array by one block of 1024 threads, 4 items per thread and round;
+// out[n] = total (saturated), total64 exact.
+__global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in, uint32_t *out, uint32_t n,
+                                               unsigned long long *total64, uint32_t *status)
 {
-    __shared__ uint32_t s_scan[34];
+    __shared__ uint32_t s_w[33];
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long carry = 0;
-    for (uint32_t base = 0; base < n; base += NT) {
-        const uint32_t idx = base + threadIdx.x;
-        const uint32_t x = idx < n ? in[idx] : 0u;
-        uint32_t total;
-        const uint32_t ex = block_excl_scan(x, s_scan, &total);
-        if (idx < n) out[idx] = (uint32_t)(carry + ex);
-        carry += total;
+    for (uint32_t base = 0; base < n; base += 4096) {
+        const uint32_t i = base + tid * 4;
+        uint32_t x[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[j] = i + j < n ? in[i + j] : 0u;
+        const uint32_t mine = x[0] + x[1] + x[2] + x[3];
+        uint32_t inc = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += y;
+        }
+        __syncthreads();
+        if (lane == 31) s_w[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint32_t t = s_w[lane];
+            uint32_t ti = t;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, ti, d);
+                if (lane >= d) ti += y;
+            }
+            s_w[lane] = ti - t;
+            if (lane == 31) s_w[32] = ti;
+        }
+        __syncthreads();
+        uint32_t ex = (uint32_t)carry + s_w[warp] + inc - mine;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (i + j < n) out[i + j] = ex;
+            ex += x[j];
+        }
+        carry += s_w[32];
     }
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         out[n] = carry > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)carry;
         *total64 = carry;
         if (carry > 0xFFFFFFF0ull) atomicOr(status, ST_SIZE_OVERFLOW);
@@ -441,27 +505,23 @@ __global__ void k_fill_through(uint32_t Wv, const uint32_t *__restrict__ blk_th,
 
 // --------------------------------------------------------------------------- host
 namespace {
-struct Scratch {
-    std::vector<void *> ptrs;
-    ~Scratch() { for (void *q : ptrs) cudaFree(q); }
+template <typename T>
+cudaError_t pool_get(VlArena &arena, T **out, size_t n, int fill, bool do_fill, cudaStream_t st)
+{
+    cudaError_t e = arena.alloc((void **)out, std::max<size_t>(n, 1) * sizeof(T));
+    if (e != cudaSuccess || !do_fill) return e;
+    return cudaMemsetAsync(*out, fill, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
+}
+struct TmpPool {
+    vl_program *p;
     template <typename T>
     cudaError_t get(T **out, size_t n, bool zero, cudaStream_t st)
     {
-        cudaError_t e = cudaMalloc((void **)out, std::max<size_t>(n, 1) * sizeof(T) + 64);
-        if (e != cudaSuccess) return e;
-        ptrs.push_back(*out);
-        if (zero) e = cudaMemsetAsync(*out, 0, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
-        return e;
+        return pool_get(p->tmp_arena, out, n, 0, zero, st);
     }
 };
-template <typename T>
-cudaError_t keep(T **out, size_t n, int fill, cudaStream_t st)
-{
-    cudaError_t e = cudaMalloc((void **)out, std::max<size_t>(n, 1) * sizeof(T) + 64);
-    if (e != cudaSuccess) return e;
-    return cudaMemsetAsync(*out, fill, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
-}
 }  // namespace
+#define keep(out, n, fill, st) pool_get(p->live_arena, out, n, fill, true, st)
 
 #define LAUNCH(kernel, grid, smem, st, ...)                          \
     do {                                                             \
@@ -494,6 +554,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
     p->use_th = (nB <= 32 && (uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
     const size_t smem2 = (size_t)2 * Wv * 4;
+    const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O) * 4 + WALK_CAP_I + 16;
 
     VL_CUDA(p, keep(&p->d_chunk_i0, nC, 0, st));
     VL_CUDA(p, keep(&p->d_chunk_i1, nC, 0, st));
@@ -514,7 +575,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     VL_CUDA(p, keep(&p->d_slotmeta, (size_t)p->nOp8 / 8, 0, st));
     VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
 
-    Scratch sc;
+    TmpPool sc{p};
     uint32_t *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry, *blk_use, *blk_def, *blk_th;
     uint32_t *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
     uint8_t *opmeta;
@@ -545,10 +606,11 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
            p->d_blk_out, p->d_status);
     LAUNCH(k_chunk_boundaries, nB, 0, st, p->d_blk_chunk_off, Wv, p->d_blk_out, chunk_use, chunk_def, chunk_end,
            chunk_entry);
-    LAUNCH(k_instr_walk<false>, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
+    if (nC) k_instr_walk<false><<<nC, 32, walk_smem, st>>>( p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
            Wv, chunk_end, lo_cnt, ev_cnt, p->d_opflags, chunk_touch, (const uint32_t *)nullptr, (uint32_t *)nullptr);
-    LAUNCH(k_scan, 1, 0, st, lo_cnt, p->d_lo_off, nI, totals + 0, p->d_status);
-    LAUNCH(k_scan, 1, 0, st, ev_cnt, ev_off, nI, totals + 1, p->d_status);
+    k_scan<<<1, 1024, 0, st>>>(lo_cnt, p->d_lo_off, nI, totals + 0, p->d_status);
+    k_scan<<<1, 1024, 0, st>>>(ev_cnt, ev_off, nI, totals + 1, p->d_status);
+    g_vl_launches.fetch_add(2);
     LAUNCH(k_block_through, nB, 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
     LAUNCH(k_chunk_entry, nC, 0, st, p->d_chunk_blk, p->d_chunk_i0, p->d_chunk_i1, Wv, blk_th, chunk_entry, ev_off,
            centry_cnt, cev);
@@ -611,9 +673,10 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     VL_CUDA(p, cudaMemcpyAsync(p->d_cev_off, h_cev_off.data(), (nC + 1) * 4, cudaMemcpyHostToDevice, st));
     VL_CUDA(p, cudaMemcpyAsync(p->d_th_off, h_th_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
 
-    LAUNCH(k_instr_walk<true>, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
+    if (nC) k_instr_walk<true><<<nC, 32, walk_smem, st>>>( p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
            Wv, chunk_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr, (uint32_t *)nullptr,
            (const uint32_t *)p->d_lo_off, p->d_lo);
+    g_vl_launches.fetch_add(2);  // the two k_instr_walk passes
     LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_first_def_instr);
     LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, st, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
