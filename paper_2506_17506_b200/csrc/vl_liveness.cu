@@ -162,6 +162,7 @@ __global__ void k_chunk_boundaries(const uint32_t *__restrict__ blk_chunk_off, u
 // population count / compaction of the live bitset.
 #define WALK_CAP_I 256
 #define WALK_CAP_O 2048
+#define WALK_CAP_L 1024
 template <bool FILL>
 __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ chunk_i0,
                                                    const uint32_t *__restrict__ chunk_i1,
@@ -176,7 +177,8 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
     uint32_t *s_off = sm + 2 * Wv;                 // [WALK_CAP_I + 1]
     uint32_t *s_lo = s_off + WALK_CAP_I + 1;       // [WALK_CAP_I] list offsets (FILL)
     uint32_t *s_ops = s_lo + WALK_CAP_I;           // [WALK_CAP_O]
-    uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_ops + WALK_CAP_O);  // [WALK_CAP_I]
+    uint32_t *s_list = s_ops + WALK_CAP_O;         // [WALK_CAP_L] one live-after list (FILL)
+    uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_list + WALK_CAP_L);  // [WALK_CAP_I]
     const uint32_t c = blockIdx.x, lane = threadIdx.x;
     const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
     for (uint32_t w = lane; w < Wv; w += 32) {
@@ -197,28 +199,31 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
     auto OFF = [&](uint32_t i) { return staged ? s_off[i - i0] : op_off[i]; };
     auto ND = [&](uint32_t i) -> uint32_t { return staged ? s_nd[i - i0] : ndefs[i]; };
     auto OP = [&](uint32_t o) { return staged ? s_ops[o - ob] : op_vreg[o]; };
-    const uint32_t per = (Wv + 31) / 32;
-    const uint32_t w0 = min(Wv, lane * per), w1 = min(Wv, w0 + per);
+    const uint32_t rounds = (Wv + 31) / 32;
     for (uint32_t i = i1; i-- > i0;) {
-        uint32_t cnt = 0;
-        for (uint32_t w = w0; w < w1; ++w) cnt += __popc(s_live[w]);
-        uint32_t inc = cnt;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += y;
-        }
-        const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+        uint32_t total = 0;
         if (FILL) {
-            uint32_t at = (staged ? s_lo[i - i0] : lo_off[i]) + inc - cnt;
-            for (uint32_t w = w0; w < w1; ++w) {
-                uint32_t x = s_live[w];
-                while (x) {
-                    const uint32_t bpos = __ffs(x) - 1;
-                    x &= x - 1;
-                    lo[at++] = w * 32 + bpos;
+            // ascending ids, 32 words per round; every non-empty word is broadcast and each lane whose
+            // bit is set writes its id at the rank of that bit: up to 32 consecutive stores per word
+            uint32_t at = staged ? s_lo[i - i0] : lo_off[i];
+            for (uint32_t r = 0; r < rounds; ++r) {
+                const uint32_t w = r * 32 + lane;
+                const uint32_t mine = w < Wv ? s_live[w] : 0u;
+                uint32_t nz = __ballot_sync(0xffffffffu, mine != 0);
+                while (nz) {
+                    const uint32_t src = __ffs(nz) - 1;
+                    nz &= nz - 1;
+                    const uint32_t x = __shfl_sync(0xffffffffu, mine, src);
+                    if ((x >> lane) & 1u) lo[at + __popc(x & ((1u << lane) - 1u))] = (r * 32 + src) * 32 + lane;
+                    at += __popc(x);
                 }
             }
+        } else {
+            uint32_t cnt = 0;
+            for (uint32_t w = lane; w < Wv; w += 32) cnt += __popc(s_live[w]);
+#pragma unroll
+            for (int d = 16; d; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+            total = cnt;
         }
         __syncwarp();
         if (lane == 0) {
@@ -554,7 +559,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
     p->use_th = (nB <= 32 && (uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
     const size_t smem2 = (size_t)2 * Wv * 4;
-    const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O) * 4 + WALK_CAP_I + 16;
+    const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O + WALK_CAP_L) * 4 + WALK_CAP_I + 16;
 
     VL_CUDA(p, keep(&p->d_chunk_i0, nC, 0, st));
     VL_CUDA(p, keep(&p->d_chunk_i1, nC, 0, st));
