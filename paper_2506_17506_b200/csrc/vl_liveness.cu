@@ -398,7 +398,7 @@ __global__ void k_instr_flags(uint32_t nI, const uint32_t *__restrict__ op_off, 
 __global__ void k_fill_noop(uint4 *dst, size_t n, uint32_t spare_vreg)
 {
     for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT)
-        dst[i] = make_uint4(spare_vreg, 0u, 0u, 0u);
+        dst[i] = make_uint4(spare_vreg, 0u, 0u, 31u);
 }
 
 __global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
@@ -448,13 +448,14 @@ __global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8
 }
 
 // A walk event is 16 bytes: x = vreg, y = bits to test, z = bits to toggle (the width-w mask
-// (1<<w)-1, or 0), w = 1 if the range may straddle a 32-bit word (w > 1).  Ranges wider than 32
-// registers carry w = 2 | width << 8 and y, z as 0/1 flags.  A no-op names the spare vreg V.
+// (1<<w)-1, or 0), w = 32 - width: the range straddles a 32-bit word iff (register & 31) > w.
+// Ranges wider than 32 registers carry w = 0x80000000 | width and y, z as 0/1 flags.
+// A no-op names the spare vreg V with empty masks.
 __device__ __forceinline__ uint4 make_event(uint32_t v, uint32_t w, bool test, bool toggle)
 {
-    if (w > 32) return make_uint4(v, test ? 1u : 0u, toggle ? 1u : 0u, 2u | (w << 8));
+    if (w > 32) return make_uint4(v, test ? 1u : 0u, toggle ? 1u : 0u, 0x80000000u | w);
     const uint32_t wm = w == 32 ? 0xFFFFFFFFu : ((1u << w) - 1u);
-    return make_uint4(v, test ? wm : 0u, toggle ? wm : 0u, w > 1 ? 1u : 0u);
+    return make_uint4(v, test ? wm : 0u, toggle ? wm : 0u, 32u - w);
 }
 
 // Walk events of one chunk: entry occupancy (ascending vreg id), then per instruction the

@@ -74,6 +74,23 @@ struct RParams {
     vl_verdict *out;
 };
 
+// Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
+// status[2 + phase]); compiled in only with -DVL_PHASE_TIMERS, for profiling builds.
+#ifdef VL_PHASE_TIMERS
+#define PT_INIT() long long pt_last = clock64()
+#define PT(idx)                                                                \
+    do {                                                                       \
+        if (threadIdx.x == 0) {                                                \
+            long long now = clock64();                                         \
+            atomicAdd(q.status + 2 + (idx), (uint32_t)((now - pt_last) >> 6)); \
+            pt_last = now;                                                     \
+        }                                                                      \
+    } while (0)
+#else
+#define PT_INIT()
+#define PT(idx)
+#endif
+
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -175,38 +192,28 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     };
     if (tid == 0)
         for (uint32_t t = 0; t < q.NS && t < q.ntiles; ++t) issue_tile(t);
+    PT_INIT();
 
-    // operand metadata of the next tile is fetched one iteration ahead (global memory, L2 latency)
-    uint4 nx_v4 = make_uint4(0, 0, 0, 0);
-    uint32_t nx_first = 0;
-    if (tid * 8 < q.nOp8) {
-        nx_v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + tid * 8);
-        nx_first = (uint32_t)q.slotmeta[tid] & 0xFFu;
-    }
-    for (uint32_t t = 0; t < q.ntiles; ++t) {
+    // Per tile: load it from the ring and store its first occurrences to the table, barrier, compare
+    // every occurrence with the table.  The compare of tile t may overlap the stores of tile t+1 by
+    // faster threads: those are first occurrences of other vregs.
+    auto wait_tile = [&](uint32_t t) {  // bounded wait
         const uint32_t stage = t % q.NS, parity = (t / q.NS) & 1;
-        const uint4 v4 = nx_v4;
-        const uint32_t first = nx_first;
-        {
-            const uint32_t o_next = (t + 1) * TILE + tid * 8;
-            if (t + 1 < q.ntiles && o_next < q.nOp8) {
-                nx_v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + o_next);
-                nx_first = (uint32_t)q.slotmeta[o_next >> 3] & 0xFFu;
+        uint32_t spins = 0;
+        const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 22);
+        while (!mbar_try_wait(&M->bar[stage], parity)) {
+            if (++spins > limit) {
+                M->abort_flag = 1;
+                atomicOr(q.status, ST_DEVICE_WAIT);
+                break;
             }
         }
-        {  // bounded wait for the tile
-            uint32_t spins = 0;
-            const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 22);
-            while (!mbar_try_wait(&M->bar[stage], parity)) {
-                if (++spins > limit) {
-                    M->abort_flag = 1;
-                    atomicOr(q.status, ST_DEVICE_WAIT);
-                    break;
-                }
-            }
-        }
-        const uint32_t o_base = t * TILE + tid * 8;
-        const bool act = o_base < q.nOp8;
+    };
+    // loads this thread's 8 operands x G candidates of tile t and transposes them to
+    // "G candidates side by side per operand"; stores the first occurrences
+    auto load_tile = [&](uint32_t t, uint64_t (&pc)[8], uint32_t (&vj)[8], const uint4 &v4, uint32_t first) {
+        const uint32_t stage = t % q.NS;
+        const bool act = t * TILE + tid * 8 < q.nOp8;
         uint32_t r[G][4];
         if (act) {
 #pragma unroll
@@ -220,8 +227,6 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
             for (int g = 0; g < G; ++g) r[g][0] = r[g][1] = r[g][2] = r[g][3] = 0;
         }
         const uint32_t vr[4] = {v4.x, v4.y, v4.z, v4.w};
-        uint64_t pc[8];
-        uint32_t vj[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int k = j >> 1;
@@ -236,44 +241,71 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
             }
             vj[j] = (j & 1) ? (vr[k] >> 16) : (vr[k] & 0xFFFFu);
         }
-        // first occurrences write the table ...
         if (act) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 if ((first >> j) & 1) t_store<G>(Tt, vj[j], pc[j]);
         }
-        __syncthreads();
-        // the stage just read is free again: refill it with the tile NS ahead
-        if (tid == 0 && t + q.NS < q.ntiles) issue_tile(t + q.NS);
-        // ... and every occurrence is compared with it (a first occurrence trivially matches;
-        // padding operands beyond n_operands are left out)
-        if (act) {
-            uint64_t acc = 0;
-            if (o_base + 8 <= q.nO) {
+    };
+    // every occurrence of tile t against the table (a first occurrence trivially matches; padding
+    // operands beyond n_operands are left out)
+    auto compare_tile = [&](uint32_t t, const uint64_t (&pc)[8], const uint32_t (&vj)[8]) {
+        const uint32_t o_base = t * TILE + tid * 8;
+        if (o_base >= q.nOp8) return;
+        uint64_t acc = 0;
+        if (o_base + 8 <= q.nO) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc |= t_load<G>(Tt, vj[j]) ^ pc[j];
-            } else {
+            for (int j = 0; j < 8; ++j) acc |= t_load<G>(Tt, vj[j]) ^ pc[j];
+        } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (o_base + j < q.nO) acc |= t_load<G>(Tt, vj[j]) ^ pc[j];
+            for (int j = 0; j < 8; ++j)
+                if (o_base + j < q.nO) acc |= t_load<G>(Tt, vj[j]) ^ pc[j];
+        }
+        if (acc) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (o_base + j >= q.nO) continue;
+                const uint64_t d = t_load<G>(Tt, vj[j]) ^ pc[j];
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (pk_get(d, g)) {
+                        atomicOr(&M->flags[g], (uint32_t)VL_INCONSISTENT);
+                        atomicMin(&M->minop[g], o_base + j);
+                    }
             }
-            if (acc) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (o_base + j >= q.nO) continue;
-                    const uint64_t d = t_load<G>(Tt, vj[j]) ^ pc[j];
-#pragma unroll
-                    for (int g = 0; g < G; ++g)
-                        if (pk_get(d, g)) {
-                            atomicOr(&M->flags[g], (uint32_t)VL_INCONSISTENT);
-                            atomicMin(&M->minop[g], o_base + j);
-                        }
-                }
-            }
+        }
+    };
+    // operand metadata (vreg ids, first-occurrence bits) comes from global memory, fetched one tile ahead
+    auto load_meta = [&](uint32_t t, uint4 &v4, uint32_t &first) {
+        const uint32_t o = t * TILE + tid * 8;
+        if (t < q.ntiles && o < q.nOp8) {
+            v4 = *reinterpret_cast<const uint4 *>(q.vreg16 + o);
+            first = (uint32_t)q.slotmeta[o >> 3] & 0xFFu;
+        } else {
+            v4 = make_uint4(0, 0, 0, 0);
+            first = 0;
+        }
+    };
+    {
+        uint64_t pc[8];
+        uint32_t vj[8];
+        uint4 m_v4, m2_v4;
+        uint32_t m_first, m2_first;
+        load_meta(0, m_v4, m_first);
+        for (uint32_t t = 0; t < q.ntiles; ++t) {
+            load_meta(t + 1, m2_v4, m2_first);
+            wait_tile(t);
+            load_tile(t, pc, vj, m_v4, m_first);
+            __syncthreads();
+            if (tid == 0 && t + q.NS < q.ntiles) issue_tile(t + q.NS);  // the stage just read is free again
+            compare_tile(t, pc, vj);
+            m_v4 = m2_v4;
+            m_first = m2_first;
         }
     }
     __syncthreads();
 
+    PT(0);
     // ------------------------------------------------- realizability, one sweep over the vregs
     for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NT) {
         uint32_t vis[4], fds[4];
@@ -303,6 +335,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         }
     }
 
+    PT(1);
     // ------------------------------- bank tally from T: instructions with 2..4 distinct sources.
     // Distinct vregs read by one instruction are live together, so a candidate whose walk sees no
     // collision has them on distinct registers and only the banks need comparing; candidates with
@@ -312,23 +345,42 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         const uint64_t BM = L1 * q.Bmask;
         uint64_t acc = 0;
         auto same = [&](uint64_t x) -> uint64_t { return ((x | (x >> 1)) & L1) ^ L1; };  // per lane: x == 0
-        for (uint32_t e = q.bank_seg[0] + tid; e < q.bank_seg[1]; e += NT) {
-            const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16);
-            acc += same((a ^ b) & BM);
+        // four list entries per thread in flight (the lists sit in global memory)
+        for (uint32_t e0 = q.bank_seg[0] + tid; e0 < q.bank_seg[1]; e0 += 4 * NT) {
+            uint2 ids[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[1] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (e0 + u * NT >= q.bank_seg[1]) break;
+                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16);
+                acc += same((a ^ b) & BM);
+            }
         }
-        for (uint32_t e = q.bank_seg[1] + tid; e < q.bank_seg[2]; e += NT) {
-            const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16),
-                           c = t_load<G>(Tt, ids.y & 0xFFFFu);
-            acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM));
+        for (uint32_t e0 = q.bank_seg[1] + tid; e0 < q.bank_seg[2]; e0 += 4 * NT) {
+            uint2 ids[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[2] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (e0 + u * NT >= q.bank_seg[2]) break;
+                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16),
+                               c = t_load<G>(Tt, ids[u].y & 0xFFFFu);
+                acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM));
+            }
         }
-        for (uint32_t e = q.bank_seg[2] + tid; e < q.bank_seg[3]; e += NT) {
-            const uint2 ids = q.bank_list[e];
-            const uint64_t a = t_load<G>(Tt, ids.x & 0xFFFFu), b = t_load<G>(Tt, ids.x >> 16),
-                           c = t_load<G>(Tt, ids.y & 0xFFFFu), d = t_load<G>(Tt, ids.y >> 16);
-            acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM)) +
-                   (same((d ^ a) & BM) | same((d ^ b) & BM) | same((d ^ c) & BM));
+        for (uint32_t e0 = q.bank_seg[2] + tid; e0 < q.bank_seg[3]; e0 += 4 * NT) {
+            uint2 ids[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[3] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (e0 + u * NT >= q.bank_seg[3]) break;
+                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16),
+                               c = t_load<G>(Tt, ids[u].y & 0xFFFFu), d = t_load<G>(Tt, ids[u].y >> 16);
+                acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM)) +
+                       (same((d ^ a) & BM) | same((d ^ b) & BM) | same((d ^ c) & BM));
+            }
         }
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -340,6 +392,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     __syncthreads();
 
+    PT(2);
     // ------------------------------------------------- hand-over to the walk
     // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
     // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
@@ -364,6 +417,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
             }
         }
     }
+    PT(3);
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
@@ -398,6 +452,12 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
 {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t atom_xor_shared(uint32_t addr, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.shared.xor.b32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {
     uint4 v;
@@ -407,7 +467,7 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
 // A range wider than 32 registers (rare): word by word.
 __device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, uint32_t tv, uint4 e)
 {
-    uint32_t viol = 0, left = e.w >> 8, pos = tv;
+    uint32_t viol = 0, left = e.w & 0xFFFFu, pos = tv;
     while (left) {
         const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
         const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
@@ -424,6 +484,7 @@ __device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, 
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
+template <bool WIDE>
 __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
 {
     extern __shared__ __align__(16) uint32_t wsm[];
@@ -496,21 +557,18 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
                 for (int u = 0; u < 8; ++u) {
                     const uint4 e = lds128(ev_addr + (s + u) * 16);
                     const uint32_t tv = t[u];
-                    if (!(e.w & 2u)) {
-                        const uint32_t a = occ_addr + ((tv >> 5) << 7);  // word (tv / 32) of this lane's mask
-                        const uint32_t o = lds32(a);
-                        viol |= o & __funnelshift_l(0u, e.y, tv);
-                        sts32(a, o ^ __funnelshift_l(0u, e.z, tv));
-                        if (e.w) {  // wider than one register: bits that spill into the next word
-                            const uint32_t m1t = __funnelshift_l(e.y, 0u, tv), m1x = __funnelshift_l(e.z, 0u, tv);
-                            if (m1t | m1x) {
-                                const uint32_t o2 = lds32(a + 128);
-                                viol |= o2 & m1t;
-                                sts32(a + 128, o2 ^ m1x);
-                            }
-                        }
-                    } else {
+                    if (WIDE && (int)e.w < 0) {
                         viol |= walk_very_wide(s_occ, lane, tv, e);
+                        continue;
+                    }
+                    const uint32_t a = occ_addr + ((tv >> 5) << 7);  // word (tv / 32) of this lane's mask
+                    // toggling returns the old word: occupied and released are both a toggle as long as
+                    // no collision has been seen (after one, the chunk is recounted exactly anyway)
+                    const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, e.z, tv));
+                    viol |= o & __funnelshift_l(0u, e.y, tv);
+                    if ((tv & 31u) > e.w) {  // the range straddles into the next word
+                        const uint32_t o2 = atom_xor_shared(a + 128, __funnelshift_l(e.z, 0u, tv));
+                        viol |= o2 & __funnelshift_l(e.y, 0u, tv);
                     }
                 }
             }
@@ -792,7 +850,9 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
     vl_program::VScratch &vs = p->vs[slot];
     cudaError_t e = cudaSuccess;
     if (walk_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
+        e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
+    if (e == cudaSuccess && walk_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
     if (e == cudaSuccess && rc_smem > 48 * 1024)
         e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rc_smem);
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
@@ -836,7 +896,8 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
             wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
             wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = ev_cap;
             wq.cstate = vs.cstate; wq.anom = vs.anom;
-            k_walk<<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
+            if (p->wmax > 32) k_walk<true><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
+            else k_walk<false><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
             e = cudaGetLastError();
             if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
             g_vl_launches.fetch_add(1);
