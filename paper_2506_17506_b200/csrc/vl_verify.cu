@@ -20,7 +20,6 @@
 #define MAX_STAGES 4
 #define WALK_WARPS 8
 #define RC_THREADS 256
-#define RC_SLICES 8
 
 // per-candidate state between the kernels (8 words)
 enum { CS_FLAGS = 0, CS_FIRST = 1, CS_BANK = 2, CS_NOUT = 3, CS_OUTV = 4, CS_OUTRAW = 5, CS_WALK = 6, CS_THCOL = 7 };
@@ -581,126 +580,124 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
 }
 
 // =========================================================================== k_finish
-// Verdicts of the candidates the walk vouches for; the others go on the work list.
-__global__ void k_finish(uint64_t K, const uint32_t *__restrict__ cstate, uint32_t *work, vl_verdict *out)
+// Verdicts of the candidates the walk vouches for.  For the others, one work item per chunk that
+// needs an exact recount, plus one for the general bank tally; racc[k][3] counts the items pending.
+// Item: (candidate, code); code = chunk | RC_ELIDED (only the definitions the walk skipped) or RC_BANK.
+#define RC_ELIDED 0x80000000u
+#define RC_BANK 0x7FFFFFFFu
+__global__ void k_finish(uint64_t K, uint32_t nC, uint32_t AW, int list_all, const uint32_t *__restrict__ cstate,
+                         const uint32_t *__restrict__ anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
+                         uint32_t *racc, vl_verdict *out)
 {
     const uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= K) return;
     const uint32_t *cs = cstate + k * 8;
-    if (cs[CS_WALK] | cs[CS_THCOL]) {
-        work[1 + atomicAdd(work, 1u)] = (uint32_t)k;
+    if (!list_all && !(cs[CS_WALK] | cs[CS_THCOL])) {
+        vl_verdict vd;
+        vd.flags = cs[CS_FLAGS] ? cs[CS_FLAGS] : (uint32_t)VL_PASS;
+        vd.first_violation_instr = cs[CS_FIRST] == 0xFFFFFFFFu ? -1 : (int32_t)cs[CS_FIRST];
+        vd.conflict_pairs = 0;
+        vd.bank_conflicts = cs[CS_BANK];
+        out[k] = vd;
         return;
     }
-    vl_verdict vd;
-    vd.flags = cs[CS_FLAGS] ? cs[CS_FLAGS] : (uint32_t)VL_PASS;
-    vd.first_violation_instr = cs[CS_FIRST] == 0xFFFFFFFFu ? -1 : (int32_t)cs[CS_FIRST];
-    vd.conflict_pairs = 0;
-    vd.bank_conflicts = cs[CS_BANK];
-    out[k] = vd;
-}
-
-// Programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction with
-// more than 4 distinct sources): every candidate goes through k_recount.
-__global__ void k_list_all(uint64_t K, uint32_t *work)
-{
-    const uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (k < K) work[1 + k] = (uint32_t)k;
-    if (k == 0) work[0] = (uint32_t)K;
+    // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
+    // a block whose through-set collided: the definitions the walk skipped (a vreg redefined from
+    // itself while it stays occupied), since everything else in it was walked exactly
+    const bool full = cs[CS_WALK] & WALK_FULL;
+    const uint32_t thcol = cs[CS_THCOL];
+    uint32_t n = 1;
+    for (uint32_t c = 0; c < nC; ++c) {
+        const bool all_defs = full || ((anom[k * AW + (c >> 5)] >> (c & 31)) & 1u);
+        const bool elided = !all_defs && thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u);
+        n += (all_defs || elided) ? 1u : 0u;
+    }
+    racc[k * 4 + 3] = n;
+    uint32_t at = atomicAdd(work, n);
+    work[2 + 2 * at] = (uint32_t)k;
+    work[3 + 2 * at] = RC_BANK;
+    ++at;
+    for (uint32_t c = 0; c < nC; ++c) {
+        const bool all_defs = full || ((anom[k * AW + (c >> 5)] >> (c & 31)) & 1u);
+        const bool elided = !all_defs && thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u);
+        if (all_defs || elided) {
+            work[2 + 2 * at] = (uint32_t)k;
+            work[3 + 2 * at] = c | (elided ? RC_ELIDED : 0u);
+            ++at;
+        }
+    }
 }
 
 // =========================================================================== k_recount
-// Exact answers for the listed candidates.  A candidate is cut into RC_SLICES slices of the chunk
-// range; one thread block handles one (candidate, slice): it copies the candidate's table column to
-// shared memory, recounts overlaps from the live-after lists in the chunks of its slice where the
-// walk could not vouch, adds its part to the candidate's accumulators, and the slice that finishes
-// last writes the verdict.  Slice 0 also does the general bank tally (distinct registers rather than
-// distinct vregs).
-// Shared memory: [T (V+1) x u16][chunks needing every definition, AW words][chunks needing only the
-// definitions the walk skipped, AW words].
+// Exact answers for the listed work items; thread blocks loop over the list.  For one item a block
+// copies the candidate's table column to shared memory, then either recounts the overlaps of one
+// chunk from the live-after lists (warps share the chunk's instructions) or does the general bank
+// tally (distinct registers rather than distinct vregs).  Results are added to the candidate's
+// accumulators; the item that finishes last writes the verdict.
 __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 {
     extern __shared__ __align__(16) uint16_t T[];
-    __shared__ uint32_t s_pairs, s_mind, s_bank, s_last;
-    uint32_t *s_all = reinterpret_cast<uint32_t *>(T + ((q.V + 1 + 7) & ~7u));
-    uint32_t *s_eli = s_all + q.AW;
+    __shared__ uint32_t s_pairs, s_mind, s_bank;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t nwork = q.work[0];
-    const uint32_t per = (q.nC + RC_SLICES - 1) / RC_SLICES;
-    for (uint32_t vi = blockIdx.x; vi < nwork * RC_SLICES; vi += gridDim.x) {
-        const uint64_t k = q.work[1 + vi / RC_SLICES];
-        const uint32_t slice = vi % RC_SLICES;
-        const uint32_t cbeg = min(q.nC, slice * per), cend = min(q.nC, cbeg + per);
+    const uint32_t nitems = q.work[0];
+    uint64_t have = ~0ull;  // candidate whose column is in shared memory
+    for (uint32_t it = blockIdx.x; it < nitems; it += gridDim.x) {
+        const uint64_t k = q.work[2 + 2 * it];
+        const uint32_t code = q.work[3 + 2 * it];
         const uint32_t *cs = q.cstate + k * 8;
-        const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
         __syncthreads();
-        for (uint32_t v = tid; v < q.V; v += RC_THREADS) T[v] = tg[(size_t)v * 32];
-        for (uint32_t i = tid; i < 2 * q.AW; i += RC_THREADS) s_all[i] = 0;
+        if (k != have) {
+            const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
+            for (uint32_t v = tid; v < q.V; v += RC_THREADS) T[v] = tg[(size_t)v * 32];
+            have = k;
+        }
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
         if (tid == 0 && cs[CS_NOUT] == 1) T[cs[CS_OUTV]] = (uint16_t)cs[CS_OUTRAW];  // the true value, not the parked one
-        const bool full = cs[CS_WALK] & WALK_FULL;
-        const uint32_t thcol = cs[CS_THCOL];
-        const uint32_t *anom = q.anom + k * q.AW;
-        // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
-        // a block whose through-set collided: the definitions the walk skipped (a vreg redefined
-        // from itself while it stays occupied), since everything else in it was walked exactly
-        for (uint32_t c = cbeg + tid; c < cend; c += RC_THREADS) {
-            const bool all_defs = full || ((anom[c >> 5] >> (c & 31)) & 1u);
-            const bool elided_only = !all_defs && ((thcol >> (q.chunk_blk[c] & 31)) & 1u);
-            if (all_defs) atomicOr(&s_all[c >> 5], 1u << (c & 31));
-            if (elided_only) atomicOr(&s_eli[c >> 5], 1u << (c & 31));
-        }
         __syncthreads();
-        for (uint32_t cw = cbeg >> 5; cw < (cend + 31) >> 5; ++cw) {
-            uint32_t bits = s_all[cw] | s_eli[cw];
-            while (bits) {
-                const uint32_t cb = __ffs(bits) - 1;
-                bits &= bits - 1;
-                const uint32_t c = cw * 32 + cb;
-                const bool elided_only = !((s_all[cw] >> cb) & 1u);
-                uint32_t pairs = 0, mind = 0xFFFFFFFFu;
-                for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += RC_THREADS / 32) {
-                    if (elided_only && !q.iflags[i]) continue;
-                    const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
-                    const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
-                    for (uint32_t d = o0; d < o0 + nd; ++d) {
-                        if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
-                        const uint32_t v = q.op_vreg[d];
-                        const uint32_t s = T[v], w = q.width[v];
-                        uint32_t cnt = 0;
-                        for (uint32_t e0 = l0; e0 < l1; e0 += 128) {  // 4 list entries per lane in flight
-                            uint32_t us[4], ws[4];
+        if (code != RC_BANK) {
+            const uint32_t c = code & ~RC_ELIDED;
+            const bool elided_only = code & RC_ELIDED;
+            uint32_t pairs = 0, mind = 0xFFFFFFFFu;
+            for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += RC_THREADS / 32) {
+                if (elided_only && !q.iflags[i]) continue;
+                const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
+                const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
+                for (uint32_t d = o0; d < o0 + nd; ++d) {
+                    if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
+                    const uint32_t v = q.op_vreg[d];
+                    const uint32_t s = T[v], w = q.width[v];
+                    uint32_t cnt = 0;
+                    for (uint32_t e0 = l0; e0 < l1; e0 += 256) {  // 8 list entries per lane in flight
+                        uint32_t us[8], ws[8];
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const uint32_t e = e0 + u * 32 + lane;
-                                us[u] = e < l1 ? q.lo[e] : v;
-                            }
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
-#pragma unroll
-                            for (int u = 0; u < 4; ++u)
-                                if (us[u] != v && ranges_overlap(s, w, T[us[u]], ws[u])) ++cnt;
-                        }
-                        // co-defined vregs that are not live after the instruction
-                        for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
-                            if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
-                            const uint32_t u = q.op_vreg[d2];
-                            if (ranges_overlap(s, w, T[u], q.width[u])) ++cnt;
+                        for (int u = 0; u < 8; ++u) {
+                            const uint32_t e = e0 + u * 32 + lane;
+                            us[u] = e < l1 ? q.lo[e] : v;
                         }
 #pragma unroll
-                        for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
-                        if (cnt) { pairs += cnt; mind = min(mind, i); }
+                        for (int u = 0; u < 8; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (us[u] != v && ranges_overlap(s, w, T[us[u]], ws[u])) ++cnt;
                     }
-                }
-                if (lane == 0 && pairs) {
-                    atomicAdd(&s_pairs, pairs);
-                    atomicMin(&s_mind, mind);
+                    // co-defined vregs that are not live after the instruction
+                    for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
+                        if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
+                        const uint32_t u = q.op_vreg[d2];
+                        if (ranges_overlap(s, w, T[u], q.width[u])) ++cnt;
+                    }
+#pragma unroll
+                    for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
+                    if (cnt) { pairs += cnt; mind = min(mind, i); }
                 }
             }
-        }
-        // general bank tally: a source counts when its register is new among the instruction's sources
-        // and its bank is not
-        if (slice == 0) {
+            if (lane == 0 && pairs) {
+                atomicAdd(&s_pairs, pairs);
+                atomicMin(&s_mind, mind);
+            }
+        } else {
+            // a source counts when its register is new among the instruction's sources and its bank is not
             uint32_t bt = 0;
             if (q.bank_fast) {
                 for (uint32_t e = tid; e < q.bank_seg[3]; e += RC_THREADS) {
@@ -746,8 +743,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             if (s_mind != 0xFFFFFFFFu) atomicMax(&acc[1], ~s_mind);  // accumulators start at 0: keep the complement
             if (s_bank) atomicAdd(&acc[2], s_bank);
             __threadfence();
-            s_last = atomicAdd(&acc[3], 1u) == RC_SLICES - 1;
-            if (s_last) {
+            if (atomicSub(&acc[3], 1u) == 1u) {  // last item of this candidate
                 __threadfence();
                 const uint32_t pairs = atomicAdd(&acc[0], 0u), mind = ~atomicMax(&acc[1], 0u),
                                bank = atomicAdd(&acc[2], 0u);
@@ -813,7 +809,7 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.work, (1 + groups * 32) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * 32 * (uint64_t)(p->nC + 1)) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
     v.rows = groups * 32;
     v.aw = aw;
@@ -841,10 +837,12 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
     const uint32_t Wp = (p->P + p->wmax + 31) / 32;
     const uint32_t ev_cap = 256;
     const uint32_t walk_smem = (Wp * 32 + WALK_WARPS * (Wp * 32 + ev_cap * 4)) * 4;
-    const uint32_t rc_smem = (uint32_t)align16((uint64_t)((p->V + 1 + 7) & ~7u) * 2 + 2ull * std::max(1u, (p->nC + 31) / 32) * 4);
+    const uint32_t rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
     if (walk_smem > SM_BYTES || rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
 
-    const uint64_t sub = std::min<uint64_t>(K, p->sub_batch);
+    // the recount work list holds up to (chunks + 1) items per candidate: keep it within 4 Mi items
+    const uint64_t sub_cap = std::max<uint64_t>(32, ((4ull << 20) / (p->nC + 1)) / 32 * 32);
+    const uint64_t sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
     int rc = ensure_scratch(p, slot, sub);
     if (rc != VL_OK) return rc;
     vl_program::VScratch &vs = p->vs[slot];
@@ -903,8 +901,10 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
             g_vl_launches.fetch_add(1);
         }
 
-        if (p->bank_fast) k_finish<<<(uint32_t)((n + 255) / 256), 256, 0, st>>>(n, vs.cstate, vs.work, d_out + kb);
-        else k_list_all<<<(uint32_t)((n + 255) / 256), 256, 0, st>>>(n, vs.work);
+        // programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction
+        // with more than 4 distinct sources) send every candidate through k_recount
+        k_finish<<<(uint32_t)((n + 127) / 128), 128, 0, st>>>(n, p->nC, (uint32_t)vs.aw, p->bank_fast ? 0 : 1, vs.cstate,
+                                                             vs.anom, p->d_chunk_blk, vs.work, vs.racc, d_out + kb);
         RParams rq{};
         rq.nI = p->nI; rq.V = p->V; rq.B = p->B; rq.nB = p->nB; rq.nC = p->nC; rq.AW = (uint32_t)vs.aw;
         rq.bank_fast = p->bank_fast; rq.K = n;
@@ -915,7 +915,7 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out + kb;
         rq.bank_list = p->d_bank_list;
         for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
-        const uint32_t rgrid = (uint32_t)std::min<uint64_t>(n, 148 * 4);
+        const uint32_t rgrid = 148 * 6;
         k_recount<<<rgrid, RC_THREADS, rc_smem, st>>>(rq);
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
