@@ -305,36 +305,48 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     __syncthreads();
 
     PT(0);
-    // ------------------------------------------------- realizability, one sweep over the vregs
-    for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NT) {
-        uint32_t vis[4], fds[4];
+    // ---- one sweep over the vregs: the table goes to global memory (32 candidates side by side per
+    // vreg; the spare entry V, looked up by no-op events, as 0) and [T, T+width) is checked against the
+    // register file (Realizability)
+    {
+        const uint64_t grp = k0 >> 5;
+        const uint32_t l0 = (uint32_t)(k0 & 31);
+        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        for (uint32_t v0 = tid; v0 <= q.V; v0 += 8 * NT) {
+            uint32_t vis[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t v = v0 + u * NT;
-            vis[u] = v < q.V ? q.vinfo[v] : 0u;
-            fds[u] = v < q.V ? q.first_def_instr[v] : 0xFFFFFFFFu;
-        }
+            for (int u = 0; u < 8; ++u) vis[u] = v0 + u * NT < q.V ? q.vinfo[v0 + u * NT] : 0u;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t v = v0 + u * NT, vi = vis[u];
-            if (!(vi & VINFO_OCCURS)) continue;
-            const uint32_t w = vi & 0xFFu;
-            const uint64_t tt = t_load<G>(Tt, v);
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t v = v0 + u * NT, vi = vis[u];
+                if (v > q.V) break;
+                const uint64_t tt = v < q.V ? t_load<G>(Tt, v) : 0ull;
+                if constexpr (G == 4) {
+                    *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2((uint32_t)tt, (uint32_t)(tt >> 32));
+                } else if constexpr (G == 2) {
+                    *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = (uint32_t)tt;
+                } else {
+                    dst[(size_t)v * 32] = (uint16_t)tt;
+                }
+                if (!(vi & VINFO_OCCURS)) continue;
+                const uint32_t w = vi & 0xFFu;
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const uint32_t tv = pk_get(tt, g);
-                if (tv + w > q.P) {
-                    if (vi & VINFO_DEFINED) {
-                        atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
-                        atomicMin(&M->minR[g], fds[u]);
+                for (int g = 0; g < G; ++g) {
+                    const uint32_t tv = pk_get(tt, g);
+                    if (tv + w > q.P) {
+                        if (vi & VINFO_DEFINED) {
+                            atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
+                            atomicMin(&M->minR[g], q.first_def_instr[v]);
+                        }
+                        if (atomicAdd(&M->nout[g], 1u) == 0) { M->out_v[g] = v; M->out_raw[g] = tv; }
                     }
-                    if (atomicAdd(&M->nout[g], 1u) == 0) { M->out_v[g] = v; M->out_raw[g] = tv; }
                 }
             }
         }
     }
-
     PT(1);
+
+    PT(2);
     // ------------------------------- bank tally from T: instructions with 2..4 distinct sources.
     // Distinct vregs read by one instruction are live together, so a candidate whose walk sees no
     // collision has them on distinct registers and only the banks need comparing; candidates with
@@ -391,32 +403,12 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     __syncthreads();
 
-    PT(2);
+    PT(3);
     // ------------------------------------------------- hand-over to the walk
     // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
     // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
-    if (tid < G) {
-        const uint32_t g = tid;
-        if (M->nout[g] == 1 && M->out_raw[g] >= q.P) Tt[(size_t)M->out_v[g] * G + g] = (uint16_t)q.P;
-        Tt[(size_t)q.V * G + g] = 0;  // the spare entry that no-op events look up
-    }
-    __syncthreads();
-    {   // tables to global memory, 32 candidates side by side per vreg
-        const uint64_t grp = k0 >> 5;
-        const uint32_t l0 = (uint32_t)(k0 & 31);
-        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
-        for (uint32_t v = tid; v <= q.V; v += NT) {
-            const uint64_t x = t_load<G>(Tt, v);
-            if constexpr (G == 4) {
-                *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2((uint32_t)x, (uint32_t)(x >> 32));
-            } else if constexpr (G == 2) {
-                *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = (uint32_t)x;
-            } else {
-                dst[(size_t)v * 32] = (uint16_t)x;
-            }
-        }
-    }
-    PT(3);
+    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P)
+        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)M->out_v[tid] * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)q.P;
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
