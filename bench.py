@@ -23,7 +23,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2506_17506_b200 import synth  # noqa: E402
+from paper_2506_17506_b200 import shard, synth  # noqa: E402
 
 METRIC = "candidate_verifications_per_sec"
 UNIT = "verifications/s"
@@ -109,7 +109,8 @@ def build_inputs(rank: int, rows: int, pinned: bool, fault_rate: float = -1.0):
         arr = np.empty((K, pitch), dtype=np.uint16)
     t0 = time.time()
     # rank r checks rows [r*K, (r+1)*K) of the same seeded candidate stream
-    synth.candidate_rows(prog, (rank + 1) * K, wl.fault_rate, wl.seeds[0], rank * K, (rank + 1) * K, out=arr, chunk=256)
+    lo, hi = shard.weak_rows(rank, K)
+    synth.candidate_rows(prog, hi, wl.fault_rate, wl.seeds[0], lo, hi, out=arr, chunk=256)
     log(f"[bench] rank {rank}: generated {K} rows x {pitch} operands in {time.time() - t0:.1f}s")
     return wl, prog, K, host, arr
 
@@ -157,6 +158,12 @@ def run_reference(args):
     }
     print(json.dumps(line), flush=True)
     return 0
+
+
+# DRAM bytes (read + write) per candidate of each kernel, from the profiler capture of a 4096-row launch
+# summarised under profiles/ (traffic grows in proportion to the rows of a launch); None = no capture of
+# the kernel as it stands.
+TRAFFIC_PER_CANDIDATE = {"k_tables": 891.17e6 / 4096, "k_walk": 86.78e6 / 4096}
 
 
 def main():
@@ -218,6 +225,7 @@ def main():
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    gp.set_option(vl.VL_OPT_KERNEL_TIMING, 1)   # events around each verify kernel, read after the timed region
     barrier()
     ev[0].record(stream)
     for s in range(args.steps):
@@ -232,14 +240,13 @@ def main():
     launches = vl.vl_kernel_launches() - launches0
     clocks = sampler.stop() if rank == 0 else None
     gp.vl_verify_status(stream)
+    kernel_ms, kernel_passes = gp.vl_kernel_times()
+    gp.set_option(vl.VL_OPT_KERNEL_TIMING, 0)
     total_ms = ev[0].elapsed_time(ev[1])
     verify_ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
     live_ms = float(np.mean([a.elapsed_time(b) for a, b in lev]))
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
-    value = world * K * args.steps / (total_ms * 1e-3)
+    rows_all, total_ms, _ = shard.job_totals(K * args.steps, total_ms, 0, torch.device("cuda", local))
+    value = shard.throughput(rows_all, total_ms)
 
     # ---- end to end through the host-buffer entry point
     e2e_steps = max(1, args.e2e_steps)
@@ -253,10 +260,8 @@ def main():
         gp.vl_verify_host(host, out_host, stream)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * K * e2e_steps / float(t.item())
+    rows_all, e2e_ms, _ = shard.job_totals(K * e2e_steps, e2e_s * 1e3, 0, torch.device("cuda", local))
+    e2e_value = shard.throughput(rows_all, e2e_ms)
 
     # sanity: device-resident and host-buffer results agree
     dev_v = vl.verdicts_to_numpy(out)
@@ -265,8 +270,20 @@ def main():
 
     if rank == 0:
         peak, peak_kind = measured_peak_gbs()
-        bytes_per_launch = 2.0 * prog.pitch * K + 16.0 * K
-        achieved = bytes_per_launch / (verify_ms * 1e-3) / 1e9
+        # algorithmic bytes: every candidate row is read once (2 bytes per operand column) and one 16-byte
+        # verdict is written; the table kernel is the one that streams the rows
+        bytes_per_step = 2.0 * prog.pitch * K + 16.0 * K
+        names = ["k_tables", "k_walk", "k_finish", "k_recount"]
+        passes = max(1, kernel_passes)
+        ksum = max(1e-9, sum(kernel_ms))
+        kernels = {n: {"ms_per_launch": kernel_ms[j] / passes, "share": kernel_ms[j] / ksum} for j, n in enumerate(names)}
+        dom = max(range(4), key=lambda j: kernel_ms[j])
+        dom_ms = kernel_ms[dom] / passes
+        bytes_per_launch = bytes_per_step * args.steps / passes
+        achieved = bytes_per_launch / (dom_ms * 1e-3) / 1e9
+        path_achieved = bytes_per_step / (verify_ms * 1e-3) / 1e9
+        per_cand = TRAFFIC_PER_CANDIDATE.get(names[dom])
+        traffic = per_cand * K * args.steps / passes if per_cand else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -278,8 +295,11 @@ def main():
             "operand_checks_per_sec": value * prog.n_operands,
             "verify_ms": verify_ms, "liveness_ms": live_ms,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "kernel": "k_verify", "of": peak_kind,
-                         "frac_of_8TBs_nominal": achieved / 8000.0},
+                         "traffic": traffic, "kernel": names[dom], "of": peak_kind,
+                         "launches": passes, "ms_per_launch": dom_ms, "bytes_per_launch": bytes_per_launch,
+                         "path": {"what": "all kernels of one vl_verify call", "achieved": path_achieved,
+                                  "frac": path_achieved / peak, "ms": verify_ms},
+                         "kernels": kernels},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(2 * prog.pitch * K),
                     "d2h_bytes_per_step": int(16 * K)},

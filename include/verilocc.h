@@ -46,7 +46,9 @@ enum {
     VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 128) */
     VL_OPT_GROUP = 2,        /* candidates per thread block: 0 = choose, else 1, 2 or 4 */
     VL_OPT_THREADS = 3,      /* threads per thread block of the table kernel: 0 = choose, else 256 or 512 */
-    VL_OPT_SUB_BATCH = 4     /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
+    VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
+    VL_OPT_KERNEL_TIMING = 5 /* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
+                                set at any time; setting it discards the events recorded so far */
 };
 
 /*
@@ -191,6 +193,15 @@ int vl_verify_status(vl_program *prog, void *cuda_stream);
 
 /* Number of kernels this library has launched in this process (all handles). */
 uint64_t vl_kernel_launches(void);
+
+/*
+ * Device time of the verify kernels since the last call (or since VL_OPT_KERNEL_TIMING was set), summed over
+ * the passes recorded (at most 4096): ms[0] table kernel (first occurrences, Consistency, Realizability, bank
+ * tally), ms[1] occupancy walk (Safety), ms[2] verdict kernel, ms[3] exact recount.  ms is HOST memory for
+ * 4 floats; *passes (HOST, may be NULL) receives the number of passes summed.  Waits for the last recorded
+ * event, then forgets the events.  Without the option everything is 0.  Errors: INVALID_ARG, CUDA.
+ */
+int vl_kernel_times(vl_program *prog, float ms[4], uint32_t *passes);
 
 /* Last CUDA error code seen by the handle (0 if none). */
 int vl_last_cuda_error(const vl_program *prog);

@@ -24,11 +24,11 @@ VL_OK = 0
 VL_ERR_INVALID_ARG, VL_ERR_MALFORMED_PROGRAM, VL_ERR_NOT_STRICT, VL_ERR_LIVENESS_NOT_RUN = -1, -2, -3, -4
 VL_ERR_UNSUPPORTED, VL_ERR_NO_CONVERGE, VL_ERR_CUDA, VL_ERR_DEVICE_WAIT = -5, -6, -7, -8
 VL_PASS, VL_INCONSISTENT, VL_OUT_OF_RANGE, VL_INTERFERENCE = 1, 2, 4, 8
-VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH = 1, 2, 3, 4
+VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERNEL_TIMING = 1, 2, 3, 4, 5
 
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
-           "vl_kernel_launches", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static"]
+           "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -47,6 +47,8 @@ _lib.vl_program_destroy.restype = None
 _lib.vl_program_destroy.argtypes = [C.c_void_p]
 _lib.vl_program_set_option.restype = C.c_int
 _lib.vl_program_set_option.argtypes = [C.c_void_p, C.c_int, C.c_uint32]
+_lib.vl_kernel_times.restype = C.c_int
+_lib.vl_kernel_times.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_uint32)]
 _lib.vl_liveness.restype = C.c_int
 _lib.vl_liveness.argtypes = [C.c_void_p, C.c_void_p]
 _lib.vl_liveness_result.restype = C.c_int
@@ -202,6 +204,13 @@ class Program:
 
     def vl_verify_status(self, stream=None):
         self._check(_lib.vl_verify_status(self._h, _stream_ptr(stream)), "vl_verify_status")
+
+    def vl_kernel_times(self):
+        """Summed device time (ms) of the four verify kernels since the last call, and the passes summed."""
+        ms = (C.c_float * 4)()
+        n = C.c_uint32(0)
+        self._check(_lib.vl_kernel_times(self._h, ms, C.byref(n)), "vl_kernel_times")
+        return [float(x) for x in ms], int(n.value)
 
     @property
     def handle(self):

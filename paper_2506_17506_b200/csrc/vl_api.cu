@@ -150,6 +150,7 @@ extern "C" void vl_program_destroy(vl_program *p)
         if (p->h_streams[j]) cudaStreamDestroy(p->h_streams[j]);
         if (p->h_events[j]) cudaEventDestroy(p->h_events[j]);
     }
+    for (cudaEvent_t ev : p->kt_ev) cudaEventDestroy(ev);
     delete p;
 }
 
@@ -169,6 +170,11 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     case VL_OPT_SUB_BATCH:
         if (value < 32 || value % 32) return VL_ERR_INVALID_ARG;
         p->sub_batch = value;
+        return VL_OK;
+    case VL_OPT_KERNEL_TIMING:
+        if (value > 1) return VL_ERR_INVALID_ARG;
+        p->ktime = (int)value;
+        p->kt_used = 0;
         return VL_OK;
     case VL_OPT_THREADS:
         if (value != 0 && value != 256 && value != 512) return VL_ERR_INVALID_ARG;
@@ -309,6 +315,26 @@ extern "C" int vl_debug_read_status(vl_program *p, uint32_t *out16)
 #endif
 
 extern "C" uint64_t vl_kernel_launches(void) { return g_vl_launches.load(); }
+
+extern "C" int vl_kernel_times(vl_program *p, float ms[4], uint32_t *passes)
+{
+    if (!p || !ms) return VL_ERR_INVALID_ARG;
+    for (int j = 0; j < 4; ++j) ms[j] = 0.f;
+    const size_t n = p->kt_used / 5;
+    if (passes) *passes = (uint32_t)n;
+    if (n) {
+        cudaSetDevice(p->device);
+        VL_CUDA(p, cudaEventSynchronize(p->kt_ev[n * 5 - 1]));
+        for (size_t i = 0; i < n; ++i)
+            for (int j = 0; j < 4; ++j) {
+                float t = 0.f;
+                VL_CUDA(p, cudaEventElapsedTime(&t, p->kt_ev[i * 5 + j], p->kt_ev[i * 5 + j + 1]));
+                ms[j] += t;
+            }
+    }
+    p->kt_used = 0;
+    return VL_OK;
+}
 
 extern "C" int vl_last_cuda_error(const vl_program *p) { return p ? p->last_cuda_error : 0; }
 

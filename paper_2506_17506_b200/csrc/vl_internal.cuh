@@ -127,6 +127,11 @@ struct vl_program {
     } vs[3];
     uint32_t sub_batch = 4096;       // candidates per pass of the three verify kernels
 
+    // opt-in per-kernel timing of vl_verify: five events per pass (before each of the four kernels, after the last)
+    int ktime = 0;
+    std::vector<cudaEvent_t> kt_ev;
+    size_t kt_used = 0;
+
     // staging for vl_verify_host
     uint16_t *d_stage[2] = {nullptr, nullptr};
     vl_verdict *d_stage_out[2] = {nullptr, nullptr};

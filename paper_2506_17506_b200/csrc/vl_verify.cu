@@ -810,6 +810,18 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
 }
 }  // namespace
 
+// Records the next timing event of the handle on `st` (no-op unless kernel timing is switched on).
+static void kt_mark(vl_program *p, cudaStream_t st)
+{
+    if (!p->ktime || p->kt_used >= 5 * 4096) return;
+    if (p->kt_used == p->kt_ev.size()) {
+        cudaEvent_t ev;
+        if (cudaEventCreate(&ev) != cudaSuccess) { p->ktime = 0; return; }
+        p->kt_ev.push_back(ev);
+    }
+    cudaEventRecord(p->kt_ev[p->kt_used++], st);
+}
+
 int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
                    cudaStream_t st, int slot)
 {
@@ -866,6 +878,7 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
         tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
         const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
+        kt_mark(p, st);
         if (pl.NT == 256) {
             if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
             else if (pl.G == 2) e = launch_tables<2, 256>(tq, tgrid, pl.smem, st);
@@ -878,6 +891,7 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
         g_vl_launches.fetch_add(1);
 
+        kt_mark(p, st);
         if (p->nItems) {
             WParams wq{};
             wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = Wp; wq.AW = (uint32_t)vs.aw;
@@ -895,6 +909,7 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
 
         // programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction
         // with more than 4 distinct sources) send every candidate through k_recount
+        kt_mark(p, st);
         k_finish<<<(uint32_t)((n + 127) / 128), 128, 0, st>>>(n, p->nC, (uint32_t)vs.aw, p->bank_fast ? 0 : 1, vs.cstate,
                                                              vs.anom, p->d_chunk_blk, vs.work, vs.racc, d_out + kb);
         RParams rq{};
@@ -908,7 +923,9 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
         rq.bank_list = p->d_bank_list;
         for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
         const uint32_t rgrid = 148 * 6;
+        kt_mark(p, st);
         k_recount<<<rgrid, RC_THREADS, rc_smem, st>>>(rq);
+        kt_mark(p, st);
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
         g_vl_launches.fetch_add(2);

@@ -1,0 +1,78 @@
+"""The several-GPU path on CPU: two `gloo` ranks split the rows, each checks its shard (the oracle stands
+in for the GPU here, this test is about the sharding and the reductions), and the union must equal
+the single-process result with the job totals reduced correctly."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch.multiprocessing as mp
+
+from paper_2506_17506_b200 import shard, synth
+
+
+def test_row_range_partitions():
+    for n_rows in (0, 1, 31, 32, 33, 1000, 4096, 10000):
+        for world in (1, 2, 3, 8):
+            prev = 0
+            sizes = []
+            for r in range(world):
+                lo, hi = shard.row_range(r, world, n_rows)
+                assert lo == prev and hi >= lo
+                if hi < n_rows:
+                    assert hi % 32 == 0
+                sizes.append(hi - lo)
+                prev = hi
+            assert prev == n_rows
+            assert max(sizes) - min(sizes) < 64
+    with pytest.raises(ValueError):
+        shard.row_range(2, 2, 10)
+    assert shard.weak_rows(3, 100) == (300, 400)
+
+
+def test_job_totals_single_process():
+    assert shard.job_totals(7, 2.5, 3) == (7, 2.5, 3)
+    assert shard.throughput(1000, 500.0) == 2000.0
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank, world, port, n_rows, tmpdir):
+    import torch.distributed as dist
+    import oracle
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        wl = synth.workload(0)
+        prog = synth.build_program(wl.shapes[0], wl.seeds[0])
+        lo, hi = shard.row_range(rank, world, n_rows)
+        rows, _ = synth.candidate_rows(prog, n_rows, 0.3, wl.seeds[0], lo, hi)
+        op = oracle.OracleProgram(prog)
+        v = op.verify(op.liveness(), rows)
+        np.save(os.path.join(tmpdir, f"v{rank}.npy"), v)
+        passing = int((v["flags"] == 1).sum())
+        total, ms, npass = shard.job_totals(hi - lo, 10.0 * (rank + 1), passing)
+        if rank == 0:
+            np.save(os.path.join(tmpdir, "totals.npy"), np.array([total, ms, npass], dtype=np.float64))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_cover_the_job(tmp_path, oracle_mod):
+    n_rows, world = 100, 2
+    mp.spawn(_rank_main, args=(world, _free_port(), n_rows, str(tmp_path)), nprocs=world, join=True)
+    wl = synth.workload(0)
+    prog = synth.build_program(wl.shapes[0], wl.seeds[0])
+    rows, _ = synth.candidate_rows(prog, n_rows, 0.3, wl.seeds[0], 0, n_rows)
+    op = oracle_mod.OracleProgram(prog)
+    want = op.verify(op.liveness(), rows)
+    got = np.concatenate([np.load(tmp_path / f"v{r}.npy") for r in range(world)])
+    assert np.array_equal(got.view(np.int32), want.view(np.int32))
+    total, ms, npass = np.load(tmp_path / "totals.npy")
+    assert total == n_rows and ms == 20.0 and npass == int((want["flags"] == 1).sum())
+    assert 0 < npass < n_rows
