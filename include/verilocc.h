@@ -46,9 +46,11 @@ enum {
     VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 128) */
     VL_OPT_GROUP = 2,        /* candidates per thread block: 0 = choose, else 1, 2 or 4 */
     VL_OPT_THREADS = 3,      /* threads per thread block of the table kernel: 0 = choose, else 256 or 512 */
-    VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
-    VL_OPT_KERNEL_TIMING = 5 /* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
+    VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 2048) */
+    VL_OPT_KERNEL_TIMING = 5,/* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
                                 set at any time; setting it discards the events recorded so far */
+    VL_OPT_LANES = 6         /* internal streams the passes of vl_verify / vl_verify_batch are spread over, 1..4
+                                (default 3); 1 = every kernel in order on the caller's stream */
 };
 
 /*
@@ -123,8 +125,12 @@ int vl_liveness_result(const vl_program *prog, const uint32_t **blk_live_in, con
  * d_cand[k * pitch_elems + o] is the physical register candidate k gives operand o.
  * Requirements: base 16-byte aligned, pitch_elems >= n_operands rounded up to 8,
  * pitch_elems % 8 == 0.  d_out is DEVICE memory for K records (4-byte aligned).
- * Buffers are borrowed for the call; the work is enqueued on `cuda_stream` and the
- * function returns without synchronising.  K == 0 is a no-op.
+ * Buffers are borrowed for the call; the work is ordered after what `cuda_stream` holds at
+ * the call, what is enqueued on `cuda_stream` later is ordered after the work, and the function
+ * returns without synchronising.  K == 0 is a no-op.  A call with more than one pass
+ * (VL_OPT_SUB_BATCH) spreads its passes over internal streams of the device (VL_OPT_LANES) that
+ * fork from and join back into `cuda_stream`, so that kernels of different passes run side by
+ * side; with VL_OPT_LANES = 1 every kernel is enqueued on `cuda_stream` itself.
  *
  * Per candidate (Section 3.4): T[v] = register at the first occurrence of v;
  * Consistency: every occurrence equals T[v]; Realizability: at every definition
@@ -198,8 +204,9 @@ uint64_t vl_kernel_launches(void);
  * Device time of the verify kernels since the last call (or since VL_OPT_KERNEL_TIMING was set), summed over
  * the passes recorded (at most 4096): ms[0] table kernel (first occurrences, Consistency, Realizability, bank
  * tally), ms[1] occupancy walk (Safety), ms[2] verdict kernel, ms[3] exact recount.  ms is HOST memory for
- * 4 floats; *passes (HOST, may be NULL) receives the number of passes summed.  Waits for the last recorded
- * event, then forgets the events.  Without the option everything is 0.  Errors: INVALID_ARG, CUDA.
+ * 4 floats; *passes (HOST, may be NULL) receives the number of passes summed.  Kernels of different passes
+ * may run side by side (VL_OPT_LANES), so the four sums can add up to more than the duration of the calls.
+ * Waits for the last recorded event, then forgets the events.  Without the option everything is 0.  Errors: INVALID_ARG, CUDA.
  */
 int vl_kernel_times(vl_program *prog, float ms[4], uint32_t *passes);
 

@@ -1,11 +1,36 @@
 // C ABI entry points: program handle, validation, host-buffer verify, error strings.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "vl_internal.cuh"
 
 std::atomic<uint64_t> g_vl_launches{0};
+
+// Lane streams are per device and shared by every handle on it; they live until the process exits.
+#define VL_MAX_DEVICES 64
+static std::mutex g_lane_mutex;
+static cudaStream_t g_lanes[VL_MAX_DEVICES][VL_LANES];
+static bool g_lanes_made[VL_MAX_DEVICES];
+
+int vl_lane_streams(vl_program *p, cudaStream_t **lanes)
+{
+    if (p->device < 0 || p->device >= VL_MAX_DEVICES) return VL_ERR_UNSUPPORTED;
+    {
+        std::lock_guard<std::mutex> lock(g_lane_mutex);
+        if (!g_lanes_made[p->device]) {
+            for (int l = 0; l < VL_LANES; ++l)
+                VL_CUDA(p, cudaStreamCreateWithFlags(&g_lanes[p->device][l], cudaStreamNonBlocking));
+            g_lanes_made[p->device] = true;
+        }
+    }
+    if (!p->ev_fork) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+    for (int l = 0; l < VL_LANES; ++l)
+        if (!p->ev_join[l]) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_join[l], cudaEventDisableTiming));
+    *lanes = g_lanes[p->device];
+    return VL_OK;
+}
 
 static int validate(const vl_program_desc *d)
 {
@@ -143,7 +168,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
-    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); }
+    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); }
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
         cudaFree(p->d_stage_out[j]);
@@ -151,6 +176,9 @@ extern "C" void vl_program_destroy(vl_program *p)
         if (p->h_events[j]) cudaEventDestroy(p->h_events[j]);
     }
     for (cudaEvent_t ev : p->kt_ev) cudaEventDestroy(ev);
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    for (cudaEvent_t ev : p->ev_join)
+        if (ev) cudaEventDestroy(ev);
     delete p;
 }
 
@@ -175,6 +203,10 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
         if (value > 1) return VL_ERR_INVALID_ARG;
         p->ktime = (int)value;
         p->kt_used = 0;
+        return VL_OK;
+    case VL_OPT_LANES:
+        if (value < 1 || value > VL_LANES) return VL_ERR_INVALID_ARG;
+        p->lanes_opt = value;
         return VL_OK;
     case VL_OPT_THREADS:
         if (value != 0 && value != 256 && value != 512) return VL_ERR_INVALID_ARG;
@@ -224,7 +256,7 @@ extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K
     if (rc != VL_OK || K == 0) return rc;
     cudaError_t e = cudaSetDevice(p->device);
     if (e != cudaSuccess) return VL_ERR_CUDA;
-    return vl_verify_impl(p, d_cand, K, pitch, d_out, (cudaStream_t)stream, 2);
+    return vl_verify_lanes(1, &p, &d_cand, &K, &pitch, &d_out, (cudaStream_t)stream);
 }
 
 extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
@@ -238,12 +270,11 @@ extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const
         if (progs[j]->device != progs[0]->device) return VL_ERR_INVALID_ARG;
     }
     if (cudaSetDevice(progs[0]->device) != cudaSuccess) return VL_ERR_CUDA;
-    for (uint32_t j = 0; j < n; ++j) {
-        if (K[j] == 0) continue;
-        int rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], (cudaStream_t)stream, 2);
-        if (rc != VL_OK) return rc;
-    }
-    return VL_OK;
+    uint32_t first = 0;  // the first program with rows lends its fork / join events
+    while (first < n && K[first] == 0) ++first;
+    if (first == n) return VL_OK;
+    return vl_verify_lanes(n - first, progs + first, d_cand + first, K + first, pitch + first, d_out + first,
+                           (cudaStream_t)stream);
 }
 
 extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K, uint64_t pitch, vl_verdict *h_out,
@@ -281,7 +312,7 @@ extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K,
         uint64_t n = std::min(rows, K - k0);
         VL_CUDA(p, cudaMemcpyAsync(p->d_stage[j], h_cand + k0 * pitch, n * pitch * 2, cudaMemcpyHostToDevice,
                                    p->h_streams[j]));
-        rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j], j);
+        rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j], VL_LANES + j);
         if (rc != VL_OK) return rc;
         VL_CUDA(p, cudaMemcpyAsync(h_out + k0, p->d_stage_out[j], n * sizeof(vl_verdict), cudaMemcpyDeviceToHost,
                                    p->h_streams[j]));

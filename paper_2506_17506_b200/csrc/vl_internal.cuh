@@ -32,6 +32,7 @@ enum : uint32_t {
 };
 
 #define VL_MAX_GROUP 4
+#define VL_LANES 4  // internal streams that the passes of a device-resident verify call are spread over
 
 // Device memory pool of a program handle: slabs are kept across calls, so that a repeated
 // vl_liveness on the same handle allocates nothing.
@@ -123,9 +124,12 @@ struct vl_program {
         uint32_t *anom = nullptr;    // [rows][AW] chunks whose walk collided
         uint32_t *work = nullptr;    // [1 + rows] count, then candidates that need the exact recount
         uint32_t *racc = nullptr;    // [rows][4] recount accumulators: pairs, lowest instruction, bank tally, slices done
+        uint32_t *grp_done = nullptr;  // [rows / 32] walk thread blocks that have finished, per group of 32 candidates
         uint64_t rows = 0, aw = 0, vregs = 0;
-    } vs[3];
-    uint32_t sub_batch = 4096;       // candidates per pass of the three verify kernels
+    } vs[VL_LANES + 2];              // one per lane, then one per staging buffer of vl_verify_host
+    uint32_t sub_batch = 2048;       // candidates per pass of the verify kernels
+    uint32_t lanes_opt = 3;          // lanes in use (1 = everything in order on the caller's stream)
+    cudaEvent_t ev_fork = nullptr, ev_join[VL_LANES] = {nullptr, nullptr, nullptr, nullptr};
 
     // opt-in per-kernel timing of vl_verify: five events per pass (before each of the four kernels, after the last)
     int ktime = 0;
@@ -154,4 +158,8 @@ extern std::atomic<uint64_t> g_vl_launches;
 int vl_liveness_impl(vl_program *p, cudaStream_t st);
 int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
                    cudaStream_t st, int slot);
+int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
+                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st);
+// The lane streams of the handle's device (created once per device) and the handle's fork / join events.
+int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);

@@ -11,8 +11,10 @@
 //            event stream is the same for all 32 lanes, the occupancy bitmask of each lane sits in
 //            shared memory at [word][lane] (Safety).  A chunk whose walk sees no collision provably
 //            has no overlap.
-// k_finish / k_recount   verdicts for clean candidates; candidates with a collision are recounted
-//            exactly from the per-instruction live-after lists, one thread block per candidate.
+//            The thread block that ends a group of 32 candidates writes the verdicts of its clean
+//            candidates and lists the others for the recount.
+// k_recount  candidates with a collision are recounted exactly from the per-instruction live-after
+//            lists, one thread block per piece of a colliding chunk.
 #include <algorithm>
 
 #include "vl_internal.cuh"
@@ -39,6 +41,9 @@ struct TParams {
     uint32_t *cstate;
     uint32_t *status;
     uint32_t NS, off_region, off_misc;
+    // per-pass state this kernel clears for the kernels after it
+    uint32_t AW;
+    uint32_t *anom, *racc, *grp_done, *work;
 };
 
 struct TMisc {
@@ -56,6 +61,11 @@ struct WParams {
     const uint16_t *tg, *tg_zero;
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
+    // hand-over to k_recount by the last thread block of each group of 32 candidates
+    int list_all;
+    const uint32_t *chunk_blk;
+    uint32_t *grp_done, *work, *racc;
+    vl_verdict *out;
 };
 
 struct RParams {
@@ -71,6 +81,7 @@ struct RParams {
     uint32_t bank_seg[4];
     uint32_t *work;
     vl_verdict *out;
+    uint32_t *status;
 };
 
 // Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
@@ -179,6 +190,11 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         for (uint32_t s = 0; s < q.NS; ++s) mbar_init(&M->bar[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // state of this pass that the walk and the recount update with atomics starts at zero
+    for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
+    if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
+    if (tid == 0 && (k0 & 31) == 0) q.grp_done[k0 >> 5] = 0;
+    if (tid == 0 && blockIdx.x == 0) q.work[0] = 0;
     __syncthreads();
 
     auto issue_tile = [&](uint32_t t) {
@@ -472,6 +488,10 @@ __device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, 
     return viol;
 }
 
+__device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_all, const uint32_t *cstate,
+                                 const uint32_t *anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
+                                 uint32_t *racc, vl_verdict *out);
+
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
@@ -569,119 +589,208 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
             atomicOr(&cs[CS_WALK], WALK_ANOM);
         }
     }
+    // the thread block that finishes a group's last item writes the verdicts of the group's clean
+    // candidates and lists the others for the recount
+    __shared__ uint32_t s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&q.grp_done[grp], 1u) == gridDim.x - 1 ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (uint32_t j = warp; j < 32; j += WALK_WARPS) {
+        const uint64_t kk = (uint64_t)grp * 32 + j;
+        if (kk < q.K) finish_candidate(kk, q.nC, q.AW, q.list_all, q.cstate, q.anom, q.chunk_blk, q.work, q.racc, q.out);
+    }
 }
 
-// =========================================================================== k_finish
-// Verdicts of the candidates the walk vouches for.  For the others, one work item per chunk that
-// needs an exact recount, plus one for the general bank tally; racc[k][3] counts the items pending.
-// Item: (candidate, code); code = chunk | RC_ELIDED (only the definitions the walk skipped) or RC_BANK.
-#define RC_ELIDED 0x80000000u
-#define RC_BANK 0x7FFFFFFFu
-__global__ void k_finish(uint64_t K, uint32_t nC, uint32_t AW, int list_all, const uint32_t *__restrict__ cstate,
-                         const uint32_t *__restrict__ anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
-                         uint32_t *racc, vl_verdict *out)
+// =========================================================================== verdicts / work list
+// Verdicts of the candidates the walk vouches for.  For the others, work items for k_recount:
+// every chunk that needs an exact recount is cut into RC_PARTS pieces, the general bank tally into
+// RC_BANK_PARTS slices; racc[k][3] counts the items pending.  An item is (candidate, code) with
+// code = kind << 30 | piece << 24 | chunk.
+#define RC_PARTS 4
+#define RC_BANK_PARTS 2
+#define RC_KIND_ALL 0u     // every definition of the piece
+#define RC_KIND_ELIDED 1u  // only the definitions the walk skipped
+#define RC_KIND_BANK 2u
+__device__ __forceinline__ uint32_t rc_code(uint32_t kind, uint32_t piece, uint32_t chunk)
 {
-    const uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= K) return;
+    return (kind << 30) | (piece << 24) | chunk;
+}
+
+// One warp finishes candidate k: the verdict if nothing is left to recount, else its work items.
+// cstate / anom words that other thread blocks updated with atomics are read from L2.
+__device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_all, const uint32_t *cstate,
+                                 const uint32_t *anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
+                                 uint32_t *racc, vl_verdict *out)
+{
+    const uint32_t lane = threadIdx.x & 31;
     const uint32_t *cs = cstate + k * 8;
-    if (!list_all && !(cs[CS_WALK] | cs[CS_THCOL])) {
-        vl_verdict vd;
-        vd.flags = cs[CS_FLAGS] ? cs[CS_FLAGS] : (uint32_t)VL_PASS;
-        vd.first_violation_instr = cs[CS_FIRST] == 0xFFFFFFFFu ? -1 : (int32_t)cs[CS_FIRST];
-        vd.conflict_pairs = 0;
-        vd.bank_conflicts = cs[CS_BANK];
-        out[k] = vd;
+    const uint32_t walk = __ldcg(cs + CS_WALK), thcol = __ldcg(cs + CS_THCOL);
+    if (!list_all && !(walk | thcol)) {
+        if (lane == 0) {
+            const uint32_t fl = __ldcg(cs + CS_FLAGS), first = __ldcg(cs + CS_FIRST);
+            vl_verdict vd;
+            vd.flags = fl ? fl : (uint32_t)VL_PASS;
+            vd.first_violation_instr = first == 0xFFFFFFFFu ? -1 : (int32_t)first;
+            vd.conflict_pairs = 0;
+            vd.bank_conflicts = __ldcg(cs + CS_BANK);
+            out[k] = vd;
+        }
         return;
     }
     // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
     // a block whose through-set collided: the definitions the walk skipped (a vreg redefined from
     // itself while it stays occupied), since everything else in it was walked exactly
-    const bool full = cs[CS_WALK] & WALK_FULL;
-    const uint32_t thcol = cs[CS_THCOL];
-    uint32_t n = 1;
-    for (uint32_t c = 0; c < nC; ++c) {
-        const bool all_defs = full || ((anom[k * AW + (c >> 5)] >> (c & 31)) & 1u);
-        const bool elided = !all_defs && thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u);
-        n += (all_defs || elided) ? 1u : 0u;
+    const bool full = walk & WALK_FULL;
+    auto kind_of = [&](uint32_t c) -> uint32_t {  // 0 none, 1 all definitions, 2 skipped definitions only
+        if (c >= nC) return 0u;
+        const bool all_defs = full || ((__ldcg(anom + k * AW + (c >> 5)) >> (c & 31)) & 1u);
+        if (all_defs) return 1u;
+        return (thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u)) ? 2u : 0u;
+    };
+    uint32_t n_chunks = 0;
+    for (uint32_t c0 = 0; c0 < nC; c0 += 32) n_chunks += __popc(__ballot_sync(0xffffffffu, kind_of(c0 + lane) != 0));
+    const uint32_t n = RC_BANK_PARTS + RC_PARTS * n_chunks;
+    uint32_t at = 0;
+    if (lane == 0) {
+        racc[k * 4 + 3] = n;
+        at = atomicAdd(work, n);
     }
-    racc[k * 4 + 3] = n;
-    uint32_t at = atomicAdd(work, n);
-    work[2 + 2 * at] = (uint32_t)k;
-    work[3 + 2 * at] = RC_BANK;
-    ++at;
-    for (uint32_t c = 0; c < nC; ++c) {
-        const bool all_defs = full || ((anom[k * AW + (c >> 5)] >> (c & 31)) & 1u);
-        const bool elided = !all_defs && thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u);
-        if (all_defs || elided) {
-            work[2 + 2 * at] = (uint32_t)k;
-            work[3 + 2 * at] = c | (elided ? RC_ELIDED : 0u);
-            ++at;
+    at = __shfl_sync(0xffffffffu, at, 0);
+    if (lane < RC_BANK_PARTS) {
+        work[2 + 2 * (at + lane)] = (uint32_t)k;
+        work[3 + 2 * (at + lane)] = rc_code(RC_KIND_BANK, lane, 0);
+    }
+    at += RC_BANK_PARTS;
+    for (uint32_t c0 = 0; c0 < nC; c0 += 32) {
+        const uint32_t kd = kind_of(c0 + lane);
+        const uint32_t m = __ballot_sync(0xffffffffu, kd != 0);
+        if (kd) {
+            const uint32_t slot = at + RC_PARTS * __popc(m & ((1u << lane) - 1u));
+#pragma unroll
+            for (uint32_t part = 0; part < RC_PARTS; ++part) {
+                work[2 + 2 * (slot + part)] = (uint32_t)k;
+                work[3 + 2 * (slot + part)] = rc_code(kd == 1 ? RC_KIND_ALL : RC_KIND_ELIDED, part, c0 + lane);
+            }
         }
+        at += RC_PARTS * __popc(m);
     }
 }
 
+// Stand-alone form for programs without walk items (no instructions): one warp per candidate.
+__global__ void k_finish(uint64_t K, uint32_t nC, uint32_t AW, int list_all, const uint32_t *cstate,
+                         const uint32_t *anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work, uint32_t *racc,
+                         vl_verdict *out)
+{
+    const uint64_t k = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (k < K) finish_candidate(k, nC, AW, list_all, cstate, anom, chunk_blk, work, racc, out);
+}
+
 // =========================================================================== k_recount
-// Exact answers for the listed work items; thread blocks loop over the list.  For one item a block
-// copies the candidate's table column to shared memory, then either recounts the overlaps of one
-// chunk from the live-after lists (warps share the chunk's instructions) or does the general bank
-// tally (distinct registers rather than distinct vregs).  Results are added to the candidate's
-// accumulators; the item that finishes last writes the verdict.
+// Exact answers for the listed work items; thread blocks loop over the list.  A chunk item recounts
+// the overlaps of one piece of a chunk from the live-after lists: the warps share the piece's
+// instructions, the lanes of a warp fetch the bookkeeping of 32 instructions at a time, and the
+// candidate's registers come straight from its table column in global memory (the live-after sets
+// of neighbouring instructions are nearly the same, so these gathers hit in L1).  A bank item
+// copies the whole column to shared memory and does a slice of the general bank tally (distinct
+// registers rather than distinct vregs).  Results are added to the candidate's accumulators; the
+// item that finishes last writes the verdict.
 __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 {
-    extern __shared__ __align__(16) uint16_t T[];
+    extern __shared__ __align__(16) uint16_t T[];  // [V + 8] registers of one candidate (bank items)
     __shared__ uint32_t s_pairs, s_mind, s_bank;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr uint32_t NW = RC_THREADS / 32;
     const uint32_t nitems = q.work[0];
     uint64_t have = ~0ull;  // candidate whose column is in shared memory
+#ifdef VL_PHASE_TIMERS
+    const long long rc_t0 = clock64();
+    if (tid == 0 && blockIdx.x == 0) atomicAdd(q.status + 8, nitems);
+#endif
     for (uint32_t it = blockIdx.x; it < nitems; it += gridDim.x) {
         const uint64_t k = q.work[2 + 2 * it];
         const uint32_t code = q.work[3 + 2 * it];
+        const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
+#ifdef VL_PHASE_TIMERS
+        if (tid == 0) atomicAdd(q.status + 11 + kind, 1u);
+#endif
         const uint32_t *cs = q.cstate + k * 8;
+        const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
+        // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
+        const uint32_t out_v = cs[CS_NOUT] == 1 ? cs[CS_OUTV] : 0xFFFFFFFFu, out_raw = cs[CS_OUTRAW];
         __syncthreads();
-        if (k != have) {
-            const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
-            for (uint32_t v = tid; v < q.V; v += RC_THREADS) T[v] = tg[(size_t)v * 32];
+        if (kind == RC_KIND_BANK && k != have) {
+            for (uint32_t v0 = tid; v0 < q.V; v0 += 8 * RC_THREADS) {
+                uint16_t t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t v = v0 + u * RC_THREADS;
+                    t[u] = v < q.V ? tg[(size_t)v * 32] : (uint16_t)0;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t v = v0 + u * RC_THREADS;
+                    if (v < q.V) T[v] = v == out_v ? (uint16_t)out_raw : t[u];
+                }
+            }
             have = k;
         }
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
-        if (tid == 0 && cs[CS_NOUT] == 1) T[cs[CS_OUTV]] = (uint16_t)cs[CS_OUTRAW];  // the true value, not the parked one
-        __syncthreads();
-        if (code != RC_BANK) {
-            const uint32_t c = code & ~RC_ELIDED;
-            const bool elided_only = code & RC_ELIDED;
+        auto reg_of = [&](uint32_t v) -> uint32_t { return v == out_v ? out_raw : (uint32_t)tg[(size_t)v * 32]; };
+        if (kind != RC_KIND_BANK) {
+            const bool elided_only = kind == RC_KIND_ELIDED;
+            const uint32_t ci0 = q.chunk_i0[c], cn = q.chunk_i1[c] - ci0;
+            const uint32_t i_lo = ci0 + (uint32_t)((uint64_t)cn * part / RC_PARTS);
+            const uint32_t i_hi = ci0 + (uint32_t)((uint64_t)cn * (part + 1) / RC_PARTS);
             uint32_t pairs = 0, mind = 0xFFFFFFFFu;
-            for (uint32_t i = q.chunk_i0[c] + warp; i < q.chunk_i1[c]; i += RC_THREADS / 32) {
-                if (elided_only && !q.iflags[i]) continue;
-                const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
-                const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
-                for (uint32_t d = o0; d < o0 + nd; ++d) {
-                    if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
-                    const uint32_t v = q.op_vreg[d];
-                    const uint32_t s = T[v], w = q.width[v];
-                    uint32_t cnt = 0;
-                    for (uint32_t e0 = l0; e0 < l1; e0 += 256) {  // 8 list entries per lane in flight
-                        uint32_t us[8], ws[8];
+            // this warp's instructions: i_lo + warp, i_lo + warp + NW, ...; 32 of them per round
+            for (uint32_t ib = i_lo + warp; ib < i_hi; ib += 32 * NW) {
+                const uint32_t my_i = ib + lane * NW;
+                uint32_t m_o0 = 0, m_nd = 0, m_l0 = 0, m_l1 = 0;
+                if (my_i < i_hi && !(elided_only && !q.iflags[my_i])) {
+                    m_o0 = q.op_off[my_i]; m_nd = q.ndefs[my_i]; m_l0 = q.lo_off[my_i]; m_l1 = q.lo_off[my_i + 1];
+                }
+                uint32_t todo = __ballot_sync(0xffffffffu, m_nd != 0);
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const uint32_t i = ib + (uint32_t)src * NW;
+                    const uint32_t o0 = __shfl_sync(0xffffffffu, m_o0, src), nd = __shfl_sync(0xffffffffu, m_nd, src);
+                    const uint32_t l0 = __shfl_sync(0xffffffffu, m_l0, src), l1 = __shfl_sync(0xffffffffu, m_l1, src);
+                    for (uint32_t d = o0; d < o0 + nd; ++d) {
+                        if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
+                        const uint32_t v = q.op_vreg[d];
+                        const uint32_t s = reg_of(v), w = q.vinfo[v] & 0xFFu;
+                        uint32_t cnt = 0;
+                        for (uint32_t e0 = l0; e0 < l1; e0 += 256) {  // 8 list entries per lane in flight
+                            uint32_t us[8], ts[8], ws[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const uint32_t e = e0 + u * 32 + lane;
-                            us[u] = e < l1 ? q.lo[e] : v;
+                            for (int u = 0; u < 8; ++u) {
+                                const uint32_t e = e0 + u * 32 + lane;
+                                us[u] = e < l1 ? q.lo[e] : v;
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                ts[u] = reg_of(us[u]);
+                                ws[u] = q.vinfo[us[u]] & 0xFFu;
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if (us[u] != v && ranges_overlap(s, w, ts[u], ws[u])) ++cnt;
+                        }
+                        // co-defined vregs that are not live after the instruction
+                        for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
+                            if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
+                            const uint32_t u = q.op_vreg[d2];
+                            if (ranges_overlap(s, w, reg_of(u), q.vinfo[u] & 0xFFu)) ++cnt;
                         }
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) ws[u] = q.vinfo[us[u]] & 0xFFu;
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if (us[u] != v && ranges_overlap(s, w, T[us[u]], ws[u])) ++cnt;
+                        for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
+                        if (cnt) { pairs += cnt; mind = min(mind, i); }
                     }
-                    // co-defined vregs that are not live after the instruction
-                    for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
-                        if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
-                        const uint32_t u = q.op_vreg[d2];
-                        if (ranges_overlap(s, w, T[u], q.width[u])) ++cnt;
-                    }
-#pragma unroll
-                    for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
-                    if (cnt) { pairs += cnt; mind = min(mind, i); }
                 }
             }
             if (lane == 0 && pairs) {
@@ -692,25 +801,39 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             // a source counts when its register is new among the instruction's sources and its bank is not
             uint32_t bt = 0;
             if (q.bank_fast) {
-                for (uint32_t e = tid; e < q.bank_seg[3]; e += RC_THREADS) {
-                    const uint2 ids = q.bank_list[e];
-                    const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
-                    uint32_t x[4];
-                    x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
+                const uint32_t n_all = q.bank_seg[3];
+                const uint32_t e_lo = (uint32_t)((uint64_t)n_all * part / RC_BANK_PARTS);
+                const uint32_t e_hi = (uint32_t)((uint64_t)n_all * (part + 1) / RC_BANK_PARTS);
+                for (uint32_t e0 = e_lo + tid; e0 < e_hi; e0 += 4 * RC_THREADS) {
+                    uint2 idv[4];
 #pragma unroll
-                    for (uint32_t a = 1; a < 4; ++a) {
-                        if (a >= n) break;
-                        bool seen_value = false, seen_bank = false;
+                    for (int u = 0; u < 4; ++u)
+                        idv[u] = e0 + u * RC_THREADS < e_hi ? q.bank_list[e0 + u * RC_THREADS] : make_uint2(0, 0);
 #pragma unroll
-                        for (uint32_t bb = 0; bb < a; ++bb) {
-                            seen_value |= (x[bb] == x[a]);
-                            seen_bank |= ((x[bb] ^ x[a]) & (q.B - 1)) == 0;
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t e = e0 + u * RC_THREADS;
+                        if (e >= e_hi) break;
+                        const uint2 ids = idv[u];
+                        const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
+                        uint32_t x[4];
+                        x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
+#pragma unroll
+                        for (uint32_t a = 1; a < 4; ++a) {
+                            if (a >= n) break;
+                            bool seen_value = false, seen_bank = false;
+#pragma unroll
+                            for (uint32_t bb = 0; bb < a; ++bb) {
+                                seen_value |= (x[bb] == x[a]);
+                                seen_bank |= ((x[bb] ^ x[a]) & (q.B - 1)) == 0;
+                            }
+                            if (!seen_value && seen_bank) ++bt;
                         }
-                        if (!seen_value && seen_bank) ++bt;
                     }
                 }
             } else {
-                for (uint32_t i = tid; i < q.nI; i += RC_THREADS) {
+                const uint32_t i_lo = (uint32_t)((uint64_t)q.nI * part / RC_BANK_PARTS);
+                const uint32_t i_hi = (uint32_t)((uint64_t)q.nI * (part + 1) / RC_BANK_PARTS);
+                for (uint32_t i = i_lo + tid; i < i_hi; i += RC_THREADS) {
                     const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
                     for (uint32_t a = u0 + 1; a < u1; ++a) {
                         const uint32_t xa = T[q.op_vreg[a]];
@@ -751,6 +874,13 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             }
         }
     }
+#ifdef VL_PHASE_TIMERS
+    if (tid == 0) {
+        const uint32_t dt = (uint32_t)((clock64() - rc_t0) >> 6);
+        atomicAdd(q.status + 9, dt);
+        atomicMax(q.status + 10, dt);
+    }
+#endif
 }
 
 // --------------------------------------------------------------------------- host
@@ -792,8 +922,8 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     const uint64_t aw = std::max(1u, (p->nC + 31) / 32);
     const uint64_t groups = (rows + 31) / 32;
     if (v.rows >= rows && v.aw == aw && v.vregs == p->V) return VL_OK;
-    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc);
-    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr;
+    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done);
+    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr; v.grp_done = nullptr;
     v.rows = 0;
     // one more group than needed: it stays all zero, for lanes that have nothing to walk
     VL_CUDA(p, cudaMalloc((void **)&v.tg, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
@@ -801,8 +931,10 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * 32 * (uint64_t)(p->nC + 1)) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work,
+                          (2 + 2 * groups * 32 * ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.grp_done, (groups + 1) * sizeof(uint32_t)));
     v.rows = groups * 32;
     v.aw = aw;
     v.vregs = p->V;
@@ -822,10 +954,16 @@ static void kt_mark(vl_program *p, cudaStream_t st)
     cudaEventRecord(p->kt_ev[p->kt_used++], st);
 }
 
-int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
-                   cudaStream_t st, int slot)
+namespace {
+struct PassPlan {
+    Plan pl;
+    uint32_t Wp, ev_cap, walk_smem, rc_smem;
+    uint64_t sub;
+};
+
+// Launch geometry of a program's passes and the shared-memory opt-ins of its kernels.
+int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
 {
-    vl_program *p = const_cast<vl_program *>(cp);  // the handle owns the working memory of its calls
     const uint32_t SM_BYTES = 227 * 1024;
     // preference: the largest group that still lets two blocks share an SM, then anything that fits
     Plan pl{};
@@ -838,97 +976,170 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
             if (pl.ok) break;
         }
     if (!pl.ok) return VL_ERR_UNSUPPORTED;
-    const uint32_t Wp = (p->P + p->wmax + 31) / 32;
-    const uint32_t ev_cap = 256;
-    const uint32_t walk_smem = (Wp * 32 + WALK_WARPS * (Wp * 32 + ev_cap * 4)) * 4;
-    const uint32_t rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
-    if (walk_smem > SM_BYTES || rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    pp->pl = pl;
+    pp->Wp = (p->P + p->wmax + 31) / 32;
+    pp->ev_cap = 256;
+    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + pp->ev_cap * 4)) * 4;
+    pp->rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
+    if (pp->walk_smem > SM_BYTES || pp->rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    // the recount work list holds up to RC_PARTS items per chunk and candidate: keep it within 8 Mi items
+    const uint64_t sub_cap =
+        std::max<uint64_t>(32, ((8ull << 20) / ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) / 32 * 32);
+    pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
+    cudaError_t e = cudaSuccess;
+    if (pp->walk_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->walk_smem);
+    if (e == cudaSuccess && pp->walk_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->walk_smem);
+    if (e == cudaSuccess && pp->rc_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
+    if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+    return VL_OK;
+}
 
-    // the recount work list holds up to (chunks + 1) items per candidate: keep it within 4 Mi items
-    const uint64_t sub_cap = std::max<uint64_t>(32, ((4ull << 20) / (p->nC + 1)) / 32 * 32);
-    const uint64_t sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
-    int rc = ensure_scratch(p, slot, sub);
+// One pass: the four kernels over n <= sub candidates, in order on `st`, with working set `slot`.
+int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t n, uint64_t pitch, vl_verdict *d_out,
+             cudaStream_t st, int slot)
+{
+    const Plan &pl = pp.pl;
+    int rc = ensure_scratch(p, slot, pp.sub);
     if (rc != VL_OK) return rc;
     vl_program::VScratch &vs = p->vs[slot];
     cudaError_t e = cudaSuccess;
-    if (walk_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
-    if (e == cudaSuccess && walk_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)walk_smem);
-    if (e == cudaSuccess && rc_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rc_smem);
+    const uint32_t ngrp = (uint32_t)((n + 31) / 32);
+
+    TParams tq{};
+    tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
+    tq.ntiles = (p->nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
+    tq.bank_fast = p->bank_fast;
+    tq.vreg16 = p->d_vreg16; tq.slotmeta = p->d_slotmeta; tq.vinfo = p->d_vinfo;
+    tq.first_def_instr = p->d_first_def_instr; tq.op_off = p->d_op_off;
+    tq.bank_list = p->d_bank_list;
+    for (int j = 0; j < 4; ++j) tq.bank_seg[j] = p->bank_seg[j];
+    tq.cand = d_cand; tq.K = n; tq.pitch = pitch;
+    tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
+    tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
+    tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
+    const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
+    kt_mark(p, st);
+    if (pl.NT == 256) {
+        if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
+        else if (pl.G == 2) e = launch_tables<2, 256>(tq, tgrid, pl.smem, st);
+        else e = launch_tables<1, 256>(tq, tgrid, pl.smem, st);
+    } else {
+        if (pl.G == 4) e = launch_tables<4, 512>(tq, tgrid, pl.smem, st);
+        else if (pl.G == 2) e = launch_tables<2, 512>(tq, tgrid, pl.smem, st);
+        else e = launch_tables<1, 512>(tq, tgrid, pl.smem, st);
+    }
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+    g_vl_launches.fetch_add(1);
 
-    for (uint64_t kb = 0; kb < K; kb += sub) {
-        const uint64_t n = std::min(sub, K - kb);
-        const uint32_t ngrp = (uint32_t)((n + 31) / 32);
-        VL_CUDA(p, cudaMemsetAsync(vs.anom, 0, (size_t)ngrp * 32 * vs.aw * 4, st));
-        VL_CUDA(p, cudaMemsetAsync(vs.work, 0, 4, st));
-        VL_CUDA(p, cudaMemsetAsync(vs.racc, 0, (size_t)ngrp * 32 * 16, st));
-
-        TParams tq{};
-        tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
-        tq.ntiles = (p->nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
-        tq.bank_fast = p->bank_fast;
-        tq.vreg16 = p->d_vreg16; tq.slotmeta = p->d_slotmeta; tq.vinfo = p->d_vinfo;
-        tq.first_def_instr = p->d_first_def_instr; tq.op_off = p->d_op_off;
-        tq.bank_list = p->d_bank_list;
-        for (int j = 0; j < 4; ++j) tq.bank_seg[j] = p->bank_seg[j];
-        tq.cand = d_cand + kb * pitch; tq.K = n; tq.pitch = pitch;
-        tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
-        tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
-        const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
-        kt_mark(p, st);
-        if (pl.NT == 256) {
-            if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
-            else if (pl.G == 2) e = launch_tables<2, 256>(tq, tgrid, pl.smem, st);
-            else e = launch_tables<1, 256>(tq, tgrid, pl.smem, st);
-        } else {
-            if (pl.G == 4) e = launch_tables<4, 512>(tq, tgrid, pl.smem, st);
-            else if (pl.G == 2) e = launch_tables<2, 512>(tq, tgrid, pl.smem, st);
-            else e = launch_tables<1, 512>(tq, tgrid, pl.smem, st);
-        }
-        if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
-        g_vl_launches.fetch_add(1);
-
-        kt_mark(p, st);
-        if (p->nItems) {
-            WParams wq{};
-            wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = Wp; wq.AW = (uint32_t)vs.aw;
-            wq.use_th = (uint32_t)p->use_th; wq.K = n;
-            wq.th_off = p->d_th_off; wq.th = p->d_th; wq.cev_off = p->d_cev_off; wq.ev = p->d_ev;
-            wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
-            wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = ev_cap;
-            wq.cstate = vs.cstate; wq.anom = vs.anom;
-            if (p->wmax > 32) k_walk<true><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
-            else k_walk<false><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, walk_smem, st>>>(wq);
-            e = cudaGetLastError();
-            if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
-            g_vl_launches.fetch_add(1);
-        }
-
-        // programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction
-        // with more than 4 distinct sources) send every candidate through k_recount
-        kt_mark(p, st);
-        k_finish<<<(uint32_t)((n + 127) / 128), 128, 0, st>>>(n, p->nC, (uint32_t)vs.aw, p->bank_fast ? 0 : 1, vs.cstate,
-                                                             vs.anom, p->d_chunk_blk, vs.work, vs.racc, d_out + kb);
-        RParams rq{};
-        rq.nI = p->nI; rq.V = p->V; rq.B = p->B; rq.nB = p->nB; rq.nC = p->nC; rq.AW = (uint32_t)vs.aw;
-        rq.bank_fast = p->bank_fast; rq.K = n;
-        rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
-        rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
-        rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
-        rq.racc = vs.racc;
-        rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out + kb;
-        rq.bank_list = p->d_bank_list;
-        for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
-        const uint32_t rgrid = 148 * 6;
-        kt_mark(p, st);
-        k_recount<<<rgrid, RC_THREADS, rc_smem, st>>>(rq);
-        kt_mark(p, st);
+    kt_mark(p, st);
+    if (p->nItems) {
+        WParams wq{};
+        wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = pp.Wp; wq.AW = (uint32_t)vs.aw;
+        wq.use_th = (uint32_t)p->use_th; wq.K = n;
+        wq.th_off = p->d_th_off; wq.th = p->d_th; wq.cev_off = p->d_cev_off; wq.ev = p->d_ev;
+        wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
+        wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = pp.ev_cap;
+        wq.cstate = vs.cstate; wq.anom = vs.anom;
+        wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
+        wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
+        if (p->wmax > 32) k_walk<true><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        else k_walk<false><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
-        g_vl_launches.fetch_add(2);
+        g_vl_launches.fetch_add(1);
+    }
+
+    // programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction
+    // with more than 4 distinct sources) send every candidate through k_recount
+    kt_mark(p, st);
+    if (!p->nItems) {  // nothing to walk: the verdict step runs on its own
+        k_finish<<<(uint32_t)((n * 32 + 127) / 128), 128, 0, st>>>(n, p->nC, (uint32_t)vs.aw, p->bank_fast ? 0 : 1,
+                                                                  vs.cstate, vs.anom, p->d_chunk_blk, vs.work, vs.racc,
+                                                                  d_out);
+        g_vl_launches.fetch_add(1);
+    }
+    RParams rq{};
+    rq.nI = p->nI; rq.V = p->V; rq.B = p->B; rq.nB = p->nB; rq.nC = p->nC; rq.AW = (uint32_t)vs.aw;
+    rq.bank_fast = p->bank_fast; rq.K = n;
+    rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
+    rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
+    rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
+    rq.racc = vs.racc; rq.status = p->d_status + 1;
+    rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out;
+    rq.bank_list = p->d_bank_list;
+    for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
+    const uint32_t rgrid = 148 * 6;
+    kt_mark(p, st);
+    k_recount<<<rgrid, RC_THREADS, pp.rc_smem, st>>>(rq);
+    kt_mark(p, st);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+    g_vl_launches.fetch_add(1);
+    return VL_OK;
+}
+}  // namespace
+
+// All passes in order on one stream, with one working set.
+int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+                   cudaStream_t st, int slot)
+{
+    vl_program *p = const_cast<vl_program *>(cp);  // the handle owns the working memory of its calls
+    PassPlan pp{};
+    int rc = plan_passes(p, K, &pp);
+    if (rc != VL_OK) return rc;
+    for (uint64_t kb = 0; kb < K; kb += pp.sub) {
+        rc = run_pass(p, pp, d_cand + kb * pitch, std::min(pp.sub, K - kb), pitch, d_out + kb, st, slot);
+        if (rc != VL_OK) return rc;
     }
     return VL_OK;
+}
+
+// Passes of one or several programs spread round-robin over the device's lane streams, so that
+// the table kernel of one pass (bound by the row stream) runs beside the walk of another (bound by
+// instruction issue).  Pass j of a program uses working set j mod lanes and runs on lane
+// (first_lane + j) mod lanes: two passes that share a working set are ordered by their stream.
+int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
+                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st)
+{
+    vl_program *p0 = const_cast<vl_program *>(progs[0]);
+    cudaStream_t *lane = nullptr;
+    int rc = vl_lane_streams(p0, &lane);
+    if (rc != VL_OK) return rc;
+    const uint32_t L = std::min<uint32_t>(VL_LANES, std::max<uint32_t>(1, p0->lanes_opt));
+    uint64_t jobs = 0;
+    for (uint32_t j = 0; j < nprog; ++j) jobs += (K[j] + progs[j]->sub_batch - 1) / progs[j]->sub_batch;
+    if (L == 1 || jobs <= 1) {
+        for (uint32_t j = 0; j < nprog; ++j) {
+            if (K[j] == 0) continue;
+            rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], st, 0);
+            if (rc != VL_OK) return rc;
+        }
+        return VL_OK;
+    }
+    VL_CUDA(p0, cudaEventRecord(p0->ev_fork, st));
+    for (uint32_t l = 0; l < L; ++l) VL_CUDA(p0, cudaStreamWaitEvent(lane[l], p0->ev_fork, 0));
+    uint64_t job = 0;
+    for (uint32_t j = 0; j < nprog && rc == VL_OK; ++j) {
+        if (K[j] == 0) continue;
+        vl_program *p = const_cast<vl_program *>(progs[j]);
+        PassPlan pp{};
+        rc = plan_passes(p, K[j], &pp);
+        if (rc != VL_OK) break;
+        // a program's passes keep to "working set s on lane (base + s) mod L"
+        const uint64_t base = job;
+        uint64_t s = 0;
+        for (uint64_t kb = 0; kb < K[j] && rc == VL_OK; kb += pp.sub, ++s, ++job)
+            rc = run_pass(p, pp, d_cand[j] + kb * pitch[j], std::min(pp.sub, K[j] - kb), pitch[j], d_out[j] + kb,
+                          lane[(base + s) % L], (int)(s % L));
+    }
+    // join even after an error, so that the caller's stream stays ordered after what was launched
+    for (uint32_t l = 0; l < L; ++l) {
+        cudaError_t e = cudaEventRecord(p0->ev_join[l], lane[l]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, p0->ev_join[l], 0);
+        if (e != cudaSuccess && rc == VL_OK) { p0->last_cuda_error = (int)e; rc = VL_ERR_CUDA; }
+    }
+    return rc;
 }
