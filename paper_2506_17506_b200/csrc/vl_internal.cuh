@@ -100,7 +100,7 @@ struct vl_program {
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
     uint32_t th_len = 0;
     uint32_t *d_cev_off = nullptr;  // [nC+1] first walk event of each chunk (every chunk padded to 8 events)
-    uint4 *d_ev = nullptr;          // walk events (16 bytes each), chunk after chunk
+    uint4 *d_ev = nullptr;          // walk events, 112 bytes per group of 8, chunk after chunk
     uint32_t ev_total = 0;
     // walk work items: a run of chunks of one block
     uint32_t nItems = 0;

@@ -395,10 +395,14 @@ __global__ void k_instr_flags(uint32_t nI, const uint32_t *__restrict__ op_off, 
     iflags[i] = f;
 }
 
-__global__ void k_fill_noop(uint4 *dst, size_t n, uint32_t spare_vreg)
+// Every event slot starts as a no-op (see put_event for the layout of a group of 8 events).
+__global__ void k_fill_noop(uint4 *dst, size_t n_groups, uint32_t spare_vreg)
 {
-    for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n; i += (size_t)gridDim.x * NT)
-        dst[i] = make_uint4(spare_vreg, 0u, 0u, 31u);
+    const uint32_t vv = spare_vreg * 64u, ww = 31u | (31u << 16);
+    for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n_groups * 7; i += (size_t)gridDim.x * NT) {
+        const uint32_t part = (uint32_t)(i % 7);
+        dst[i] = part < 2 ? make_uint4(vv, vv, vv, vv) : (part == 6 ? make_uint4(ww, ww, ww, ww) : make_uint4(0, 0, 0, 0));
+    }
 }
 
 __global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
@@ -447,15 +451,21 @@ __global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8
     slotmeta[s] = m;
 }
 
-// A walk event is 16 bytes: x = vreg, y = bits to test, z = bits to toggle (the width-w mask
-// (1<<w)-1, or 0), w = 32 - width: the range straddles a 32-bit word iff (register & 31) > w.
-// Ranges wider than 32 registers carry w = 0x80000000 | width and y, z as 0/1 flags.
-// A no-op names the spare vreg V with empty masks.
-__device__ __forceinline__ uint4 make_event(uint32_t v, uint32_t w, bool test, bool toggle)
+// Walk events are stored in groups of 8, 112 bytes per group, field by field so that the walk
+// fetches a group with 16-byte loads: off[8] (32 bit: byte offset of the vreg's row in a table of
+// 32 16-bit entries per vreg), toggle[8] (32 bit: the width-w mask (1<<w)-1, or 0), test[8]
+// (likewise), wl[8] (16 bit: 32 - width; the range straddles a 32-bit word iff
+// (register & 31) > wl).  Ranges wider than 32 registers carry wl = 0x8000 | width and
+// toggle, test as 0/1 flags.  A no-op names the spare vreg V with empty masks.
+__device__ __forceinline__ void put_event(uint4 *ev, size_t idx, uint32_t v, uint32_t w, bool test, bool toggle)
 {
-    if (w > 32) return make_uint4(v, test ? 1u : 0u, toggle ? 1u : 0u, 0x80000000u | w);
-    const uint32_t wm = w == 32 ? 0xFFFFFFFFu : ((1u << w) - 1u);
-    return make_uint4(v, test ? wm : 0u, toggle ? wm : 0u, 32u - w);
+    unsigned char *g = reinterpret_cast<unsigned char *>(ev) + (idx >> 3) * 112;
+    const uint32_t slot = (uint32_t)(idx & 7);
+    const uint32_t wm = w > 32 ? 1u : (w == 32 ? 0xFFFFFFFFu : ((1u << w) - 1u));
+    reinterpret_cast<uint32_t *>(g)[slot] = v * 64u;
+    reinterpret_cast<uint32_t *>(g + 32)[slot] = toggle ? wm : 0u;
+    reinterpret_cast<uint32_t *>(g + 64)[slot] = test ? wm : 0u;
+    reinterpret_cast<uint16_t *>(g + 96)[slot] = (uint16_t)(w > 32 ? (0x8000u | w) : (32u - w));
 }
 
 // Walk events of one chunk: entry occupancy (ascending vreg id), then per instruction the
@@ -473,7 +483,7 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
     const size_t base = cev_off[c];
     uint32_t total;
     compact_bits(chunk_entry + (size_t)c * Wv, Wv, s_scan, &total, [&](uint32_t rank, uint32_t v) {
-        ev[base + rank] = make_event(v, width[v], true, true);
+        put_event(ev, base + rank, v, width[v], true, true);
     });
     const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
     const uint32_t e_base = centry_cnt[c];
@@ -483,17 +493,17 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
         for (uint32_t o = o0 + nd; o < o1; ++o)
             if (opflags[o] & OPF_KILL) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (e++)] = make_event(v, width[v], false, true);
+                put_event(ev, base + (e++), v, width[v], false, true);
             }
         for (uint32_t o = o0; o < o0 + nd; ++o)
             if (!(opflags[o] & OPF_ELIDE)) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (e++)] = make_event(v, width[v], true, (opflags[o] & OPF_SET) != 0);
+                put_event(ev, base + (e++), v, width[v], true, (opflags[o] & OPF_SET) != 0);
             }
         for (uint32_t o = o0; o < o0 + nd; ++o)
             if ((opflags[o] & OPF_POST) && !(opflags[o] & OPF_ELIDE)) {
                 const uint32_t v = op_vreg[o];
-                ev[base + (e++)] = make_event(v, width[v], false, true);
+                put_event(ev, base + (e++), v, width[v], false, true);
             }
     }
 }
@@ -660,10 +670,10 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     p->th_len = (uint32_t)thn;
 
     VL_CUDA(p, keep(&p->d_lo, (size_t)p->lo_len, 0, st));
-    VL_CUDA(p, keep(&p->d_ev, (size_t)steps, 0, st));
+    VL_CUDA(p, keep(&p->d_ev, (size_t)(steps / 8) * 7, 0, st));
     VL_CUDA(p, keep(&p->d_vinfo, (size_t)V, 0, st));
     VL_CUDA(p, keep(&p->d_iflags, (size_t)nI, 0, st));
-    LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)steps,
+    LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)(steps / 8),
            V);  // every slot starts as a no-op event
     VL_CUDA(p, keep(&p->d_th, (size_t)thn, 0, st));
     VL_CUDA(p, keep(&p->d_cev_off, (size_t)nC + 1, 0, st));

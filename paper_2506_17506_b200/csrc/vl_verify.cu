@@ -41,6 +41,9 @@ struct TParams {
     uint32_t *cstate;
     uint32_t *status;
     uint32_t NS, off_region, off_misc;
+    // 1: bit 15 of a table entry handed to the walk marks a range that reaches into the next 32-bit
+    // word of the occupancy mask (possible when every in-file register number is below 2^15)
+    uint32_t flag15;
     // per-pass state this kernel clears for the kernels after it
     uint32_t AW;
     uint32_t *anom, *racc, *grp_done, *work;
@@ -61,6 +64,7 @@ struct WParams {
     const uint16_t *tg, *tg_zero;
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
+    uint32_t tmask;  // 0x7FFF when bit 15 of a table entry is the straddle mark, else 0xFFFF
     // hand-over to k_recount by the last thread block of each group of 32 candidates
     int list_all;
     const uint32_t *chunk_blk;
@@ -82,6 +86,7 @@ struct RParams {
     uint32_t *work;
     vl_verdict *out;
     uint32_t *status;
+    uint32_t tmask;  // see WParams
 };
 
 // Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
@@ -337,12 +342,19 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
                 const uint32_t v = v0 + u * NT, vi = vis[u];
                 if (v > q.V) break;
                 const uint64_t tt = v < q.V ? t_load<G>(Tt, v) : 0ull;
+                uint32_t lo = (uint32_t)tt, hi = (uint32_t)(tt >> 32);
+                if (q.flag15) {
+                    // per 16-bit entry: bit 15 := ((register & 31) + width > 32); 0x7FDF = 0x8000 - 33
+                    const uint32_t wc = (vi & 0xFFu) * 0x10001u + 0x7FDF7FDFu;
+                    lo = (lo & 0x7FFF7FFFu) | (((lo & 0x001F001Fu) + wc) & 0x80008000u);
+                    hi = (hi & 0x7FFF7FFFu) | (((hi & 0x001F001Fu) + wc) & 0x80008000u);
+                }
                 if constexpr (G == 4) {
-                    *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2((uint32_t)tt, (uint32_t)(tt >> 32));
+                    *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2(lo, hi);
                 } else if constexpr (G == 2) {
-                    *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = (uint32_t)tt;
+                    *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = lo;
                 } else {
-                    dst[(size_t)v * 32] = (uint16_t)tt;
+                    dst[(size_t)v * 32] = (uint16_t)lo;
                 }
                 if (!(vi & VINFO_OCCURS)) continue;
                 const uint32_t w = vi & 0xFFu;
@@ -423,8 +435,20 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     // ------------------------------------------------- hand-over to the walk
     // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
     // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
-    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P)
-        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)M->out_v[tid] * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)q.P;
+    // (such a candidate does not take part in the walk: it gets its table back without the marks)
+    if (q.flag15) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            if (M->nout[g] < 2) continue;
+            uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
+            for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk_get(t_load<G>(Tt, v), g);
+        }
+    }
+    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
+        const uint32_t ov = M->out_v[tid];
+        const uint32_t mark = (q.flag15 && (q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
+        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)ov * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)(q.P | mark);
+    }
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
@@ -472,16 +496,17 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 // A range wider than 32 registers (rare): word by word.
-__device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, uint32_t tv, uint4 e)
+__device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, uint32_t tv, uint32_t width,
+                                                uint32_t test, uint32_t toggle)
 {
-    uint32_t viol = 0, left = e.w & 0xFFFFu, pos = tv;
+    uint32_t viol = 0, left = width, pos = tv;
     while (left) {
         const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
         const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
         uint32_t *a = s_occ + (pos >> 5) * 32 + lane;
         const uint32_t o = *a;
-        if (e.y) viol |= o & m;
-        if (e.z) *a = o ^ m;
+        if (test) viol |= o & m;
+        if (toggle) *a = o ^ m;
         pos += nn;
         left -= nn;
     }
@@ -492,18 +517,98 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
                                  const uint32_t *anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
                                  uint32_t *racc, vl_verdict *out);
 
+// An event group in shared memory is 112 bytes: off[8] (byte offset of the vreg's table row),
+// toggle[8], test[8] (32-bit masks), wl[8] (16 bit).  Constant offsets go into the instruction.
+template <int OFF>
+__device__ __forceinline__ uint4 lds128_at(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4 + %5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr), "n"(OFF)
+                 : "memory");
+    return v;
+}
+
+// Table entries (this lane's candidate) of the 8 vregs of the event group at shared address ga.
+__device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tgb, uint32_t (&t)[8])
+{
+    const uint4 a = lds128_at<0>(ga), b = lds128_at<16>(ga);
+    const uint32_t off[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = *reinterpret_cast<const uint16_t *>(tgb + off[u]);
+}
+
+// Applies the 8 events of the group at shared address ga to this lane's occupancy mask; returns the
+// occupied bits that a test found.  Toggling returns the old word: occupied and released are both
+// a toggle as long as no collision has been seen (after one, the chunk is recounted exactly
+// anyway).  The common case, no range of the group reaching into the next 32-bit word for any
+// lane, is decided before anything is applied and takes one atomic per event.  F15: the table
+// entries carry that fact in bit 15; otherwise it is worked out from the event's width.
+template <bool WIDE, bool F15>
+__device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, uint32_t *s_occ,
+                                                uint32_t lane)
+{
+    const uint4 z0 = lds128_at<32>(ga), z1 = lds128_at<48>(ga), y0 = lds128_at<64>(ga), y1 = lds128_at<80>(ga);
+    const uint32_t ez[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+    const uint32_t ey[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+    bool slow;
+    if (F15 && !WIDE) {
+        slow = ((t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & 0x8000u) != 0;
+    } else {
+        const uint4 w4 = lds128_at<96>(ga);
+        const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
+        slow = false;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t wl = (u & 1) ? (ew[u >> 1] >> 16) : (ew[u >> 1] & 0xFFFFu);
+            slow |= ((t[u] & 31u) > wl) || (WIDE && (wl & 0x8000u));
+        }
+    }
+    uint32_t viol = 0;
+    if (!__any_sync(0xffffffffu, slow)) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t tv = t[u];
+            const uint32_t a = occ_addr + (tv & (F15 ? 0x7FE0u : 0xFFE0u)) * 4u;  // word (tv / 32) of this lane's mask
+            const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, ez[u], tv));
+            viol |= o & __funnelshift_l(0u, ey[u], tv);
+        }
+        return viol;
+    }
+    const uint4 w4 = lds128_at<96>(ga);
+    const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const uint32_t tv = F15 ? (t[u] & 0x7FFFu) : t[u];
+        const uint32_t wl = (u & 1) ? (ew[u >> 1] >> 16) : (ew[u >> 1] & 0xFFFFu);
+        if (WIDE && (wl & 0x8000u)) {
+            viol |= walk_very_wide(s_occ, lane, tv, wl & 0xFFu, ey[u], ez[u]);
+            continue;
+        }
+        const uint32_t a = occ_addr + ((tv >> 5) << 7);
+        const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, ez[u], tv));
+        viol |= o & __funnelshift_l(0u, ey[u], tv);
+        if ((tv & 31u) > wl) {  // the range straddles into the next word
+            const uint32_t o2 = atom_xor_shared(a + 128, __funnelshift_l(ez[u], 0u, tv));
+            viol |= o2 & __funnelshift_l(ey[u], 0u, tv);
+        }
+    }
+    return viol;
+}
+
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
-template <bool WIDE>
-__global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
+template <bool WIDE, bool F15>
+__global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
 {
     extern __shared__ __align__(16) uint32_t wsm[];
     uint32_t *s_th = wsm;  // [Wp][32]
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t per_warp = q.Wp * 32 + q.ev_cap * 4;  // words
+    const uint32_t per_warp = q.Wp * 32 + (q.ev_cap >> 3) * 28;  // words: 112 bytes per group of 8 events
     uint32_t *s_occ = wsm + q.Wp * 32 + (size_t)warp * per_warp;  // [Wp][32]
-    uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap]
+    uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap / 8] groups of 7 x 16 bytes
     const uint32_t item = blockIdx.x, grp = blockIdx.y;
     const uint32_t b = q.item_blk[item], c0 = q.item_c0[item], c1 = q.item_c1[item];
     const uint64_t k = (uint64_t)grp * 32 + lane;
@@ -512,6 +617,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
     // hold anything), read an all-zero table instead
     const bool walked = k < q.K && !(cs[CS_WALK] & WALK_FULL);
     const uint16_t *tg = walked ? q.tg + (uint64_t)grp * (q.V + 1) * 32 + lane : q.tg_zero + lane;
+    const unsigned char *tgb = reinterpret_cast<const unsigned char *>(tg);
 
     for (uint32_t i = threadIdx.x; i < q.Wp * 32; i += WALK_WARPS * 32) s_th[i] = 0;
     __syncthreads();
@@ -527,7 +633,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
             for (int u = 0; u < 8; ++u) t[u] = tg[(size_t)(x[u] & 0xFFFFu) * 32];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                uint32_t pos = t[u], left = x[u] >> 16;
+                uint32_t pos = t[u] & q.tmask, left = x[u] >> 16;
                 while (left) {
                     const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
                     const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
@@ -542,45 +648,29 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) k_walk(const WParams q)
         __syncthreads();
     }
 
+    const uint32_t occ_addr = smem_u32(s_occ) + lane * 4, ev_addr = smem_u32(s_ev);
     for (uint32_t c = c0 + warp; c < c1; c += WALK_WARPS) {
         for (uint32_t wd = 0; wd < q.Wp; ++wd) s_occ[wd * 32 + lane] = s_th[wd * 32 + lane];
         uint32_t viol = 0;
-        const uint32_t occ_addr = smem_u32(s_occ) + lane * 4, ev_addr = smem_u32(s_ev);
         const uint32_t s0 = q.cev_off[c], n_ev = q.cev_off[c + 1] - s0;  // a multiple of 8 events
         for (uint32_t done = 0; done < n_ev; done += q.ev_cap) {
-            const uint32_t n = min(q.ev_cap, n_ev - done);
+            const uint32_t n = min(q.ev_cap, n_ev - done), ng = n >> 3;
             __syncwarp();
-            for (uint32_t i = lane; i < n; i += 32) s_ev[i] = q.ev[s0 + done + i];  // events of this piece, once
+            {   // events of this piece, once: 7 x 16 bytes per group of 8
+                const uint4 *src = q.ev + (size_t)((s0 + done) >> 3) * 7;
+                for (uint32_t i = lane; i < ng * 7; i += 32) s_ev[i] = src[i];
+            }
             __syncwarp();
-            // table entries of the next 8 events are fetched while the current 8 are applied
-            uint32_t tn[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) tn[u] = tg[(size_t)s_ev[u].x * 32];
-            for (uint32_t s = 0; s < n; s += 8) {
-                uint32_t t[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) t[u] = tn[u];
-                if (s + 8 < n) {
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) tn[u] = tg[(size_t)s_ev[s + 8 + u].x * 32];
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint4 e = lds128(ev_addr + (s + u) * 16);
-                    const uint32_t tv = t[u];
-                    if (WIDE && (int)e.w < 0) {
-                        viol |= walk_very_wide(s_occ, lane, tv, e);
-                        continue;
-                    }
-                    const uint32_t a = occ_addr + ((tv >> 5) << 7);  // word (tv / 32) of this lane's mask
-                    // toggling returns the old word: occupied and released are both a toggle as long as
-                    // no collision has been seen (after one, the chunk is recounted exactly anyway)
-                    const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, e.z, tv));
-                    viol |= o & __funnelshift_l(0u, e.y, tv);
-                    if ((tv & 31u) > e.w) {  // the range straddles into the next word
-                        const uint32_t o2 = atom_xor_shared(a + 128, __funnelshift_l(e.z, 0u, tv));
-                        viol |= o2 & __funnelshift_l(e.y, 0u, tv);
-                    }
+            // table entries of the next group are fetched while the current group is applied
+            uint32_t ta[8], tb[8];
+            fetch_group(ev_addr, tgb, ta);
+            for (uint32_t g = 0; g < ng; g += 2) {
+                const uint32_t ga = ev_addr + g * 112;
+                if (g + 1 < ng) fetch_group(ga + 112, tgb, tb);
+                viol |= apply_group<WIDE, F15>(ga, ta, occ_addr, s_occ, lane);
+                if (g + 1 < ng) {
+                    if (g + 2 < ng) fetch_group(ga + 224, tgb, ta);
+                    viol |= apply_group<WIDE, F15>(ga + 112, tb, occ_addr, s_occ, lane);
                 }
             }
         }
@@ -720,6 +810,8 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
         // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
         const uint32_t out_v = cs[CS_NOUT] == 1 ? cs[CS_OUTV] : 0xFFFFFFFFu, out_raw = cs[CS_OUTRAW];
+        // a candidate with several out-of-file vregs was not walked and keeps its table unmarked
+        const uint32_t tmask = (cs[CS_WALK] & WALK_FULL) ? 0xFFFFu : q.tmask;
         __syncthreads();
         if (kind == RC_KIND_BANK && k != have) {
             for (uint32_t v0 = tid; v0 < q.V; v0 += 8 * RC_THREADS) {
@@ -732,14 +824,16 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const uint32_t v = v0 + u * RC_THREADS;
-                    if (v < q.V) T[v] = v == out_v ? (uint16_t)out_raw : t[u];
+                    if (v < q.V) T[v] = v == out_v ? (uint16_t)out_raw : (uint16_t)(t[u] & tmask);
                 }
             }
             have = k;
         }
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
-        auto reg_of = [&](uint32_t v) -> uint32_t { return v == out_v ? out_raw : (uint32_t)tg[(size_t)v * 32]; };
+        auto reg_of = [&](uint32_t v) -> uint32_t {
+            return v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * 32] & tmask);
+        };
         if (kind != RC_KIND_BANK) {
             const bool elided_only = kind == RC_KIND_ELIDED;
             const uint32_t ci0 = q.chunk_i0[c], cn = q.chunk_i1[c] - ci0;
@@ -957,7 +1051,7 @@ static void kt_mark(vl_program *p, cudaStream_t st)
 namespace {
 struct PassPlan {
     Plan pl;
-    uint32_t Wp, ev_cap, walk_smem, rc_smem;
+    uint32_t Wp, ev_cap, walk_smem, rc_smem, flag15;
     uint64_t sub;
 };
 
@@ -979,7 +1073,7 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->pl = pl;
     pp->Wp = (p->P + p->wmax + 31) / 32;
     pp->ev_cap = 256;
-    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + pp->ev_cap * 4)) * 4;
+    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + (pp->ev_cap >> 3) * 28)) * 4;
     pp->rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
     if (pp->walk_smem > SM_BYTES || pp->rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
     // the recount work list holds up to RC_PARTS items per chunk and candidate: keep it within 8 Mi items
@@ -987,10 +1081,14 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
         std::max<uint64_t>(32, ((8ull << 20) / ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) / 32 * 32);
     pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
     cudaError_t e = cudaSuccess;
-    if (pp->walk_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->walk_smem);
-    if (e == cudaSuccess && pp->walk_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->walk_smem);
+    pp->flag15 = p->P + p->wmax <= 32768u ? 1u : 0u;
+    if (pp->walk_smem > 48 * 1024) {
+        const int sm = (int)pp->walk_smem;
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    }
     if (e == cudaSuccess && pp->rc_smem > 48 * 1024)
         e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
@@ -1019,6 +1117,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.cand = d_cand; tq.K = n; tq.pitch = pitch;
     tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
+    tq.flag15 = pp.flag15;
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
@@ -1045,8 +1144,15 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
         wq.cstate = vs.cstate; wq.anom = vs.anom;
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
-        if (p->wmax > 32) k_walk<true><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-        else k_walk<false><<<dim3(p->nItems, ngrp), WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        wq.tmask = pp.flag15 ? 0x7FFFu : 0xFFFFu;
+        const dim3 wgrid(p->nItems, ngrp);
+        if (p->wmax > 32) {
+            if (pp.flag15) k_walk<true, true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+            else k_walk<true, false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        } else {
+            if (pp.flag15) k_walk<false, true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+            else k_walk<false, false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        }
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
         g_vl_launches.fetch_add(1);
@@ -1067,7 +1173,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
     rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
     rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
-    rq.racc = vs.racc; rq.status = p->d_status + 1;
+    rq.racc = vs.racc; rq.status = p->d_status + 1; rq.tmask = pp.flag15 ? 0x7FFFu : 0xFFFFu;
     rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out;
     rq.bank_list = p->d_bank_list;
     for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
