@@ -41,9 +41,6 @@ struct TParams {
     uint32_t *cstate;
     uint32_t *status;
     uint32_t NS, off_region, off_misc;
-    // 1: bit 15 of a table entry handed to the walk marks a range that reaches into the next 32-bit
-    // word of the occupancy mask (possible when every in-file register number is below 2^15)
-    uint32_t flag15;
     // per-pass state this kernel clears for the kernels after it
     uint32_t AW;
     uint32_t *anom, *racc, *grp_done, *work;
@@ -64,7 +61,6 @@ struct WParams {
     const uint16_t *tg, *tg_zero;
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
-    uint32_t tmask;  // 0x7FFF when bit 15 of a table entry is the straddle mark, else 0xFFFF
     // hand-over to k_recount by the last thread block of each group of 32 candidates
     int list_all;
     const uint32_t *chunk_blk;
@@ -86,7 +82,6 @@ struct RParams {
     uint32_t *work;
     vl_verdict *out;
     uint32_t *status;
-    uint32_t tmask;  // see WParams
 };
 
 // Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
@@ -343,8 +338,9 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
                 if (v > q.V) break;
                 const uint64_t tt = v < q.V ? t_load<G>(Tt, v) : 0ull;
                 uint32_t lo = (uint32_t)tt, hi = (uint32_t)(tt >> 32);
-                if (q.flag15) {
-                    // per 16-bit entry: bit 15 := ((register & 31) + width > 32); 0x7FDF = 0x8000 - 33
+                {   // bit 15 of an entry handed to the walk marks a range that reaches into the next 32-bit
+                    // word of the occupancy mask (every in-file register number is below 2^15):
+                    // per 16-bit entry bit 15 := ((register & 31) + width > 32); 0x7FDF = 0x8000 - 33
                     const uint32_t wc = (vi & 0xFFu) * 0x10001u + 0x7FDF7FDFu;
                     lo = (lo & 0x7FFF7FFFu) | (((lo & 0x001F001Fu) + wc) & 0x80008000u);
                     hi = (hi & 0x7FFF7FFFu) | (((hi & 0x001F001Fu) + wc) & 0x80008000u);
@@ -436,17 +432,15 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
     // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
     // (such a candidate does not take part in the walk: it gets its table back without the marks)
-    if (q.flag15) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            if (M->nout[g] < 2) continue;
-            uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
-            for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk_get(t_load<G>(Tt, v), g);
-        }
+    for (int g = 0; g < G; ++g) {
+        if (M->nout[g] < 2) continue;
+        uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
+        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk_get(t_load<G>(Tt, v), g);
     }
     if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
         const uint32_t ov = M->out_v[tid];
-        const uint32_t mark = (q.flag15 && (q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
+        const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
         q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)ov * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)(q.P | mark);
     }
     if (tid < G && k0 + tid < q.K) {
@@ -543,9 +537,9 @@ __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tg
 // occupied bits that a test found.  Toggling returns the old word: occupied and released are both
 // a toggle as long as no collision has been seen (after one, the chunk is recounted exactly
 // anyway).  The common case, no range of the group reaching into the next 32-bit word for any
-// lane, is decided before anything is applied and takes one atomic per event.  F15: the table
-// entries carry that fact in bit 15; otherwise it is worked out from the event's width.
-template <bool WIDE, bool F15>
+// lane, is decided before anything is applied and takes one atomic per event: the table entries
+// carry that fact in bit 15 (very wide ranges are found from the event's width).
+template <bool WIDE>
 __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, uint32_t *s_occ,
                                                 uint32_t lane)
 {
@@ -553,7 +547,7 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
     const uint32_t ez[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
     const uint32_t ey[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
     bool slow;
-    if (F15 && !WIDE) {
+    if (!WIDE) {
         slow = ((t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & 0x8000u) != 0;
     } else {
         const uint4 w4 = lds128_at<96>(ga);
@@ -570,7 +564,7 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const uint32_t tv = t[u];
-            const uint32_t a = occ_addr + (tv & (F15 ? 0x7FE0u : 0xFFE0u)) * 4u;  // word (tv / 32) of this lane's mask
+            const uint32_t a = occ_addr + (tv & 0x7FE0u) * 4u;  // word (tv / 32) of this lane's mask
             const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, ez[u], tv));
             viol |= o & __funnelshift_l(0u, ey[u], tv);
         }
@@ -580,7 +574,7 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
     const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-        const uint32_t tv = F15 ? (t[u] & 0x7FFFu) : t[u];
+        const uint32_t tv = t[u] & 0x7FFFu;
         const uint32_t wl = (u & 1) ? (ew[u >> 1] >> 16) : (ew[u >> 1] & 0xFFFFu);
         if (WIDE && (wl & 0x8000u)) {
             viol |= walk_very_wide(s_occ, lane, tv, wl & 0xFFu, ey[u], ez[u]);
@@ -600,7 +594,7 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
-template <bool WIDE, bool F15>
+template <bool WIDE>
 __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
 {
     extern __shared__ __align__(16) uint32_t wsm[];
@@ -633,7 +627,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
             for (int u = 0; u < 8; ++u) t[u] = tg[(size_t)(x[u] & 0xFFFFu) * 32];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                uint32_t pos = t[u] & q.tmask, left = x[u] >> 16;
+                uint32_t pos = t[u] & 0x7FFFu, left = x[u] >> 16;
                 while (left) {
                     const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
                     const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
@@ -667,10 +661,10 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
             for (uint32_t g = 0; g < ng; g += 2) {
                 const uint32_t ga = ev_addr + g * 112;
                 if (g + 1 < ng) fetch_group(ga + 112, tgb, tb);
-                viol |= apply_group<WIDE, F15>(ga, ta, occ_addr, s_occ, lane);
+                viol |= apply_group<WIDE>(ga, ta, occ_addr, s_occ, lane);
                 if (g + 1 < ng) {
                     if (g + 2 < ng) fetch_group(ga + 224, tgb, ta);
-                    viol |= apply_group<WIDE, F15>(ga + 112, tb, occ_addr, s_occ, lane);
+                    viol |= apply_group<WIDE>(ga + 112, tb, occ_addr, s_occ, lane);
                 }
             }
         }
@@ -811,7 +805,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
         const uint32_t out_v = cs[CS_NOUT] == 1 ? cs[CS_OUTV] : 0xFFFFFFFFu, out_raw = cs[CS_OUTRAW];
         // a candidate with several out-of-file vregs was not walked and keeps its table unmarked
-        const uint32_t tmask = (cs[CS_WALK] & WALK_FULL) ? 0xFFFFu : q.tmask;
+        const uint32_t tmask = (cs[CS_WALK] & WALK_FULL) ? 0xFFFFu : 0x7FFFu;
         __syncthreads();
         if (kind == RC_KIND_BANK && k != have) {
             for (uint32_t v0 = tid; v0 < q.V; v0 += 8 * RC_THREADS) {
@@ -1051,7 +1045,7 @@ static void kt_mark(vl_program *p, cudaStream_t st)
 namespace {
 struct PassPlan {
     Plan pl;
-    uint32_t Wp, ev_cap, walk_smem, rc_smem, flag15;
+    uint32_t Wp, ev_cap, walk_smem, rc_smem;
     uint64_t sub;
 };
 
@@ -1076,18 +1070,18 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + (pp->ev_cap >> 3) * 28)) * 4;
     pp->rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
     if (pp->walk_smem > SM_BYTES || pp->rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    // the walk's table entries keep bit 15 for a mark: every in-file register number must be below 2^15
+    // (the occupancy masks of a register file that large would not fit shared memory anyway)
+    if (p->P + p->wmax > 32768u) return VL_ERR_UNSUPPORTED;
     // the recount work list holds up to RC_PARTS items per chunk and candidate: keep it within 8 Mi items
     const uint64_t sub_cap =
         std::max<uint64_t>(32, ((8ull << 20) / ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) / 32 * 32);
     pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
     cudaError_t e = cudaSuccess;
-    pp->flag15 = p->P + p->wmax <= 32768u ? 1u : 0u;
     if (pp->walk_smem > 48 * 1024) {
         const int sm = (int)pp->walk_smem;
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
     }
     if (e == cudaSuccess && pp->rc_smem > 48 * 1024)
         e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
@@ -1117,7 +1111,6 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.cand = d_cand; tq.K = n; tq.pitch = pitch;
     tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
-    tq.flag15 = pp.flag15;
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
@@ -1144,15 +1137,9 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
         wq.cstate = vs.cstate; wq.anom = vs.anom;
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
-        wq.tmask = pp.flag15 ? 0x7FFFu : 0xFFFFu;
         const dim3 wgrid(p->nItems, ngrp);
-        if (p->wmax > 32) {
-            if (pp.flag15) k_walk<true, true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-            else k_walk<true, false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-        } else {
-            if (pp.flag15) k_walk<false, true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-            else k_walk<false, false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-        }
+        if (p->wmax > 32) k_walk<true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        else k_walk<false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
         g_vl_launches.fetch_add(1);
@@ -1173,7 +1160,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
     rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
     rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
-    rq.racc = vs.racc; rq.status = p->d_status + 1; rq.tmask = pp.flag15 ? 0x7FFFu : 0xFFFFu;
+    rq.racc = vs.racc; rq.status = p->d_status + 1;
     rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out;
     rq.bank_list = p->d_bank_list;
     for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];

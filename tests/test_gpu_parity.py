@@ -161,6 +161,58 @@ def test_options_do_not_change_results(B, oracle_mod, chunk, G, threads):
     gp.close()
 
 
+@pytest.mark.parametrize("P,widths", [(4000, (1, 2, 8)), (5000, (1, 3, 40)), (300, (1, 5, 40, 64)), (97, (1, 2, 33)),
+                                      (1000, (1, 2, 255))])
+def test_large_files_and_very_wide_tuples(B, oracle_mod, P, widths):
+    """Register files of many mask words, tuples wider than one 32-bit mask word, and packed tables
+    whose ranges keep crossing word boundaries."""
+    for seed in range(4):
+        p = H.random_program(9000 + seed, strict=True, reachable=True, max_instrs=50, max_vregs=16, P=P,
+                             widths=widths, B=4)
+        gp, lv = _check_liveness(B, oracle_mod, p)
+        rng = np.random.default_rng(seed)
+        rows = [_garbage_rows(p, 12, seed)]
+        tabs = np.zeros((20, p.n_vregs), dtype=np.int64)
+        for k in range(20):                                # packed tables that tend to straddle mask words
+            base = int(rng.integers(0, 64)) if k % 2 else int(rng.integers(max(1, P - 200), P))
+            pos = base
+            for v in rng.permutation(p.n_vregs):
+                tabs[k, v] = min(pos, 65535)
+                pos += int(p.vreg_width[v]) if k % 4 < 3 else 1
+        rows.append(np.stack([H.row_from_table(p, t) for t in tabs]))
+        rows = np.concatenate(rows)
+        want = oracle_mod.OracleProgram(p).verify(lv, rows)
+        _assert_same(_gpu_verify(B, gp, rows), want, f"P {P} seed {seed}")
+        gp.close()
+
+
+def test_register_file_too_large_is_refused(B):
+    p = H.random_program(1, strict=True, P=40000)
+    gp = B.Program(p)
+    gp.vl_liveness()
+    import torch
+    with pytest.raises(B.VlError) as e:
+        gp.vl_verify(torch.zeros((4, p.pitch), dtype=torch.uint16, device="cuda"))
+    assert e.value.code == B.VL_ERR_UNSUPPORTED
+    gp.close()
+
+
+@pytest.mark.parametrize("lanes,sub", [(1, 64), (2, 32), (3, 96), (4, 32), (4, 4096)])
+def test_passes_over_lanes(B, oracle_mod, lanes, sub):
+    """Many passes spread over the internal streams give the records of a single pass."""
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    rows, _ = synth.candidate_rows(p, 500, 0.3, 11)
+    rows = np.concatenate([rows[:487], _garbage_rows(p, 12, 5)])     # 499 rows: ragged last pass
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    gp.set_option(B.VL_OPT_LANES, lanes)
+    gp.set_option(B.VL_OPT_SUB_BATCH, sub)
+    for _ in range(2):                                               # working sets reused by the next call
+        _assert_same(_gpu_verify(B, gp, rows), want, f"lanes {lanes} sub {sub}")
+    gp.close()
+
+
 def test_batch_call(B, oracle_mod):
     """Workload 4 (256 independent programs): a sample of members through vl_verify_batch."""
     import torch
