@@ -120,7 +120,7 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
             }
             if (many) { p->bank_many = 1; continue; }
             if (n < 2) continue;
-            for (uint32_t k = n; k < 4; ++k) ids[k] = 0;
+            for (uint32_t k = n; k < 4; ++k) ids[k] = ids[0];  // unused slots repeat the first source
             cls[n - 2].push_back(make_uint2(ids[0] | (ids[1] << 16), ids[2] | (ids[3] << 16)));
         }
         std::vector<uint2> all;

@@ -35,6 +35,7 @@ struct TParams {
     const uint32_t *vinfo, *first_def_instr, *op_off;
     const uint2 *bank_list;
     uint32_t bank_seg[4];  // entries with n = 2, 3, 4 distinct sources: [seg[n-2], seg[n-1])
+    uint32_t bank_total;   // distinct sources summed over the listed instructions
     const uint16_t *cand;
     uint64_t K, pitch;
     uint16_t *tg;
@@ -173,6 +174,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     extern __shared__ __align__(16) unsigned char smem[];
     uint16_t *Tt = reinterpret_cast<uint16_t *>(smem);
     unsigned char *region = smem + q.off_region;
+    uint16_t *Hb = reinterpret_cast<uint16_t *>(region);  // [V] after the rows have been streamed: bank nibbles
     TMisc *M = reinterpret_cast<TMisc *>(smem + q.off_misc);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31;
@@ -328,16 +330,29 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         const uint64_t grp = k0 >> 5;
         const uint32_t l0 = (uint32_t)(k0 & 31);
         uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        uint32_t vis_next[8];  // the vreg descriptors of the next round are fetched during the current one
+#pragma unroll
+        for (int u = 0; u < 8; ++u) vis_next[u] = tid + u * NT < q.V ? q.vinfo[tid + u * NT] : 0u;
         for (uint32_t v0 = tid; v0 <= q.V; v0 += 8 * NT) {
             uint32_t vis[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) vis[u] = v0 + u * NT < q.V ? q.vinfo[v0 + u * NT] : 0u;
+            for (int u = 0; u < 8; ++u) {
+                vis[u] = vis_next[u];
+                const uint32_t vn = v0 + 8 * NT + u * NT;
+                vis_next[u] = vn < q.V ? q.vinfo[vn] : 0u;
+            }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const uint32_t v = v0 + u * NT, vi = vis[u];
                 if (v > q.V) break;
                 const uint64_t tt = v < q.V ? t_load<G>(Tt, v) : 0ull;
                 uint32_t lo = (uint32_t)tt, hi = (uint32_t)(tt >> 32);
+                if (q.bank_fast && v < q.V) {  // one-hot bank nibbles of the G candidates
+                    uint32_t h = (1u << (lo & q.Bmask));
+                    if constexpr (G >= 2) h |= 16u << ((lo >> 16) & q.Bmask);
+                    if constexpr (G == 4) h |= (256u << (hi & q.Bmask)) | (4096u << ((hi >> 16) & q.Bmask));
+                    Hb[v] = (uint16_t)h;
+                }
                 {   // bit 15 of an entry handed to the walk marks a range that reaches into the next 32-bit
                     // word of the occupancy mask (every in-file register number is below 2^15):
                     // per 16-bit entry bit 15 := ((register & 31) + width > 32); 0x7FDF = 0x8000 - 33
@@ -370,56 +385,71 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     PT(1);
 
+    __syncthreads();
     PT(2);
-    // ------------------------------- bank tally from T: instructions with 2..4 distinct sources.
+    // ------------------------------- bank tally: instructions with 2..4 distinct sources.
     // Distinct vregs read by one instruction are live together, so a candidate whose walk sees no
-    // collision has them on distinct registers and only the banks need comparing; candidates with
-    // a collision get the general tally in k_recount.
+    // collision has them on distinct registers, and its tally for one instruction is the number of
+    // sources minus the number of banks they touch.  Hb[v] holds, per candidate, the bank of T[v]
+    // as a one-hot nibble: the banks touched are the bits of the OR over the sources (list entries
+    // repeat their first source in unused slots).  The bits are counted with carry-save adders, 8
+    // entries per round.  Candidates with a collision get the general tally in k_recount.
     if (q.bank_fast) {
-        constexpr uint64_t L1 = 0x0001000100010001ull;
-        const uint64_t BM = L1 * q.Bmask;
-        uint64_t acc = 0;
-        auto same = [&](uint64_t x) -> uint64_t { return ((x | (x >> 1)) & L1) ^ L1; };  // per lane: x == 0
-        // four list entries per thread in flight (the lists sit in global memory)
-        for (uint32_t e0 = q.bank_seg[0] + tid; e0 < q.bank_seg[1]; e0 += 4 * NT) {
-            uint2 ids[4];
+        auto csa = [](uint32_t &h, uint32_t &l, uint32_t a, uint32_t b, uint32_t c) {
+            const uint32_t u = a ^ b;
+            h = (a & b) | (u & c);
+            l = u ^ c;
+        };
+        // per nibble of the low 16 bits: its population count, as four byte fields (nibbles 0, 2, 1, 3)
+        auto nibble_counts = [](uint32_t x) -> uint32_t {
+            uint32_t y = (x & 0x0F0Fu) | ((x & 0xF0F0u) << 12);
+            y = y - ((y >> 1) & 0x55555555u);
+            return (y & 0x33333333u) + ((y >> 2) & 0x33333333u);
+        };
+        auto field = [](uint32_t c, int g) -> uint32_t { return (c >> ((g & 1) * 16 + (g >> 1) * 8)) & 0xFFu; };
+        uint32_t ones = 0, twos = 0, fours = 0, acc8 = 0, rounds = 0;
+        uint32_t sum[G];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[1] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
+        for (int g = 0; g < G; ++g) sum[g] = 0;
+        const uint32_t n_ent = q.bank_seg[3];
+        uint2 ids_next[8];  // list entries of the next round are fetched during the current one
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (e0 + u * NT >= q.bank_seg[1]) break;
-                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16);
-                acc += same((a ^ b) & BM);
+        for (int u = 0; u < 8; ++u) ids_next[u] = tid + u * NT < n_ent ? q.bank_list[tid + u * NT] : make_uint2(0, 0);
+        for (uint32_t e0 = tid; e0 < n_ent; e0 += 8 * NT) {
+            uint2 ids[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                ids[u] = ids_next[u];
+                const uint32_t en = e0 + 8 * NT + u * NT;
+                ids_next[u] = en < n_ent ? q.bank_list[en] : make_uint2(0, 0);
+            }
+            uint32_t x[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t o = (uint32_t)Hb[ids[u].x & 0xFFFFu] | Hb[ids[u].x >> 16] | Hb[ids[u].y & 0xFFFFu] |
+                                   Hb[ids[u].y >> 16];
+                x[u] = e0 + u * NT < n_ent ? o : 0u;
+            }
+            uint32_t ta, tb, fa, fb, eights;
+            csa(ta, ones, ones, x[0], x[1]);
+            csa(tb, ones, ones, x[2], x[3]);
+            csa(fa, twos, twos, ta, tb);
+            csa(ta, ones, ones, x[4], x[5]);
+            csa(tb, ones, ones, x[6], x[7]);
+            csa(fb, twos, twos, ta, tb);
+            csa(eights, fours, fours, fa, fb);
+            acc8 += nibble_counts(eights);
+            if (++rounds == 32) {  // the byte fields of acc8 hold at most 4 per round
+#pragma unroll
+                for (int g = 0; g < G; ++g) sum[g] += 8u * field(acc8, g);
+                acc8 = 0;
+                rounds = 0;
             }
         }
-        for (uint32_t e0 = q.bank_seg[1] + tid; e0 < q.bank_seg[2]; e0 += 4 * NT) {
-            uint2 ids[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[2] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (e0 + u * NT >= q.bank_seg[2]) break;
-                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16),
-                               c = t_load<G>(Tt, ids[u].y & 0xFFFFu);
-                acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM));
-            }
-        }
-        for (uint32_t e0 = q.bank_seg[2] + tid; e0 < q.bank_seg[3]; e0 += 4 * NT) {
-            uint2 ids[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) ids[u] = e0 + u * NT < q.bank_seg[3] ? q.bank_list[e0 + u * NT] : make_uint2(0, 0);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (e0 + u * NT >= q.bank_seg[3]) break;
-                const uint64_t a = t_load<G>(Tt, ids[u].x & 0xFFFFu), b = t_load<G>(Tt, ids[u].x >> 16),
-                               c = t_load<G>(Tt, ids[u].y & 0xFFFFu), d = t_load<G>(Tt, ids[u].y >> 16);
-                acc += same((a ^ b) & BM) + (same((c ^ a) & BM) | same((c ^ b) & BM)) +
-                       (same((d ^ a) & BM) | same((d ^ b) & BM) | same((d ^ c) & BM));
-            }
-        }
+        const uint32_t c4 = nibble_counts(fours), c2 = nibble_counts(twos), c1 = nibble_counts(ones);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-            uint32_t x = pk_get(acc, g);
+            uint32_t x = sum[g] + 8u * field(acc8, g) + 4u * field(c4, g) + 2u * field(c2, g) + field(c1, g);
 #pragma unroll
             for (int d = 16; d; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
             if (lane == 0 && x) atomicAdd(&M->bank[g], x);
@@ -458,7 +488,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         uint32_t *cs = q.cstate + (k0 + g) * 8;
         cs[CS_FLAGS] = M->flags[g];
         cs[CS_FIRST] = min(first, M->minR[g]);
-        cs[CS_BANK] = M->bank[g];
+        cs[CS_BANK] = q.bank_fast ? q.bank_total - M->bank[g] : 0u;
         cs[CS_NOUT] = M->nout[g];
         cs[CS_OUTV] = M->out_v[g];
         cs[CS_OUTRAW] = M->out_raw[g];
@@ -693,8 +723,8 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
 // every chunk that needs an exact recount is cut into RC_PARTS pieces, the general bank tally into
 // RC_BANK_PARTS slices; racc[k][3] counts the items pending.  An item is (candidate, code) with
 // code = kind << 30 | piece << 24 | chunk.
-#define RC_PARTS 4
-#define RC_BANK_PARTS 2
+#define RC_PARTS 2
+#define RC_BANK_PARTS 4
 #define RC_KIND_ALL 0u     // every definition of the piece
 #define RC_KIND_ELIDED 1u  // only the definitions the walk skipped
 #define RC_KIND_BANK 2u
@@ -774,21 +804,22 @@ __global__ void k_finish(uint64_t K, uint32_t nC, uint32_t AW, int list_all, con
 
 // =========================================================================== k_recount
 // Exact answers for the listed work items; thread blocks loop over the list.  A chunk item recounts
-// the overlaps of one piece of a chunk from the live-after lists: the warps share the piece's
-// instructions, the lanes of a warp fetch the bookkeeping of 32 instructions at a time, and the
-// candidate's registers come straight from its table column in global memory (the live-after sets
-// of neighbouring instructions are nearly the same, so these gathers hit in L1).  A bank item
-// copies the whole column to shared memory and does a slice of the general bank tally (distinct
-// registers rather than distinct vregs).  Results are added to the candidate's accumulators; the
-// item that finishes last writes the verdict.
+// the overlaps of one piece of a chunk from the live-after lists (the warps share the piece's
+// instructions; the lanes of a warp fetch the bookkeeping of 32 instructions at a time); a bank
+// item does a slice of the general bank tally (distinct registers rather than distinct vregs).
+// The candidate's register and the width of a vreg are fetched from global memory the first time
+// an item needs them and kept in a shared-memory cache (CACHE; one word per vreg, valid bit 31):
+// the live-after sets of neighbouring instructions are nearly the same, so a piece touches a few
+// hundred vregs, not the whole table column.  Results are added to the candidate's accumulators;
+// the item that finishes last writes the verdict.
+template <bool CACHE>
 __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 {
-    extern __shared__ __align__(16) uint16_t T[];  // [V + 8] registers of one candidate (bank items)
+    extern __shared__ __align__(16) uint32_t Cv[];  // [V] register | width << 16 | valid << 31
     __shared__ uint32_t s_pairs, s_mind, s_bank;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr uint32_t NW = RC_THREADS / 32;
     const uint32_t nitems = q.work[0];
-    uint64_t have = ~0ull;  // candidate whose column is in shared memory
 #ifdef VL_PHASE_TIMERS
     const long long rc_t0 = clock64();
     if (tid == 0 && blockIdx.x == 0) atomicAdd(q.status + 8, nitems);
@@ -797,9 +828,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         const uint64_t k = q.work[2 + 2 * it];
         const uint32_t code = q.work[3 + 2 * it];
         const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
-#ifdef VL_PHASE_TIMERS
-        if (tid == 0) atomicAdd(q.status + 11 + kind, 1u);
-#endif
         const uint32_t *cs = q.cstate + k * 8;
         const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
         // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
@@ -807,26 +835,23 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         // a candidate with several out-of-file vregs was not walked and keeps its table unmarked
         const uint32_t tmask = (cs[CS_WALK] & WALK_FULL) ? 0xFFFFu : 0x7FFFu;
         __syncthreads();
-        if (kind == RC_KIND_BANK && k != have) {
-            for (uint32_t v0 = tid; v0 < q.V; v0 += 8 * RC_THREADS) {
-                uint16_t t[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t v = v0 + u * RC_THREADS;
-                    t[u] = v < q.V ? tg[(size_t)v * 32] : (uint16_t)0;
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t v = v0 + u * RC_THREADS;
-                    if (v < q.V) T[v] = v == out_v ? (uint16_t)out_raw : (uint16_t)(t[u] & tmask);
-                }
-            }
-            have = k;
-        }
+        if (CACHE)
+            for (uint32_t v = tid; v < q.V; v += RC_THREADS) Cv[v] = 0;
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
-        auto reg_of = [&](uint32_t v) -> uint32_t {
-            return v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * 32] & tmask);
+        // register (low 16 bits) and width (bits 16..23) of vreg v for this candidate
+        auto fetch = [&](uint32_t v) -> uint32_t {
+            const uint32_t r = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * 32] & tmask);
+            return r | ((q.vinfo[v] & 0xFFu) << 16);
+        };
+        auto reg_w = [&](uint32_t v) -> uint32_t {
+            if (!CACHE) return fetch(v);
+            uint32_t x = Cv[v];
+            if (!(x >> 31)) {
+                x = fetch(v) | 0x80000000u;
+                Cv[v] = x;  // several threads may store the same word
+            }
+            return x;
         };
         if (kind != RC_KIND_BANK) {
             const bool elided_only = kind == RC_KIND_ELIDED;
@@ -841,39 +866,58 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 if (my_i < i_hi && !(elided_only && !q.iflags[my_i])) {
                     m_o0 = q.op_off[my_i]; m_nd = q.ndefs[my_i]; m_l0 = q.lo_off[my_i]; m_l1 = q.lo_off[my_i + 1];
                 }
+                // first defined vreg of each instruction, fetched by the lane that holds its bookkeeping
+                uint32_t m_v0 = 0;
+                if (m_nd) m_v0 = q.op_vreg[m_o0];
                 uint32_t todo = __ballot_sync(0xffffffffu, m_nd != 0);
+                // the first 256 entries of the next instruction's live-after list are fetched while the
+                // current instruction is recounted
+                uint32_t us_nx[8];
+                auto fetch_list = [&](int src) {
+                    const uint32_t l0 = __shfl_sync(0xffffffffu, m_l0, src), l1 = __shfl_sync(0xffffffffu, m_l1, src);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t e = l0 + u * 32 + lane;
+                        us_nx[u] = e < l1 ? q.lo[e] : 0xFFFFFFFFu;
+                    }
+                };
+                if (todo) fetch_list(__ffs(todo) - 1);
                 while (todo) {
                     const int src = __ffs(todo) - 1;
                     todo &= todo - 1;
+                    uint32_t us0[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) us0[u] = us_nx[u];
+                    if (todo) fetch_list(__ffs(todo) - 1);
                     const uint32_t i = ib + (uint32_t)src * NW;
                     const uint32_t o0 = __shfl_sync(0xffffffffu, m_o0, src), nd = __shfl_sync(0xffffffffu, m_nd, src);
                     const uint32_t l0 = __shfl_sync(0xffffffffu, m_l0, src), l1 = __shfl_sync(0xffffffffu, m_l1, src);
+                    const uint32_t v0 = __shfl_sync(0xffffffffu, m_v0, src);
                     for (uint32_t d = o0; d < o0 + nd; ++d) {
                         if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
-                        const uint32_t v = q.op_vreg[d];
-                        const uint32_t s = reg_of(v), w = q.vinfo[v] & 0xFFu;
+                        const uint32_t v = d == o0 ? v0 : q.op_vreg[d];
+                        const uint32_t sw = reg_w(v);
+                        const uint32_t s = sw & 0xFFFFu, w = (sw >> 16) & 0xFFu;
                         uint32_t cnt = 0;
                         for (uint32_t e0 = l0; e0 < l1; e0 += 256) {  // 8 list entries per lane in flight
-                            uint32_t us[8], ts[8], ws[8];
+                            uint32_t us[8], xs[8];
 #pragma unroll
                             for (int u = 0; u < 8; ++u) {
                                 const uint32_t e = e0 + u * 32 + lane;
-                                us[u] = e < l1 ? q.lo[e] : v;
+                                us[u] = e0 == l0 ? us0[u] : (e < l1 ? q.lo[e] : 0xFFFFFFFFu);
+                                if (us[u] == 0xFFFFFFFFu) us[u] = v;
                             }
 #pragma unroll
-                            for (int u = 0; u < 8; ++u) {
-                                ts[u] = reg_of(us[u]);
-                                ws[u] = q.vinfo[us[u]] & 0xFFu;
-                            }
+                            for (int u = 0; u < 8; ++u) xs[u] = reg_w(us[u]);
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
-                                if (us[u] != v && ranges_overlap(s, w, ts[u], ws[u])) ++cnt;
+                                if (us[u] != v && ranges_overlap(s, w, xs[u] & 0xFFFFu, (xs[u] >> 16) & 0xFFu)) ++cnt;
                         }
                         // co-defined vregs that are not live after the instruction
                         for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
                             if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
-                            const uint32_t u = q.op_vreg[d2];
-                            if (ranges_overlap(s, w, reg_of(u), q.vinfo[u] & 0xFFu)) ++cnt;
+                            const uint32_t x = reg_w(q.op_vreg[d2]);
+                            if (ranges_overlap(s, w, x & 0xFFFFu, (x >> 16) & 0xFFu)) ++cnt;
                         }
 #pragma unroll
                         for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
@@ -904,7 +948,8 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                         const uint2 ids = idv[u];
                         const uint32_t n = e < q.bank_seg[1] ? 2u : (e < q.bank_seg[2] ? 3u : 4u);
                         uint32_t x[4];
-                        x[0] = T[ids.x & 0xFFFFu]; x[1] = T[ids.x >> 16]; x[2] = T[ids.y & 0xFFFFu]; x[3] = T[ids.y >> 16];
+                        x[0] = reg_w(ids.x & 0xFFFFu) & 0xFFFFu; x[1] = reg_w(ids.x >> 16) & 0xFFFFu;
+                        x[2] = reg_w(ids.y & 0xFFFFu) & 0xFFFFu; x[3] = reg_w(ids.y >> 16) & 0xFFFFu;
 #pragma unroll
                         for (uint32_t a = 1; a < 4; ++a) {
                             if (a >= n) break;
@@ -924,10 +969,10 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 for (uint32_t i = i_lo + tid; i < i_hi; i += RC_THREADS) {
                     const uint32_t u0 = q.op_off[i] + q.ndefs[i], u1 = q.op_off[i + 1];
                     for (uint32_t a = u0 + 1; a < u1; ++a) {
-                        const uint32_t xa = T[q.op_vreg[a]];
+                        const uint32_t xa = reg_w(q.op_vreg[a]) & 0xFFFFu;
                         bool seen_value = false, seen_bank = false;
                         for (uint32_t bb = u0; bb < a; ++bb) {
-                            const uint32_t xb = T[q.op_vreg[bb]];
+                            const uint32_t xb = reg_w(q.op_vreg[bb]) & 0xFFFFu;
                             seen_value |= (xb == xa);
                             seen_bank |= (xb % q.B == xa % q.B);
                         }
@@ -985,11 +1030,12 @@ Plan make_plan(const vl_program *p, uint32_t G, uint32_t NT, uint32_t budget)
     const uint64_t stage = (uint64_t)NT * 8 * 2 * G;
     const uint64_t tbytes = align16((uint64_t)(p->V + 1) * G * 2);
     const uint64_t misc = align16(sizeof(TMisc));
+    const uint64_t hbytes = align16((uint64_t)(p->V + 1) * 2);  // the bank nibbles reuse the copy ring
     pl.ok = false;
-    if (tbytes + misc + 2 * stage > budget) return pl;
+    if (tbytes + misc + std::max(2 * stage, hbytes) > budget) return pl;
     pl.NS = (uint32_t)std::min<uint64_t>(MAX_STAGES, (budget - tbytes - misc) / stage);
     pl.off_region = (uint32_t)tbytes;
-    pl.off_misc = (uint32_t)(tbytes + pl.NS * stage);
+    pl.off_misc = (uint32_t)(tbytes + std::max(pl.NS * stage, hbytes));
     pl.smem = pl.off_misc + (uint32_t)misc;
     pl.ok = true;
     return pl;
@@ -1068,8 +1114,10 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->Wp = (p->P + p->wmax + 31) / 32;
     pp->ev_cap = 256;
     pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + (pp->ev_cap >> 3) * 28)) * 4;
-    pp->rc_smem = (uint32_t)align16((uint64_t)(p->V + 8) * 2);
-    if (pp->walk_smem > SM_BYTES || pp->rc_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    if (pp->walk_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    // the recount keeps one cache word per vreg in shared memory when that leaves room for several
+    // thread blocks per SM, else it fetches from global memory every time
+    pp->rc_smem = (uint64_t)p->V * 4 <= 72 * 1024 ? (uint32_t)align16((uint64_t)(p->V + 4) * 4) : 0u;
     // the walk's table entries keep bit 15 for a mark: every in-file register number must be below 2^15
     // (the occupancy masks of a register file that large would not fit shared memory anyway)
     if (p->P + p->wmax > 32768u) return VL_ERR_UNSUPPORTED;
@@ -1084,7 +1132,7 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
     }
     if (e == cudaSuccess && pp->rc_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_recount, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
+        e = cudaFuncSetAttribute(k_recount<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
     return VL_OK;
 }
@@ -1108,6 +1156,8 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.first_def_instr = p->d_first_def_instr; tq.op_off = p->d_op_off;
     tq.bank_list = p->d_bank_list;
     for (int j = 0; j < 4; ++j) tq.bank_seg[j] = p->bank_seg[j];
+    tq.bank_total = 2 * (p->bank_seg[1] - p->bank_seg[0]) + 3 * (p->bank_seg[2] - p->bank_seg[1]) +
+                    4 * (p->bank_seg[3] - p->bank_seg[2]);
     tq.cand = d_cand; tq.K = n; tq.pitch = pitch;
     tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
@@ -1166,7 +1216,8 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
     const uint32_t rgrid = 148 * 6;
     kt_mark(p, st);
-    k_recount<<<rgrid, RC_THREADS, pp.rc_smem, st>>>(rq);
+    if (pp.rc_smem) k_recount<true><<<rgrid, RC_THREADS, pp.rc_smem, st>>>(rq);
+    else k_recount<false><<<rgrid, RC_THREADS, 0, st>>>(rq);
     kt_mark(p, st);
     e = cudaGetLastError();
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
