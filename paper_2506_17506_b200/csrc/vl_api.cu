@@ -147,13 +147,11 @@ void vl_free_liveness(vl_program *p)
     // everything below lives in the handle's pools, which are rewound, not freed
     p->live_arena.reset();
     p->tmp_arena.reset();
-    p->d_chunk_i0 = p->d_chunk_i1 = p->d_chunk_blk = p->d_blk_chunk_off = nullptr;
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
     p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_iflags = nullptr;
     p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
-    p->d_item_blk = p->d_item_c0 = p->d_item_c1 = nullptr;
     p->live_ok = false;
     p->lo_len = 0;
 }
@@ -165,6 +163,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     vl_free_liveness(p);
     p->live_arena.release();
     p->tmp_arena.release();
+    p->layout_arena.release();
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);

@@ -76,15 +76,19 @@ struct vl_program {
     uint32_t chunk_instrs = 128;
     uint32_t group_opt = 0;
 
-    // chunks: every chunk lies inside one block
-    uint32_t nC = 0;
-    std::vector<uint32_t> h_chunk_i0, h_chunk_i1, h_chunk_blk, h_blk_chunk_off;
+    // chunks: every chunk lies inside one block; pieces: every piece lies inside one chunk
+    uint32_t nC = 0, nP = 0;
+    uint32_t layout_chunk_instrs = 0;  // chunk size the device copies of the layout were made for (0: none)
     std::vector<uint32_t> h_blk_off, h_op_off;
+    // list lengths of the last liveness run with this layout: the next run allocates from them
+    bool sizes_known = false;
+    uint64_t known_lo_len = 0, known_steps = 0, known_thn = 0;
 
     // device copies of the program
     uint32_t *d_blk_off = nullptr, *d_succ_off = nullptr, *d_succ = nullptr, *d_op_off = nullptr, *d_op_vreg = nullptr;
     uint8_t *d_ndefs = nullptr, *d_width = nullptr;
     uint32_t *d_chunk_i0 = nullptr, *d_chunk_i1 = nullptr, *d_chunk_blk = nullptr, *d_blk_chunk_off = nullptr;
+    uint32_t *d_piece_i0 = nullptr, *d_piece_i1 = nullptr, *d_piece_chunk = nullptr, *d_chunk_piece_off = nullptr;
 
     // liveness results
     uint32_t *d_blk_in = nullptr, *d_blk_out = nullptr, *d_lo_off = nullptr, *d_lo = nullptr;
@@ -113,6 +117,7 @@ struct vl_program {
     int use_th = 0;
 
     VlArena live_arena, tmp_arena;  // liveness results and tables / liveness working sets
+    VlArena layout_arena;           // chunks, pieces, walk items
     uint32_t *d_status = nullptr;  // [16] device status words
     int last_cuda_error = 0;
     bool live_ok = false;

@@ -1,16 +1,19 @@
 // Liveness on the GPU and the per-program tables the verify kernels consume.
 //
-// Pipeline (all kernels on the caller's stream):
-//   chunk read/write sets -> block sets -> fixed point over blocks (one thread per
-//   bitset word) -> live set at every chunk boundary -> backward walk of every chunk
-//   (count, then fill) giving the per-instruction live-after lists in CSR form and the
-//   per-operand flags -> operand metadata, walk events, through-sets.
+// Pipeline (all kernels on the caller's stream).  Every block is cut into chunks (the unit of the
+// verify walk) and every chunk into pieces of at most PIECE_INSTRS instructions (the unit of the
+// backward instruction walk here, so that a few thousand warps share it):
+//   piece read/write sets -> chunk sets -> block sets -> fixed point over blocks (one thread per
+//   bitset word) -> live set at every chunk boundary -> at every piece boundary -> backward walk
+//   of every piece (count, then fill) giving the per-instruction live-after lists in CSR form and
+//   the per-operand flags -> operand metadata, walk events, through-sets.
 #include <algorithm>
 #include <vector>
 
 #include "vl_internal.cuh"
 
 #define NT 128  // threads per block in every kernel of this file
+#define PIECE_INSTRS 16
 
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ bool bit_get(const uint32_t *s, uint32_t v) { return (s[v >> 5] >> (v & 31)) & 1u; }
@@ -68,7 +71,7 @@ __device__ void compact_bits(const uint32_t *words, uint32_t nwords, uint32_t *s
 }
 
 // ------------------------------------------------------------------------- kernels
-// Per chunk: use = vregs read before any write inside the chunk, def = vregs written.
+// Per span of instructions (a piece): use = vregs read before any write inside the span, def = vregs written.
 __global__ void k_chunk_sets(const uint32_t *__restrict__ chunk_i0, const uint32_t *__restrict__ chunk_i1,
                              const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
                              const uint32_t *__restrict__ op_vreg, uint32_t Wv, uint32_t *chunk_use,
@@ -96,7 +99,7 @@ __global__ void k_chunk_sets(const uint32_t *__restrict__ chunk_i0, const uint32
     }
 }
 
-// Per block: compose the chunk sets in order.
+// Per parent (a block over its chunks, a chunk over its pieces): compose the children's sets in order.
 __global__ void k_block_sets(const uint32_t *__restrict__ blk_chunk_off, uint32_t Wv,
                              const uint32_t *__restrict__ chunk_use, const uint32_t *__restrict__ chunk_def,
                              uint32_t *blk_use, uint32_t *blk_def)
@@ -104,6 +107,7 @@ __global__ void k_block_sets(const uint32_t *__restrict__ blk_chunk_off, uint32_
     const uint32_t b = blockIdx.x;
     for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
         uint32_t u = 0, d = 0;
+#pragma unroll 8
         for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) {
             u |= chunk_use[(size_t)c * Wv + w] & ~d;
             d |= chunk_def[(size_t)c * Wv + w];
@@ -139,37 +143,41 @@ __global__ void k_fixed_point(uint32_t nB, uint32_t Wv, const uint32_t *__restri
     if (live_in[w] != 0) atomicOr(status, ST_NOT_STRICT);  // block 0 is the entry
 }
 
-// Live set after the last instruction of every chunk (chunk_end) and before its first (chunk_entry).
+// Live set after the last instruction of every child (chunk_end) and before its first (chunk_entry,
+// may be null), walking a parent's children backwards from the parent's live-out set: chunks of a
+// block, or pieces of a chunk.
 __global__ void k_chunk_boundaries(const uint32_t *__restrict__ blk_chunk_off, uint32_t Wv,
                                    const uint32_t *__restrict__ live_out, const uint32_t *__restrict__ chunk_use,
                                    const uint32_t *__restrict__ chunk_def, uint32_t *chunk_end, uint32_t *chunk_entry)
 {
     const uint32_t b = blockIdx.x;
+    const uint32_t c_lo = blk_chunk_off[b], c_hi = blk_chunk_off[b + 1];
     for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
         uint32_t live = live_out[(size_t)b * Wv + w];
-        for (uint32_t c = blk_chunk_off[b + 1]; c-- > blk_chunk_off[b];) {
+#pragma unroll 8
+        for (uint32_t c = c_hi; c-- > c_lo;) {
             chunk_end[(size_t)c * Wv + w] = live;
             live = chunk_use[(size_t)c * Wv + w] | (live & ~chunk_def[(size_t)c * Wv + w]);
-            chunk_entry[(size_t)c * Wv + w] = live;
+            if (chunk_entry) chunk_entry[(size_t)c * Wv + w] = live;
         }
     }
 }
 
-// Backward walk of one chunk by one warp.  FILL = false: list sizes, per-operand flags, walk-event
+// Backward walk of one piece by one warp.  FILL = false: list sizes, per-operand flags, walk-event
 // counts, and the set of vregs whose occupancy changes inside the chunk.  FILL = true: the lists.
 // The chunk's slice of the operand arrays is staged in shared memory when it fits (WALK_CAP_I
 // instructions, WALK_CAP_O operands); lane 0 does the per-instruction bookkeeping, all lanes the
 // population count / compaction of the live bitset.
-#define WALK_CAP_I 256
-#define WALK_CAP_O 2048
-#define WALK_CAP_L 1024
+#define WALK_CAP_I 32
+#define WALK_CAP_O 256
 template <bool FILL>
 __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ chunk_i0,
                                                    const uint32_t *__restrict__ chunk_i1,
                                                    const uint32_t *__restrict__ op_off, const uint8_t *__restrict__ ndefs,
                                                    const uint32_t *__restrict__ op_vreg, uint32_t Wv,
                                                    const uint32_t *__restrict__ chunk_end, uint32_t *lo_cnt,
-                                                   uint32_t *ev_cnt, uint8_t *opflags, uint32_t *chunk_touch,
+                                                   uint32_t *ev_cnt, uint8_t *opflags,
+                                                   const uint32_t *__restrict__ piece_chunk, uint32_t *chunk_touch,
                                                    const uint32_t *__restrict__ lo_off, uint32_t *lo)
 {
     extern __shared__ uint32_t sm[];
@@ -177,8 +185,7 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
     uint32_t *s_off = sm + 2 * Wv;                 // [WALK_CAP_I + 1]
     uint32_t *s_lo = s_off + WALK_CAP_I + 1;       // [WALK_CAP_I] list offsets (FILL)
     uint32_t *s_ops = s_lo + WALK_CAP_I;           // [WALK_CAP_O]
-    uint32_t *s_list = s_ops + WALK_CAP_O;         // [WALK_CAP_L] one live-after list (FILL)
-    uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_list + WALK_CAP_L);  // [WALK_CAP_I]
+    uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_ops + WALK_CAP_O);  // [WALK_CAP_I]
     const uint32_t c = blockIdx.x, lane = threadIdx.x;
     const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
     for (uint32_t w = lane; w < Wv; w += 32) {
@@ -259,8 +266,11 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
         }
         __syncwarp();
     }
-    if (!FILL)
-        for (uint32_t w = lane; w < Wv; w += 32) chunk_touch[(size_t)c * Wv + w] = s_touch[w];
+    if (!FILL) {  // the vregs whose occupancy changes somewhere in the chunk this piece belongs to
+        const size_t row = (size_t)piece_chunk[c] * Wv;
+        for (uint32_t w = lane; w < Wv; w += 32)
+            if (s_touch[w]) atomicOr(&chunk_touch[row + w], s_touch[w]);
+    }
 }
 
 // Exclusive scan of a u32 array by one block of 1024 threads, 4 items per thread and round;
@@ -321,6 +331,7 @@ __global__ void k_block_through(const uint32_t *__restrict__ blk_chunk_off, uint
     const uint32_t b = blockIdx.x;
     for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
         uint32_t t = 0;
+#pragma unroll 8
         for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) t |= chunk_touch[(size_t)c * Wv + w];
         blk_th[(size_t)b * Wv + w] = use_th ? (live_in[(size_t)b * Wv + w] & ~t) : 0u;
     }
@@ -519,25 +530,52 @@ __global__ void k_fill_through(uint32_t Wv, const uint32_t *__restrict__ blk_th,
                  [&](uint32_t rank, uint32_t v) { th[base + rank] = v | ((uint32_t)width[v] << 16); });
 }
 
+// First walk event of every chunk (each chunk padded to a multiple of 8 events), first through-set
+// entry of every block, and both totals: totals[2] = events with padding, totals[3] = through entries.
+// One thread block; the arrays are short (chunks, blocks).
+__global__ void k_offsets(uint32_t nC, uint32_t nB, const uint32_t *__restrict__ cev, const uint32_t *__restrict__ th_cnt,
+                          uint32_t *cev_off, uint32_t *th_off, unsigned long long *totals)
+{
+    __shared__ uint32_t s_scan[34];
+    __shared__ unsigned long long s_carry;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int which = 0; which < 2; ++which) {
+        const uint32_t n = which == 0 ? nC : nB;
+        const uint32_t *src = which == 0 ? cev : th_cnt;
+        uint32_t *dst = which == 0 ? cev_off : th_off;
+        for (uint32_t base = 0; base < n; base += NT) {
+            const uint32_t i = base + threadIdx.x;
+            uint32_t x = i < n ? src[i] : 0u;
+            if (which == 0) x = (x + 7u) / 8u * 8u;
+            uint32_t total;
+            const uint32_t ex = block_excl_scan(x, s_scan, &total);
+            const unsigned long long carry = s_carry;
+            if (i < n) dst[i] = (uint32_t)(carry + ex);
+            __syncthreads();
+            if (threadIdx.x == 0) s_carry = carry + total;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            dst[n] = s_carry > 0xFFFFFFF0ull ? 0xFFFFFFF0u : (uint32_t)s_carry;
+            totals[2 + which] = s_carry;
+            s_carry = 0;
+        }
+        __syncthreads();
+    }
+}
+
 // --------------------------------------------------------------------------- host
 namespace {
 template <typename T>
-cudaError_t pool_get(VlArena &arena, T **out, size_t n, int fill, bool do_fill, cudaStream_t st)
+cudaError_t pool_get(VlArena &arena, T **out, size_t n)
 {
-    cudaError_t e = arena.alloc((void **)out, std::max<size_t>(n, 1) * sizeof(T));
-    if (e != cudaSuccess || !do_fill) return e;
-    return cudaMemsetAsync(*out, fill, std::max<size_t>(n, 1) * sizeof(T) + 64, st);
+    return arena.alloc((void **)out, std::max<size_t>(n, 1) * sizeof(T) + 64);
 }
-struct TmpPool {
-    vl_program *p;
-    template <typename T>
-    cudaError_t get(T **out, size_t n, bool zero, cudaStream_t st)
-    {
-        return pool_get(p->tmp_arena, out, n, 0, zero, st);
-    }
-};
 }  // namespace
-#define keep(out, n, fill, st) pool_get(p->live_arena, out, n, fill, true, st)
+#define KEEP(out, n) VL_CUDA(p, pool_get(p->live_arena, out, n))
+#define TMP(out, n) VL_CUDA(p, pool_get(p->tmp_arena, out, n))
+#define LAYOUT(out, n) VL_CUDA(p, pool_get(p->layout_arena, out, n))
 
 #define LAUNCH(kernel, grid, smem, st, ...)                          \
     do {                                                             \
@@ -547,152 +585,172 @@ struct TmpPool {
         }                                                            \
     } while (0)
 
-int vl_liveness_impl(vl_program *p, cudaStream_t st)
+// Chunks, pieces and walk items depend on the program and on the chunk size only: they are laid
+// out (and uploaded) when the chunk size changes, not on every call.
+static int vl_layout(vl_program *p, cudaStream_t st)
 {
-    vl_free_liveness(p);
-    const uint32_t nB = p->nB, nI = p->nI, V = p->V, nO = p->nO, Wv = p->Wv;
-
-    // ---- chunks: split every block into pieces of about chunk_instrs instructions
-    p->h_chunk_i0.clear(); p->h_chunk_i1.clear(); p->h_chunk_blk.clear();
-    p->h_blk_chunk_off.assign(nB + 1, 0);
+    if (p->layout_chunk_instrs == p->chunk_instrs) return VL_OK;
+    const uint32_t nB = p->nB;
+    p->layout_chunk_instrs = 0;
+    p->sizes_known = false;
+    VL_CUDA(p, cudaStreamSynchronize(st));  // earlier work on the stream may still read the old layout
+    p->layout_arena.reset();
+    std::vector<uint32_t> c_i0, c_i1, c_blk, blk_c_off(nB + 1, 0), p_i0, p_i1, p_chunk, c_p_off;
     for (uint32_t b = 0; b < nB; ++b) {
         const uint64_t s = p->h_blk_off[b], n = p->h_blk_off[b + 1] - s;
         const uint64_t nc = (n + p->chunk_instrs - 1) / p->chunk_instrs;
         for (uint64_t j = 0; j < nc; ++j) {
-            p->h_chunk_i0.push_back((uint32_t)(s + j * n / nc));
-            p->h_chunk_i1.push_back((uint32_t)(s + (j + 1) * n / nc));
-            p->h_chunk_blk.push_back(b);
+            const uint32_t i0 = (uint32_t)(s + j * n / nc), i1 = (uint32_t)(s + (j + 1) * n / nc);
+            c_p_off.push_back((uint32_t)p_i0.size());
+            for (uint32_t q0 = i0; q0 < i1; q0 += PIECE_INSTRS) {
+                p_i0.push_back(q0);
+                p_i1.push_back(std::min(i1, q0 + PIECE_INSTRS));
+                p_chunk.push_back((uint32_t)c_i0.size());
+            }
+            c_i0.push_back(i0);
+            c_i1.push_back(i1);
+            c_blk.push_back(b);
         }
-        p->h_blk_chunk_off[b + 1] = (uint32_t)p->h_chunk_i0.size();
+        blk_c_off[b + 1] = (uint32_t)c_i0.size();
     }
-    const uint32_t nC = p->nC = (uint32_t)p->h_chunk_i0.size();
-
+    c_p_off.push_back((uint32_t)p_i0.size());
+    const uint32_t nC = p->nC = (uint32_t)c_i0.size();
+    p->nP = (uint32_t)p_i0.size();
+    // walk work items: runs of at most 16 chunks of one block
+    std::vector<uint32_t> it_blk, it_c0, it_c1;
+    for (uint32_t b = 0; b < nB; ++b)
+        for (uint32_t c = blk_c_off[b]; c < blk_c_off[b + 1]; c += 16) {
+            it_blk.push_back(b);
+            it_c0.push_back(c);
+            it_c1.push_back(std::min(c + 16, blk_c_off[b + 1]));
+        }
+    p->nItems = (uint32_t)it_blk.size();
+    auto up = [&](uint32_t **dst, const std::vector<uint32_t> &v) -> int {
+        LAYOUT(dst, v.size());
+        if (!v.empty()) VL_CUDA(p, cudaMemcpy(*dst, v.data(), v.size() * 4, cudaMemcpyHostToDevice));
+        return VL_OK;
+    };
+    int rc;
+    if ((rc = up(&p->d_chunk_i0, c_i0)) || (rc = up(&p->d_chunk_i1, c_i1)) || (rc = up(&p->d_chunk_blk, c_blk)) ||
+        (rc = up(&p->d_blk_chunk_off, blk_c_off)) || (rc = up(&p->d_piece_i0, p_i0)) || (rc = up(&p->d_piece_i1, p_i1)) ||
+        (rc = up(&p->d_piece_chunk, p_chunk)) || (rc = up(&p->d_chunk_piece_off, c_p_off)) ||
+        (rc = up(&p->d_item_blk, it_blk)) || (rc = up(&p->d_item_c0, it_c0)) || (rc = up(&p->d_item_c1, it_c1)))
+        return rc;
     const uint32_t Wp = (p->P + p->wmax + 31) / 32 + 1;
     p->use_th = (nB <= 32 && (uint64_t)nB * VL_MAX_GROUP * Wp * 4 <= 24 * 1024) ? 1 : 0;
+    p->layout_chunk_instrs = p->chunk_instrs;
+    (void)nC;
+    return VL_OK;
+}
+
+int vl_liveness_impl(vl_program *p, cudaStream_t st)
+{
+    vl_free_liveness(p);
+    int rc = vl_layout(p, st);
+    if (rc != VL_OK) return rc;
+    const uint32_t nB = p->nB, nI = p->nI, V = p->V, nO = p->nO, Wv = p->Wv, nC = p->nC, nP = p->nP;
     const size_t smem2 = (size_t)2 * Wv * 4;
-    const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O + WALK_CAP_L) * 4 + WALK_CAP_I + 16;
+    const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O) * 4 + WALK_CAP_I + 16;
 
-    VL_CUDA(p, keep(&p->d_chunk_i0, nC, 0, st));
-    VL_CUDA(p, keep(&p->d_chunk_i1, nC, 0, st));
-    VL_CUDA(p, keep(&p->d_chunk_blk, nC, 0, st));
-    VL_CUDA(p, keep(&p->d_blk_chunk_off, (size_t)nB + 1, 0, st));
-    if (nC) {
-        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_i0, p->h_chunk_i0.data(), nC * 4, cudaMemcpyHostToDevice, st));
-        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_i1, p->h_chunk_i1.data(), nC * 4, cudaMemcpyHostToDevice, st));
-        VL_CUDA(p, cudaMemcpyAsync(p->d_chunk_blk, p->h_chunk_blk.data(), nC * 4, cudaMemcpyHostToDevice, st));
-    }
-    VL_CUDA(p, cudaMemcpyAsync(p->d_blk_chunk_off, p->h_blk_chunk_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
-    VL_CUDA(p, keep(&p->d_blk_in, (size_t)nB * Wv, 0, st));
-    VL_CUDA(p, keep(&p->d_blk_out, (size_t)nB * Wv, 0, st));
-    VL_CUDA(p, keep(&p->d_lo_off, (size_t)nI + 1, 0, st));
-    VL_CUDA(p, keep(&p->d_opflags, (size_t)nO, 0, st));
-    VL_CUDA(p, keep(&p->d_first_def_instr, (size_t)V, 0xFF, st));
-    VL_CUDA(p, keep(&p->d_vreg16, (size_t)p->nOp8 + 8, 0, st));
-    VL_CUDA(p, keep(&p->d_slotmeta, (size_t)p->nOp8 / 8, 0, st));
-    VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
+    // ---- results and tables that do not depend on the list lengths
+    KEEP(&p->d_blk_in, (size_t)2 * nB * Wv);  // live-in rows, then live-out rows
+    p->d_blk_out = p->d_blk_in + (size_t)nB * Wv;
+    KEEP(&p->d_lo_off, (size_t)nI + 1);
+    KEEP(&p->d_opflags, (size_t)nO);
+    KEEP(&p->d_first_def_instr, (size_t)V);
+    KEEP(&p->d_vreg16, (size_t)p->nOp8 + 8);
+    KEEP(&p->d_slotmeta, (size_t)p->nOp8 / 8);
+    KEEP(&p->d_vinfo, (size_t)V);
+    KEEP(&p->d_iflags, (size_t)nI);
+    KEEP(&p->d_cev_off, (size_t)nC + 1);
+    KEEP(&p->d_th_off, (size_t)nB + 1);
 
-    TmpPool sc{p};
-    uint32_t *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry, *blk_use, *blk_def, *blk_th;
-    uint32_t *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
+    uint32_t *piece_use, *piece_def, *piece_end, *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry;
+    uint32_t *blk_use, *blk_def, *blk_th, *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
     uint8_t *opmeta;
     unsigned long long *totals;
-    VL_CUDA(p, sc.get(&chunk_use, (size_t)nC * Wv, false, st));
-    VL_CUDA(p, sc.get(&chunk_def, (size_t)nC * Wv, false, st));
-    VL_CUDA(p, sc.get(&chunk_touch, (size_t)nC * Wv, false, st));
-    VL_CUDA(p, sc.get(&chunk_end, (size_t)nC * Wv, false, st));
-    VL_CUDA(p, sc.get(&chunk_entry, (size_t)nC * Wv, false, st));
-    VL_CUDA(p, sc.get(&blk_use, (size_t)nB * Wv, false, st));
-    VL_CUDA(p, sc.get(&blk_def, (size_t)nB * Wv, false, st));
-    VL_CUDA(p, sc.get(&blk_th, (size_t)nB * Wv, false, st));
-    VL_CUDA(p, sc.get(&lo_cnt, (size_t)nI + 1, true, st));
-    VL_CUDA(p, sc.get(&ev_cnt, (size_t)nI + 1, true, st));
-    VL_CUDA(p, sc.get(&ev_off, (size_t)nI + 1, true, st));
-    VL_CUDA(p, sc.get(&centry_cnt, (size_t)nC, true, st));
-    VL_CUDA(p, sc.get(&cev, (size_t)nC, true, st));
-    VL_CUDA(p, sc.get(&th_cnt, (size_t)nB, true, st));
-    VL_CUDA(p, sc.get(&first_occ, (size_t)V, false, st));
+    TMP(&piece_use, (size_t)nP * Wv);
+    TMP(&piece_def, (size_t)nP * Wv);
+    TMP(&piece_end, (size_t)nP * Wv);
+    TMP(&chunk_use, (size_t)nC * Wv);
+    TMP(&chunk_def, (size_t)nC * Wv);
+    TMP(&chunk_end, (size_t)nC * Wv);
+    TMP(&chunk_entry, (size_t)nC * Wv);
+    TMP(&blk_use, (size_t)nB * Wv);
+    TMP(&blk_def, (size_t)nB * Wv);
+    TMP(&blk_th, (size_t)nB * Wv);
+    TMP(&lo_cnt, (size_t)nI + 1);
+    TMP(&ev_cnt, (size_t)nI + 1);
+    TMP(&ev_off, (size_t)nI + 1);
+    TMP(&centry_cnt, (size_t)nC);
+    TMP(&cev, (size_t)nC);
+    TMP(&th_cnt, (size_t)nB);
+    TMP(&first_occ, (size_t)V);
+    TMP(&opmeta, (size_t)nO);
+    TMP(&chunk_touch, (size_t)nC * Wv + 16);  // followed by the totals: one memset clears both
+    totals = reinterpret_cast<unsigned long long *>(chunk_touch + (((size_t)nC * Wv + 1) & ~(size_t)1));
+    // what has to start from a known value: the fixed point's sets, the touch sets (updated with
+    // atomics), the totals, the status word, and the two "lowest index so far" arrays
+    VL_CUDA(p, cudaMemsetAsync(p->d_blk_in, 0, (size_t)2 * nB * Wv * 4, st));
+    VL_CUDA(p, cudaMemsetAsync(chunk_touch, 0, ((size_t)nC * Wv + 16) * 4, st));
+    VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
     VL_CUDA(p, cudaMemsetAsync(first_occ, 0xFF, std::max<size_t>(V, 1) * 4, st));
-    VL_CUDA(p, sc.get(&opmeta, (size_t)nO, true, st));
-    VL_CUDA(p, sc.get(&totals, 4, true, st));
+    VL_CUDA(p, cudaMemsetAsync(p->d_first_def_instr, 0xFF, std::max<size_t>(V, 1) * 4, st));
 
-    LAUNCH(k_chunk_sets, nC, smem2, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, Wv,
-           chunk_use, chunk_def);
+    LAUNCH(k_chunk_sets, nP, smem2, st, p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, Wv,
+           piece_use, piece_def);
+    LAUNCH(k_block_sets, nC, 0, st, p->d_chunk_piece_off, Wv, piece_use, piece_def, chunk_use, chunk_def);
     LAUNCH(k_block_sets, nB, 0, st, p->d_blk_chunk_off, Wv, chunk_use, chunk_def, blk_use, blk_def);
     LAUNCH(k_fixed_point, (Wv + NT - 1) / NT, 0, st, nB, Wv, p->d_succ_off, p->d_succ, blk_use, blk_def, p->d_blk_in,
            p->d_blk_out, p->d_status);
     LAUNCH(k_chunk_boundaries, nB, 0, st, p->d_blk_chunk_off, Wv, p->d_blk_out, chunk_use, chunk_def, chunk_end,
            chunk_entry);
-    if (nC) k_instr_walk<false><<<nC, 32, walk_smem, st>>>( p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
-           Wv, chunk_end, lo_cnt, ev_cnt, p->d_opflags, chunk_touch, (const uint32_t *)nullptr, (uint32_t *)nullptr);
+    LAUNCH(k_chunk_boundaries, nC, 0, st, p->d_chunk_piece_off, Wv, chunk_end, piece_use, piece_def, piece_end,
+           (uint32_t *)nullptr);
+    if (nP) k_instr_walk<false><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
+           p->d_op_vreg, Wv, piece_end, lo_cnt, ev_cnt, p->d_opflags, p->d_piece_chunk, chunk_touch,
+           (const uint32_t *)nullptr, (uint32_t *)nullptr);
     k_scan<<<1, 1024, 0, st>>>(lo_cnt, p->d_lo_off, nI, totals + 0, p->d_status);
     k_scan<<<1, 1024, 0, st>>>(ev_cnt, ev_off, nI, totals + 1, p->d_status);
-    g_vl_launches.fetch_add(2);
+    g_vl_launches.fetch_add(nP ? 3 : 2);
     LAUNCH(k_block_through, nB, 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
     LAUNCH(k_chunk_entry, nC, 0, st, p->d_chunk_blk, p->d_chunk_i0, p->d_chunk_i1, Wv, blk_th, chunk_entry, ev_off,
            centry_cnt, cev);
     LAUNCH(k_row_popc, nB, 0, st, Wv, blk_th, th_cnt);
+    k_offsets<<<1, NT, 0, st>>>(nC, nB, cev, th_cnt, p->d_cev_off, p->d_th_off, totals);
+    g_vl_launches.fetch_add(1);
 
-    // ---- read back sizes and status
+    // ---- list lengths: read back on the first run with this layout; later runs allocate from the
+    // lengths they remember (same program, same layout) and only compare at the end
     uint32_t status = 0;
-    unsigned long long h_tot[2] = {0, 0};
-    std::vector<uint32_t> h_cev(nC), h_thc(nB);
-    VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 16, cudaMemcpyDeviceToHost, st));
-    if (nC) VL_CUDA(p, cudaMemcpyAsync(h_cev.data(), cev, nC * 4, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaMemcpyAsync(h_thc.data(), th_cnt, nB * 4, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaStreamSynchronize(st));
-    if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
-    if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
-    if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
-    p->lo_len = h_tot[0];
-
-    std::vector<uint32_t> h_cev_off(nC + 1, 0), h_th_off(nB + 1, 0);
-    uint64_t steps = 0;  // walk events in total, every chunk padded to a multiple of 8 with no-ops
-    for (uint32_t c = 0; c < nC; ++c) {
-        h_cev_off[c] = (uint32_t)steps;
-        steps += (h_cev[c] + 7) / 8 * 8;
+    unsigned long long h_tot[4] = {0, 0, 0, 0};
+    if (!p->sizes_known) {
+        VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
+        VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 32, cudaMemcpyDeviceToHost, st));
+        VL_CUDA(p, cudaStreamSynchronize(st));
+        if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
+        if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
+        if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
+        if (h_tot[2] > 0xFFFFFFF0ull) return VL_ERR_UNSUPPORTED;
+        p->known_lo_len = h_tot[0];
+        p->known_steps = h_tot[2];
+        p->known_thn = h_tot[3];
     }
-    h_cev_off[nC] = (uint32_t)steps;
-    // walk work items: runs of at most 16 chunks of one block
-    std::vector<uint32_t> it_blk, it_c0, it_c1;
-    for (uint32_t b = 0; b < nB; ++b)
-        for (uint32_t c = p->h_blk_chunk_off[b]; c < p->h_blk_chunk_off[b + 1]; c += 16) {
-            it_blk.push_back(b);
-            it_c0.push_back(c);
-            it_c1.push_back(std::min(c + 16, p->h_blk_chunk_off[b + 1]));
-        }
-    p->nItems = (uint32_t)it_blk.size();
-    uint64_t thn = 0;
-    for (uint32_t b = 0; b < nB; ++b) { h_th_off[b] = (uint32_t)thn; thn += h_thc[b]; }
-    h_th_off[nB] = (uint32_t)thn;
-    if (steps > 0xFFFFFFF0ull) return VL_ERR_UNSUPPORTED;
+    p->lo_len = p->known_lo_len;
+    const uint64_t steps = p->known_steps;  // walk events in total, every chunk padded to a multiple of 8 with no-ops
     p->ev_total = (uint32_t)steps;
-    p->th_len = (uint32_t)thn;
+    p->th_len = (uint32_t)p->known_thn;
 
-    VL_CUDA(p, keep(&p->d_lo, (size_t)p->lo_len, 0, st));
-    VL_CUDA(p, keep(&p->d_ev, (size_t)(steps / 8) * 7, 0, st));
-    VL_CUDA(p, keep(&p->d_vinfo, (size_t)V, 0, st));
-    VL_CUDA(p, keep(&p->d_iflags, (size_t)nI, 0, st));
+    KEEP(&p->d_lo, (size_t)p->lo_len);
+    KEEP(&p->d_ev, (size_t)(steps / 8) * 7);
+    KEEP(&p->d_th, (size_t)p->known_thn);
     LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)(steps / 8),
            V);  // every slot starts as a no-op event
-    VL_CUDA(p, keep(&p->d_th, (size_t)thn, 0, st));
-    VL_CUDA(p, keep(&p->d_cev_off, (size_t)nC + 1, 0, st));
-    VL_CUDA(p, keep(&p->d_item_blk, (size_t)p->nItems, 0, st));
-    VL_CUDA(p, keep(&p->d_item_c0, (size_t)p->nItems, 0, st));
-    VL_CUDA(p, keep(&p->d_item_c1, (size_t)p->nItems, 0, st));
-    if (p->nItems) {
-        VL_CUDA(p, cudaMemcpyAsync(p->d_item_blk, it_blk.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
-        VL_CUDA(p, cudaMemcpyAsync(p->d_item_c0, it_c0.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
-        VL_CUDA(p, cudaMemcpyAsync(p->d_item_c1, it_c1.data(), p->nItems * 4, cudaMemcpyHostToDevice, st));
-    }
-    VL_CUDA(p, keep(&p->d_th_off, (size_t)nB + 1, 0, st));
-    VL_CUDA(p, cudaMemcpyAsync(p->d_cev_off, h_cev_off.data(), (nC + 1) * 4, cudaMemcpyHostToDevice, st));
-    VL_CUDA(p, cudaMemcpyAsync(p->d_th_off, h_th_off.data(), (nB + 1) * 4, cudaMemcpyHostToDevice, st));
 
-    if (nC) k_instr_walk<true><<<nC, 32, walk_smem, st>>>( p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg,
-           Wv, chunk_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr, (uint32_t *)nullptr,
-           (const uint32_t *)p->d_lo_off, p->d_lo);
-    g_vl_launches.fetch_add(2);  // the two k_instr_walk passes
+    if (nP) k_instr_walk<true><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
+           p->d_op_vreg, Wv, piece_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr,
+           (const uint32_t *)nullptr, (uint32_t *)nullptr, (const uint32_t *)p->d_lo_off, p->d_lo);
+    if (nP) g_vl_launches.fetch_add(1);
     LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_first_def_instr);
     LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, st, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
@@ -704,8 +762,19 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 32, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaStreamSynchronize(st));
     VL_CUDA(p, cudaGetLastError());
+    if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
+    if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
+    if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
+    if (h_tot[0] != p->known_lo_len || h_tot[2] != p->known_steps || h_tot[3] != p->known_thn) {
+        // the remembered lengths do not fit what was just computed: measure again
+        const bool retry = p->sizes_known;
+        p->sizes_known = false;
+        return retry ? vl_liveness_impl(p, st) : VL_ERR_CUDA;
+    }
+    p->sizes_known = true;
     p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     p->live_ok = true;
     return VL_OK;
