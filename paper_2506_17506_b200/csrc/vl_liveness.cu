@@ -13,7 +13,7 @@
 #include "vl_internal.cuh"
 
 #define NT 128  // threads per block in every kernel of this file
-#define PIECE_INSTRS 16
+#define PIECE_INSTRS 8
 
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ bool bit_get(const uint32_t *s, uint32_t v) { return (s[v >> 5] >> (v & 31)) & 1u; }
@@ -104,27 +104,66 @@ __global__ void k_block_sets(const uint32_t *__restrict__ blk_chunk_off, uint32_
                              const uint32_t *__restrict__ chunk_use, const uint32_t *__restrict__ chunk_def,
                              uint32_t *blk_use, uint32_t *blk_def)
 {
-    const uint32_t b = blockIdx.x;
-    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
-        uint32_t u = 0, d = 0;
+    const uint32_t b = blockIdx.y, w = blockIdx.x * NT + threadIdx.x;  // one bitset word per thread
+    if (w >= Wv) return;
+    const uint32_t c_lo = blk_chunk_off[b], c_hi = blk_chunk_off[b + 1];
+    uint32_t u = 0, d = 0;
 #pragma unroll 8
-        for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) {
-            u |= chunk_use[(size_t)c * Wv + w] & ~d;
-            d |= chunk_def[(size_t)c * Wv + w];
-        }
-        blk_use[(size_t)b * Wv + w] = u;
-        blk_def[(size_t)b * Wv + w] = d;
+    for (uint32_t c = c_lo; c < c_hi; ++c) {
+        u |= chunk_use[(size_t)c * Wv + w] & ~d;
+        d |= chunk_def[(size_t)c * Wv + w];
     }
+    blk_use[(size_t)b * Wv + w] = u;
+    blk_def[(size_t)b * Wv + w] = d;
 }
 
 // Backward dataflow to the least fixed point.  Bitset words are independent of each other,
 // so one thread iterates one word column over all blocks until nothing changes; no barrier.
-__global__ void k_fixed_point(uint32_t nB, uint32_t Wv, const uint32_t *__restrict__ succ_off,
+// SMEM: the four sets of this thread's word column and the successor lists sit in shared memory
+// ([4][nB][NT] words, then succ_off[nB + 1] and succ[nE]); otherwise everything stays in global memory.
+template <bool SMEM>
+__global__ void k_fixed_point(uint32_t nB, uint32_t nE, uint32_t Wv, const uint32_t *__restrict__ succ_off,
                               const uint32_t *__restrict__ succ, const uint32_t *__restrict__ blk_use,
                               const uint32_t *__restrict__ blk_def, uint32_t *live_in, uint32_t *live_out,
                               uint32_t *status)
 {
     const uint32_t w = blockIdx.x * NT + threadIdx.x;
+    if (SMEM) {
+        extern __shared__ uint32_t fsm[];
+        uint32_t *s_use = fsm, *s_def = fsm + nB * NT, *s_in = fsm + 2 * nB * NT, *s_out = fsm + 3 * nB * NT;
+        uint32_t *s_so = fsm + 4 * nB * NT, *s_su = s_so + nB + 1;
+        for (uint32_t i = threadIdx.x; i <= nB; i += NT) s_so[i] = succ_off[i];
+        for (uint32_t i = threadIdx.x; i < nE; i += NT) s_su[i] = succ[i];
+        const uint32_t t = threadIdx.x;
+        for (uint32_t b = 0; b < nB; ++b) {
+            s_use[b * NT + t] = w < Wv ? blk_use[(size_t)b * Wv + w] : 0u;
+            s_def[b * NT + t] = w < Wv ? blk_def[(size_t)b * Wv + w] : 0u;
+            s_in[b * NT + t] = 0;
+            s_out[b * NT + t] = 0;
+        }
+        __syncthreads();
+        if (w >= Wv) return;
+        bool changed = true;
+        for (uint32_t sweep = 0; sweep < nB + 2 && changed; ++sweep) {
+            changed = false;
+            for (uint32_t n = 0; n < nB; ++n) {
+                const uint32_t b = nB - 1 - n;
+                uint32_t o = 0;
+                for (uint32_t e = s_so[b]; e < s_so[b + 1]; ++e) o |= s_in[s_su[e] * NT + t];
+                const uint32_t in = s_use[b * NT + t] | (o & ~s_def[b * NT + t]);
+                if (o != s_out[b * NT + t] || in != s_in[b * NT + t]) changed = true;
+                s_out[b * NT + t] = o;
+                s_in[b * NT + t] = in;
+            }
+        }
+        for (uint32_t b = 0; b < nB; ++b) {
+            live_in[(size_t)b * Wv + w] = s_in[b * NT + t];
+            live_out[(size_t)b * Wv + w] = s_out[b * NT + t];
+        }
+        if (changed) atomicOr(status, ST_NO_CONVERGE);
+        if (s_in[t] != 0) atomicOr(status, ST_NOT_STRICT);  // block 0 is the entry
+        return;
+    }
     if (w >= Wv) return;
     bool changed = true;
     for (uint32_t sweep = 0; sweep < nB + 2 && changed; ++sweep) {
@@ -150,15 +189,22 @@ __global__ void k_chunk_boundaries(const uint32_t *__restrict__ blk_chunk_off, u
                                    const uint32_t *__restrict__ live_out, const uint32_t *__restrict__ chunk_use,
                                    const uint32_t *__restrict__ chunk_def, uint32_t *chunk_end, uint32_t *chunk_entry)
 {
-    const uint32_t b = blockIdx.x;
+    const uint32_t b = blockIdx.y, w = blockIdx.x * NT + threadIdx.x;  // one bitset word per thread
+    if (w >= Wv) return;
     const uint32_t c_lo = blk_chunk_off[b], c_hi = blk_chunk_off[b + 1];
-    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
-        uint32_t live = live_out[(size_t)b * Wv + w];
+    uint32_t live = live_out[(size_t)b * Wv + w];
+    if (chunk_entry) {
 #pragma unroll 8
         for (uint32_t c = c_hi; c-- > c_lo;) {
             chunk_end[(size_t)c * Wv + w] = live;
             live = chunk_use[(size_t)c * Wv + w] | (live & ~chunk_def[(size_t)c * Wv + w]);
-            if (chunk_entry) chunk_entry[(size_t)c * Wv + w] = live;
+            chunk_entry[(size_t)c * Wv + w] = live;
+        }
+    } else {
+#pragma unroll 8
+        for (uint32_t c = c_hi; c-- > c_lo;) {
+            chunk_end[(size_t)c * Wv + w] = live;
+            live = chunk_use[(size_t)c * Wv + w] | (live & ~chunk_def[(size_t)c * Wv + w]);
         }
     }
 }
@@ -275,9 +321,14 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
 
 // Exclusive scan of a u32 array by one block of 1024 threads, 4 items per thread and round;
 // out[n] = total (saturated), total64 exact.
-__global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in, uint32_t *out, uint32_t n,
-                                               unsigned long long *total64, uint32_t *status)
+// Block b of the grid scans in_b into out_b (two arrays per launch).
+__global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in0, uint32_t *out0,
+                                               const uint32_t *__restrict__ in1, uint32_t *out1, uint32_t n,
+                                               unsigned long long *totals, uint32_t *status)
 {
+    const uint32_t *__restrict__ in = blockIdx.x ? in1 : in0;
+    uint32_t *out = blockIdx.x ? out1 : out0;
+    unsigned long long *total64 = totals + blockIdx.x;
     __shared__ uint32_t s_w[33];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long carry = 0;
@@ -328,13 +379,13 @@ __global__ void k_block_through(const uint32_t *__restrict__ blk_chunk_off, uint
                                 const uint32_t *__restrict__ live_in, const uint32_t *__restrict__ chunk_touch,
                                 uint32_t *blk_th)
 {
-    const uint32_t b = blockIdx.x;
-    for (uint32_t w = threadIdx.x; w < Wv; w += NT) {
-        uint32_t t = 0;
+    const uint32_t b = blockIdx.y, w = blockIdx.x * NT + threadIdx.x;  // one bitset word per thread
+    if (w >= Wv) return;
+    const uint32_t c_lo = blk_chunk_off[b], c_hi = blk_chunk_off[b + 1];
+    uint32_t t = 0;
 #pragma unroll 8
-        for (uint32_t c = blk_chunk_off[b]; c < blk_chunk_off[b + 1]; ++c) t |= chunk_touch[(size_t)c * Wv + w];
-        blk_th[(size_t)b * Wv + w] = use_th ? (live_in[(size_t)b * Wv + w] & ~t) : 0u;
-    }
+    for (uint32_t c = c_lo; c < c_hi; ++c) t |= chunk_touch[(size_t)c * Wv + w];
+    blk_th[(size_t)b * Wv + w] = use_th ? (live_in[(size_t)b * Wv + w] & ~t) : 0u;
 }
 
 // chunk_entry &= ~through(block); entry count; events of the chunk = entries + instruction events.
@@ -577,9 +628,11 @@ cudaError_t pool_get(VlArena &arena, T **out, size_t n)
 #define TMP(out, n) VL_CUDA(p, pool_get(p->tmp_arena, out, n))
 #define LAYOUT(out, n) VL_CUDA(p, pool_get(p->layout_arena, out, n))
 
+static inline bool grid_nonempty(uint32_t g) { return g > 0; }
+static inline bool grid_nonempty(dim3 g) { return g.x > 0 && g.y > 0 && g.z > 0; }
 #define LAUNCH(kernel, grid, smem, st, ...)                          \
     do {                                                             \
-        if ((grid) > 0) {                                            \
+        if (grid_nonempty(grid)) {                                   \
             kernel<<<(grid), NT, (smem), (st)>>>(__VA_ARGS__);       \
             g_vl_launches.fetch_add(1);                              \
         }                                                            \
@@ -699,21 +752,28 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
 
     LAUNCH(k_chunk_sets, nP, smem2, st, p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, Wv,
            piece_use, piece_def);
-    LAUNCH(k_block_sets, nC, 0, st, p->d_chunk_piece_off, Wv, piece_use, piece_def, chunk_use, chunk_def);
-    LAUNCH(k_block_sets, nB, 0, st, p->d_blk_chunk_off, Wv, chunk_use, chunk_def, blk_use, blk_def);
-    LAUNCH(k_fixed_point, (Wv + NT - 1) / NT, 0, st, nB, Wv, p->d_succ_off, p->d_succ, blk_use, blk_def, p->d_blk_in,
-           p->d_blk_out, p->d_status);
-    LAUNCH(k_chunk_boundaries, nB, 0, st, p->d_blk_chunk_off, Wv, p->d_blk_out, chunk_use, chunk_def, chunk_end,
-           chunk_entry);
-    LAUNCH(k_chunk_boundaries, nC, 0, st, p->d_chunk_piece_off, Wv, chunk_end, piece_use, piece_def, piece_end,
-           (uint32_t *)nullptr);
+    const uint32_t wgrid = (Wv + NT - 1) / NT;
+    if (nC) LAUNCH(k_block_sets, dim3(wgrid, nC), 0, st, p->d_chunk_piece_off, Wv, piece_use, piece_def, chunk_use, chunk_def);
+    LAUNCH(k_block_sets, dim3(wgrid, nB), 0, st, p->d_blk_chunk_off, Wv, chunk_use, chunk_def, blk_use, blk_def);
+    {
+        const size_t fp_smem = ((size_t)4 * nB * NT + nB + 1 + p->nE) * 4;
+        if (fp_smem <= 48 * 1024)
+            LAUNCH(k_fixed_point<true>, wgrid, fp_smem, st, nB, p->nE, Wv, p->d_succ_off, p->d_succ, blk_use, blk_def,
+                   p->d_blk_in, p->d_blk_out, p->d_status);
+        else
+            LAUNCH(k_fixed_point<false>, wgrid, 0, st, nB, p->nE, Wv, p->d_succ_off, p->d_succ, blk_use, blk_def,
+                   p->d_blk_in, p->d_blk_out, p->d_status);
+    }
+    LAUNCH(k_chunk_boundaries, dim3(wgrid, nB), 0, st, p->d_blk_chunk_off, Wv, p->d_blk_out, chunk_use, chunk_def,
+           chunk_end, chunk_entry);
+    if (nC) LAUNCH(k_chunk_boundaries, dim3(wgrid, nC), 0, st, p->d_chunk_piece_off, Wv, chunk_end, piece_use, piece_def,
+                   piece_end, (uint32_t *)nullptr);
     if (nP) k_instr_walk<false><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
            p->d_op_vreg, Wv, piece_end, lo_cnt, ev_cnt, p->d_opflags, p->d_piece_chunk, chunk_touch,
            (const uint32_t *)nullptr, (uint32_t *)nullptr);
-    k_scan<<<1, 1024, 0, st>>>(lo_cnt, p->d_lo_off, nI, totals + 0, p->d_status);
-    k_scan<<<1, 1024, 0, st>>>(ev_cnt, ev_off, nI, totals + 1, p->d_status);
-    g_vl_launches.fetch_add(nP ? 3 : 2);
-    LAUNCH(k_block_through, nB, 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
+    k_scan<<<2, 1024, 0, st>>>(lo_cnt, p->d_lo_off, ev_cnt, ev_off, nI, totals, p->d_status);
+    g_vl_launches.fetch_add(nP ? 2 : 1);
+    LAUNCH(k_block_through, dim3(wgrid, nB), 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
     LAUNCH(k_chunk_entry, nC, 0, st, p->d_chunk_blk, p->d_chunk_i0, p->d_chunk_i1, Wv, blk_th, chunk_entry, ev_off,
            centry_cnt, cev);
     LAUNCH(k_row_popc, nB, 0, st, Wv, blk_th, th_cnt);
