@@ -152,6 +152,7 @@ void vl_free_liveness(vl_program *p)
     p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
+    p->d_el = nullptr; p->d_el_count = nullptr;
     p->live_ok = false;
     p->lo_len = 0;
 }

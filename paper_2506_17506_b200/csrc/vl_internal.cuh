@@ -102,6 +102,8 @@ struct vl_program {
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
     uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
+    uint4 *d_el = nullptr;          // definitions without a walk event: {instruction, chunk, vreg, block}, any order
+    uint32_t *d_el_count = nullptr;
     uint32_t th_len = 0;
     uint32_t *d_cev_off = nullptr;  // [nC+1] first walk event of each chunk (every chunk padded to 8 events)
     uint4 *d_ev = nullptr;          // walk events, 112 bytes per group of 8, chunk after chunk

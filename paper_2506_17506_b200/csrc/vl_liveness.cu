@@ -538,7 +538,7 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
                               const uint8_t *__restrict__ opflags, uint32_t Wv,
                               const uint32_t *__restrict__ chunk_entry, const uint32_t *__restrict__ centry_cnt,
                               const uint32_t *__restrict__ ev_off, const uint32_t *__restrict__ cev_off,
-                              uint4 *ev)
+                              uint4 *ev, const uint32_t *__restrict__ chunk_blk, uint4 *el, uint32_t *el_count)
 {
     __shared__ uint32_t s_scan[34];
     const uint32_t c = blockIdx.x;
@@ -561,6 +561,8 @@ __global__ void k_fill_events(const uint32_t *__restrict__ chunk_i0, const uint3
             if (!(opflags[o] & OPF_ELIDE)) {
                 const uint32_t v = op_vreg[o];
                 put_event(ev, base + (e++), v, width[v], true, (opflags[o] & OPF_SET) != 0);
+            } else {  // no event: listed (in any order) for the recount of through-set collisions
+                el[atomicAdd(el_count, 1u)] = make_uint4(i, c, op_vreg[o], chunk_blk[c]);
             }
         for (uint32_t o = o0; o < o0 + nd; ++o)
             if ((opflags[o] & OPF_POST) && !(opflags[o] & OPF_ELIDE)) {
@@ -717,6 +719,8 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     KEEP(&p->d_iflags, (size_t)nI);
     KEEP(&p->d_cev_off, (size_t)nC + 1);
     KEEP(&p->d_th_off, (size_t)nB + 1);
+    KEEP(&p->d_el, (size_t)nO);  // at most one entry per definition
+    KEEP(&p->d_el_count, 1);
 
     uint32_t *piece_use, *piece_def, *piece_end, *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry;
     uint32_t *blk_use, *blk_def, *blk_th, *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
@@ -747,6 +751,7 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     VL_CUDA(p, cudaMemsetAsync(p->d_blk_in, 0, (size_t)2 * nB * Wv * 4, st));
     VL_CUDA(p, cudaMemsetAsync(chunk_touch, 0, ((size_t)nC * Wv + 16) * 4, st));
     VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
+    VL_CUDA(p, cudaMemsetAsync(p->d_el_count, 0, 4, st));
     VL_CUDA(p, cudaMemsetAsync(first_occ, 0xFF, std::max<size_t>(V, 1) * 4, st));
     VL_CUDA(p, cudaMemsetAsync(p->d_first_def_instr, 0xFF, std::max<size_t>(V, 1) * 4, st));
 
@@ -818,7 +823,8 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
            p->d_opflags, p->d_vreg16, opmeta, p->d_status);
     LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, st, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
     LAUNCH(k_fill_events, nC, 0, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
-           p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev);
+           p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev, p->d_chunk_blk, p->d_el,
+           p->d_el_count);
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));

@@ -73,7 +73,7 @@ struct RParams {
     uint32_t nI, V, B, nB, nC, AW;
     int bank_fast;
     uint64_t K;
-    const uint32_t *vinfo, *chunk_i0, *chunk_i1, *chunk_blk, *op_off, *op_vreg, *lo_off, *lo;
+    const uint32_t *vinfo, *chunk_i0, *chunk_i1, *chunk_blk, *blk_chunk_off, *th_off, *th, *op_off, *op_vreg, *lo_off, *lo;
     const uint8_t *ndefs, *width, *opflags, *iflags;
     const uint16_t *tg;
     const uint32_t *cstate, *anom;
@@ -83,6 +83,8 @@ struct RParams {
     uint32_t *work;
     vl_verdict *out;
     uint32_t *status;
+    const uint4 *el;           // the definitions the walk skips: {instruction, chunk, vreg, block}
+    const uint32_t *el_count;
 };
 
 // Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
@@ -721,12 +723,13 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
 // =========================================================================== verdicts / work list
 // Verdicts of the candidates the walk vouches for.  For the others, work items for k_recount:
 // every chunk that needs an exact recount is cut into RC_PARTS pieces, the general bank tally into
-// RC_BANK_PARTS slices; racc[k][3] counts the items pending.  An item is (candidate, code) with
-// code = kind << 30 | piece << 24 | chunk.
+// RC_BANK_PARTS slices, and every block whose through-set collided gets one item for the
+// definitions the walk skipped in its other chunks; racc[k][3] counts the items pending.  An item
+// is (candidate, code) with code = kind << 30 | piece << 24 | chunk (or block).
 #define RC_PARTS 2
 #define RC_BANK_PARTS 4
 #define RC_KIND_ALL 0u     // every definition of the piece
-#define RC_KIND_ELIDED 1u  // only the definitions the walk skipped
+#define RC_KIND_THROUGH 1u // a block whose through-set collided: the definitions the walk skipped, chunk = block
 #define RC_KIND_BANK 2u
 __device__ __forceinline__ uint32_t rc_code(uint32_t kind, uint32_t piece, uint32_t chunk)
 {
@@ -755,18 +758,17 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
         return;
     }
     // a chunk that collided (or a candidate with several out-of-file vregs): every definition;
-    // a block whose through-set collided: the definitions the walk skipped (a vreg redefined from
-    // itself while it stays occupied), since everything else in it was walked exactly
+    // a block whose through-set collided: the definitions the walk skipped in its other chunks (a
+    // vreg redefined from itself while it stays occupied), since everything else in them was walked
+    // exactly
     const bool full = walk & WALK_FULL;
-    auto kind_of = [&](uint32_t c) -> uint32_t {  // 0 none, 1 all definitions, 2 skipped definitions only
-        if (c >= nC) return 0u;
-        const bool all_defs = full || ((__ldcg(anom + k * AW + (c >> 5)) >> (c & 31)) & 1u);
-        if (all_defs) return 1u;
-        return (thcol && ((thcol >> (chunk_blk[c] & 31)) & 1u)) ? 2u : 0u;
+    auto all_defs = [&](uint32_t c) -> bool {
+        return c < nC && (full || ((__ldcg(anom + k * AW + (c >> 5)) >> (c & 31)) & 1u));
     };
     uint32_t n_chunks = 0;
-    for (uint32_t c0 = 0; c0 < nC; c0 += 32) n_chunks += __popc(__ballot_sync(0xffffffffu, kind_of(c0 + lane) != 0));
-    const uint32_t n = RC_BANK_PARTS + RC_PARTS * n_chunks;
+    for (uint32_t c0 = 0; c0 < nC; c0 += 32) n_chunks += __popc(__ballot_sync(0xffffffffu, all_defs(c0 + lane)));
+    const uint32_t n_blocks = full ? 0u : __popc(thcol);
+    const uint32_t n = RC_BANK_PARTS + RC_PARTS * n_chunks + n_blocks;
     uint32_t at = 0;
     if (lane == 0) {
         racc[k * 4 + 3] = n;
@@ -778,15 +780,21 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
         work[3 + 2 * (at + lane)] = rc_code(RC_KIND_BANK, lane, 0);
     }
     at += RC_BANK_PARTS;
+    if (!full && ((thcol >> lane) & 1u)) {  // through-sets are used only if the program has at most 32 blocks
+        const uint32_t slot = at + __popc(thcol & ((1u << lane) - 1u));
+        work[2 + 2 * slot] = (uint32_t)k;
+        work[3 + 2 * slot] = rc_code(RC_KIND_THROUGH, 0, lane);
+    }
+    at += n_blocks;
     for (uint32_t c0 = 0; c0 < nC; c0 += 32) {
-        const uint32_t kd = kind_of(c0 + lane);
-        const uint32_t m = __ballot_sync(0xffffffffu, kd != 0);
+        const bool kd = all_defs(c0 + lane);
+        const uint32_t m = __ballot_sync(0xffffffffu, kd);
         if (kd) {
             const uint32_t slot = at + RC_PARTS * __popc(m & ((1u << lane) - 1u));
 #pragma unroll
             for (uint32_t part = 0; part < RC_PARTS; ++part) {
                 work[2 + 2 * (slot + part)] = (uint32_t)k;
-                work[3 + 2 * (slot + part)] = rc_code(kd == 1 ? RC_KIND_ALL : RC_KIND_ELIDED, part, c0 + lane);
+                work[3 + 2 * (slot + part)] = rc_code(RC_KIND_ALL, part, c0 + lane);
             }
         }
         at += RC_PARTS * __popc(m);
@@ -853,8 +861,71 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             }
             return x;
         };
-        if (kind != RC_KIND_BANK) {
-            const bool elided_only = kind == RC_KIND_ELIDED;
+        if (kind == RC_KIND_THROUGH) {
+            // The through-set of block c collided.  In a chunk of the block whose own walk was clean,
+            // everything else that is live is disjoint from the through-set and from each other, so a
+            // skipped definition of a through-set vreg overlaps exactly the through-set members that
+            // overlap it, whatever the instruction: count those once per member, then add them up over
+            // the skipped definitions.  (Chunks that did collide are recounted in full by their own items.)
+            const uint32_t t0 = q.th_off[c], n_th = q.th_off[c + 1] - t0;
+            uint32_t *ids = Cv;  // [n_th] member vreg ids (ascending), [n_th] register | width << 16, [n_th] counts
+            uint32_t *mem = Cv + n_th, *cnt_th = Cv + 2 * n_th;
+            const bool fits = CACHE && 3 * n_th <= q.V;
+            if (fits) {
+                __syncthreads();
+                for (uint32_t j = tid; j < n_th; j += RC_THREADS) {
+                    const uint32_t v = q.th[t0 + j] & 0xFFFFu;
+                    ids[j] = v;
+                    mem[j] = fetch(v);
+                }
+                __syncthreads();
+                for (uint32_t j = tid; j < n_th; j += RC_THREADS) {
+                    const uint32_t s = mem[j] & 0xFFFFu, w = (mem[j] >> 16) & 0xFFu;
+                    uint32_t cc = 0;
+                    for (uint32_t u = 0; u < n_th; ++u)
+                        if (u != j && ranges_overlap(s, w, mem[u] & 0xFFFFu, (mem[u] >> 16) & 0xFFu)) ++cc;
+                    cnt_th[j] = cc;
+                }
+                __syncthreads();
+            }
+            // overlap count of through-set member v (0 if v is not a member): the list is ascending
+            auto count_of = [&](uint32_t v) -> uint32_t {
+                uint32_t lo_j = 0, hi_j = n_th;
+                while (lo_j < hi_j) {
+                    const uint32_t mid = (lo_j + hi_j) >> 1;
+                    if ((fits ? ids[mid] : (q.th[t0 + mid] & 0xFFFFu)) < v) lo_j = mid + 1; else hi_j = mid;
+                }
+                if (lo_j >= n_th || (fits ? ids[lo_j] : (q.th[t0 + lo_j] & 0xFFFFu)) != v) return 0u;
+                if (fits) return cnt_th[lo_j];
+                const uint32_t x = fetch(v);
+                uint32_t cc = 0;
+                for (uint32_t u = 0; u < n_th; ++u) {
+                    if (u == lo_j) continue;
+                    const uint32_t y = fetch(q.th[t0 + u] & 0xFFFFu);
+                    if (ranges_overlap(x & 0xFFFFu, (x >> 16) & 0xFFu, y & 0xFFFFu, (y >> 16) & 0xFFu)) ++cc;
+                }
+                return cc;
+            };
+            // the program's skipped definitions are listed as {instruction, chunk, vreg, block}
+            uint32_t pairs = 0, mind = 0xFFFFFFFFu;
+            const uint32_t n_el = *q.el_count;
+            for (uint32_t e = tid; e < n_el; e += RC_THREADS) {
+                const uint4 x = q.el[e];
+                if (x.w != c) continue;
+                if ((q.anom[k * q.AW + (x.y >> 5)] >> (x.y & 31)) & 1u) continue;
+                const uint32_t cn = count_of(x.z);
+                if (cn) { pairs += cn; mind = min(mind, x.x); }
+            }
+#pragma unroll
+            for (int dd = 16; dd; dd >>= 1) {
+                pairs += __shfl_xor_sync(0xffffffffu, pairs, dd);
+                mind = min(mind, __shfl_xor_sync(0xffffffffu, mind, dd));
+            }
+            if (lane == 0 && pairs) {
+                atomicAdd(&s_pairs, pairs);
+                atomicMin(&s_mind, mind);
+            }
+        } else if (kind != RC_KIND_BANK) {
             const uint32_t ci0 = q.chunk_i0[c], cn = q.chunk_i1[c] - ci0;
             const uint32_t i_lo = ci0 + (uint32_t)((uint64_t)cn * part / RC_PARTS);
             const uint32_t i_hi = ci0 + (uint32_t)((uint64_t)cn * (part + 1) / RC_PARTS);
@@ -863,7 +934,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             for (uint32_t ib = i_lo + warp; ib < i_hi; ib += 32 * NW) {
                 const uint32_t my_i = ib + lane * NW;
                 uint32_t m_o0 = 0, m_nd = 0, m_l0 = 0, m_l1 = 0;
-                if (my_i < i_hi && !(elided_only && !q.iflags[my_i])) {
+                if (my_i < i_hi) {
                     m_o0 = q.op_off[my_i]; m_nd = q.ndefs[my_i]; m_l0 = q.lo_off[my_i]; m_l1 = q.lo_off[my_i + 1];
                 }
                 // first defined vreg of each instruction, fetched by the lane that holds its bookkeeping
@@ -894,7 +965,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                     const uint32_t l0 = __shfl_sync(0xffffffffu, m_l0, src), l1 = __shfl_sync(0xffffffffu, m_l1, src);
                     const uint32_t v0 = __shfl_sync(0xffffffffu, m_v0, src);
                     for (uint32_t d = o0; d < o0 + nd; ++d) {
-                        if (elided_only && !(q.opflags[d] & OPF_ELIDE)) continue;
                         const uint32_t v = d == o0 ? v0 : q.op_vreg[d];
                         const uint32_t sw = reg_w(v);
                         const uint32_t s = sw & 0xFFFFu, w = (sw >> 16) & 0xFFu;
@@ -1207,6 +1277,8 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     RParams rq{};
     rq.nI = p->nI; rq.V = p->V; rq.B = p->B; rq.nB = p->nB; rq.nC = p->nC; rq.AW = (uint32_t)vs.aw;
     rq.bank_fast = p->bank_fast; rq.K = n;
+    rq.blk_chunk_off = p->d_blk_chunk_off; rq.th_off = p->d_th_off; rq.th = p->d_th;
+    rq.el = p->d_el; rq.el_count = p->d_el_count;
     rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
     rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
     rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
