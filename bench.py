@@ -4,7 +4,10 @@ instructions / 10,000 vregs, K = 10,000 per-operand uint16 candidate rows, about
 
 A step is the whole path for one batch: vl_liveness on the program, then vl_verify over the
 K rows.  `value` is measured with the rows resident in HBM; `e2e` goes through vl_verify_host
-with pinned host buffers, copies inside the timed region.  Prints one JSON line (rank 0).
+with pinned host buffers, copies inside the timed region.  vl_verify spreads its passes over
+internal streams, so its kernels overlap in the timed region; the per-kernel durations behind
+`roofline` come from a second timed loop with the passes in order on one stream
+(VL_OPT_LANES = 1), where a kernel's duration is its own.  Prints one JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--rows R]
 """
@@ -163,7 +166,7 @@ def run_reference(args):
 # DRAM bytes (read + write) per candidate of each kernel, from the profiler capture of a 4096-row launch
 # summarised under profiles/ (traffic grows in proportion to the rows of a launch); None = no capture of
 # the kernel as it stands.
-TRAFFIC_PER_CANDIDATE = {"k_tables": 891.17e6 / 4096, "k_walk": 86.78e6 / 4096}
+TRAFFIC_PER_CANDIDATE = {"k_tables": None, "k_walk": None}
 
 
 def main():
@@ -175,6 +178,8 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="candidate rows per GPU (default: the workload's 10,000)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--group", type=int, default=0)
+    ap.add_argument("--lanes", type=int, default=0, help="internal streams of vl_verify (default: the library's)")
+    ap.add_argument("--sub-batch", type=int, default=0, help="candidates per pass (default: the library's)")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--fault-rate", type=float, default=-1.0, help="override the workload's faulted fraction")
@@ -199,6 +204,10 @@ def main():
         gp.set_option(vl.VL_OPT_GROUP, args.group)
     if args.chunk:
         gp.set_option(vl.VL_OPT_CHUNK_INSTRS, args.chunk)
+    if args.lanes:
+        gp.set_option(vl.VL_OPT_LANES, args.lanes)
+    if args.sub_batch:
+        gp.set_option(vl.VL_OPT_SUB_BATCH, args.sub_batch)
     dev_rows = host.cuda().view(torch.uint16)
     out = torch.empty((K, 4), dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
@@ -238,11 +247,28 @@ def main():
     ev[1].record(stream)
     barrier()
     launches = vl.vl_kernel_launches() - launches0
-    clocks = sampler.stop() if rank == 0 else None
     gp.vl_verify_status(stream)
-    kernel_ms, kernel_passes = gp.vl_kernel_times()
-    gp.set_option(vl.VL_OPT_KERNEL_TIMING, 0)
+    overlap_ms, overlap_passes = gp.vl_kernel_times()
     total_ms = ev[0].elapsed_time(ev[1])
+    # ---- second timed loop, same rows: passes in order on one stream, so that the events around a
+    # kernel time that kernel alone (the clock sampler keeps running)
+    iso_steps = max(3, min(args.steps, 30))
+    gp.set_option(vl.VL_OPT_LANES, 1)
+    for _ in range(3):
+        gp.vl_verify(dev_rows, out, stream)
+    barrier()
+    gp.set_option(vl.VL_OPT_KERNEL_TIMING, 1)
+    iso_ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    iso_ev[0].record(stream)
+    for _ in range(iso_steps):
+        gp.vl_verify(dev_rows, out, stream)
+    iso_ev[1].record(stream)
+    barrier()
+    kernel_ms, kernel_passes = gp.vl_kernel_times()
+    iso_verify_ms = iso_ev[0].elapsed_time(iso_ev[1]) / iso_steps
+    gp.set_option(vl.VL_OPT_KERNEL_TIMING, 0)
+    gp.set_option(vl.VL_OPT_LANES, args.lanes or 3)
+    clocks = sampler.stop() if rank == 0 else None
     verify_ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
     live_ms = float(np.mean([a.elapsed_time(b) for a, b in lev]))
     rows_all, total_ms, _ = shard.job_totals(K * args.steps, total_ms, 0, torch.device("cuda", local))
@@ -277,13 +303,16 @@ def main():
         passes = max(1, kernel_passes)
         ksum = max(1e-9, sum(kernel_ms))
         kernels = {n: {"ms_per_launch": kernel_ms[j] / passes, "share": kernel_ms[j] / ksum} for j, n in enumerate(names)}
+        osum = max(1e-9, sum(overlap_ms))
+        overlapped = {n: {"ms_per_launch": overlap_ms[j] / max(1, overlap_passes), "share": overlap_ms[j] / osum}
+                      for j, n in enumerate(names)}
         dom = max(range(4), key=lambda j: kernel_ms[j])
         dom_ms = kernel_ms[dom] / passes
-        bytes_per_launch = bytes_per_step * args.steps / passes
+        bytes_per_launch = bytes_per_step * iso_steps / passes
         achieved = bytes_per_launch / (dom_ms * 1e-3) / 1e9
         path_achieved = bytes_per_step / (verify_ms * 1e-3) / 1e9
         per_cand = TRAFFIC_PER_CANDIDATE.get(names[dom])
-        traffic = per_cand * K * args.steps / passes if per_cand else None
+        traffic = per_cand * K * iso_steps / passes if per_cand else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -297,9 +326,14 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "kernel": names[dom], "of": peak_kind,
                          "launches": passes, "ms_per_launch": dom_ms, "bytes_per_launch": bytes_per_launch,
-                         "path": {"what": "all kernels of one vl_verify call", "achieved": path_achieved,
-                                  "frac": path_achieved / peak, "ms": verify_ms},
-                         "kernels": kernels},
+                         "how": f"CUDA events around every launch, {iso_steps} vl_verify calls with their passes in order "
+                                "on one stream (VL_OPT_LANES=1), so that no other kernel runs beside the timed one",
+                         "path": {"what": "one vl_verify call as the timed region runs it (passes spread over the "
+                                          "library's internal streams, kernels overlapping)",
+                                  "achieved": path_achieved, "frac": path_achieved / peak, "ms": verify_ms},
+                         "path_in_order": {"what": "one vl_verify call with VL_OPT_LANES=1", "ms": iso_verify_ms,
+                                           "frac": bytes_per_step / (iso_verify_ms * 1e-3) / 1e9 / peak},
+                         "kernels": kernels, "kernels_in_timed_region": overlapped},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(2 * prog.pitch * K),
                     "d2h_bytes_per_step": int(16 * K)},
@@ -308,7 +342,7 @@ def main():
         }
         if not args.no_cpu_baseline and world == 1:
             threads = os.cpu_count() or 1
-            sample = min(K, max(threads * 16, 256))
+            sample = min(K, max(threads * 256, 1024))
             rate, dt, t_live, ov, _ = oracle_rate(prog, arr, sample, threads)
             line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
                                     "sample": f"first {sample} rows of the same workload, {dt:.1f}s on {threads} threads "
