@@ -14,6 +14,9 @@
 
 #define NT 128  // threads per block in every kernel of this file
 #define PIECE_INSTRS 8
+#ifndef VL_ITEM_CHUNKS
+#define VL_ITEM_CHUNKS 16  // chunks per walk work item
+#endif
 
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ bool bit_get(const uint32_t *s, uint32_t v) { return (s[v >> 5] >> (v & 31)) & 1u; }
@@ -674,10 +677,10 @@ static int vl_layout(vl_program *p, cudaStream_t st)
     // walk work items: runs of at most 16 chunks of one block
     std::vector<uint32_t> it_blk, it_c0, it_c1;
     for (uint32_t b = 0; b < nB; ++b)
-        for (uint32_t c = blk_c_off[b]; c < blk_c_off[b + 1]; c += 16) {
+        for (uint32_t c = blk_c_off[b]; c < blk_c_off[b + 1]; c += VL_ITEM_CHUNKS) {
             it_blk.push_back(b);
             it_c0.push_back(c);
-            it_c1.push_back(std::min(c + 16, blk_c_off[b + 1]));
+            it_c1.push_back(std::min(c + VL_ITEM_CHUNKS, blk_c_off[b + 1]));
         }
     p->nItems = (uint32_t)it_blk.size();
     auto up = [&](uint32_t **dst, const std::vector<uint32_t> &v) -> int {

@@ -562,7 +562,13 @@ __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tg
     const uint4 a = lds128_at<0>(ga), b = lds128_at<16>(ga);
     const uint32_t off[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-    for (int u = 0; u < 8; ++u) t[u] = *reinterpret_cast<const uint16_t *>(tgb + off[u]);
+    for (int u = 0; u < 8; ++u) {
+        // base + offset as one multiply-add: the integer ALU pipe is the walk's bottleneck, the
+        // multiply-add pipe has room
+        unsigned long long addr;
+        asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(addr) : "r"(off[u]), "l"(tgb));
+        t[u] = *reinterpret_cast<const uint16_t *>(addr);
+    }
 }
 
 // Applies the 8 events of the group at shared address ga to this lane's occupancy mask; returns the
@@ -596,9 +602,15 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const uint32_t tv = t[u];
-            const uint32_t a = occ_addr + (tv & 0x7FE0u) * 4u;  // word (tv / 32) of this lane's mask
-            const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, ez[u], tv));
-            viol |= o & __funnelshift_l(0u, ey[u], tv);
+            // word (tv / 32) of this lane's mask; the masks are moved to bit (tv & 31) by a multiplication
+            // with 1 << (tv & 31), again to spare the integer ALU pipe
+            uint32_t a, mz, my;
+            const uint32_t p2 = __funnelshift_l(0u, 1u, tv);
+            asm("mad.lo.u32 %0, %1, 4, %2;" : "=r"(a) : "r"(tv & 0x7FE0u), "r"(occ_addr));
+            asm("mul.lo.u32 %0, %1, %2;" : "=r"(mz) : "r"(ez[u]), "r"(p2));
+            asm("mul.lo.u32 %0, %1, %2;" : "=r"(my) : "r"(ey[u]), "r"(p2));
+            const uint32_t o = atom_xor_shared(a, mz);
+            viol |= o & my;
         }
         return viol;
     }
