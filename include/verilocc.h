@@ -49,8 +49,9 @@ enum {
     VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
     VL_OPT_KERNEL_TIMING = 5,/* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
                                 set at any time; setting it discards the events recorded so far */
-    VL_OPT_LANES = 6         /* internal streams the passes of vl_verify / vl_verify_batch are spread over, 1..4
-                                (default 3); 1 = every kernel in order on the caller's stream */
+    VL_OPT_LANES = 6         /* internal streams the passes of vl_verify are spread over, 1..8 (default 3);
+                                1 = every kernel in order on the caller's stream.  vl_verify_batch reads the
+                                option of its first program: 1 = in order, anything else = all 8 streams */
 };
 
 /*

@@ -32,7 +32,7 @@ enum : uint32_t {
 };
 
 #define VL_MAX_GROUP 4
-#define VL_LANES 4  // internal streams that the passes of a device-resident verify call are spread over
+#define VL_LANES 8  // internal streams that the passes of device-resident verify calls can be spread over
 
 // Device memory pool of a program handle: slabs are kept across calls, so that a repeated
 // vl_liveness on the same handle allocates nothing.
@@ -136,7 +136,7 @@ struct vl_program {
     } vs[VL_LANES + 2];              // one per lane, then one per staging buffer of vl_verify_host
     uint32_t sub_batch = 4096;       // candidates per pass of the verify kernels
     uint32_t lanes_opt = 3;          // lanes in use (1 = everything in order on the caller's stream)
-    cudaEvent_t ev_fork = nullptr, ev_join[VL_LANES] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_fork = nullptr, ev_join[VL_LANES] = {};
 
     // opt-in per-kernel timing of vl_verify: five events per pass (before each of the four kernels, after the last)
     int ktime = 0;

@@ -16,6 +16,7 @@
 // k_recount  candidates with a collision are recounted exactly from the per-instruction live-after
 //            lists, one thread block per piece of a colliding chunk.
 #include <algorithm>
+#include <mutex>
 
 #include "vl_internal.cuh"
 
@@ -1126,8 +1127,6 @@ Plan make_plan(const vl_program *p, uint32_t G, uint32_t NT, uint32_t budget)
 template <int G, int NT>
 cudaError_t launch_tables(const TParams &q, uint32_t grid, uint32_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(k_tables<G, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     k_tables<G, NT><<<grid, NT, smem, st>>>(q);
     return cudaGetLastError();
 }
@@ -1196,7 +1195,7 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->Wp = (p->P + p->wmax + 31) / 32;
     pp->ev_cap = 256;
     pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + (pp->ev_cap >> 3) * 28)) * 4;
-    if (pp->walk_smem > SM_BYTES) return VL_ERR_UNSUPPORTED;
+    if (pp->walk_smem > SM_BYTES - 1024) return VL_ERR_UNSUPPORTED;
     // the recount keeps one cache word per vreg in shared memory when that leaves room for several
     // thread blocks per SM, else it fetches from global memory every time
     pp->rc_smem = (uint64_t)p->V * 4 <= 72 * 1024 ? (uint32_t)align16((uint64_t)(p->V + 4) * 4) : 0u;
@@ -1207,15 +1206,28 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     const uint64_t sub_cap =
         std::max<uint64_t>(32, ((8ull << 20) / ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) / 32 * 32);
     pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
-    cudaError_t e = cudaSuccess;
-    if (pp->walk_smem > 48 * 1024) {
-        const int sm = (int)pp->walk_smem;
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    // once per device: every verify kernel may use the whole shared memory of an SM
+    static std::mutex attr_mutex;
+    static bool attr_done[64];
+    if (p->device >= 0 && p->device < 64) {
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (!attr_done[p->device]) {
+            const int sm = (int)SM_BYTES;
+            const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+            // (the walk and the recount also have a few bytes of static shared memory)
+            cudaError_t e = cudaFuncSetAttribute(k_walk<true>, at, sm - 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false>, at, sm - 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_recount<true>, at, sm - 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<4, 256>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<2, 256>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<1, 256>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<4, 512>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<2, 512>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<1, 512>, at, sm);
+            if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+            attr_done[p->device] = true;
+        }
     }
-    if (e == cudaSuccess && pp->rc_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(k_recount<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pp->rc_smem);
-    if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
     return VL_OK;
 }
 
@@ -1336,7 +1348,8 @@ int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16
     cudaStream_t *lane = nullptr;
     int rc = vl_lane_streams(p0, &lane);
     if (rc != VL_OK) return rc;
-    const uint32_t L = std::min<uint32_t>(VL_LANES, std::max<uint32_t>(1, p0->lanes_opt));
+    // several programs in one call are small jobs bound by launch latency: they take every lane
+    const uint32_t L = p0->lanes_opt == 1 ? 1u : (nprog > 1 ? (uint32_t)VL_LANES : std::min<uint32_t>(VL_LANES, p0->lanes_opt));
     uint64_t jobs = 0;
     for (uint32_t j = 0; j < nprog; ++j) jobs += (K[j] + progs[j]->sub_batch - 1) / progs[j]->sub_batch;
     if (L == 1 || jobs <= 1) {

@@ -1,0 +1,104 @@
+"""Throughput of vl_liveness + vl_verify on the five synthetic workloads, one line per workload.
+
+    python -m paper_2506_17506_b200.workloads_report [--steps N]
+
+For every workload: candidate verifications per second and operand checks per second with the rows
+resident in device memory (CUDA events around `steps` repetitions of liveness + verify, after
+warm-up), the same for vl_verify alone, the algorithmic bytes per second (2 bytes per operand
+column + a 16-byte verdict per candidate) and their fraction of the measured copy bandwidth.  The
+small workloads move kilobytes per call and are bound by launch latency: read their latency, not
+their bandwidth fraction.  Workload 4 (256 independent programs) goes through vl_verify_batch.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+from . import synth
+
+
+def peak_gbs() -> float:
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--workloads", default="1,2,3,4,5")
+    args = ap.parse_args()
+    import torch
+    from . import binding as vl
+
+    peak = peak_gbs()
+    stream = torch.cuda.current_stream()
+    for idx in [int(x) - 1 for x in args.workloads.split(",")]:
+        wl = synth.workload(idx)
+        progs, gps, cands, outs = [], [], [], []
+        for shape, seed in zip(wl.shapes, wl.seeds):
+            p = synth.build_program(shape, seed)
+            rows = np.empty((wl.K, p.pitch), dtype=np.uint16)
+            synth.candidate_rows(p, wl.K, wl.fault_rate, seed, 0, wl.K, out=rows, chunk=256)
+            progs.append(p)
+            gps.append(vl.Program(p))
+            cands.append(torch.from_numpy(rows.view(np.int16)).cuda().view(torch.uint16))
+            outs.append(torch.empty((wl.K, 4), dtype=torch.int32, device="cuda"))
+
+        def liveness():
+            for gp in gps:
+                gp.vl_liveness(stream)
+
+        def verify():
+            if len(gps) == 1:
+                gps[0].vl_verify(cands[0], outs[0], stream)
+            else:
+                vl.vl_verify_batch(gps, cands, outs, stream)
+
+        for _ in range(3):
+            liveness()
+            verify()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        ev[0].record(stream)
+        for _ in range(args.steps):
+            liveness()
+            verify()
+        ev[1].record(stream)
+        ev[2].record(stream)
+        for _ in range(args.steps):
+            verify()
+        ev[3].record(stream)
+        torch.cuda.synchronize()
+        for gp in gps:
+            gp.vl_verify_status(stream)
+        step_ms = ev[0].elapsed_time(ev[1]) / args.steps
+        verify_ms = ev[2].elapsed_time(ev[3]) / args.steps
+        n_cand = wl.K * len(progs)
+        n_checks = sum(p.n_operands for p in progs) * wl.K
+        n_bytes = sum(2 * p.pitch + 16 for p in progs) * wl.K
+        n_pass = sum(int((o[:, 0] == vl.VL_PASS).sum()) for o in outs)
+        print(json.dumps({
+            "workload": idx + 1, "name": wl.name, "programs": len(progs), "candidates": n_cand,
+            "operand_columns": int(sum(p.n_operands for p in progs)), "rows_passing": n_pass,
+            "step_ms": step_ms, "verify_ms": verify_ms,
+            "verifications_per_sec": n_cand / (step_ms * 1e-3),
+            "operand_checks_per_sec": n_checks / (step_ms * 1e-3),
+            "verify_only_verifications_per_sec": n_cand / (verify_ms * 1e-3),
+            "verify_only_gb_per_sec": n_bytes / (verify_ms * 1e-3) / 1e9,
+            "verify_only_frac_of_measured_copy_peak": n_bytes / (verify_ms * 1e-3) / 1e9 / peak,
+        }), flush=True)
+        for gp in gps:
+            gp.close()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

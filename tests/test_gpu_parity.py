@@ -197,7 +197,7 @@ def test_register_file_too_large_is_refused(B):
     gp.close()
 
 
-@pytest.mark.parametrize("lanes,sub", [(1, 64), (2, 32), (3, 96), (4, 32), (4, 4096)])
+@pytest.mark.parametrize("lanes,sub", [(1, 64), (2, 32), (3, 96), (4, 32), (8, 32), (4, 4096)])
 def test_passes_over_lanes(B, oracle_mod, lanes, sub):
     """Many passes spread over the internal streams give the records of a single pass."""
     wl = synth.workload(1)
