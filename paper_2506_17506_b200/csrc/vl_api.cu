@@ -161,7 +161,10 @@ extern "C" void vl_program_destroy(vl_program *p)
 {
     if (!p) return;
     cudaSetDevice(p->device);
+    vl_live_settle(p);
     vl_free_liveness(p);
+    if (p->h_live) cudaFreeHost(p->h_live);
+    if (p->ev_live) cudaEventDestroy(p->ev_live);
     p->live_arena.release();
     p->tmp_arena.release();
     p->layout_arena.release();
@@ -188,6 +191,7 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     switch (option) {
     case VL_OPT_CHUNK_INSTRS:
         if (value < 8 || value > 65536) return VL_ERR_INVALID_ARG;
+        vl_live_settle(p);
         p->chunk_instrs = value;
         p->live_ok = false;
         return VL_OK;
@@ -228,6 +232,10 @@ extern "C" int vl_liveness_result(const vl_program *p, const uint32_t **blk_live
                                   const uint32_t **lo_off, const uint32_t **lo, uint64_t *lo_len)
 {
     if (!p) return VL_ERR_INVALID_ARG;
+    if (p->live_pending) {
+        const int rc = vl_live_settle(const_cast<vl_program *>(p));
+        if (rc != VL_OK) return rc;
+    }
     if (!p->live_ok) return VL_ERR_LIVENESS_NOT_RUN;
     if (blk_live_in) *blk_live_in = p->d_blk_in;
     if (blk_live_out) *blk_live_out = p->d_blk_out;
@@ -256,7 +264,11 @@ extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K
     if (rc != VL_OK || K == 0) return rc;
     cudaError_t e = cudaSetDevice(p->device);
     if (e != cudaSuccess) return VL_ERR_CUDA;
-    return vl_verify_lanes(1, &p, &d_cand, &K, &pitch, &d_out, (cudaStream_t)stream);
+    rc = vl_verify_lanes(1, &p, &d_cand, &K, &pitch, &d_out, (cudaStream_t)stream);
+    // a repeated liveness run may still be in flight: the kernels above are ordered behind it on the
+    // stream; its outcome is checked here, after they have been enqueued
+    const int rl = vl_live_settle(const_cast<vl_program *>(p));
+    return rc != VL_OK ? rc : rl;
 }
 
 extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
@@ -273,8 +285,13 @@ extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const
     uint32_t first = 0;  // the first program with rows lends its fork / join events
     while (first < n && K[first] == 0) ++first;
     if (first == n) return VL_OK;
-    return vl_verify_lanes(n - first, progs + first, d_cand + first, K + first, pitch + first, d_out + first,
-                           (cudaStream_t)stream);
+    int rc = vl_verify_lanes(n - first, progs + first, d_cand + first, K + first, pitch + first, d_out + first,
+                             (cudaStream_t)stream);
+    for (uint32_t j = 0; j < n; ++j) {
+        const int rl = vl_live_settle(const_cast<vl_program *>(progs[j]));
+        if (rc == VL_OK) rc = rl;
+    }
+    return rc;
 }
 
 extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K, uint64_t pitch, vl_verdict *h_out,
@@ -283,6 +300,7 @@ extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K,
     int rc = check_verify_args(p, h_cand, K, pitch, h_out);
     if (rc != VL_OK || K == 0) return rc;
     VL_CUDA(p, cudaSetDevice(p->device));
+    if ((rc = vl_live_settle(p)) != VL_OK) return rc;
     // slabs of about 64 MiB, a multiple of 4 rows
     uint64_t rows = std::max<uint64_t>(4, ((64ull << 20) / (pitch * 2)) / 4 * 4);
     rows = std::min<uint64_t>(rows, (K + 3) / 4 * 4);

@@ -123,6 +123,12 @@ struct vl_program {
     uint32_t *d_status = nullptr;  // [16] device status words
     int last_cuda_error = 0;
     bool live_ok = false;
+    // A repeated liveness run (same layout, lengths remembered) does not wait for the GPU: its status
+    // word and list lengths are copied to pinned host memory behind the kernels, and the next call
+    // that needs the results on the host side (vl_live_settle) waits for the copy and checks them.
+    uint32_t *h_live = nullptr;      // pinned: [0] status, [2..9] four 64-bit totals
+    cudaEvent_t ev_live = nullptr;
+    bool live_pending = false;
 
     // per-call working memory of vl_verify (one set per internal stream slot), grown on demand
     struct VScratch {
@@ -170,3 +176,5 @@ int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16
 // The lane streams of the handle's device (created once per device) and the handle's fork / join events.
 int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);
+// Waits for a liveness run that is still in flight and checks its outcome; VL_OK if none is pending.
+int vl_live_settle(vl_program *p);

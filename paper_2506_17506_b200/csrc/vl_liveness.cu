@@ -8,6 +8,7 @@
 //   of every piece (count, then fill) giving the per-instruction live-after lists in CSR form and
 //   the per-operand flags -> operand metadata, walk events, through-sets.
 #include <algorithm>
+#include <cstring>
 #include <vector>
 
 #include "vl_internal.cuh"
@@ -703,6 +704,7 @@ static int vl_layout(vl_program *p, cudaStream_t st)
 
 int vl_liveness_impl(vl_program *p, cudaStream_t st)
 {
+    vl_live_settle(p);  // the pinned words of an earlier run are about to be reused
     vl_free_liveness(p);
     int rc = vl_layout(p, st);
     if (rc != VL_OK) return rc;
@@ -830,21 +832,38 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
            p->d_el_count);
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
-    VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 32, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaStreamSynchronize(st));
+    p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
+    if (!p->h_live) VL_CUDA(p, cudaHostAlloc((void **)&p->h_live, 64, cudaHostAllocDefault));
+    if (!p->ev_live) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_live, cudaEventDisableTiming));
+    VL_CUDA(p, cudaMemcpyAsync(p->h_live, p->d_status, 4, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 32, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaEventRecord(p->ev_live, st));
     VL_CUDA(p, cudaGetLastError());
+    p->live_pending = true;
+    p->live_ok = true;
+    if (p->sizes_known) return VL_OK;  // lengths remembered from an earlier run: checked when the results are used
+    rc = vl_live_settle(p);
+    if (rc == VL_OK) p->sizes_known = true;
+    return rc;
+}
+
+int vl_live_settle(vl_program *p)
+{
+    if (!p->live_pending) return VL_OK;
+    p->live_pending = false;
+    p->live_ok = false;
+    VL_CUDA(p, cudaEventSynchronize(p->ev_live));
+    const uint32_t status = p->h_live[0];
+    unsigned long long h_tot[4];
+    memcpy(h_tot, p->h_live + 2, 32);
     if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
     if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
     if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
     if (h_tot[0] != p->known_lo_len || h_tot[2] != p->known_steps || h_tot[3] != p->known_thn) {
-        // the remembered lengths do not fit what was just computed: measure again
-        const bool retry = p->sizes_known;
+        // the lengths the run allocated from do not fit what it computed: the next run measures again
         p->sizes_known = false;
-        return retry ? vl_liveness_impl(p, st) : VL_ERR_CUDA;
+        return VL_ERR_CUDA;
     }
-    p->sizes_known = true;
-    p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     p->live_ok = true;
     return VL_OK;
 }
