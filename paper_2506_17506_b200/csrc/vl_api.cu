@@ -162,6 +162,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     if (!p) return;
     cudaSetDevice(p->device);
     vl_live_settle(p);
+    vl_drop_live_graph(p);
     vl_free_liveness(p);
     if (p->h_live) cudaFreeHost(p->h_live);
     if (p->ev_live) cudaEventDestroy(p->ev_live);

@@ -129,6 +129,11 @@ struct vl_program {
     uint32_t *h_live = nullptr;      // pinned: [0] status, [2..9] four 64-bit totals
     cudaEvent_t ev_live = nullptr;
     bool live_pending = false;
+    // the recorded form of a liveness run with settled layout and lengths (see vl_liveness_impl)
+    cudaGraphExec_t live_graph = nullptr;
+    uint64_t live_graph_launches = 0;
+    uint32_t settled_runs = 0;
+    int graph_opt = 1;
 
     // per-call working memory of vl_verify (one set per internal stream slot), grown on demand
     struct VScratch {
@@ -178,3 +183,4 @@ int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);
 // Waits for a liveness run that is still in flight and checks its outcome; VL_OK if none is pending.
 int vl_live_settle(vl_program *p);
+void vl_drop_live_graph(vl_program *p);

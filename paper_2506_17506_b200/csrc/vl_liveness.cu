@@ -702,12 +702,13 @@ static int vl_layout(vl_program *p, cudaStream_t st)
     return VL_OK;
 }
 
-int vl_liveness_impl(vl_program *p, cudaStream_t st)
+// Enqueues one complete liveness run on st (every kernel, the clears before them, the copy of the
+// status word and the list lengths to pinned host memory behind them).  Without remembered list
+// lengths it waits once in the middle to read them.
+static int live_enqueue(vl_program *p, cudaStream_t st)
 {
-    vl_live_settle(p);  // the pinned words of an earlier run are about to be reused
     vl_free_liveness(p);
-    int rc = vl_layout(p, st);
-    if (rc != VL_OK) return rc;
+    int rc = VL_OK;
     const uint32_t nB = p->nB, nI = p->nI, V = p->V, nO = p->nO, Wv = p->Wv, nC = p->nC, nP = p->nP;
     const size_t smem2 = (size_t)2 * Wv * 4;
     const size_t walk_smem = smem2 + (size_t)(2 * WALK_CAP_I + 1 + WALK_CAP_O) * 4 + WALK_CAP_I + 16;
@@ -833,18 +834,81 @@ int vl_liveness_impl(vl_program *p, cudaStream_t st)
     LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
-    if (!p->h_live) VL_CUDA(p, cudaHostAlloc((void **)&p->h_live, 64, cudaHostAllocDefault));
-    if (!p->ev_live) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_live, cudaEventDisableTiming));
     VL_CUDA(p, cudaMemcpyAsync(p->h_live, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 32, cudaMemcpyDeviceToHost, st));
+    return rc;
+}
+
+// A run is the same sequence of launches with the same arguments every time once the layout and
+// the list lengths are settled (the pools hand out the same addresses after a rewind).  The third
+// run with settled lengths is therefore recorded as a CUDA graph while it is enqueued, and later
+// runs replay the graph: one launch call instead of about thirty, which is what small programs and
+// batches of programs spend their time on.  Everything is recomputed on the device on every run.
+int vl_liveness_impl(vl_program *p, cudaStream_t st)
+{
+    vl_live_settle(p);  // the pinned words of an earlier run are about to be reused
+    int rc = vl_layout(p, st);
+    if (rc != VL_OK) return rc;
+    if (!p->h_live) VL_CUDA(p, cudaHostAlloc((void **)&p->h_live, 64, cudaHostAllocDefault));
+    if (!p->ev_live) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_live, cudaEventDisableTiming));
+    if (!p->sizes_known) vl_drop_live_graph(p);
+    bool replayed = false;
+    if (p->sizes_known && p->live_graph) {
+        if (cudaGraphLaunch(p->live_graph, st) == cudaSuccess) {
+            g_vl_launches.fetch_add(p->live_graph_launches);
+            replayed = true;
+        } else {
+            cudaGetLastError();
+            vl_drop_live_graph(p);
+        }
+    }
+    if (!replayed) {
+        bool capturing = false;
+        cudaStream_t rec = st;
+        if (p->sizes_known && p->graph_opt && ++p->settled_runs >= 2) {
+            // recorded on an internal stream (the caller's may be the legacy default stream, which
+            // cannot record; nothing runs while recording), then launched on the caller's
+            cudaStream_t *lanes = nullptr;
+            if (vl_lane_streams(p, &lanes) == VL_OK) {
+                rec = lanes[0];
+                capturing = cudaStreamBeginCapture(rec, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+            }
+            if (!capturing) { cudaGetLastError(); p->graph_opt = 0; rec = st; }
+        }
+        const uint64_t launches0 = g_vl_launches.load();
+        rc = live_enqueue(p, rec);
+        if (capturing) {
+            cudaGraph_t graph = nullptr;
+            cudaError_t e = cudaStreamEndCapture(rec, &graph);
+            if (e == cudaSuccess && rc == VL_OK) e = cudaGraphInstantiate(&p->live_graph, graph, 0);
+            if (graph) cudaGraphDestroy(graph);
+            if (e != cudaSuccess || rc != VL_OK) {
+                cudaGetLastError();
+                vl_drop_live_graph(p);
+                p->graph_opt = 0;  // recording does not work here: enqueue directly from now on
+                if (rc == VL_OK) rc = live_enqueue(p, st);
+            } else {
+                p->live_graph_launches = g_vl_launches.load() - launches0;
+                VL_CUDA(p, cudaGraphLaunch(p->live_graph, st));  // what was recorded has not run yet
+            }
+        }
+        if (rc != VL_OK) return rc;
+    }
     VL_CUDA(p, cudaEventRecord(p->ev_live, st));
     VL_CUDA(p, cudaGetLastError());
     p->live_pending = true;
     p->live_ok = true;
     if (p->sizes_known) return VL_OK;  // lengths remembered from an earlier run: checked when the results are used
     rc = vl_live_settle(p);
-    if (rc == VL_OK) p->sizes_known = true;
+    if (rc == VL_OK) { p->sizes_known = true; p->settled_runs = 0; }
     return rc;
+}
+
+void vl_drop_live_graph(vl_program *p)
+{
+    if (p->live_graph) cudaGraphExecDestroy(p->live_graph);
+    p->live_graph = nullptr;
+    p->settled_runs = 0;
 }
 
 int vl_live_settle(vl_program *p)
