@@ -106,11 +106,24 @@ int vl_program_set_option(vl_program *prog, int option, uint32_t value);
  * rest on): per-block read/write bitsets, backward dataflow to the least fixed point,
  * then the set of vregs live after every instruction as CSR lists (ascending ids),
  * plus the per-program tables vl_verify consumes.  Runs on `cuda_stream`
- * (a cudaStream_t, may be NULL) and synchronises it before returning, because list
- * lengths and the status word are read back.
+ * (a cudaStream_t, may be NULL).  The first run of a handle (and the first after the chunk
+ * size changed) synchronises the stream before returning, because list lengths and the
+ * status word are read back; it is the run that reports NOT_STRICT or NO_CONVERGE.  Later
+ * runs recompute everything on the device but allocate from the remembered lengths and
+ * return without waiting: their outcome is checked by the next call that uses the results
+ * (vl_verify*, vl_liveness_result, vl_liveness), which may then return the error.  From the
+ * third such run on the sequence of kernels is replayed as a CUDA graph.
  * Errors: NOT_STRICT, NO_CONVERGE, UNSUPPORTED, CUDA.
  */
 int vl_liveness(vl_program *prog, void *cuda_stream);
+
+/*
+ * vl_liveness for n independent programs (all on the device of the first) in one call: the
+ * runs are spread over internal streams that fork from and join back into `cuda_stream`, so
+ * that the short kernels of different programs run side by side.  `progs` is HOST memory.
+ * Stops at the first error and returns it.  Errors: as vl_liveness, INVALID_ARG.
+ */
+int vl_liveness_batch(uint32_t n, vl_program *const *progs, void *cuda_stream);
 
 /*
  * Device pointers to the liveness results; owned by the handle, valid until

@@ -26,7 +26,7 @@ VL_ERR_UNSUPPORTED, VL_ERR_NO_CONVERGE, VL_ERR_CUDA, VL_ERR_DEVICE_WAIT = -5, -6
 VL_PASS, VL_INCONSISTENT, VL_OUT_OF_RANGE, VL_INTERFERENCE = 1, 2, 4, 8
 VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERNEL_TIMING, VL_OPT_LANES = 1, 2, 3, 4, 5, 6
 
-EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness",
+EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
            "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static"]
 
@@ -51,6 +51,8 @@ _lib.vl_kernel_times.restype = C.c_int
 _lib.vl_kernel_times.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_uint32)]
 _lib.vl_liveness.restype = C.c_int
 _lib.vl_liveness.argtypes = [C.c_void_p, C.c_void_p]
+_lib.vl_liveness_batch.restype = C.c_int
+_lib.vl_liveness_batch.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p]
 _lib.vl_liveness_result.restype = C.c_int
 _lib.vl_liveness_result.argtypes = [C.c_void_p] + [C.POINTER(C.c_void_p)] * 4 + [C.POINTER(C.c_uint64)]
 _lib.vl_verify.restype = C.c_int
@@ -238,6 +240,15 @@ def vl_block_liveness_static(n_blocks, n_vregs, block_instr_off, succ_off, succ,
     return int(_lib.vl_block_liveness_static(device, n_blocks, n_vregs, ptr(block_instr_off), ptr(succ_off), ptr(succ),
                                              ptr(instr_op_off), ptr(instr_n_defs), ptr(op_vreg), ptr(live_in),
                                              ptr(live_out), _stream_ptr(stream)))
+
+
+def vl_liveness_batch(programs, stream=None):
+    """vl_liveness on every program of the list in one call."""
+    n = len(programs)
+    hp = (C.c_void_p * n)(*[p.handle for p in programs])
+    rc = _lib.vl_liveness_batch(n, hp, _stream_ptr(stream))
+    if rc != VL_OK:
+        raise VlError(rc, "vl_liveness_batch")
 
 
 def vl_verify_batch(programs, cands, outs=None, stream=None):

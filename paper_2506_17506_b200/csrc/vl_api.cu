@@ -229,6 +229,31 @@ extern "C" int vl_liveness(vl_program *p, void *stream)
     return vl_liveness_impl(p, (cudaStream_t)stream);
 }
 
+extern "C" int vl_liveness_batch(uint32_t n, vl_program *const *progs, void *stream)
+{
+    if (n == 0) return VL_OK;
+    if (!progs) return VL_ERR_INVALID_ARG;
+    for (uint32_t j = 0; j < n; ++j)
+        if (!progs[j] || progs[j]->device != progs[0]->device) return VL_ERR_INVALID_ARG;
+    vl_program *p0 = progs[0];
+    VL_CUDA(p0, cudaSetDevice(p0->device));
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaStream_t *lane = nullptr;
+    int rc = vl_lane_streams(p0, &lane);
+    if (rc != VL_OK) return rc;
+    if (n == 1) return vl_liveness_impl(p0, st);
+    VL_CUDA(p0, cudaEventRecord(p0->ev_fork, st));
+    for (uint32_t l = 0; l < VL_LANES; ++l) VL_CUDA(p0, cudaStreamWaitEvent(lane[l], p0->ev_fork, 0));
+    for (uint32_t j = 0; j < n && rc == VL_OK; ++j) rc = vl_liveness_impl(progs[j], lane[j % VL_LANES]);
+    // join even after an error, so that the caller's stream stays ordered after what was launched
+    for (uint32_t l = 0; l < VL_LANES; ++l) {
+        cudaError_t e = cudaEventRecord(p0->ev_join[l], lane[l]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, p0->ev_join[l], 0);
+        if (e != cudaSuccess && rc == VL_OK) { p0->last_cuda_error = (int)e; rc = VL_ERR_CUDA; }
+    }
+    return rc;
+}
+
 extern "C" int vl_liveness_result(const vl_program *p, const uint32_t **blk_live_in, const uint32_t **blk_live_out,
                                   const uint32_t **lo_off, const uint32_t **lo, uint64_t *lo_len)
 {

@@ -7,7 +7,8 @@ resident in device memory (CUDA events around `steps` repetitions of liveness + 
 warm-up), the same for vl_verify alone, the algorithmic bytes per second (2 bytes per operand
 column + a 16-byte verdict per candidate) and their fraction of the measured copy bandwidth.  The
 small workloads move kilobytes per call and are bound by launch latency: read their latency, not
-their bandwidth fraction.  Workload 4 (256 independent programs) goes through vl_verify_batch.
+their bandwidth fraction.  Workload 4 (256 independent programs) goes through vl_liveness_batch
+and vl_verify_batch.
 """
 from __future__ import annotations
 
@@ -53,8 +54,10 @@ def main() -> int:
             outs.append(torch.empty((wl.K, 4), dtype=torch.int32, device="cuda"))
 
         def liveness():
-            for gp in gps:
-                gp.vl_liveness(stream)
+            if len(gps) == 1:
+                gps[0].vl_liveness(stream)
+            else:
+                vl.vl_liveness_batch(gps, stream)
 
         def verify():
             if len(gps) == 1:

@@ -39,6 +39,10 @@ def _assert_same(got, want, what=""):
 def _check_liveness(B, oracle_mod, p, gp=None):
     gp = gp or B.Program(p)
     gp.vl_liveness()
+    return _check_liveness_result(B, oracle_mod, gp, p)
+
+
+def _check_liveness_result(B, oracle_mod, gp, p):
     bin_, bout, lo_off, lo = gp.vl_liveness_result()
     lv = oracle_mod.OracleProgram(p).liveness()
     assert np.array_equal(bin_, lv.packed("in"))
@@ -229,6 +233,16 @@ def test_batch_call(B, oracle_mod):
     torch.cuda.synchronize()
     for j, o, w in zip(members, outs, wants):
         _assert_same(B.verdicts_to_numpy(o), w, f"batch member {j}")
+    # liveness of all members in one call, several times (the later runs are replayed recordings):
+    # same liveness results, same verdicts
+    for _ in range(4):
+        B.vl_liveness_batch(gps)
+    for gp, p in zip(gps, progs):
+        _check_liveness_result(B, oracle_mod, gp, p)
+    outs = B.vl_verify_batch(gps, cands)
+    torch.cuda.synchronize()
+    for j, o, w in zip(members, outs, wants):
+        _assert_same(B.verdicts_to_numpy(o), w, f"batch member {j} after vl_liveness_batch")
     for gp in gps:
         gp.close()
 
