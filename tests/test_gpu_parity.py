@@ -266,6 +266,28 @@ def test_stress_workload_sampled(B, oracle_mod):
     gp.close()
 
 
+def test_repeated_liveness_runs(B, oracle_mod):
+    """Later liveness runs of a handle return without waiting for the GPU and are replayed from a
+    recording: the results stay those of the first run, a changed chunk size starts over, and the
+    verdicts computed behind an unsettled run are right."""
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    rows, _ = synth.candidate_rows(p, 64, 0.4, 3)
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    for run in range(6):
+        gp.vl_liveness()
+        if run % 2:
+            _check_liveness_result(B, oracle_mod, gp, p)
+        _assert_same(_gpu_verify(B, gp, rows), want, f"run {run}")
+    gp.set_option(B.VL_OPT_CHUNK_INSTRS, 40)
+    for run in range(5):
+        gp.vl_liveness()
+        _assert_same(_gpu_verify(B, gp, rows), want, f"chunk 40 run {run}")
+    _check_liveness_result(B, oracle_mod, gp, p)
+    gp.close()
+
+
 def test_determinism(B):
     wl = synth.workload(1)
     p = synth.build_program(wl.shapes[0], wl.seeds[0])

@@ -91,3 +91,9 @@ def test_null_arguments(B):
     lib.vl_verify.restype = C.c_int
     lib.vl_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
     assert lib.vl_verify(None, None, 1, 8, None, None) == B.VL_ERR_INVALID_ARG
+    lib.vl_liveness_batch.restype = C.c_int
+    lib.vl_liveness_batch.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p]
+    assert lib.vl_liveness_batch(0, None, None) == B.VL_OK
+    assert lib.vl_liveness_batch(2, None, None) == B.VL_ERR_INVALID_ARG
+    two_nulls = (C.c_void_p * 2)(None, None)
+    assert lib.vl_liveness_batch(2, two_nulls, None) == B.VL_ERR_INVALID_ARG
