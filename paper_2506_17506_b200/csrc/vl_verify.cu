@@ -582,9 +582,6 @@ template <bool WIDE>
 __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, uint32_t *s_occ,
                                                 uint32_t lane)
 {
-    const uint4 z0 = lds128_at<32>(ga), z1 = lds128_at<48>(ga), y0 = lds128_at<64>(ga), y1 = lds128_at<80>(ga);
-    const uint32_t ez[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
-    const uint32_t ey[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
     bool slow;
     if (!WIDE) {
         slow = ((t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & 0x8000u) != 0;
@@ -601,20 +598,28 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
     uint32_t viol = 0;
     if (!__any_sync(0xffffffffu, slow)) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const uint32_t tv = t[u];
-            // word (tv / 32) of this lane's mask; the masks are moved to bit (tv & 31) by a multiplication
-            // with 1 << (tv & 31), again to spare the integer ALU pipe
-            uint32_t a, mz, my;
-            const uint32_t p2 = __funnelshift_l(0u, 1u, tv);
-            asm("mad.lo.u32 %0, %1, 4, %2;" : "=r"(a) : "r"(tv & 0x7FE0u), "r"(occ_addr));
-            asm("mul.lo.u32 %0, %1, %2;" : "=r"(mz) : "r"(ez[u]), "r"(p2));
-            asm("mul.lo.u32 %0, %1, %2;" : "=r"(my) : "r"(ey[u]), "r"(p2));
-            const uint32_t o = atom_xor_shared(a, mz);
-            viol |= o & my;
+        for (int h = 0; h < 2; ++h) {  // the masks of four events at a time: fewer registers held
+            const uint4 z4 = h ? lds128_at<48>(ga) : lds128_at<32>(ga), y4 = h ? lds128_at<80>(ga) : lds128_at<64>(ga);
+            const uint32_t hz[4] = {z4.x, z4.y, z4.z, z4.w}, hy[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t tv = t[4 * h + u];
+                // word (tv / 32) of this lane's mask; the masks are moved to bit (tv & 31) by a
+                // multiplication with 1 << (tv & 31), again to spare the integer ALU pipe
+                uint32_t a, mz, my;
+                const uint32_t p2 = __funnelshift_l(0u, 1u, tv);
+                asm("mad.lo.u32 %0, %1, 4, %2;" : "=r"(a) : "r"(tv & 0x7FE0u), "r"(occ_addr));
+                asm("mul.lo.u32 %0, %1, %2;" : "=r"(mz) : "r"(hz[u]), "r"(p2));
+                asm("mul.lo.u32 %0, %1, %2;" : "=r"(my) : "r"(hy[u]), "r"(p2));
+                const uint32_t o = atom_xor_shared(a, mz);
+                viol |= o & my;
+            }
         }
         return viol;
     }
+    const uint4 z0 = lds128_at<32>(ga), z1 = lds128_at<48>(ga), y0 = lds128_at<64>(ga), y1 = lds128_at<80>(ga);
+    const uint32_t ez[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+    const uint32_t ey[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
     const uint4 w4 = lds128_at<96>(ga);
     const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
@@ -700,16 +705,21 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
                 for (uint32_t i = lane; i < ng * 7; i += 32) s_ev[i] = src[i];
             }
             __syncwarp();
-            // table entries of the next group are fetched while the current group is applied
-            uint32_t ta[8], tb[8];
+            // table entries are fetched two groups ahead of the group that is applied
+            uint32_t ta[8], tb[8], tc[8];
             fetch_group(ev_addr, tgb, ta);
-            for (uint32_t g = 0; g < ng; g += 2) {
+            if (ng > 1) fetch_group(ev_addr + 112, tgb, tb);
+            for (uint32_t g = 0; g < ng; g += 3) {
                 const uint32_t ga = ev_addr + g * 112;
-                if (g + 1 < ng) fetch_group(ga + 112, tgb, tb);
+                if (g + 2 < ng) fetch_group(ga + 224, tgb, tc);
                 viol |= apply_group<WIDE>(ga, ta, occ_addr, s_occ, lane);
                 if (g + 1 < ng) {
-                    if (g + 2 < ng) fetch_group(ga + 224, tgb, ta);
+                    if (g + 3 < ng) fetch_group(ga + 336, tgb, ta);
                     viol |= apply_group<WIDE>(ga + 112, tb, occ_addr, s_occ, lane);
+                }
+                if (g + 2 < ng) {
+                    if (g + 4 < ng) fetch_group(ga + 448, tgb, tb);
+                    viol |= apply_group<WIDE>(ga + 224, tc, occ_addr, s_occ, lane);
                 }
             }
         }
