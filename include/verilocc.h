@@ -43,7 +43,7 @@ enum { VL_PASS = 1u, VL_INCONSISTENT = 2u, VL_OUT_OF_RANGE = 4u, VL_INTERFERENCE
 
 /* Tunables for vl_program_set_option (set before vl_liveness). */
 enum {
-    VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 128) */
+    VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 160; long blocks get a chunk count that is a multiple of 8) */
     VL_OPT_GROUP = 2,        /* candidates per thread block: 0 = choose, else 1, 2 or 4 */
     VL_OPT_THREADS = 3,      /* threads per thread block of the table kernel: 0 = choose, else 256 or 512 */
     VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */

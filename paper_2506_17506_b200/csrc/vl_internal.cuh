@@ -73,7 +73,7 @@ struct vl_program {
     uint32_t Wv = 0;    // 32-bit words per vreg bitset
     uint32_t nOp8 = 0;  // n_operands rounded up to 8 (at least 8)
     uint32_t wmax = 1;  // widest vreg
-    uint32_t chunk_instrs = 128;
+    uint32_t chunk_instrs = 160;
     uint32_t group_opt = 0;
 
     // chunks: every chunk lies inside one block; pieces: every piece lies inside one chunk

@@ -657,7 +657,10 @@ static int vl_layout(vl_program *p, cudaStream_t st)
     std::vector<uint32_t> c_i0, c_i1, c_blk, blk_c_off(nB + 1, 0), p_i0, p_i1, p_chunk, c_p_off;
     for (uint32_t b = 0; b < nB; ++b) {
         const uint64_t s = p->h_blk_off[b], n = p->h_blk_off[b + 1] - s;
-        const uint64_t nc = (n + p->chunk_instrs - 1) / p->chunk_instrs;
+        uint64_t nc = (n + p->chunk_instrs - 1) / p->chunk_instrs;
+        // a walk item is shared by 8 warps, one chunk each at a time: a chunk count that is a multiple
+        // of 8 keeps them equally busy (the chunks get a little shorter than asked for)
+        if (nc > 4 && n >= 8 * 16) nc = (nc + 7) / 8 * 8;
         for (uint64_t j = 0; j < nc; ++j) {
             const uint32_t i0 = (uint32_t)(s + j * n / nc), i1 = (uint32_t)(s + (j + 1) * n / nc);
             c_p_off.push_back((uint32_t)p_i0.size());
