@@ -16,7 +16,7 @@
 #define NT 128  // threads per block in every kernel of this file
 #define PIECE_INSTRS 8
 #ifndef VL_ITEM_CHUNKS
-#define VL_ITEM_CHUNKS 16  // chunks per walk work item
+#define VL_ITEM_CHUNKS 32  // chunks per walk work item
 #endif
 
 // ------------------------------------------------------------------ device helpers
@@ -678,7 +678,7 @@ static int vl_layout(vl_program *p, cudaStream_t st)
     c_p_off.push_back((uint32_t)p_i0.size());
     const uint32_t nC = p->nC = (uint32_t)c_i0.size();
     p->nP = (uint32_t)p_i0.size();
-    // walk work items: runs of at most 16 chunks of one block
+    // walk work items: runs of at most VL_ITEM_CHUNKS chunks of one block
     std::vector<uint32_t> it_blk, it_c0, it_c1;
     for (uint32_t b = 0; b < nB; ++b)
         for (uint32_t c = blk_c_off[b]; c < blk_c_off[b + 1]; c += VL_ITEM_CHUNKS) {
