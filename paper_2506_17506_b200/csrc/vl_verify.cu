@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
     if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
     if (tid == 0 && (k0 & 31) == 0) q.grp_done[k0 >> 5] = 0;
-    if (tid == 0 && blockIdx.x == 0) q.work[0] = 0;
+    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
     __syncthreads();
 
     auto issue_tile = [&](uint32_t t) {
@@ -855,7 +855,20 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
     const long long rc_t0 = clock64();
     if (tid == 0 && blockIdx.x == 0) atomicAdd(q.status + 8, nitems);
 #endif
-    for (uint32_t it = blockIdx.x; it < nitems; it += gridDim.x) {
+    __shared__ uint32_t s_item;
+    for (;;) {
+        // the items differ a lot in length: thread blocks take the next one from a shared cursor
+        __syncthreads();
+        if (tid == 0) s_item = atomicAdd(q.work + 1, 1u);
+        __syncthreads();
+        const uint32_t it = s_item;
+        if (it >= nitems) break;
+#ifdef VL_PHASE_TIMERS
+        long long rt = clock64();
+#define RT(idx) do { if (tid == 0) { long long n_ = clock64(); atomicAdd(q.status + (idx), (uint32_t)((n_ - rt) >> 4)); rt = n_; } } while (0)
+#else
+#define RT(idx)
+#endif
         const uint64_t k = q.work[2 + 2 * it];
         const uint32_t code = q.work[3 + 2 * it];
         const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
@@ -870,6 +883,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             for (uint32_t v = tid; v < q.V; v += RC_THREADS) Cv[v] = 0;
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
+        RT(11);
         // register (low 16 bits) and width (bits 16..23) of vreg v for this candidate
         auto fetch = [&](uint32_t v) -> uint32_t {
             const uint32_t r = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * 32] & tmask);
@@ -953,6 +967,26 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             const uint32_t i_lo = ci0 + (uint32_t)((uint64_t)cn * part / RC_PARTS);
             const uint32_t i_hi = ci0 + (uint32_t)((uint64_t)cn * (part + 1) / RC_PARTS);
             uint32_t pairs = 0, mind = 0xFFFFFFFFu;
+            if (CACHE && i_lo < i_hi) {
+                // Every vreg that is live after an instruction of the piece is live after its first
+                // instruction or defined inside the piece: the whole block fetches those into the cache in
+                // one go, so that the instruction-by-instruction recount below finds them there instead of
+                // waiting for global memory once per instruction.
+                const uint32_t l0 = q.lo_off[i_lo], l1 = q.lo_off[i_lo + 1];
+                for (uint32_t e = l0 + tid; e < l1; e += RC_THREADS) {
+                    const uint32_t v = q.lo[e];
+                    Cv[v] = fetch(v) | 0x80000000u;
+                }
+                for (uint32_t i = i_lo + tid; i < i_hi; i += RC_THREADS) {
+                    const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
+                    for (uint32_t d = o0; d < o0 + nd; ++d) {
+                        const uint32_t v = q.op_vreg[d];
+                        Cv[v] = fetch(v) | 0x80000000u;
+                    }
+                }
+                __syncthreads();
+            }
+            RT(12);
             // this warp's instructions: i_lo + warp, i_lo + warp + NW, ...; 32 of them per round
             for (uint32_t ib = i_lo + warp; ib < i_hi; ib += 32 * NW) {
                 const uint32_t my_i = ib + lane * NW;
@@ -1000,18 +1034,20 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                                 us[u] = e0 == l0 ? us0[u] : (e < l1 ? q.lo[e] : 0xFFFFFFFFu);
                                 if (us[u] == 0xFFFFFFFFu) us[u] = v;
                             }
+                            // (with the cache, every entry of the list and v itself were fetched up front)
 #pragma unroll
-                            for (int u = 0; u < 8; ++u) xs[u] = reg_w(us[u]);
+                            for (int u = 0; u < 8; ++u) xs[u] = CACHE ? Cv[us[u]] : fetch(us[u]);
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
                                 if (us[u] != v && ranges_overlap(s, w, xs[u] & 0xFFFFu, (xs[u] >> 16) & 0xFFu)) ++cnt;
                         }
                         // co-defined vregs that are not live after the instruction
-                        for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
-                            if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
-                            const uint32_t x = reg_w(q.op_vreg[d2]);
-                            if (ranges_overlap(s, w, x & 0xFFFFu, (x >> 16) & 0xFFu)) ++cnt;
-                        }
+                        if (nd > 1)
+                            for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {
+                                if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
+                                const uint32_t x = reg_w(q.op_vreg[d2]);
+                                if (ranges_overlap(s, w, x & 0xFFFFu, (x >> 16) & 0xFFu)) ++cnt;
+                            }
 #pragma unroll
                         for (int dd = 16; dd; dd >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, dd);
                         if (cnt) { pairs += cnt; mind = min(mind, i); }
@@ -1078,6 +1114,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             if (lane == 0 && bt) atomicAdd(&s_bank, bt);
         }
         __syncthreads();
+        RT(kind == RC_KIND_BANK ? 6 : (kind == RC_KIND_THROUGH ? 7 : 13));
         if (tid == 0) {
             uint32_t *acc = q.racc + k * 4;
             if (s_pairs) atomicAdd(&acc[0], s_pairs);
@@ -1099,6 +1136,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 q.out[k] = vd;
             }
         }
+        RT(14);
     }
 #ifdef VL_PHASE_TIMERS
     if (tid == 0) {
