@@ -153,6 +153,7 @@ void vl_free_liveness(vl_program *p)
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
     p->d_el = nullptr; p->d_el_count = nullptr;
+    p->d_ls = p->d_ls_adj = p->d_th_cnt = p->d_blk_th = nullptr;
     p->live_ok = false;
     p->lo_len = 0;
 }

@@ -82,7 +82,7 @@ struct vl_program {
     std::vector<uint32_t> h_blk_off, h_op_off;
     // list lengths of the last liveness run with this layout: the next run allocates from them
     bool sizes_known = false;
-    uint64_t known_lo_len = 0, known_steps = 0, known_thn = 0;
+    uint64_t known_lo_len = 0, known_steps = 0, known_thn = 0, known_ls_len = 0;
 
     // device copies of the program
     uint32_t *d_blk_off = nullptr, *d_succ_off = nullptr, *d_succ = nullptr, *d_op_off = nullptr, *d_op_vreg = nullptr;
@@ -102,6 +102,9 @@ struct vl_program {
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
     uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
+    // live-after lists without the block's through-set, for the recount: the list of instruction i of
+    // block b is ls[lo_off[i] - ls_adj[b] - i * th_cnt[b] ...), |live-after| - th_cnt[b] entries
+    uint32_t *d_ls = nullptr, *d_ls_adj = nullptr, *d_th_cnt = nullptr, *d_blk_th = nullptr;
     uint4 *d_el = nullptr;          // definitions without a walk event: {instruction, chunk, vreg, block}, any order
     uint32_t *d_el_count = nullptr;
     uint32_t th_len = 0;

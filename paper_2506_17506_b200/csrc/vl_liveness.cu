@@ -228,7 +228,11 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
                                                    const uint32_t *__restrict__ chunk_end, uint32_t *lo_cnt,
                                                    uint32_t *ev_cnt, uint8_t *opflags,
                                                    const uint32_t *__restrict__ piece_chunk, uint32_t *chunk_touch,
-                                                   const uint32_t *__restrict__ lo_off, uint32_t *lo)
+                                                   const uint32_t *__restrict__ lo_off, uint32_t *lo,
+                                                   const uint32_t *__restrict__ chunk_blk,
+                                                   const uint32_t *__restrict__ blk_th,
+                                                   const uint32_t *__restrict__ ls_adj,
+                                                   const uint32_t *__restrict__ th_cnt, uint32_t *ls)
 {
     extern __shared__ uint32_t sm[];
     uint32_t *s_live = sm, *s_touch = sm + Wv;
@@ -238,6 +242,16 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
     uint8_t *s_nd = reinterpret_cast<uint8_t *>(s_ops + WALK_CAP_O);  // [WALK_CAP_I]
     const uint32_t c = blockIdx.x, lane = threadIdx.x;
     const uint32_t i0 = chunk_i0[c], i1 = chunk_i1[c];
+    // FILL: second list per instruction without the vregs that stay occupied through the whole block
+    // (s_touch then holds the block's through-set); every instruction of the block has all of them in
+    // its live-after set, so the short list of instruction i starts at lo_off[i] - ls_adj[b] - i * th_cnt[b]
+    uint32_t ls_sub = 0, ls_mul = 0;
+    if (FILL) {
+        const uint32_t b = chunk_blk[piece_chunk[c]];
+        ls_sub = ls_adj[b];
+        ls_mul = th_cnt[b];
+        for (uint32_t w = lane; w < Wv; w += 32) s_touch[w] = blk_th[(size_t)b * Wv + w];
+    }
     for (uint32_t w = lane; w < Wv; w += 32) {
         s_live[w] = chunk_end[(size_t)c * Wv + w];
         if (!FILL) s_touch[w] = 0;
@@ -263,16 +277,22 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
             // ascending ids, 32 words per round; every non-empty word is broadcast and each lane whose
             // bit is set writes its id at the rank of that bit: up to 32 consecutive stores per word
             uint32_t at = staged ? s_lo[i - i0] : lo_off[i];
+            uint32_t at_s = at - ls_sub - i * ls_mul;
             for (uint32_t r = 0; r < rounds; ++r) {
                 const uint32_t w = r * 32 + lane;
                 const uint32_t mine = w < Wv ? s_live[w] : 0u;
+                const uint32_t mine_th = w < Wv ? s_touch[w] : 0u;
                 uint32_t nz = __ballot_sync(0xffffffffu, mine != 0);
                 while (nz) {
                     const uint32_t src = __ffs(nz) - 1;
                     nz &= nz - 1;
                     const uint32_t x = __shfl_sync(0xffffffffu, mine, src);
-                    if ((x >> lane) & 1u) lo[at + __popc(x & ((1u << lane) - 1u))] = (r * 32 + src) * 32 + lane;
+                    const uint32_t y = x & ~__shfl_sync(0xffffffffu, mine_th, src);
+                    const uint32_t id = (r * 32 + src) * 32 + lane, below = (1u << lane) - 1u;
+                    if ((x >> lane) & 1u) lo[at + __popc(x & below)] = id;
+                    if ((y >> lane) & 1u) ls[at_s + __popc(y & below)] = id;
                     at += __popc(x);
+                    at_s += __popc(y);
                 }
             }
         } else {
@@ -590,8 +610,10 @@ __global__ void k_fill_through(uint32_t Wv, const uint32_t *__restrict__ blk_th,
 // First walk event of every chunk (each chunk padded to a multiple of 8 events), first through-set
 // entry of every block, and both totals: totals[2] = events with padding, totals[3] = through entries.
 // One thread block; the arrays are short (chunks, blocks).
+// Also ls_adj[b] (see k_instr_walk) and totals[4] = length of all short live-after lists.
 __global__ void k_offsets(uint32_t nC, uint32_t nB, const uint32_t *__restrict__ cev, const uint32_t *__restrict__ th_cnt,
-                          uint32_t *cev_off, uint32_t *th_off, unsigned long long *totals)
+                          uint32_t *cev_off, uint32_t *th_off, unsigned long long *totals,
+                          const uint32_t *__restrict__ blk_off, uint32_t *ls_adj)
 {
     __shared__ uint32_t s_scan[34];
     __shared__ unsigned long long s_carry;
@@ -619,6 +641,14 @@ __global__ void k_offsets(uint32_t nC, uint32_t nB, const uint32_t *__restrict__
             s_carry = 0;
         }
         __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        unsigned long long pre = 0;  // through-set entries of all instructions of the blocks before b
+        for (uint32_t b = 0; b < nB; ++b) {
+            ls_adj[b] = (uint32_t)pre - blk_off[b] * th_cnt[b];
+            pre += (unsigned long long)(blk_off[b + 1] - blk_off[b]) * th_cnt[b];
+        }
+        totals[4] = totals[0] - pre;
     }
 }
 
@@ -728,11 +758,15 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     KEEP(&p->d_iflags, (size_t)nI);
     KEEP(&p->d_cev_off, (size_t)nC + 1);
     KEEP(&p->d_th_off, (size_t)nB + 1);
+    KEEP(&p->d_th_cnt, (size_t)nB);
+    KEEP(&p->d_ls_adj, (size_t)nB);
+    KEEP(&p->d_blk_th, (size_t)nB * Wv);
     KEEP(&p->d_el, (size_t)nO);  // at most one entry per definition
     KEEP(&p->d_el_count, 1);
 
     uint32_t *piece_use, *piece_def, *piece_end, *chunk_use, *chunk_def, *chunk_touch, *chunk_end, *chunk_entry;
-    uint32_t *blk_use, *blk_def, *blk_th, *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *th_cnt, *first_occ;
+    uint32_t *blk_use, *blk_def, *lo_cnt, *ev_cnt, *ev_off, *centry_cnt, *cev, *first_occ;
+    uint32_t *const blk_th = p->d_blk_th, *const th_cnt = p->d_th_cnt;
     uint8_t *opmeta;
     unsigned long long *totals;
     TMP(&piece_use, (size_t)nP * Wv);
@@ -744,13 +778,11 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     TMP(&chunk_entry, (size_t)nC * Wv);
     TMP(&blk_use, (size_t)nB * Wv);
     TMP(&blk_def, (size_t)nB * Wv);
-    TMP(&blk_th, (size_t)nB * Wv);
     TMP(&lo_cnt, (size_t)nI + 1);
     TMP(&ev_cnt, (size_t)nI + 1);
     TMP(&ev_off, (size_t)nI + 1);
     TMP(&centry_cnt, (size_t)nC);
     TMP(&cev, (size_t)nC);
-    TMP(&th_cnt, (size_t)nB);
     TMP(&first_occ, (size_t)V);
     TMP(&opmeta, (size_t)nO);
     TMP(&chunk_touch, (size_t)nC * Wv + 16);  // followed by the totals: one memset clears both
@@ -784,23 +816,24 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
                    piece_end, (uint32_t *)nullptr);
     if (nP) k_instr_walk<false><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
            p->d_op_vreg, Wv, piece_end, lo_cnt, ev_cnt, p->d_opflags, p->d_piece_chunk, chunk_touch,
-           (const uint32_t *)nullptr, (uint32_t *)nullptr);
+           (const uint32_t *)nullptr, (uint32_t *)nullptr, (const uint32_t *)nullptr, (const uint32_t *)nullptr,
+           (const uint32_t *)nullptr, (const uint32_t *)nullptr, (uint32_t *)nullptr);
     k_scan<<<2, 1024, 0, st>>>(lo_cnt, p->d_lo_off, ev_cnt, ev_off, nI, totals, p->d_status);
     g_vl_launches.fetch_add(nP ? 2 : 1);
     LAUNCH(k_block_through, dim3(wgrid, nB), 0, st, p->d_blk_chunk_off, Wv, p->use_th, p->d_blk_in, chunk_touch, blk_th);
     LAUNCH(k_chunk_entry, nC, 0, st, p->d_chunk_blk, p->d_chunk_i0, p->d_chunk_i1, Wv, blk_th, chunk_entry, ev_off,
            centry_cnt, cev);
     LAUNCH(k_row_popc, nB, 0, st, Wv, blk_th, th_cnt);
-    k_offsets<<<1, NT, 0, st>>>(nC, nB, cev, th_cnt, p->d_cev_off, p->d_th_off, totals);
+    k_offsets<<<1, NT, 0, st>>>(nC, nB, cev, th_cnt, p->d_cev_off, p->d_th_off, totals, p->d_blk_off, p->d_ls_adj);
     g_vl_launches.fetch_add(1);
 
     // ---- list lengths: read back on the first run with this layout; later runs allocate from the
     // lengths they remember (same program, same layout) and only compare at the end
     uint32_t status = 0;
-    unsigned long long h_tot[4] = {0, 0, 0, 0};
+    unsigned long long h_tot[5] = {0, 0, 0, 0, 0};
     if (!p->sizes_known) {
         VL_CUDA(p, cudaMemcpyAsync(&status, p->d_status, 4, cudaMemcpyDeviceToHost, st));
-        VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 32, cudaMemcpyDeviceToHost, st));
+        VL_CUDA(p, cudaMemcpyAsync(h_tot, totals, 40, cudaMemcpyDeviceToHost, st));
         VL_CUDA(p, cudaStreamSynchronize(st));
         if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
         if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
@@ -809,6 +842,7 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
         p->known_lo_len = h_tot[0];
         p->known_steps = h_tot[2];
         p->known_thn = h_tot[3];
+        p->known_ls_len = h_tot[4];
     }
     p->lo_len = p->known_lo_len;
     const uint64_t steps = p->known_steps;  // walk events in total, every chunk padded to a multiple of 8 with no-ops
@@ -816,6 +850,7 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     p->th_len = (uint32_t)p->known_thn;
 
     KEEP(&p->d_lo, (size_t)p->lo_len);
+    KEEP(&p->d_ls, (size_t)p->known_ls_len);
     KEEP(&p->d_ev, (size_t)(steps / 8) * 7);
     KEEP(&p->d_th, (size_t)p->known_thn);
     LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)(steps / 8),
@@ -823,7 +858,9 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
 
     if (nP) k_instr_walk<true><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
            p->d_op_vreg, Wv, piece_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr,
-           (const uint32_t *)nullptr, (uint32_t *)nullptr, (const uint32_t *)p->d_lo_off, p->d_lo);
+           (const uint32_t *)p->d_piece_chunk, (uint32_t *)nullptr, (const uint32_t *)p->d_lo_off, p->d_lo,
+           (const uint32_t *)p->d_chunk_blk, (const uint32_t *)blk_th, (const uint32_t *)p->d_ls_adj,
+           (const uint32_t *)th_cnt, p->d_ls);
     if (nP) g_vl_launches.fetch_add(1);
     LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_first_def_instr);
@@ -838,7 +875,7 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     VL_CUDA(p, cudaMemcpyAsync(p->h_live, p->d_status, 4, cudaMemcpyDeviceToHost, st));
-    VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 32, cudaMemcpyDeviceToHost, st));
+    VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 40, cudaMemcpyDeviceToHost, st));
     return rc;
 }
 
@@ -921,12 +958,13 @@ int vl_live_settle(vl_program *p)
     p->live_ok = false;
     VL_CUDA(p, cudaEventSynchronize(p->ev_live));
     const uint32_t status = p->h_live[0];
-    unsigned long long h_tot[4];
-    memcpy(h_tot, p->h_live + 2, 32);
+    unsigned long long h_tot[5];
+    memcpy(h_tot, p->h_live + 2, 40);
     if (status & ST_NO_CONVERGE) return VL_ERR_NO_CONVERGE;
     if (status & ST_NOT_STRICT) return VL_ERR_NOT_STRICT;
     if (status & ST_SIZE_OVERFLOW) return VL_ERR_UNSUPPORTED;
-    if (h_tot[0] != p->known_lo_len || h_tot[2] != p->known_steps || h_tot[3] != p->known_thn) {
+    if (h_tot[0] != p->known_lo_len || h_tot[2] != p->known_steps || h_tot[3] != p->known_thn ||
+        h_tot[4] != p->known_ls_len) {
         // the lengths the run allocated from do not fit what it computed: the next run measures again
         p->sizes_known = false;
         return VL_ERR_CUDA;

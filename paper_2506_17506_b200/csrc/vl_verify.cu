@@ -86,6 +86,8 @@ struct RParams {
     uint32_t *status;
     const uint4 *el;           // the definitions the walk skips: {instruction, chunk, vreg, block}
     const uint32_t *el_count;
+    const uint32_t *ls, *ls_adj, *th_cnt;  // live-after lists without the through-sets (see vl_program)
+    uint32_t R;                            // registers covered by the recount's through-set counters
 };
 
 // Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
@@ -847,7 +849,7 @@ template <bool CACHE>
 __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 {
     extern __shared__ __align__(16) uint32_t Cv[];  // [V] register | width << 16 | valid << 31
-    __shared__ uint32_t s_pairs, s_mind, s_bank;
+    __shared__ uint32_t s_pairs, s_mind, s_bank, s_big;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr uint32_t NW = RC_THREADS / 32;
     const uint32_t nitems = q.work[0];
@@ -967,21 +969,56 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             const uint32_t i_lo = ci0 + (uint32_t)((uint64_t)cn * part / RC_PARTS);
             const uint32_t i_hi = ci0 + (uint32_t)((uint64_t)cn * (part + 1) / RC_PARTS);
             uint32_t pairs = 0, mind = 0xFFFFFFFFu;
+            // The vregs that stay occupied through the whole block (its through-set) are live after every
+            // instruction of it.  Rather than meeting them again in every live-after list, the block
+            // counts them once into two arrays over the registers (cover[r]: members whose range holds r,
+            // start[r]: members whose range starts at r); a definition with range [s, s+w) then overlaps
+            // cover[s] + start[s+1] + ... + start[s+w-1] of them, and only the short list (live after,
+            // not in the through-set) is scanned entry by entry.  Needs every member inside the arrays
+            // (R registers: the file plus the widest vreg); otherwise the full lists are scanned.
+            const uint32_t blk = q.chunk_blk[c];
+            const uint32_t t0 = q.th_off[blk], n_th = q.th_off[blk + 1] - t0;
+            const uint32_t ls_sub = q.ls_adj[blk], ls_mul = q.th_cnt[blk];
+            uint32_t *cover = Cv + q.V + 4, *start = cover + q.R;
+            bool use_short = CACHE && n_th > 0 && ls_mul == n_th;
+            if (use_short) {
+                for (uint32_t r = tid; r < 2 * q.R; r += RC_THREADS) cover[r] = 0;
+                if (tid == 0) s_big = 0;
+                __syncthreads();
+                for (uint32_t j = tid; j < n_th; j += RC_THREADS) {
+                    const uint32_t v = q.th[t0 + j] & 0xFFFFu;
+                    const uint32_t f = fetch(v), reg = f & 0xFFFFu, w = (f >> 16) & 0xFFu;
+                    Cv[v] = f | 0xC0000000u;  // valid, member of the through-set
+                    if (reg + w <= q.R) {
+                        atomicAdd(&start[reg], 1u);
+                        for (uint32_t r = reg; r < reg + w; ++r) atomicAdd(&cover[r], 1u);
+                    } else {
+                        s_big = 1;
+                    }
+                }
+                __syncthreads();
+                use_short = s_big == 0;
+            }
+            const uint32_t *lst = use_short ? q.ls : q.lo;
+            // first entry and length of instruction i's list, from its two live-after offsets
+            auto list_lo = [&](uint32_t i, uint32_t off_i) { return use_short ? off_i - ls_sub - i * ls_mul : off_i; };
+            auto list_n = [&](uint32_t off_i, uint32_t off_i1) { return off_i1 - off_i - (use_short ? ls_mul : 0u); };
             if (CACHE && i_lo < i_hi) {
                 // Every vreg that is live after an instruction of the piece is live after its first
                 // instruction or defined inside the piece: the whole block fetches those into the cache in
                 // one go, so that the instruction-by-instruction recount below finds them there instead of
                 // waiting for global memory once per instruction.
-                const uint32_t l0 = q.lo_off[i_lo], l1 = q.lo_off[i_lo + 1];
+                const uint32_t f0 = q.lo_off[i_lo], f1 = q.lo_off[i_lo + 1];
+                const uint32_t l0 = list_lo(i_lo, f0), l1 = l0 + list_n(f0, f1);
                 for (uint32_t e = l0 + tid; e < l1; e += RC_THREADS) {
-                    const uint32_t v = q.lo[e];
-                    Cv[v] = fetch(v) | 0x80000000u;
+                    const uint32_t v = lst[e];
+                    if (!(Cv[v] >> 31)) Cv[v] = fetch(v) | 0x80000000u;
                 }
                 for (uint32_t i = i_lo + tid; i < i_hi; i += RC_THREADS) {
                     const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
                     for (uint32_t d = o0; d < o0 + nd; ++d) {
                         const uint32_t v = q.op_vreg[d];
-                        Cv[v] = fetch(v) | 0x80000000u;
+                        if (!(Cv[v] >> 31)) Cv[v] = fetch(v) | 0x80000000u;
                     }
                 }
                 __syncthreads();
@@ -992,21 +1029,24 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 const uint32_t my_i = ib + lane * NW;
                 uint32_t m_o0 = 0, m_nd = 0, m_l0 = 0, m_l1 = 0;
                 if (my_i < i_hi) {
-                    m_o0 = q.op_off[my_i]; m_nd = q.ndefs[my_i]; m_l0 = q.lo_off[my_i]; m_l1 = q.lo_off[my_i + 1];
+                    m_o0 = q.op_off[my_i]; m_nd = q.ndefs[my_i];
+                    const uint32_t f0 = q.lo_off[my_i], f1 = q.lo_off[my_i + 1];
+                    m_l0 = list_lo(my_i, f0);
+                    m_l1 = m_l0 + list_n(f0, f1);
                 }
                 // first defined vreg of each instruction, fetched by the lane that holds its bookkeeping
                 uint32_t m_v0 = 0;
                 if (m_nd) m_v0 = q.op_vreg[m_o0];
                 uint32_t todo = __ballot_sync(0xffffffffu, m_nd != 0);
-                // the first 256 entries of the next instruction's live-after list are fetched while the
-                // current instruction is recounted
+                // the first 256 entries of the next instruction's list are fetched while the current
+                // instruction is recounted
                 uint32_t us_nx[8];
                 auto fetch_list = [&](int src) {
                     const uint32_t l0 = __shfl_sync(0xffffffffu, m_l0, src), l1 = __shfl_sync(0xffffffffu, m_l1, src);
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         const uint32_t e = l0 + u * 32 + lane;
-                        us_nx[u] = e < l1 ? q.lo[e] : 0xFFFFFFFFu;
+                        us_nx[u] = e < l1 ? lst[e] : 0xFFFFFFFFu;
                     }
                 };
                 if (todo) fetch_list(__ffs(todo) - 1);
@@ -1026,12 +1066,16 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                         const uint32_t sw = reg_w(v);
                         const uint32_t s = sw & 0xFFFFu, w = (sw >> 16) & 0xFFu;
                         uint32_t cnt = 0;
+                        if (use_short && s < q.R) {  // the through-set members that overlap [s, s+w), v itself excepted
+                            if (lane == 0) cnt = cover[s] - ((sw >> 30) & 1u);
+                            for (uint32_t r = s + 1 + lane; r < min(s + w, q.R); r += 32) cnt += start[r];
+                        }
                         for (uint32_t e0 = l0; e0 < l1; e0 += 256) {  // 8 list entries per lane in flight
                             uint32_t us[8], xs[8];
 #pragma unroll
                             for (int u = 0; u < 8; ++u) {
                                 const uint32_t e = e0 + u * 32 + lane;
-                                us[u] = e0 == l0 ? us0[u] : (e < l1 ? q.lo[e] : 0xFFFFFFFFu);
+                                us[u] = e0 == l0 ? us0[u] : (e < l1 ? lst[e] : 0xFFFFFFFFu);
                                 if (us[u] == 0xFFFFFFFFu) us[u] = v;
                             }
                             // (with the cache, every entry of the list and v itself were fetched up front)
@@ -1246,7 +1290,8 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     if (pp->walk_smem > SM_BYTES - 1024) return VL_ERR_UNSUPPORTED;
     // the recount keeps one cache word per vreg in shared memory when that leaves room for several
     // thread blocks per SM, else it fetches from global memory every time
-    pp->rc_smem = (uint64_t)p->V * 4 <= 72 * 1024 ? (uint32_t)align16((uint64_t)(p->V + 4) * 4) : 0u;
+    pp->rc_smem = (uint64_t)p->V * 4 <= 72 * 1024
+                      ? (uint32_t)align16(((uint64_t)(p->V + 4) + 2ull * (p->P + p->wmax + 2)) * 4) : 0u;
     // the walk's table entries keep bit 15 for a mark: every in-file register number must be below 2^15
     // (the occupancy masks of a register file that large would not fit shared memory anyway)
     if (p->P + p->wmax > 32768u) return VL_ERR_UNSUPPORTED;
@@ -1351,6 +1396,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     rq.bank_fast = p->bank_fast; rq.K = n;
     rq.blk_chunk_off = p->d_blk_chunk_off; rq.th_off = p->d_th_off; rq.th = p->d_th;
     rq.el = p->d_el; rq.el_count = p->d_el_count;
+    rq.ls = p->d_ls; rq.ls_adj = p->d_ls_adj; rq.th_cnt = p->d_th_cnt; rq.R = p->P + p->wmax + 2;
     rq.vinfo = p->d_vinfo; rq.chunk_i0 = p->d_chunk_i0; rq.chunk_i1 = p->d_chunk_i1; rq.chunk_blk = p->d_chunk_blk;
     rq.op_off = p->d_op_off; rq.op_vreg = p->d_op_vreg; rq.lo_off = p->d_lo_off; rq.lo = p->d_lo;
     rq.ndefs = p->d_ndefs; rq.width = p->d_width; rq.opflags = p->d_opflags; rq.iflags = p->d_iflags;
