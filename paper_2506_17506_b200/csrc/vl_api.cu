@@ -11,7 +11,7 @@ std::atomic<uint64_t> g_vl_launches{0};
 // Lane streams are per device and shared by every handle on it; they live until the process exits.
 #define VL_MAX_DEVICES 64
 static std::mutex g_lane_mutex;
-static cudaStream_t g_lanes[VL_MAX_DEVICES][VL_LANES];
+static cudaStream_t g_lanes[VL_MAX_DEVICES][VL_LANES + 2];  // the lanes, then two side streams for liveness
 static bool g_lanes_made[VL_MAX_DEVICES];
 
 int vl_lane_streams(vl_program *p, cudaStream_t **lanes)
@@ -20,12 +20,14 @@ int vl_lane_streams(vl_program *p, cudaStream_t **lanes)
     {
         std::lock_guard<std::mutex> lock(g_lane_mutex);
         if (!g_lanes_made[p->device]) {
-            for (int l = 0; l < VL_LANES; ++l)
+            for (int l = 0; l < VL_LANES + 2; ++l)
                 VL_CUDA(p, cudaStreamCreateWithFlags(&g_lanes[p->device][l], cudaStreamNonBlocking));
             g_lanes_made[p->device] = true;
         }
     }
     if (!p->ev_fork) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+    for (int l = 0; l < 3; ++l)
+        if (!p->ev_side[l]) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_side[l], cudaEventDisableTiming));
     for (int l = 0; l < VL_LANES; ++l)
         if (!p->ev_join[l]) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_join[l], cudaEventDisableTiming));
     *lanes = g_lanes[p->device];
@@ -182,6 +184,8 @@ extern "C" void vl_program_destroy(vl_program *p)
     }
     for (cudaEvent_t ev : p->kt_ev) cudaEventDestroy(ev);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    for (cudaEvent_t ev : p->ev_side)
+        if (ev) cudaEventDestroy(ev);
     for (cudaEvent_t ev : p->ev_join)
         if (ev) cudaEventDestroy(ev);
     delete p;

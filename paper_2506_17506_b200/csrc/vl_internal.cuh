@@ -151,6 +151,7 @@ struct vl_program {
     uint32_t sub_batch = 4096;       // candidates per pass of the verify kernels
     uint32_t lanes_opt = 3;          // lanes in use (1 = everything in order on the caller's stream)
     cudaEvent_t ev_fork = nullptr, ev_join[VL_LANES] = {};
+    cudaEvent_t ev_side[3] = {};     // fork and two joins of the side streams of a liveness run
 
     // opt-in per-kernel timing of vl_verify: five events per pass (before each of the four kernels, after the last)
     int ktime = 0;
@@ -181,7 +182,8 @@ int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint
                    cudaStream_t st, int slot);
 int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
                     const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st);
-// The lane streams of the handle's device (created once per device) and the handle's fork / join events.
+// The lane streams of the handle's device (created once per device; two side streams for liveness
+// follow the VL_LANES lanes in the array) and the handle's fork / join events.
 int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);
 // Waits for a liveness run that is still in flight and checks its outcome; VL_OK if none is pending.

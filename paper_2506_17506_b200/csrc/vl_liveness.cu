@@ -856,23 +856,36 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)(steps / 8),
            V);  // every slot starts as a no-op event
 
+    // The list fill, the operand tables and the walk events do not depend on each other: the latter
+    // two run on side streams beside the fill (as parallel branches when the run is recorded).
+    cudaStream_t *lanes = nullptr;
+    rc = vl_lane_streams(p, &lanes);
+    if (rc != VL_OK) return rc;
+    cudaStream_t sa = lanes[VL_LANES], sb = lanes[VL_LANES + 1];
+    VL_CUDA(p, cudaEventRecord(p->ev_side[0], st));
+    VL_CUDA(p, cudaStreamWaitEvent(sa, p->ev_side[0], 0));
+    VL_CUDA(p, cudaStreamWaitEvent(sb, p->ev_side[0], 0));
     if (nP) k_instr_walk<true><<<nP, 32, walk_smem, st>>>(p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs,
            p->d_op_vreg, Wv, piece_end, (uint32_t *)nullptr, (uint32_t *)nullptr, (uint8_t *)nullptr,
            (const uint32_t *)p->d_piece_chunk, (uint32_t *)nullptr, (const uint32_t *)p->d_lo_off, p->d_lo,
            (const uint32_t *)p->d_chunk_blk, (const uint32_t *)blk_th, (const uint32_t *)p->d_ls_adj,
            (const uint32_t *)th_cnt, p->d_ls);
     if (nP) g_vl_launches.fetch_add(1);
-    LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+    LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_first_def_instr);
-    LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, st, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
-    LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+    LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, sa, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
+    LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_opflags, p->d_vreg16, opmeta, p->d_status);
-    LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, st, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
-    LAUNCH(k_fill_events, nC, 0, st, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
+    LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
+    LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
+    LAUNCH(k_fill_events, nC, 0, sb, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
            p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev, p->d_chunk_blk, p->d_el,
            p->d_el_count);
-    LAUNCH(k_fill_through, nB, 0, st, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
-    LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, st, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
+    LAUNCH(k_fill_through, nB, 0, sb, Wv, blk_th, p->d_width, p->d_th_off, p->d_th);
+    VL_CUDA(p, cudaEventRecord(p->ev_side[1], sa));
+    VL_CUDA(p, cudaEventRecord(p->ev_side[2], sb));
+    VL_CUDA(p, cudaStreamWaitEvent(st, p->ev_side[1], 0));
+    VL_CUDA(p, cudaStreamWaitEvent(st, p->ev_side[2], 0));
     p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     VL_CUDA(p, cudaMemcpyAsync(p->h_live, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 40, cudaMemcpyDeviceToHost, st));
