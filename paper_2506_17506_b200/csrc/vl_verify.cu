@@ -56,7 +56,7 @@ struct TMisc {
 };
 
 struct WParams {
-    uint32_t V, P, nB, nC, Wp, AW, use_th;
+    uint32_t V, P, nB, nC, Wp, AW, use_th, split;
     uint64_t K;
     const uint32_t *th_off, *th, *cev_off, *item_blk, *item_c0, *item_c1;
     const uint4 *ev;
@@ -655,8 +655,15 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
     const uint32_t per_warp = q.Wp * 32 + (q.ev_cap >> 3) * 28;  // words: 112 bytes per group of 8 events
     uint32_t *s_occ = wsm + q.Wp * 32 + (size_t)warp * per_warp;  // [Wp][32]
     uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap / 8] groups of 7 x 16 bytes
-    const uint32_t item = blockIdx.x, grp = blockIdx.y;
-    const uint32_t b = q.item_blk[item], c0 = q.item_c0[item], c1 = q.item_c1[item];
+    // with few candidates an item is cut into q.split parts, one thread block each
+    const uint32_t item = blockIdx.x / q.split, part = blockIdx.x % q.split, grp = blockIdx.y;
+    const uint32_t b = q.item_blk[item];
+    uint32_t c0 = q.item_c0[item], c1 = q.item_c1[item];
+    {
+        const uint32_t per = (c1 - c0 + q.split - 1) / q.split;
+        c0 = min(c1, c0 + part * per);
+        c1 = min(c1, c0 + per);
+    }
     const uint64_t k = (uint64_t)grp * 32 + lane;
     uint32_t *cs = q.cstate + k * 8;  // rows beyond K exist in the working buffers (whole groups)
     // lanes without a candidate, and candidates that are recounted in full anyway (their table may
@@ -1374,7 +1381,11 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
         wq.cstate = vs.cstate; wq.anom = vs.anom;
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
-        const dim3 wgrid(p->nItems, ngrp);
+        // few candidates: more, shorter thread blocks, so that the walk still fills the GPU
+        uint32_t split = 1;
+        while (split < 4 && (uint64_t)p->nItems * split * ngrp < 1184) split *= 2;
+        wq.split = split;
+        const dim3 wgrid(p->nItems * split, ngrp);
         if (p->wmax > 32) k_walk<true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
         else k_walk<false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
         e = cudaGetLastError();
