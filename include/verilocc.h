@@ -151,6 +151,9 @@ int vl_liveness_result(const vl_program *prog, const uint32_t **blk_live_in, con
  * [T[v], T[v]+width) lies inside [0, P); Safety: at every definition of v the range of
  * v is disjoint from the range of every other vreg live after that instruction or
  * defined by it.  Bank tally per Section 2 with B banks.
+ * UNSUPPORTED: the occupancy masks of the walk, (P + widest vreg) / 32 + 1 words for each of 32
+ * candidates and 9 copies, do not fit the shared memory of an SM (P up to about 6,000 fits), or the
+ * packed table of one candidate, 2 (n_vregs + 1) bytes, does not.
  * Errors: INVALID_ARG, LIVENESS_NOT_RUN, UNSUPPORTED, CUDA.
  */
 int vl_verify(const vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pitch_elems,
