@@ -171,7 +171,8 @@ int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *
 /*
  * End-to-end form with HOST buffers: h_cand (K rows, same layout rules, ideally
  * pinned) is copied to the device in slabs through two staging buffers owned by the
- * handle, each slab is checked, and the verdicts are copied back to h_out.  Copies and
+ * handle, each slab is checked, and the verdicts are copied back (through pinned memory of the
+ * handle) to h_out.  Copies and
  * kernels of successive slabs overlap on two internal streams; the call returns after
  * everything has finished (it synchronises).  `cuda_stream` orders the start of the work.
  * Errors: as vl_verify.

@@ -168,6 +168,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     vl_drop_live_graph(p);
     vl_free_liveness(p);
     if (p->h_live) cudaFreeHost(p->h_live);
+    if (p->h_out_pinned) cudaFreeHost(p->h_out_pinned);
     if (p->ev_live) cudaEventDestroy(p->ev_live);
     p->live_arena.release();
     p->tmp_arena.release();
@@ -353,6 +354,15 @@ extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K,
         if (!p->h_streams[j]) VL_CUDA(p, cudaStreamCreateWithFlags(&p->h_streams[j], cudaStreamNonBlocking));
         if (!p->h_events[j]) VL_CUDA(p, cudaEventCreateWithFlags(&p->h_events[j], cudaEventDisableTiming));
     }
+    // The verdicts come back through pinned memory of the handle: a copy straight into pageable
+    // caller memory would make every slab wait for its kernels before the next slab's rows are sent.
+    if (p->h_out_cap < K) {
+        if (p->h_out_pinned) cudaFreeHost(p->h_out_pinned);
+        p->h_out_pinned = nullptr;
+        p->h_out_cap = 0;
+        VL_CUDA(p, cudaHostAlloc((void **)&p->h_out_pinned, K * sizeof(vl_verdict), cudaHostAllocDefault));
+        p->h_out_cap = K;
+    }
     VL_CUDA(p, cudaEventRecord(p->h_events[0], (cudaStream_t)stream));
     for (int j = 0; j < 2; ++j) VL_CUDA(p, cudaStreamWaitEvent(p->h_streams[j], p->h_events[0], 0));
     uint64_t slab = 0;
@@ -363,10 +373,11 @@ extern "C" int vl_verify_host(vl_program *p, const uint16_t *h_cand, uint64_t K,
                                    p->h_streams[j]));
         rc = vl_verify_impl(p, p->d_stage[j], n, pitch, p->d_stage_out[j], p->h_streams[j], VL_LANES + j);
         if (rc != VL_OK) return rc;
-        VL_CUDA(p, cudaMemcpyAsync(h_out + k0, p->d_stage_out[j], n * sizeof(vl_verdict), cudaMemcpyDeviceToHost,
-                                   p->h_streams[j]));
+        VL_CUDA(p, cudaMemcpyAsync(p->h_out_pinned + k0, p->d_stage_out[j], n * sizeof(vl_verdict),
+                                   cudaMemcpyDeviceToHost, p->h_streams[j]));
     }
     for (int j = 0; j < 2; ++j) VL_CUDA(p, cudaStreamSynchronize(p->h_streams[j]));
+    memcpy(h_out, p->h_out_pinned, K * sizeof(vl_verdict));
     return VL_OK;
 }
 

@@ -162,6 +162,8 @@ struct vl_program {
     uint16_t *d_stage[2] = {nullptr, nullptr};
     vl_verdict *d_stage_out[2] = {nullptr, nullptr};
     uint64_t stage_rows = 0, stage_pitch = 0;
+    vl_verdict *h_out_pinned = nullptr;  // verdicts of a vl_verify_host call on their way back
+    uint64_t h_out_cap = 0;
     cudaStream_t h_streams[2] = {nullptr, nullptr};
     cudaEvent_t h_events[2] = {nullptr, nullptr};
 };
