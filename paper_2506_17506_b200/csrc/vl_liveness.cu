@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(32) k_instr_walk(const uint32_t *__restrict__ 
     }
 }
 
-// Exclusive scan of a u32 array by one block of 1024 threads, 4 items per thread and round;
+// Exclusive scan of a u32 array (16-byte aligned) by one block of 1024 threads, 32 items per thread and round;
 // out[n] = total (saturated), total64 exact.
 // Block b of the grid scans in_b into out_b (two arrays per launch).
 __global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in0, uint32_t *out0,
@@ -356,12 +356,23 @@ __global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in0,
     __shared__ uint32_t s_w[33];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long carry = 0;
-    for (uint32_t base = 0; base < n; base += 4096) {
-        const uint32_t i = base + tid * 4;
-        uint32_t x[4];
+    constexpr int IT = 32;
+    for (uint32_t base = 0; base < n; base += 1024 * IT) {
+        const uint32_t i = base + tid * IT;
+        uint32_t x[IT];
+        if (i + IT <= n) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) x[j] = i + j < n ? in[i + j] : 0u;
-        const uint32_t mine = x[0] + x[1] + x[2] + x[3];
+            for (int j = 0; j < IT; j += 4) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(in + i + j);
+                x[j] = v.x; x[j + 1] = v.y; x[j + 2] = v.z; x[j + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < IT; ++j) x[j] = i + j < n ? in[i + j] : 0u;
+        }
+        uint32_t mine = 0;
+#pragma unroll
+        for (int j = 0; j < IT; ++j) mine += x[j];
         uint32_t inc = mine;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -384,10 +395,22 @@ __global__ void __launch_bounds__(1024) k_scan(const uint32_t *__restrict__ in0,
         }
         __syncthreads();
         uint32_t ex = (uint32_t)carry + s_w[warp] + inc - mine;
+        if (i + IT <= n) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (i + j < n) out[i + j] = ex;
-            ex += x[j];
+            for (int j = 0; j < IT; j += 4) {
+                uint4 v;
+                v.x = ex; ex += x[j];
+                v.y = ex; ex += x[j + 1];
+                v.z = ex; ex += x[j + 2];
+                v.w = ex; ex += x[j + 3];
+                *reinterpret_cast<uint4 *>(out + i + j) = v;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < IT; ++j) {
+                if (i + j < n) out[i + j] = ex;
+                ex += x[j];
+            }
         }
         carry += s_w[32];
     }
