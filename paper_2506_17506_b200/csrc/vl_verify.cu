@@ -204,8 +204,9 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
     __syncthreads();
 
-    auto issue_tile = [&](uint32_t t) {
-        const uint32_t stage = t % q.NS;
+    // The ring stage and the barrier phase of the current tile are kept as running counters (stage
+    // wraps at NS, the phase flips with it): no division in the loop.
+    auto issue_tile = [&](uint32_t t, uint32_t stage) {
         const uint32_t bytes = min(TILE, q.nOp8 - t * TILE) * 2;
         mbar_expect_tx(&M->bar[stage], bytes * G);
 #pragma unroll
@@ -213,14 +214,13 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
             bulk_g2s(region + (size_t)(stage * G + g) * STAGE_BYTES, rows[g] + (size_t)t * TILE, bytes, &M->bar[stage]);
     };
     if (tid == 0)
-        for (uint32_t t = 0; t < q.NS && t < q.ntiles; ++t) issue_tile(t);
+        for (uint32_t t = 0; t < q.NS && t < q.ntiles; ++t) issue_tile(t, t);
     PT_INIT();
 
     // Per tile: load it from the ring and store its first occurrences to the table, barrier, compare
     // every occurrence with the table.  The compare of tile t may overlap the stores of tile t+1 by
     // faster threads: those are first occurrences of other vregs.
-    auto wait_tile = [&](uint32_t t) {  // bounded wait
-        const uint32_t stage = t % q.NS, parity = (t / q.NS) & 1;
+    auto wait_tile = [&](uint32_t stage, uint32_t parity) {  // bounded wait
         uint32_t spins = 0;
         const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 22);
         while (!mbar_try_wait(&M->bar[stage], parity)) {
@@ -233,8 +233,8 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     };
     // loads this thread's 8 operands x G candidates of tile t and transposes them to
     // "G candidates side by side per operand"; stores the first occurrences
-    auto load_tile = [&](uint32_t t, uint64_t (&pc)[8], uint32_t (&vj)[8], const uint4 &v4, uint32_t first) {
-        const uint32_t stage = t % q.NS;
+    auto load_tile = [&](uint32_t t, uint32_t stage, uint64_t (&pc)[8], uint32_t (&vj)[8], const uint4 &v4,
+                         uint32_t first) {
         const bool act = t * TILE + tid * 8 < q.nOp8;
         uint32_t r[G][4];
         if (act) {
@@ -314,15 +314,17 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         uint4 m_v4, m2_v4;
         uint32_t m_first, m2_first;
         load_meta(0, m_v4, m_first);
+        uint32_t stage = 0, parity = 0;
         for (uint32_t t = 0; t < q.ntiles; ++t) {
             load_meta(t + 1, m2_v4, m2_first);
-            wait_tile(t);
-            load_tile(t, pc, vj, m_v4, m_first);
+            wait_tile(stage, parity);
+            load_tile(t, stage, pc, vj, m_v4, m_first);
             __syncthreads();
-            if (tid == 0 && t + q.NS < q.ntiles) issue_tile(t + q.NS);  // the stage just read is free again
+            if (tid == 0 && t + q.NS < q.ntiles) issue_tile(t + q.NS, stage);  // the stage just read is free again
             compare_tile(t, pc, vj);
             m_v4 = m2_v4;
             m_first = m2_first;
+            if (++stage == q.NS) { stage = 0; parity ^= 1; }
         }
     }
     __syncthreads();
