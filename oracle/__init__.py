@@ -23,6 +23,8 @@ if os.environ.get("VL_ORACLE_MUTANT_SRC"):
 
 PASS, INCONSISTENT, OUT_OF_RANGE, INTERFERENCE = 1, 2, 4, 8
 
+SAMPLE_STATS_DTYPE = np.dtype([("first_pass", "<u8"), ("n_pass", "<u8")])
+
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
 
@@ -57,6 +59,10 @@ def _load():
         lib.vlo_violations.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.vlo_conflicts.restype = C.c_uint64
         lib.vlo_conflicts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        lib.vlo_sample_stats_of.restype = None
+        lib.vlo_sample_stats_of.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        lib.vlo_resample_summary.restype = None
+        lib.vlo_resample_summary.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -146,3 +152,26 @@ class OracleProgram:
         tr = np.zeros((max(int(n), 1), 3), dtype=np.uint32)
         lib.vlo_conflicts(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(tr), n)
         return tr[: int(n)]
+
+
+def sample_stats(verdicts: np.ndarray) -> np.ndarray:
+    """First passing row (K if none) and number of passing rows of one verdict array."""
+    lib = _load()
+    v = np.ascontiguousarray(verdicts, dtype=VERDICT_DTYPE)
+    out = np.zeros(1, dtype=SAMPLE_STATS_DTYPE)
+    keep = v if len(v) else np.zeros(1, dtype=VERDICT_DTYPE)
+    lib.vlo_sample_stats_of(_ptr(keep), len(v), _ptr(out))
+    return out[0]
+
+
+def resample_summary(stats: np.ndarray, K, ks) -> dict:
+    """Pass@k counts, attempts summed / largest over the solved test cases (Section 4 of the paper)."""
+    lib = _load()
+    n = len(stats)
+    st = np.ascontiguousarray(stats, dtype=SAMPLE_STATS_DTYPE) if n else np.zeros(1, dtype=SAMPLE_STATS_DTYPE)
+    Ks = np.ascontiguousarray(K, dtype=np.uint64) if n else np.zeros(1, dtype=np.uint64)
+    kk = np.ascontiguousarray(ks, dtype=np.uint32) if len(ks) else np.zeros(1, dtype=np.uint32)
+    out = np.zeros(4 + len(ks), dtype=np.uint64)
+    lib.vlo_resample_summary(n, _ptr(st), _ptr(Ks), len(ks), _ptr(kk), _ptr(out))
+    return dict(n_cases=int(out[0]), n_solved=int(out[1]), sum_tries=int(out[2]), max_tries=int(out[3]),
+                pass_at=[int(x) for x in out[4:]])

@@ -291,3 +291,51 @@ uint64_t vlo_conflicts(const vlo_program *p, const uint64_t *lo_off, const uint3
     walk(p, lo_off, lo, row, &v, NULL, triples, cap, &n);
     return n;
 }
+
+/* ------------------------------------------------- re-sampling statistics */
+
+/*
+ * The verifier sits in a loop that samples the model again until a candidate
+ * passes or the attempts run out (paper, Section 3.4, last paragraph).  The
+ * figures the paper reports about that loop (Section 4, before "Main
+ * Results"): Pass@k, the share of test cases with a passing candidate among
+ * their first k attempts; AvgTry and MaxTry, the average and the largest
+ * number of attempts up to and including the first passing one, over the test
+ * cases that reached one.  Rows are attempts, in order.
+ */
+typedef struct {
+    uint64_t first_pass; /* row of the first passing verdict, K if there is none */
+    uint64_t n_pass;     /* passing verdicts among the K rows */
+} vlo_sample_stats;
+
+void vlo_sample_stats_of(const vlo_verdict *out, uint64_t K, vlo_sample_stats *s)
+{
+    s->first_pass = K;
+    s->n_pass = 0;
+    for (uint64_t k = 0; k < K; ++k) {
+        if (!(out[k].flags & VLO_PASS)) continue;
+        if (s->first_pass == K) s->first_pass = k;
+        s->n_pass += 1;
+    }
+}
+
+/*
+ * summary[0] = test cases, [1] = solved ones, [2] = sum of attempts over the
+ * solved ones, [3] = largest number of attempts of a solved one (0 if none),
+ * [4 + j] = test cases solved within their first k[j] attempts.
+ */
+void vlo_resample_summary(uint32_t n, const vlo_sample_stats *s, const uint64_t *K,
+                          uint32_t n_k, const uint32_t *k, uint64_t *summary)
+{
+    for (uint32_t j = 0; j < 4 + n_k; ++j) summary[j] = 0;
+    summary[0] = n;
+    for (uint32_t c = 0; c < n; ++c) {
+        if (s[c].first_pass >= K[c]) continue; /* never passed */
+        const uint64_t attempts = s[c].first_pass + 1;
+        summary[1] += 1;
+        summary[2] += attempts;
+        if (attempts > summary[3]) summary[3] = attempts;
+        for (uint32_t j = 0; j < n_k; ++j)
+            if (attempts <= k[j]) summary[4 + j] += 1;
+    }
+}

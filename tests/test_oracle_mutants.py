@@ -24,6 +24,10 @@ MUTANTS = [
     ("bank cost n instead of n-1", "bank += n - 1;", "bank += n;"),
     ("last occurrence wins", "if (T[v] < 0) T[v] = row[o];", "if (T[v] < 0 || 1) T[v] = row[o];"),
     ("co-defined vregs ignored", "if (in_live) continue;", "continue;"),
+    ("Pass@k leaves out the k-th attempt", "if (attempts <= k[j]) summary[4 + j] += 1;",
+     "if (attempts < k[j]) summary[4 + j] += 1;"),
+    ("test cases that never pass counted among the attempts", "if (s[c].first_pass >= K[c]) continue; /* never passed */", ""),
+    ("last passing attempt instead of the first", "if (s->first_pass == K) s->first_pass = k;", "s->first_pass = k;"),
 ]
 
 

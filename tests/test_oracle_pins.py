@@ -322,3 +322,74 @@ def test_generator_batch_members_and_stress_sample(oracle_mod):
     op, lv = _oracle(oracle_mod, p)
     vd = op.verify(lv, rows)
     assert np.array_equal(vd["flags"] == PASS, faults[:, 0] == 0)
+
+
+# ------------------------------------------------------- re-sampling statistics
+def _verdicts(oracle_mod, pass_rows, K):
+    v = np.zeros(K, dtype=oracle_mod.VERDICT_DTYPE)
+    v["flags"] = INTERF
+    v["first_violation_instr"] = 0
+    v["flags"][list(pass_rows)] = PASS
+    return v
+
+
+def test_pass_rate_matches_the_paper_table(oracle_mod):
+    # Table 2: one greedy attempt per test case; the printed rate is passing / all, to two decimals.
+    with open(os.path.join(GOLDEN, "table2_pass_rates.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    assert len(rows) == 10
+    for n_pass, n_fail, printed in rows:
+        n_pass, n_fail = int(n_pass), int(n_fail)
+        stats = np.array([oracle_mod.sample_stats(_verdicts(oracle_mod, [0] if c < n_pass else [], 1))
+                          for c in range(n_pass + n_fail)])
+        s = oracle_mod.resample_summary(stats, [1] * len(stats), [1, 100])
+        assert s["n_cases"] == n_pass + n_fail and s["n_solved"] == n_pass
+        assert s["pass_at"] == [n_pass, n_pass]
+        assert f"{100.0 * s['pass_at'][0] / s['n_cases']:.2f}" == printed
+        assert (s["sum_tries"], s["max_tries"]) == (n_pass, 1 if n_pass else 0)
+
+
+def test_first_passing_attempt_closed_forms(oracle_mod):
+    K = 250
+    # case c passes first at attempt c*c + 1 (rows are attempts in order), later rows mixed
+    firsts = [c * c for c in range(15)]                     # 0, 1, 4, ..., 196
+    stats = []
+    for f0 in firsts:
+        rows = [f0] + [r for r in range(f0 + 1, K) if (r * 7 + f0) % 5 == 0]
+        st = oracle_mod.sample_stats(_verdicts(oracle_mod, rows, K))
+        assert (int(st["first_pass"]), int(st["n_pass"])) == (f0, len(rows))
+        stats.append(st)
+    never = oracle_mod.sample_stats(_verdicts(oracle_mod, [], K))
+    assert (int(never["first_pass"]), int(never["n_pass"])) == (K, 0)
+    stats += [never, never]
+    s = oracle_mod.resample_summary(np.array(stats), [K] * len(stats), [1, 10, 100, 197, 250])
+    attempts = [f0 + 1 for f0 in firsts]
+    assert s["n_cases"] == 17 and s["n_solved"] == 15
+    assert s["sum_tries"] == sum(attempts) and s["max_tries"] == 197
+    # attempts 1, 2, 5, 10 are within 10; squares up to 81 (+1) within 100; 197 is the last
+    assert s["pass_at"] == [1, 4, 10, 15, 15]
+    # Pass@k never decreases in k and ends at the solved count
+    assert all(a <= b for a, b in zip(s["pass_at"], s["pass_at"][1:])) and s["pass_at"][-1] == s["n_solved"]
+
+
+def test_resample_statistics_edge_cases(oracle_mod):
+    empty = oracle_mod.sample_stats(np.zeros(0, dtype=oracle_mod.VERDICT_DTYPE))
+    assert (int(empty["first_pass"]), int(empty["n_pass"])) == (0, 0)
+    s = oracle_mod.resample_summary(np.array([empty]), [0], [1])
+    assert (s["n_cases"], s["n_solved"], s["sum_tries"], s["max_tries"], s["pass_at"]) == (1, 0, 0, 0, [0])
+    s = oracle_mod.resample_summary(np.zeros(0, dtype=oracle_mod.SAMPLE_STATS_DTYPE), [], [1, 10])
+    assert (s["n_cases"], s["n_solved"], s["pass_at"]) == (0, 0, [0, 0])
+    # a verdict that carries the pass bit together with nothing else counts; kind bits alone never do
+    v = np.zeros(4, dtype=oracle_mod.VERDICT_DTYPE)
+    v["flags"] = [INCONS, RANGE | INTERF, INCONS | RANGE | INTERF, PASS]
+    st = oracle_mod.sample_stats(v)
+    assert (int(st["first_pass"]), int(st["n_pass"])) == (3, 1)
+    # statistics over real verdicts: a generated workload, rows in order
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    rows, _faults = synth.candidate_rows(p, 100, wl.fault_rate, wl.seeds[0])
+    op, live = _oracle(oracle_mod, p)
+    out = op.verify(live, rows)
+    passing = np.flatnonzero(out["flags"] == PASS)
+    st = oracle_mod.sample_stats(out)
+    assert int(st["n_pass"]) == len(passing) and int(st["first_pass"]) == (passing[0] if len(passing) else 100)
