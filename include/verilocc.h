@@ -181,6 +181,52 @@ int vl_verify_host(vl_program *prog, const uint16_t *h_cand, uint64_t K, uint64_
                    vl_verdict *h_out, void *cuda_stream);
 
 /*
+ * Statistics of the re-sampling loop (Section 3.4, last paragraph: the model is sampled again until
+ * a candidate passes or the attempts run out; Section 4: Pass@k, AvgTry, MaxTry).  The rows of a
+ * verdict array are the attempts of one test case, in order.
+ */
+typedef struct {
+    uint64_t first_pass; /* row of the first verdict with VL_PASS; K if there is none */
+    uint64_t n_pass;     /* verdicts with VL_PASS among the K rows */
+} vl_sample_stats;
+
+#define VL_MAX_PASS_AT 8
+typedef struct {
+    uint64_t n_cases;                 /* test cases summarised */
+    uint64_t n_solved;                /* test cases with a passing row */
+    uint64_t sum_tries;               /* attempts up to and including the first passing one, summed over
+                                         the solved test cases: AvgTry = sum_tries / n_solved */
+    uint64_t max_tries;               /* the largest such number of attempts (MaxTry); 0 if none solved */
+    uint64_t pass_at[VL_MAX_PASS_AT]; /* pass_at[j]: test cases solved within their first k[j] attempts
+                                         (Pass@k[j] = pass_at[j] / n_cases); 0 for j >= n_k */
+} vl_resample_summary;
+
+/*
+ * For each of n test cases: the record of d_out[j] (K[j] verdicts in DEVICE memory, 16-byte aligned,
+ * as vl_verify wrote them) into d_stats[j]; then, unless d_summary is NULL, the summary of the n
+ * records for the n_k <= VL_MAX_PASS_AT attempt limits k[].  d_out, K and k are HOST arrays, read
+ * during the call; d_stats ([n]) and d_summary are DEVICE memory, 8-byte aligned, owned by the
+ * caller.  A test case with K[j] == 0 counts as unsolved.  Stream-ordered on `cuda_stream` of
+ * `device`, no synchronisation, no allocation.  Errors: INVALID_ARG, CUDA.
+ */
+int vl_resample_stats(int device, uint32_t n, const vl_verdict *const *d_out, const uint64_t *K, uint32_t n_k,
+                      const uint32_t *k, vl_sample_stats *d_stats, vl_resample_summary *d_summary,
+                      void *cuda_stream);
+
+/*
+ * The re-sampling loop with early exit: checks the rows of d_cand (as vl_verify) in batches of
+ * batch_rows, in order, and stops after the first batch that holds a passing row.  *rows_checked
+ * (HOST) receives the number of rows checked, a multiple of batch_rows or K; *first_pass (HOST) the
+ * row of the first passing candidate, K if none passed.  Verdicts of the rows checked are in d_out
+ * (16-byte aligned); those of later rows are not written.  The call waits for the stream after every
+ * batch (the caller needs the answer to stop sampling); the first call allocates one record in
+ * device and in pinned host memory.  Errors: as vl_verify.
+ */
+int vl_verify_until_pass(vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pitch_elems,
+                         uint64_t batch_rows, vl_verdict *d_out, uint64_t *rows_checked, uint64_t *first_pass,
+                         void *cuda_stream);
+
+/*
  * Block-level liveness without any allocation.  (The paper has no counterpart; this exists for
  * hosts that cannot allocate device memory when they call in: a process that handed all of HBM to
  * its own pools at start-up, a plugin under a memory budget it does not control, or a loop that

@@ -28,7 +28,8 @@ VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERN
 
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
-           "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static"]
+           "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static",
+           "vl_resample_stats", "vl_verify_until_pass"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -74,6 +75,14 @@ _lib.vl_strerror.argtypes = [C.c_int]
 _lib.vl_block_liveness_static.restype = C.c_int
 _lib.vl_block_liveness_static.argtypes = [C.c_int, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9
 VL_STATIC_SCRATCH_WORDS = 1 << 18
+_lib.vl_resample_stats.restype = C.c_int
+_lib.vl_resample_stats.argtypes = [C.c_int, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_void_p]
+_lib.vl_verify_until_pass.restype = C.c_int
+_lib.vl_verify_until_pass.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p]
+VL_MAX_PASS_AT = 8
+SAMPLE_STATS_DTYPE = np.dtype([("first_pass", "<u8"), ("n_pass", "<u8")])
 
 
 class VlError(RuntimeError):
@@ -204,6 +213,19 @@ class Program:
         self._check(_lib.vl_verify_host(self._h, ptr, K, pitch, optr, _stream_ptr(stream)), "vl_verify_host")
         return out
 
+    def vl_verify_until_pass(self, cand, batch_rows: int, out=None, stream=None):
+        """The re-sampling loop with early exit over a CUDA uint16 [K, pitch] tensor; returns
+        (verdict tensor, rows checked, first passing row or K)."""
+        import torch
+        assert cand.is_cuda and cand.dtype in (torch.uint16, torch.int16) and cand.dim() == 2 and cand.is_contiguous()
+        K, pitch = cand.shape
+        if out is None:
+            out = torch.zeros((K, 4), dtype=torch.int32, device=cand.device)
+        done, first = C.c_uint64(0), C.c_uint64(0)
+        self._check(_lib.vl_verify_until_pass(self._h, cand.data_ptr(), K, pitch, batch_rows, out.data_ptr(),
+                                              C.byref(done), C.byref(first), _stream_ptr(stream)), "vl_verify_until_pass")
+        return out, int(done.value), int(first.value)
+
     def vl_verify_status(self, stream=None):
         self._check(_lib.vl_verify_status(self._h, _stream_ptr(stream)), "vl_verify_status")
 
@@ -266,6 +288,27 @@ def vl_verify_batch(programs, cands, outs=None, stream=None):
     if rc != VL_OK:
         raise VlError(rc, "vl_verify_batch")
     return outs
+
+
+def vl_resample_stats(outs, ks=(1, 10, 100), device: int = 0, stream=None):
+    """Per test case (one CUDA int32 [K_j, 4] verdict tensor each) the first passing row and the
+    number of passing rows, and the summary over the test cases for the attempt limits ``ks``.
+    Returns (records as a numpy array, summary as a dict); waits for the stream to read them back."""
+    import torch
+    n = len(outs)
+    stats = torch.zeros((max(n, 1), 2), dtype=torch.int64, device=f"cuda:{device}")
+    summ = torch.zeros(4 + VL_MAX_PASS_AT, dtype=torch.int64, device=f"cuda:{device}")
+    op = (C.c_void_p * max(n, 1))(*[o.data_ptr() if o.numel() else None for o in outs])
+    Ks = (C.c_uint64 * max(n, 1))(*[o.shape[0] for o in outs])
+    kk = (C.c_uint32 * max(len(ks), 1))(*ks)
+    rc = _lib.vl_resample_stats(device, n, op, Ks, len(ks), kk, stats.data_ptr(), summ.data_ptr(), _stream_ptr(stream))
+    if rc != VL_OK:
+        raise VlError(rc, "vl_resample_stats")
+    torch.cuda.synchronize(device)
+    rec = stats[:n].cpu().numpy().view(np.uint64).copy().view(SAMPLE_STATS_DTYPE).reshape(-1)
+    s = summ.cpu().numpy().view(np.uint64)
+    return rec, dict(n_cases=int(s[0]), n_solved=int(s[1]), sum_tries=int(s[2]), max_tries=int(s[3]),
+                     pass_at=[int(x) for x in s[4:4 + len(ks)]])
 
 
 def verdicts_to_numpy(t) -> np.ndarray:

@@ -169,6 +169,8 @@ extern "C" void vl_program_destroy(vl_program *p)
     vl_free_liveness(p);
     if (p->h_live) cudaFreeHost(p->h_live);
     if (p->h_out_pinned) cudaFreeHost(p->h_out_pinned);
+    if (p->h_rs) cudaFreeHost(p->h_rs);
+    cudaFree(p->d_rs);
     if (p->ev_live) cudaEventDestroy(p->ev_live);
     p->live_arena.release();
     p->tmp_arena.release();

@@ -166,6 +166,8 @@ struct vl_program {
     uint64_t h_out_cap = 0;
     cudaStream_t h_streams[2] = {nullptr, nullptr};
     cudaEvent_t h_events[2] = {nullptr, nullptr};
+    // one record for vl_verify_until_pass: device copy and its pinned landing place
+    vl_sample_stats *d_rs = nullptr, *h_rs = nullptr;
 };
 
 extern std::atomic<uint64_t> g_vl_launches;

@@ -97,3 +97,26 @@ def test_null_arguments(B):
     assert lib.vl_liveness_batch(2, None, None) == B.VL_ERR_INVALID_ARG
     two_nulls = (C.c_void_p * 2)(None, None)
     assert lib.vl_liveness_batch(2, two_nulls, None) == B.VL_ERR_INVALID_ARG
+
+
+def test_resample_argument_checks(B):
+    lib = C.CDLL(B.LIB_PATH)
+    f = lib.vl_resample_stats
+    f.restype = C.c_int
+    f.argtypes = [C.c_int, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    ks = (C.c_uint32 * 9)(*range(1, 10))
+    assert f(0, 0, None, None, 0, None, None, None, None) == B.VL_OK              # nothing to do
+    assert f(0, 0, None, None, 9, ks, None, None, None) == B.VL_ERR_INVALID_ARG   # too many attempt limits
+    assert f(0, 0, None, None, 2, None, None, None, None) == B.VL_ERR_INVALID_ARG # limits announced, none given
+    assert f(0, 1, None, None, 0, None, None, None, None) == B.VL_ERR_INVALID_ARG # a test case without arrays
+    outs, K = (C.c_void_p * 1)(None), (C.c_uint64 * 1)(5)
+    assert f(0, 1, outs, K, 0, None, C.c_void_p(64), None, None) == B.VL_ERR_INVALID_ARG   # rows announced, no verdicts
+    outs = (C.c_void_p * 1)(C.c_void_p(72))
+    assert f(0, 1, outs, K, 0, None, C.c_void_p(64), None, None) == B.VL_ERR_INVALID_ARG   # verdicts not 16-byte aligned
+    outs = (C.c_void_p * 1)(C.c_void_p(64))
+    assert f(0, 1, outs, K, 0, None, C.c_void_p(68), None, None) == B.VL_ERR_INVALID_ARG   # records not 8-byte aligned
+    g = lib.vl_verify_until_pass
+    g.restype = C.c_int
+    g.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    n = C.c_uint64(0)
+    assert g(None, None, 1, 8, 1, None, C.byref(n), C.byref(n), None) == B.VL_ERR_INVALID_ARG
