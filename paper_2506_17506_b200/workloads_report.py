@@ -8,7 +8,10 @@ warm-up), the same for vl_verify alone, the algorithmic bytes per second (2 byte
 column + a 16-byte verdict per candidate) and their fraction of the measured copy bandwidth.  The
 small workloads move kilobytes per call and are bound by launch latency: read their latency, not
 their bandwidth fraction.  Workload 4 (256 independent programs) goes through vl_liveness_batch
-and vl_verify_batch.
+and vl_verify_batch.  Also per workload: the time of one vl_resample_stats call over the verdict
+arrays (launch-latency bound: three or more small kernels), the statistics it returns (test cases
+solved, attempts summed and largest, Pass@1/10/100 counts), and the time of the early-exit loop
+vl_verify_until_pass in batches of 100 rows (it stops after the first batch with a passing row).
 """
 from __future__ import annotations
 
@@ -82,6 +85,37 @@ def main() -> int:
         torch.cuda.synchronize()
         for gp in gps:
             gp.vl_verify_status(stream)
+        # re-sampling statistics over the verdicts just written, and the early-exit loop
+        n = len(outs)
+        stats = torch.zeros((n, 2), dtype=torch.int64, device="cuda")
+        summ = torch.zeros(4 + vl.VL_MAX_PASS_AT, dtype=torch.int64, device="cuda")
+        import ctypes as C
+        op = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+        Ks = (C.c_uint64 * n)(*[o.shape[0] for o in outs])
+        kk = (C.c_uint32 * 3)(1, 10, 100)
+        sp = C.c_void_p(stream.cuda_stream)
+
+        def resample():
+            rc = vl._lib.vl_resample_stats(0, n, op, Ks, 3, kk, stats.data_ptr(), summ.data_ptr(), sp)
+            assert rc == vl.VL_OK, rc
+
+        for _ in range(3):
+            resample()
+        er = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        er[0].record(stream)
+        for _ in range(args.steps):
+            resample()
+        er[1].record(stream)
+        torch.cuda.synchronize()
+        _, summary = vl.vl_resample_stats(outs, (1, 10, 100), stream=stream)
+        gps[0].vl_verify_until_pass(cands[0], 100, outs[0], stream)
+        er[2].record(stream)
+        for _ in range(args.steps):
+            _, rows_done, first_pass = gps[0].vl_verify_until_pass(cands[0], 100, outs[0], stream)
+        er[3].record(stream)
+        torch.cuda.synchronize()
+        resample_us = er[0].elapsed_time(er[1]) / args.steps * 1e3
+        until_ms = er[2].elapsed_time(er[3]) / args.steps
         step_ms = ev[0].elapsed_time(ev[1]) / args.steps
         verify_ms = ev[2].elapsed_time(ev[3]) / args.steps
         n_cand = wl.K * len(progs)
@@ -97,6 +131,9 @@ def main() -> int:
             "verify_only_verifications_per_sec": n_cand / (verify_ms * 1e-3),
             "verify_only_gb_per_sec": n_bytes / (verify_ms * 1e-3) / 1e9,
             "verify_only_frac_of_measured_copy_peak": n_bytes / (verify_ms * 1e-3) / 1e9 / peak,
+            "resample_stats_us": resample_us, "resample_summary": summary,
+            "until_pass_batch100_ms": until_ms, "until_pass_rows_checked": rows_done,
+            "until_pass_first_passing_row": first_pass,
         }), flush=True)
         for gp in gps:
             gp.close()
