@@ -39,7 +39,8 @@ class _Prog(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("n_blocks", "n_instrs", "n_vregs", "n_operands", "n_edges", "P", "B")] + [
         ("block_instr_off", C.c_void_p), ("succ_off", C.c_void_p), ("succ", C.c_void_p),
         ("instr_op_off", C.c_void_p), ("instr_n_defs", C.c_void_p), ("op_vreg", C.c_void_p),
-        ("vreg_width", C.c_void_p)]
+        ("vreg_width", C.c_void_p), ("vreg_align", C.c_void_p), ("vreg_class", C.c_void_p),
+        ("class_lo", C.c_void_p), ("class_hi", C.c_void_p), ("reserved", C.c_void_p)]
 
 
 _lib = None
@@ -110,6 +111,29 @@ class OracleProgram:
                        *[self.arrays[k].ctypes.data for k in
                          ("block_instr_off", "succ_off", "succ", "instr_op_off", "instr_n_defs", "op_vreg", "vreg_width")])
         self.n_blocks, self.n_instrs, self.n_vregs = prog.n_blocks, prog.n_instrs, prog.n_vregs
+        self.P = prog.P
+
+    def set_constraints(self, vreg_align=None, vreg_class=None, class_ranges=None, reserved=None):
+        """Optional hardware rules for the Realizability check: per-vreg alignment of the base
+        register, per-vreg register class with the half-open register range of every class, and
+        the set of reserved registers (any iterable of register numbers).  None switches one off."""
+        a = self.arrays
+        for k in ("vreg_align", "vreg_class", "class_lo", "class_hi", "reserved"):
+            a.pop(k, None)
+            setattr(self.c, k, None)
+        if vreg_align is not None:
+            a["vreg_align"] = np.ascontiguousarray(np.concatenate([vreg_align, [1]]), dtype=np.uint8)
+        if vreg_class is not None:
+            a["vreg_class"] = np.ascontiguousarray(np.concatenate([vreg_class, [0]]), dtype=np.uint8)
+            a["class_lo"] = np.ascontiguousarray([r[0] for r in class_ranges], dtype=np.uint32)
+            a["class_hi"] = np.ascontiguousarray([r[1] for r in class_ranges], dtype=np.uint32)
+        if reserved is not None:
+            m = np.zeros(self.P + 1, dtype=np.uint8)
+            m[[r for r in reserved if r < self.P]] = 1
+            a["reserved"] = m
+        for k in ("vreg_align", "vreg_class", "class_lo", "class_hi", "reserved"):
+            if k in a:
+                setattr(self.c, k, a[k].ctypes.data)
 
     def liveness(self, order: int = 0) -> Liveness:
         lib = _load()

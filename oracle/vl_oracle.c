@@ -17,6 +17,9 @@
  *   C          every occurrence of a virtual register carries the physical
  *              register of its first occurrence (the table T);
  *   R          at every definition of v: [T[v], T[v]+width(v)) lies in [0,P);
+ *              optionally also: T[v] is a multiple of the vreg's alignment, the
+ *              range lies inside the registers of the vreg's class and holds no
+ *              reserved register;
  *   I          at every definition of v at instruction i: that range is
  *              disjoint from the range of every other virtual register that
  *              is live after i or also defined by i;
@@ -45,6 +48,14 @@ typedef struct {
     const uint8_t *instr_n_defs;     /* [n_instrs]   */
     const uint32_t *op_vreg;         /* [n_operands] */
     const uint8_t *vreg_width;       /* [n_vregs]    */
+    /* Optional hardware constraints (Section 1: register file sizes and reserved registers;
+     * Section 3.2: scalar / vector register classes; Section 4.5: hardware rules on register
+     * tuples).  A null pointer switches the constraint off. */
+    const uint8_t *vreg_align;       /* [n_vregs] the base register is a multiple of this (>= 1) */
+    const uint8_t *vreg_class;       /* [n_vregs] register class of the vreg */
+    const uint32_t *class_lo;        /* [classes] class c owns the registers [class_lo[c], class_hi[c]) */
+    const uint32_t *class_hi;
+    const uint8_t *reserved;         /* [P] 1 = no vreg may occupy this register */
 } vlo_program;
 
 typedef struct {
@@ -197,8 +208,17 @@ static void walk(const vlo_program *p, const uint64_t *lo_off, const uint32_t *l
             uint32_t v = p->op_vreg[d];
             uint32_t s = (uint32_t)T[v], w = p->vreg_width[v];
             int bad = 0;
-            /* realizability: the tuple fits in the register file */
-            if (s + w > p->P) {
+            /* realizability: the tuple fits in the register file and keeps the hardware rules */
+            int unreal = s + w > p->P;
+            if (p->vreg_align && s % p->vreg_align[v] != 0) unreal = 1;
+            if (p->vreg_class) {
+                uint32_t c = p->vreg_class[v];
+                if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;
+            }
+            if (p->reserved)
+                for (uint32_t r = s; r < s + w && r < p->P; ++r)
+                    if (p->reserved[r]) unreal = 1;
+            if (unreal) {
                 flags |= VLO_OUT_OF_RANGE;
                 if (kinds) kinds[i] |= VLO_OUT_OF_RANGE;
                 bad = 1;

@@ -28,6 +28,14 @@ MUTANTS = [
      "if (attempts < k[j]) summary[4 + j] += 1;"),
     ("test cases that never pass counted among the attempts", "if (s[c].first_pass >= K[c]) continue; /* never passed */", ""),
     ("last passing attempt instead of the first", "if (s->first_pass == K) s->first_pass = k;", "s->first_pass = k;"),
+    ("alignment tested on the end of the tuple", "if (p->vreg_align && s % p->vreg_align[v] != 0) unreal = 1;",
+     "if (p->vreg_align && (s + w) % p->vreg_align[v] != 0) unreal = 1;"),
+    ("class range closed at the top", "if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;",
+     "if (s < p->class_lo[c] || s + w > p->class_hi[c] + 1) unreal = 1;"),
+    ("class lower bound dropped", "if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;",
+     "if (s + w > p->class_hi[c]) unreal = 1;"),
+    ("reserved check leaves out the last register of a tuple", "for (uint32_t r = s; r < s + w && r < p->P; ++r)",
+     "for (uint32_t r = s; r + 1 < s + w && r < p->P; ++r)"),
 ]
 
 

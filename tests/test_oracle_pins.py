@@ -393,3 +393,99 @@ def test_resample_statistics_edge_cases(oracle_mod):
     passing = np.flatnonzero(out["flags"] == PASS)
     st = oracle_mod.sample_stats(out)
     assert int(st["n_pass"]) == len(passing) and int(st["first_pass"]) == (passing[0] if len(passing) else 100)
+
+
+# ------------------------------------------------- hardware rules (fuller Realizability)
+def _defs_then_use(widths, P):
+    """v0, v1, ... defined one per instruction, all read by a last instruction (all live together)."""
+    n = len(widths)
+    blocks = [[([v], []) for v in range(n)] + [([], list(range(n)))]]
+    return synth.program_from_lists(blocks, [], n, widths, P)
+
+
+def test_hardware_rules_hand_cases(oracle_mod):
+    p = _defs_then_use([2, 2, 1, 8], 32)
+    op, lv = _oracle(oracle_mod, p)
+
+    def verdict(T):
+        return op.verify(lv, H.row_from_table(p, T))[0]
+
+    base = [0, 2, 4, 8]
+    assert verdict(base)["flags"] == PASS
+    # alignment: pairs on even registers, the 8-tuple on a multiple of 8, singles anywhere
+    op.set_constraints(vreg_align=[2, 2, 1, 8])
+    assert verdict(base)["flags"] == PASS
+    assert verdict([0, 2, 5, 8])["flags"] == PASS                      # width 1 may sit on an odd register
+    vd = verdict([0, 3, 5, 8])                                         # pair on an odd register
+    assert (vd["flags"], vd["first_violation_instr"], vd["conflict_pairs"]) == (RANGE, 1, 0)
+    vd = verdict([0, 2, 4, 12])                                        # 8-tuple on 12: inside the file, misaligned
+    assert (vd["flags"], vd["first_violation_instr"]) == (RANGE, 3)
+    assert verdict([0, 2, 4, 24])["flags"] == PASS                     # last aligned place in the file
+    # reserved registers: a tuple may sit beside one, not on one; its last register counts too
+    op.set_constraints(reserved=[6, 7, 31])
+    assert verdict(base)["flags"] == PASS                              # 4 and 8.. are beside 6, 7
+    vd = verdict([0, 2, 6, 8])
+    assert (vd["flags"], vd["first_violation_instr"]) == (RANGE, 2)
+    vd = verdict([0, 5, 4, 8])                                         # pair 5..6 ends on a reserved register
+    assert (vd["flags"], vd["first_violation_instr"], vd["conflict_pairs"]) == (RANGE, 1, 0)
+    assert verdict([0, 2, 4, 23])["flags"] == PASS                     # 23..30 stops before 31
+    assert verdict([0, 2, 4, 24])["flags"] == RANGE                    # 24..31 holds 31
+    # classes: v0, v1 scalar in [0, 8); v2, v3 vector in [8, 32)
+    op.set_constraints(vreg_class=[0, 0, 1, 1], class_ranges=[(0, 8), (8, 32)])
+    assert verdict([0, 2, 8, 9])["flags"] == PASS
+    assert verdict([0, 6, 8, 24])["flags"] == PASS                     # both classes filled to their last register
+    vd = verdict([0, 7, 9, 16])                                        # scalar pair 7..8 leaves its class
+    assert (vd["flags"], vd["first_violation_instr"]) == (RANGE, 1)
+    vd = verdict([0, 2, 7, 16])                                        # vector single below its class
+    assert (vd["flags"], vd["first_violation_instr"]) == (RANGE, 2)
+    assert verdict([0, 2, 8, 25])["flags"] == RANGE                    # 25..32 beyond the class and the file
+    # all rules off again: the plain range check is all that is left
+    op.set_constraints()
+    assert verdict([0, 3, 7, 24])["flags"] == PASS
+
+
+def test_hardware_rules_hand_case_overlap_is_still_counted(oracle_mod):
+    # a misplaced tuple is compared with the others where it is (no special treatment)
+    p = _defs_then_use([2, 2], 16)
+    op, lv = _oracle(oracle_mod, p)
+    op.set_constraints(vreg_align=[2, 2], reserved=[9])
+    vd = op.verify(lv, H.row_from_table(p, [4, 5]))[0]                 # v1 misaligned and on v0's second register
+    assert (vd["flags"], vd["first_violation_instr"], vd["conflict_pairs"]) == (RANGE | INTERF, 1, 1)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_hardware_rules_equal_register_by_register_definition(oracle_mod, seed):
+    """A definition is realizable iff its base is a multiple of the alignment and every register it
+    occupies exists, belongs to the vreg's class and is not reserved: enumerate registers in Python."""
+    rng = np.random.default_rng(900 + seed)
+    p = H.random_program(7000 + seed, strict=True, reachable=True, max_instrs=40, max_vregs=14, P=32,
+                         widths=(1, 2, 2, 4))
+    op, lv = _oracle(oracle_mod, p)
+    V = p.n_vregs
+    align = rng.choice([1, 2, 4], size=V)
+    cls = rng.integers(0, 3, size=V)
+    ranges = [(0, 12), (12, 32), (4, 28)]
+    reserved = sorted(set(rng.integers(0, 32, size=3).tolist()))
+    op.set_constraints(vreg_align=align, vreg_class=cls, class_ranges=ranges, reserved=reserved)
+    first_def = {}
+    for i in range(p.n_instrs):
+        for o in range(p.instr_op_off[i], p.instr_op_off[i] + p.instr_n_defs[i]):
+            first_def.setdefault(int(p.op_vreg[o]), i)
+    plain = oracle_mod.OracleProgram(p)
+    for _ in range(30):
+        T = rng.integers(0, 36, size=V)
+        row = H.row_from_table(p, T)
+        got = op.verify(lv, row)[0]
+        ref = plain.verify(lv, row)[0]                                  # same row without the rules
+        bad_instrs = []
+        for v, i in first_def.items():
+            regs = range(int(T[v]), int(T[v]) + int(p.vreg_width[v]))
+            ok = T[v] % align[v] == 0 and all(r < 32 and ranges[cls[v]][0] <= r < ranges[cls[v]][1] and r not in reserved
+                                              for r in regs)
+            if not ok:
+                bad_instrs.append(i)
+        assert bool(got["flags"] & RANGE) == bool(bad_instrs)
+        assert got["conflict_pairs"] == ref["conflict_pairs"] and got["bank_conflicts"] == ref["bank_conflicts"]
+        assert (got["flags"] & (INTERF | INCONS)) == (ref["flags"] & (INTERF | INCONS))
+        firsts = bad_instrs + ([int(ref["first_violation_instr"])] if ref["flags"] & (INTERF | INCONS | RANGE) else [])
+        assert got["first_violation_instr"] == (min(firsts) if firsts else -1)
