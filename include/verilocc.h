@@ -181,6 +181,33 @@ int vl_verify_host(vl_program *prog, const uint16_t *h_cand, uint64_t K, uint64_
                    vl_verdict *h_out, void *cuda_stream);
 
 /*
+ * Optional hardware rules for the Realizability check (Section 1: register file sizes and reserved
+ * registers; Section 3.2: scalar and vector register classes; Section 4.5: hardware rules on register
+ * tuples).  With rules set, a definition of v violates Realizability (VL_OUT_OF_RANGE, reported at the
+ * instruction of the definition) also when T[v] is not a multiple of vreg_align[v], when
+ * [T[v], T[v]+width) is not inside [class_lo[c], class_hi[c]) for c = vreg_class[v], or when it holds a
+ * reserved register.  Classes are ranges of the one register numbering 0..P-1; Safety and the bank
+ * tally are unchanged (a misplaced tuple is compared with the others where it sits).
+ * All pointers are HOST memory, read during the call; a NULL member switches that rule off.
+ */
+#define VL_MAX_CLASSES 8
+typedef struct {
+    const uint8_t *vreg_align;     /* [n_vregs], each >= 1 */
+    const uint8_t *vreg_class;     /* [n_vregs], each < n_classes */
+    uint32_t n_classes;            /* 1..VL_MAX_CLASSES when vreg_class is given */
+    const uint32_t *class_lo;      /* [n_classes] */
+    const uint32_t *class_hi;      /* [n_classes], class_lo <= class_hi <= P */
+    const uint32_t *reserved_mask; /* ceil(P/32) words, bit (r & 31) of word r / 32: register r is reserved */
+} vl_constraints;
+
+/*
+ * Sets (or, with rules == NULL or all members NULL, clears) the rules of the handle for later
+ * vl_verify* calls.  Waits for the device, then replaces the handle's copies.
+ * Errors: INVALID_ARG (alignment 0, class out of range, bad class range), CUDA.
+ */
+int vl_program_set_constraints(vl_program *prog, const vl_constraints *rules);
+
+/*
  * Statistics of the re-sampling loop (Section 3.4, last paragraph: the model is sampled again until
  * a candidate passes or the attempts run out; Section 4: Pass@k, AvgTry, MaxTry).  The rows of a
  * verdict array are the attempts of one test case, in order.

@@ -29,7 +29,7 @@ VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERN
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
            "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static",
-           "vl_resample_stats", "vl_verify_until_pass"]
+           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -82,6 +82,16 @@ _lib.vl_verify_until_pass.restype = C.c_int
 _lib.vl_verify_until_pass.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_void_p]
 VL_MAX_PASS_AT = 8
+VL_MAX_CLASSES = 8
+
+
+class vl_constraints(C.Structure):
+    _fields_ = [("vreg_align", C.c_void_p), ("vreg_class", C.c_void_p), ("n_classes", C.c_uint32),
+                ("class_lo", C.c_void_p), ("class_hi", C.c_void_p), ("reserved_mask", C.c_void_p)]
+
+
+_lib.vl_program_set_constraints.restype = C.c_int
+_lib.vl_program_set_constraints.argtypes = [C.c_void_p, C.c_void_p]
 SAMPLE_STATS_DTYPE = np.dtype([("first_pass", "<u8"), ("n_pass", "<u8")])
 
 
@@ -164,6 +174,27 @@ class Program:
 
     def set_option(self, option: int, value: int):
         self._check(_lib.vl_program_set_option(self._h, option, value), "vl_program_set_option")
+
+    def set_constraints(self, vreg_align=None, vreg_class=None, class_ranges=None, reserved=None, P=None):
+        """Hardware rules for the Realizability check: per-vreg alignment, per-vreg class with the
+        half-open register range of every class, reserved register numbers.  No argument clears them."""
+        keep = []
+        c = vl_constraints()
+        if vreg_align is not None:
+            a = np.ascontiguousarray(vreg_align, dtype=np.uint8); keep.append(a); c.vreg_align = a.ctypes.data
+        if vreg_class is not None:
+            a = np.ascontiguousarray(vreg_class, dtype=np.uint8); keep.append(a); c.vreg_class = a.ctypes.data
+            lo = np.ascontiguousarray([r[0] for r in class_ranges], dtype=np.uint32)
+            hi = np.ascontiguousarray([r[1] for r in class_ranges], dtype=np.uint32)
+            keep += [lo, hi]
+            c.n_classes, c.class_lo, c.class_hi = len(lo), lo.ctypes.data, hi.ctypes.data
+        if reserved is not None:
+            m = np.zeros((P + 31) // 32 + 1, dtype=np.uint32)
+            for r in reserved:
+                if r < P:
+                    m[r >> 5] |= np.uint32(1 << (r & 31))
+            keep.append(m); c.reserved_mask = m.ctypes.data
+        self._check(_lib.vl_program_set_constraints(self._h, C.byref(c)), "vl_program_set_constraints")
 
     def vl_liveness(self, stream=None):
         self._check(_lib.vl_liveness(self._h, _stream_ptr(stream)), "vl_liveness")

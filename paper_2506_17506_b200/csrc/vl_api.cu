@@ -178,6 +178,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
+    cudaFree(p->d_vcons); cudaFree(p->d_rs_prefix);
     for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); }
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
@@ -228,6 +229,55 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     default:
         return VL_ERR_INVALID_ARG;
     }
+}
+
+extern "C" int vl_program_set_constraints(vl_program *p, const vl_constraints *c)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    const uint32_t V = p->V, P = p->P;
+    std::vector<uint4> vcons;
+    std::vector<uint16_t> prefix;
+    uint32_t lo[VL_MAX_CLASSES] = {0}, hi[VL_MAX_CLASSES] = {0};
+    hi[0] = P;
+    const bool any = c && (c->vreg_align || c->vreg_class || c->reserved_mask);
+    if (any) {
+        if (c->vreg_class) {
+            if (c->n_classes == 0 || c->n_classes > VL_MAX_CLASSES || !c->class_lo || !c->class_hi) return VL_ERR_INVALID_ARG;
+            for (uint32_t j = 0; j < c->n_classes; ++j) {
+                if (c->class_lo[j] > c->class_hi[j] || c->class_hi[j] > P) return VL_ERR_INVALID_ARG;
+                lo[j] = c->class_lo[j];
+                hi[j] = c->class_hi[j];
+            }
+        }
+        vcons.resize(V ? V : 1);
+        for (uint32_t v = 0; v < V; ++v) {
+            const uint32_t al = c->vreg_align ? c->vreg_align[v] : 1u;
+            const uint32_t cl = c->vreg_class ? c->vreg_class[v] : 0u;
+            if (al == 0 || (c->vreg_class && cl >= c->n_classes)) return VL_ERR_INVALID_ARG;
+            vcons[v] = make_uint4(lo[cl] | (hi[cl] << 16), al, al > 1 ? (uint32_t)((0x100000000ull + al - 1) / al) : 0u, 0u);
+        }
+        if (c->reserved_mask) {
+            prefix.resize((size_t)P + 1);
+            uint32_t n = 0;
+            for (uint32_t r = 0; r < P; ++r) {
+                prefix[r] = (uint16_t)n;
+                n += (c->reserved_mask[r >> 5] >> (r & 31)) & 1u;
+            }
+            prefix[P] = (uint16_t)n;  // P <= 65535, so the count fits
+        }
+    }
+    VL_CUDA(p, cudaSetDevice(p->device));
+    VL_CUDA(p, cudaDeviceSynchronize());  // verify kernels in flight still read the old rules
+    cudaFree(p->d_vcons); p->d_vcons = nullptr;
+    cudaFree(p->d_rs_prefix); p->d_rs_prefix = nullptr;
+    if (!any) return VL_OK;
+    VL_CUDA(p, cudaMalloc(&p->d_vcons, vcons.size() * sizeof(uint4)));
+    VL_CUDA(p, cudaMemcpy(p->d_vcons, vcons.data(), vcons.size() * sizeof(uint4), cudaMemcpyHostToDevice));
+    if (!prefix.empty()) {
+        VL_CUDA(p, cudaMalloc(&p->d_rs_prefix, prefix.size() * sizeof(uint16_t)));
+        VL_CUDA(p, cudaMemcpy(p->d_rs_prefix, prefix.data(), prefix.size() * sizeof(uint16_t), cudaMemcpyHostToDevice));
+    }
+    return VL_OK;
 }
 
 extern "C" int vl_liveness(vl_program *p, void *stream)

@@ -101,6 +101,9 @@ struct vl_program {
     uint8_t *d_iflags = nullptr;            // [nI] 1 if the instruction has a definition the walk skips
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
     uint32_t *d_vinfo = nullptr;            // [V] width | VINFO_OCCURS | VINFO_DEFINED
+    // optional hardware rules of the Realizability check (vl_program_set_constraints)
+    uint4 *d_vcons = nullptr;               // [V] (class first | class end << 16, alignment, ceil(2^32 / alignment), 0); null = no rules
+    uint16_t *d_rs_prefix = nullptr;        // [P+1] reserved registers below r; null = none reserved
     uint32_t *d_th_off = nullptr, *d_th = nullptr;  // per block: vregs occupied through the whole block
     // live-after lists without the block's through-set, for the recount: the list of instruction i of
     // block b is ls[lo_off[i] - ls_adj[b] - i * th_cnt[b] ...), |live-after| - th_cnt[b] entries

@@ -46,6 +46,11 @@ struct TParams {
     // per-pass state this kernel clears for the kernels after it
     uint32_t AW;
     uint32_t *anom, *racc, *grp_done, *work;
+    // optional hardware rules: per vreg (first | end << 16 of its class's registers, alignment,
+    // ceil(2^32 / alignment)), and
+    // the number of reserved registers below every register
+    const uint4 *vcons;
+    const uint16_t *rs_prefix;
 };
 
 struct TMisc {
@@ -168,6 +173,46 @@ __device__ __forceinline__ uint32_t pk_get(uint64_t x, int g) { return (uint32_t
 __device__ __forceinline__ bool ranges_overlap(uint32_t a, uint32_t wa, uint32_t b, uint32_t wb)
 {
     return a < b + wb && b < a + wa;
+}
+
+// Hardware rules on where the tuples may sit (alignment, registers of the vreg's class, reserved
+// registers) for the G candidates of a block: a sweep of its own over the vregs, run only for
+// programs that have rules, four vregs per thread and round so that the loads of a round are in
+// flight together.  Kept out of line, so the kernel's other phases keep their registers.  The
+// remainder uses the reciprocal the host stored (exact for 16-bit values and alignments up to 255).
+template <int G, int NT>
+__device__ __noinline__ void rules_sweep(const uint4 *vcons, const uint16_t *rs_prefix, const uint32_t *vinfo,
+                                         const uint32_t *first_def_instr, uint32_t V, uint32_t P,
+                                         const uint16_t *Tt, TMisc *M)
+{
+    for (uint32_t v0 = threadIdx.x; v0 < V; v0 += 4 * NT) {
+        uint4 vc[4];
+        uint32_t vi[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t v = v0 + u * NT;
+            vc[u] = v < V ? vcons[v] : make_uint4(0, 0, 0, 0);
+            vi[u] = v < V ? vinfo[v] : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t v = v0 + u * NT;
+            if (v >= V || !(vi[u] & VINFO_DEFINED)) continue;
+            const uint32_t clo = vc[u].x & 0xFFFFu, chi = vc[u].x >> 16, al = vc[u].y, recip = vc[u].z;
+            const uint32_t w = vi[u] & 0xFFu;
+            const uint64_t tt = t_load<G>(Tt, v);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const uint32_t tv = pk_get(tt, g);
+                bool bad = (al > 1 && tv != __umulhi(tv, recip) * al) || tv < clo || tv + w > chi;
+                if (!bad && rs_prefix) bad = rs_prefix[min(tv + w, P)] != rs_prefix[min(tv, P)];
+                if (bad) {
+                    atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
+                    atomicMin(&M->minR[g], first_def_instr[v]);
+                }
+            }
+        }
+    }
 }
 
 // =========================================================================== k_tables
@@ -391,6 +436,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         }
     }
     PT(1);
+    if (q.vcons) rules_sweep<G, NT>(q.vcons, q.rs_prefix, q.vinfo, q.first_def_instr, q.V, q.P, Tt, M);
 
     __syncthreads();
     PT(2);
@@ -1358,6 +1404,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.tg = vs.tg; tq.cstate = vs.cstate; tq.status = p->d_status + 1;
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
+    tq.vcons = p->d_vcons; tq.rs_prefix = p->d_rs_prefix;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
     if (pl.NT == 256) {

@@ -120,3 +120,7 @@ def test_resample_argument_checks(B):
     g.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     n = C.c_uint64(0)
     assert g(None, None, 1, 8, 1, None, C.byref(n), C.byref(n), None) == B.VL_ERR_INVALID_ARG
+    h = lib.vl_program_set_constraints
+    h.restype = C.c_int
+    h.argtypes = [C.c_void_p, C.c_void_p]
+    assert h(None, None) == B.VL_ERR_INVALID_ARG

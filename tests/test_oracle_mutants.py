@@ -11,7 +11,7 @@ SRC = os.path.join(ROOT, "oracle", "vl_oracle.c")
 
 MUTANTS = [
     ("overlap uses <= (touching ranges collide)", "return a < b + wb && b < a + wa;", "return a <= b + wb && b < a + wa;"),
-    ("range check off by one", "if (s + w > p->P)", "if (s + w >= p->P)"),
+    ("range check off by one", "int unreal = s + w > p->P;", "int unreal = s + w >= p->P;"),
     ("definition compared with itself", "if (u == v) continue;", ""),
     ("kill dropped from the block transfer function",
      "uint8_t in = use[(size_t)b * V + v] | (o & !def[(size_t)b * V + v]);", "uint8_t in = use[(size_t)b * V + v] | o;"),
