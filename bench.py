@@ -166,7 +166,7 @@ def run_reference(args):
 # DRAM bytes (read + write) per candidate of each kernel, from the profiler capture of a 4096-row launch
 # summarised under profiles/ (traffic grows in proportion to the rows of a launch); None = no capture of
 # the kernel as it stands.
-TRAFFIC_PER_CANDIDATE = {"k_tables": 891.86e6 / 4096, "k_walk": 86.36e6 / 4096}
+TRAFFIC_PER_CANDIDATE = {"k_tables": 891.05e6 / 4096, "k_walk": 86.28e6 / 4096}
 
 
 def main():
