@@ -60,6 +60,8 @@ def _load():
         lib.vlo_violations.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.vlo_conflicts.restype = C.c_uint64
         lib.vlo_conflicts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        lib.vlo_bank_histogram.restype = None
+        lib.vlo_bank_histogram.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.vlo_sample_stats_of.restype = None
         lib.vlo_sample_stats_of.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         lib.vlo_resample_summary.restype = None
@@ -166,6 +168,15 @@ class OracleProgram:
         lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
         lib.vlo_violations(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(kinds))
         return kinds[: self.n_instrs]
+
+    def bank_histogram(self, live: Liveness, row: np.ndarray) -> np.ndarray:
+        """Extra read cycles of one row per register bank (their sum is the verdict's bank_conflicts)."""
+        lib = _load()
+        row = np.ascontiguousarray(row, dtype=np.uint16)
+        hist = np.zeros(self.src.B, dtype=np.uint64)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        lib.vlo_bank_histogram(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(hist))
+        return hist
 
     def conflicts(self, live: Liveness, row: np.ndarray) -> np.ndarray:
         """All (instruction, defined vreg, other vreg) overlap records of one row."""

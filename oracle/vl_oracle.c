@@ -178,7 +178,7 @@ static int ranges_overlap(uint32_t a, uint32_t wa, uint32_t b, uint32_t wb)
  */
 static void walk(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
                  const uint16_t *row, vlo_verdict *out, uint8_t *kinds,
-                 uint32_t *triples, uint64_t cap, uint64_t *n_triples)
+                 uint32_t *triples, uint64_t cap, uint64_t *n_triples, uint64_t *bank_hist)
 {
     const uint32_t V = p->n_vregs, nI = p->n_instrs;
     int32_t *T = malloc(((size_t)V + 1) * sizeof(int32_t));
@@ -270,6 +270,7 @@ static void walk(const vlo_program *p, const uint64_t *lo_off, const uint32_t *l
             uint32_t n = 0;
             for (uint32_t r = 0; r < nq; ++r) if (Q[r] % p->B == Q[q] % p->B) ++n;
             bank += n - 1;
+            if (bank_hist) bank_hist[Q[q] % p->B] += n - 1;
         }
     }
     free(Q);
@@ -285,13 +286,13 @@ static void walk(const vlo_program *p, const uint64_t *lo_off, const uint32_t *l
 void vlo_verify(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
                 const uint16_t *row, vlo_verdict *out)
 {
-    walk(p, lo_off, lo, row, out, NULL, NULL, 0, NULL);
+    walk(p, lo_off, lo, row, out, NULL, NULL, 0, NULL, NULL);
 }
 
 void vlo_verify_rows(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
                      const uint16_t *rows, uint64_t K, uint64_t pitch, vlo_verdict *out)
 {
-    for (uint64_t k = 0; k < K; ++k) walk(p, lo_off, lo, rows + k * pitch, out + k, NULL, NULL, 0, NULL);
+    for (uint64_t k = 0; k < K; ++k) walk(p, lo_off, lo, rows + k * pitch, out + k, NULL, NULL, 0, NULL, NULL);
 }
 
 /* per-instruction violation kinds for one row */
@@ -299,7 +300,7 @@ void vlo_violations(const vlo_program *p, const uint64_t *lo_off, const uint32_t
                     const uint16_t *row, uint8_t *kinds)
 {
     vlo_verdict v;
-    walk(p, lo_off, lo, row, &v, kinds, NULL, 0, NULL);
+    walk(p, lo_off, lo, row, &v, kinds, NULL, 0, NULL, NULL);
 }
 
 /* every (instruction, defined vreg, other vreg) overlap of one row; returns the total */
@@ -308,8 +309,18 @@ uint64_t vlo_conflicts(const vlo_program *p, const uint64_t *lo_off, const uint3
 {
     vlo_verdict v;
     uint64_t n = 0;
-    walk(p, lo_off, lo, row, &v, NULL, triples, cap, &n);
+    walk(p, lo_off, lo, row, &v, NULL, triples, cap, &n, NULL);
     return n;
+}
+
+/* extra read cycles of one row per register bank: hist[b] sums, over the instructions, the
+ * distinct source registers in bank b beyond the first (hist must hold B zeroed counters) */
+void vlo_bank_histogram(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                        const uint16_t *row, uint64_t *hist)
+{
+    vlo_verdict v;
+    for (uint32_t b = 0; b < p->B; ++b) hist[b] = 0;
+    walk(p, lo_off, lo, row, &v, NULL, NULL, 0, NULL, hist);
 }
 
 /* ------------------------------------------------- re-sampling statistics */

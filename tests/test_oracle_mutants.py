@@ -28,6 +28,8 @@ MUTANTS = [
      "if (attempts < k[j]) summary[4 + j] += 1;"),
     ("test cases that never pass counted among the attempts", "if (s[c].first_pass >= K[c]) continue; /* never passed */", ""),
     ("last passing attempt instead of the first", "if (s->first_pass == K) s->first_pass = k;", "s->first_pass = k;"),
+    ("bank histogram charges the wrong bank", "if (bank_hist) bank_hist[Q[q] % p->B] += n - 1;",
+     "if (bank_hist) bank_hist[Q[q] / p->B % p->B] += n - 1;"),
     ("alignment tested on the end of the tuple", "if (p->vreg_align && s % p->vreg_align[v] != 0) unreal = 1;",
      "if (p->vreg_align && (s + w) % p->vreg_align[v] != 0) unreal = 1;"),
     ("class range closed at the top", "if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;",

@@ -489,3 +489,49 @@ def test_hardware_rules_equal_register_by_register_definition(oracle_mod, seed):
         assert (got["flags"] & (INTERF | INCONS)) == (ref["flags"] & (INTERF | INCONS))
         firsts = bad_instrs + ([int(ref["first_violation_instr"])] if ref["flags"] & (INTERF | INCONS | RANGE) else [])
         assert got["first_violation_instr"] == (min(firsts) if firsts else -1)
+
+
+# ------------------------------------------------------------ per-candidate diagnostics
+def test_bank_histogram_hand_cases(oracle_mod):
+    def hist(regs, B=4, P=16):
+        n = len(regs)
+        blocks = [[([v], []) for v in range(n)] + [([n], list(range(n)))]]
+        p = synth.program_from_lists(blocks, [], n + 1, [1] * (n + 1), P, B)
+        free = [r for r in range(P) if r not in regs][0]
+        op, lv = _oracle(oracle_mod, p)
+        row = H.row_from_table(p, list(regs) + [free])
+        h = op.bank_histogram(lv, row)
+        assert int(h.sum()) == int(op.verify(lv, row)[0]["bank_conflicts"])
+        return h.tolist()
+
+    assert hist([4, 6, 9]) == [0, 0, 0, 0]              # Section 2: R4, R6, R9 sit in separate banks
+    assert hist([4, 8]) == [1, 0, 0, 0]
+    assert hist([4, 8, 12, 5, 9]) == [2, 1, 0, 0]
+    assert hist([3, 7, 11, 15]) == [0, 0, 0, 3]
+    assert hist([4, 4, 8]) == [1, 0, 0, 0]              # the same register read twice counts once
+    assert hist([1, 4, 7, 10], B=3) == [0, 3, 0]
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_diagnostics_agree_with_the_verdict(oracle_mod, seed):
+    """Conflict records, per-instruction kinds and the bank histogram of a row add up to its verdict."""
+    rng = np.random.default_rng(4100 + seed)
+    p = H.random_program(8000 + seed, strict=True, reachable=True, max_instrs=50, max_vregs=16, P=24,
+                         widths=(1, 2, 4), B=[4, 3, 2][seed % 3])
+    op, lv = _oracle(oracle_mod, p)
+    for _ in range(10):
+        row = H.row_from_table(p, rng.integers(0, 28, size=p.n_vregs))
+        if rng.random() < 0.5:
+            row[rng.integers(0, p.n_operands)] ^= 1
+        vd = op.verify(lv, row)[0]
+        tr = op.conflicts(lv, row)
+        kinds = op.violations(lv, row)
+        assert len(tr) == vd["conflict_pairs"]
+        assert int(op.bank_histogram(lv, row).sum()) == vd["bank_conflicts"]
+        assert int(np.bitwise_or.reduce(kinds)) == (0 if vd["flags"] == PASS else int(vd["flags"]))
+        bad = np.flatnonzero(kinds)
+        assert vd["first_violation_instr"] == (int(bad[0]) if len(bad) else -1)
+        assert set(np.flatnonzero(kinds & INTERF).tolist()) == set(tr[:, 0].tolist())
+        for i, v, u in tr:                              # every record is a definition of v at i that overlaps u
+            defs = p.op_vreg[p.instr_op_off[i]: p.instr_op_off[i] + p.instr_n_defs[i]]
+            assert v in defs and u != v
