@@ -254,6 +254,25 @@ int vl_verify_until_pass(vl_program *prog, const uint16_t *d_cand, uint64_t K, u
                          void *cuda_stream);
 
 /*
+ * Diagnostics of one candidate, as feedback for the sampler (Section 4.5 sorts failures into dataflow
+ * and hardware-constraint violations; Section 6 proposes the verifier's findings as a training signal).
+ * For the row d_row (DEVICE, n_operands entries): every Safety violation as a record (instruction,
+ * defined vreg, other vreg) into d_conflicts (DEVICE, room for `cap` records, in no particular order;
+ * records beyond `cap` are counted, not stored) with the total in *d_n_conflicts (DEVICE, 8-byte aligned;
+ * equals the verdict's conflict_pairs); unless NULL, d_kinds[i] (DEVICE, n_instrs bytes) receives the OR
+ * of the violation bits raised at instruction i (the lowest i with a bit is first_violation_instr) and
+ * d_bank_hist[b] (DEVICE, B counters) the extra read cycles charged to bank b (their sum is
+ * bank_conflicts).  Rules set with vl_program_set_constraints apply.  Not a hot path: one thread per
+ * instruction over the live-after lists.  Stream-ordered, no synchronisation; the first call allocates
+ * 8 * n_vregs bytes in the handle.  Errors: INVALID_ARG, LIVENESS_NOT_RUN, CUDA.
+ */
+typedef struct {
+    uint32_t instr, vreg, other;
+} vl_conflict;
+int vl_diagnose(vl_program *prog, const uint16_t *d_row, uint64_t cap, vl_conflict *d_conflicts,
+                uint64_t *d_n_conflicts, uint8_t *d_kinds, uint64_t *d_bank_hist, void *cuda_stream);
+
+/*
  * Block-level liveness without any allocation.  (The paper has no counterpart; this exists for
  * hosts that cannot allocate device memory when they call in: a process that handed all of HBM to
  * its own pools at start-up, a plugin under a memory budget it does not control, or a loop that

@@ -29,7 +29,7 @@ VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERN
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
            "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static",
-           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints"]
+           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints", "vl_diagnose"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -90,6 +90,8 @@ class vl_constraints(C.Structure):
                 ("class_lo", C.c_void_p), ("class_hi", C.c_void_p), ("reserved_mask", C.c_void_p)]
 
 
+_lib.vl_diagnose.restype = C.c_int
+_lib.vl_diagnose.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.vl_program_set_constraints.restype = C.c_int
 _lib.vl_program_set_constraints.argtypes = [C.c_void_p, C.c_void_p]
 SAMPLE_STATS_DTYPE = np.dtype([("first_pass", "<u8"), ("n_pass", "<u8")])
@@ -256,6 +258,22 @@ class Program:
         self._check(_lib.vl_verify_until_pass(self._h, cand.data_ptr(), K, pitch, batch_rows, out.data_ptr(),
                                               C.byref(done), C.byref(first), _stream_ptr(stream)), "vl_verify_until_pass")
         return out, int(done.value), int(first.value)
+
+    def vl_diagnose(self, row, cap: int = 1 << 16, n_banks: int = 4, stream=None):
+        """Diagnostics of one candidate (CUDA uint16 tensor of n_operands entries or more): returns
+        (conflict records [n, 3] as numpy, total count, kinds per instruction, bank histogram)."""
+        import torch
+        dev = row.device
+        rec = torch.zeros((max(cap, 1), 3), dtype=torch.int32, device=dev)
+        cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+        kinds = torch.zeros(max(self.n_instrs, 1), dtype=torch.uint8, device=dev)
+        hist = torch.zeros(n_banks, dtype=torch.int64, device=dev)
+        self._check(_lib.vl_diagnose(self._h, row.data_ptr(), cap, rec.data_ptr(), cnt.data_ptr(), kinds.data_ptr(),
+                                     hist.data_ptr(), _stream_ptr(stream)), "vl_diagnose")
+        torch.cuda.synchronize(dev)
+        n = int(cnt.item())
+        return (rec[: min(n, cap)].cpu().numpy().view(np.uint32), n, kinds[: self.n_instrs].cpu().numpy(),
+                hist.cpu().numpy().view(np.uint64))
 
     def vl_verify_status(self, stream=None):
         self._check(_lib.vl_verify_status(self._h, _stream_ptr(stream)), "vl_verify_status")

@@ -171,6 +171,7 @@ struct vl_program {
     cudaEvent_t h_events[2] = {nullptr, nullptr};
     // one record for vl_verify_until_pass: device copy and its pinned landing place
     vl_sample_stats *d_rs = nullptr, *h_rs = nullptr;
+    unsigned long long *d_diag_T = nullptr;  // [V] scratch of vl_diagnose: (first occurrence << 16) | value
 };
 
 extern std::atomic<uint64_t> g_vl_launches;

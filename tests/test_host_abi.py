@@ -124,3 +124,7 @@ def test_resample_argument_checks(B):
     h.restype = C.c_int
     h.argtypes = [C.c_void_p, C.c_void_p]
     assert h(None, None) == B.VL_ERR_INVALID_ARG
+    d = lib.vl_diagnose
+    d.restype = C.c_int
+    d.argtypes = [C.c_void_p] * 2 + [C.c_uint64] + [C.c_void_p] * 5
+    assert d(None, None, 0, None, None, None, None, None) == B.VL_ERR_INVALID_ARG
