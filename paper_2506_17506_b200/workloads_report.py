@@ -11,7 +11,8 @@ their bandwidth fraction.  Workload 4 (256 independent programs) goes through vl
 and vl_verify_batch.  Also per workload: the time of one vl_resample_stats call over the verdict
 arrays (launch-latency bound: three or more small kernels), the statistics it returns (test cases
 solved, attempts summed and largest, Pass@1/10/100 counts), and the time of the early-exit loop
-vl_verify_until_pass in batches of 100 rows (it stops after the first batch with a passing row).
+vl_verify_until_pass in batches of 100 rows (it stops after the first batch with a passing row),
+and the time of vl_diagnose on one row.
 """
 from __future__ import annotations
 
@@ -114,6 +115,26 @@ def main() -> int:
             _, rows_done, first_pass = gps[0].vl_verify_until_pass(cands[0], 100, outs[0], stream)
         er[3].record(stream)
         torch.cuda.synchronize()
+        # diagnostics of the first row of the first program
+        rec = torch.zeros((4096, 3), dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(1, dtype=torch.int64, device="cuda")
+        kinds = torch.zeros(progs[0].n_instrs, dtype=torch.uint8, device="cuda")
+        hist = torch.zeros(progs[0].B, dtype=torch.int64, device="cuda")
+
+        def diagnose():
+            rc = vl._lib.vl_diagnose(gps[0].handle, cands[0].data_ptr(), 4096, rec.data_ptr(), cnt.data_ptr(),
+                                     kinds.data_ptr(), hist.data_ptr(), sp)
+            assert rc == vl.VL_OK, rc
+
+        for _ in range(3):
+            diagnose()
+        ed = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        ed[0].record(stream)
+        for _ in range(args.steps):
+            diagnose()
+        ed[1].record(stream)
+        torch.cuda.synchronize()
+        diagnose_us = ed[0].elapsed_time(ed[1]) / args.steps * 1e3
         resample_us = er[0].elapsed_time(er[1]) / args.steps * 1e3
         until_ms = er[2].elapsed_time(er[3]) / args.steps
         step_ms = ev[0].elapsed_time(ev[1]) / args.steps
@@ -134,6 +155,7 @@ def main() -> int:
             "resample_stats_us": resample_us, "resample_summary": summary,
             "until_pass_batch100_ms": until_ms, "until_pass_rows_checked": rows_done,
             "until_pass_first_passing_row": first_pass,
+            "diagnose_one_row_us": diagnose_us,
         }), flush=True)
         for gp in gps:
             gp.close()
