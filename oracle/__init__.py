@@ -62,6 +62,8 @@ def _load():
         lib.vlo_conflicts.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
         lib.vlo_bank_histogram.restype = None
         lib.vlo_bank_histogram.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.vlo_occupied.restype = None
+        lib.vlo_occupied.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.vlo_sample_stats_of.restype = None
         lib.vlo_sample_stats_of.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         lib.vlo_resample_summary.restype = None
@@ -177,6 +179,15 @@ class OracleProgram:
         lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
         lib.vlo_bank_histogram(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(hist))
         return hist
+
+    def occupied(self, live: Liveness, row: np.ndarray) -> np.ndarray:
+        """uint8 [n_instrs, P]: registers the definitions of every instruction must keep off."""
+        lib = _load()
+        row = np.ascontiguousarray(row, dtype=np.uint16)
+        occ = np.zeros((max(self.n_instrs, 1), self.P), dtype=np.uint8)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        lib.vlo_occupied(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(row), _ptr(occ))
+        return occ[: self.n_instrs]
 
     def conflicts(self, live: Liveness, row: np.ndarray) -> np.ndarray:
         """All (instruction, defined vreg, other vreg) overlap records of one row."""

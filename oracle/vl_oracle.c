@@ -323,6 +323,37 @@ void vlo_bank_histogram(const vlo_program *p, const uint64_t *lo_off, const uint
     walk(p, lo_off, lo, row, &v, NULL, NULL, 0, NULL, hist);
 }
 
+/*
+ * Registers the definitions of instruction i must keep off (Section 4.5 proposes decoding that masks
+ * out the registers occupied at that point): occ[i * P + r] = 1 iff register r < P belongs to the
+ * range of a vreg that is live after i and not defined by i, or is reserved.  A vreg whose table
+ * entry is P or more (not assigned yet) contributes nothing.
+ */
+void vlo_occupied(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                  const uint16_t *row, uint8_t *occ)
+{
+    const uint32_t V = p->n_vregs, nI = p->n_instrs, P = p->P;
+    int32_t *T = malloc(((size_t)V + 1) * sizeof(int32_t));
+    for (uint32_t v = 0; v < V; ++v) T[v] = -1;
+    for (uint32_t o = 0; o < p->n_operands; ++o)
+        if (T[p->op_vreg[o]] < 0) T[p->op_vreg[o]] = row[o];
+    memset(occ, 0, (size_t)nI * P);
+    for (uint32_t i = 0; i < nI; ++i) {
+        uint32_t o0 = p->instr_op_off[i], nd = p->instr_n_defs[i];
+        for (uint64_t e = lo_off[i]; e < lo_off[i + 1]; ++e) {
+            uint32_t u = lo[e];
+            int own = 0;
+            for (uint32_t d = o0; d < o0 + nd; ++d) if (p->op_vreg[d] == u) own = 1;
+            if (own) continue;
+            for (uint32_t r = (uint32_t)T[u]; r < (uint32_t)T[u] + p->vreg_width[u]; ++r)
+                if (r < P) occ[(size_t)i * P + r] = 1;
+        }
+        if (p->reserved)
+            for (uint32_t r = 0; r < P; ++r) if (p->reserved[r]) occ[(size_t)i * P + r] = 1;
+    }
+    free(T);
+}
+
 /* ------------------------------------------------- re-sampling statistics */
 
 /*

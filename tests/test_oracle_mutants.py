@@ -30,6 +30,10 @@ MUTANTS = [
     ("last passing attempt instead of the first", "if (s->first_pass == K) s->first_pass = k;", "s->first_pass = k;"),
     ("bank histogram charges the wrong bank", "if (bank_hist) bank_hist[Q[q] % p->B] += n - 1;",
      "if (bank_hist) bank_hist[Q[q] / p->B % p->B] += n - 1;"),
+    ("own definitions kept in the occupied mask", "if (own) continue;", ""),
+    ("occupied mask drops the last register of a tuple",
+     "for (uint32_t r = (uint32_t)T[u]; r < (uint32_t)T[u] + p->vreg_width[u]; ++r)",
+     "for (uint32_t r = (uint32_t)T[u]; r + 1 < (uint32_t)T[u] + p->vreg_width[u]; ++r)"),
     ("alignment tested on the end of the tuple", "if (p->vreg_align && s % p->vreg_align[v] != 0) unreal = 1;",
      "if (p->vreg_align && (s + w) % p->vreg_align[v] != 0) unreal = 1;"),
     ("class range closed at the top", "if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;",

@@ -535,3 +535,54 @@ def test_diagnostics_agree_with_the_verdict(oracle_mod, seed):
         for i, v, u in tr:                              # every record is a definition of v at i that overlaps u
             defs = p.op_vreg[p.instr_op_off[i]: p.instr_op_off[i] + p.instr_n_defs[i]]
             assert v in defs and u != v
+
+
+# --------------------------------------------------- occupied registers at every definition point
+def test_occupied_registers_hand_case(oracle_mod):
+    # v0 (w2) and v1 (w1) defined, v2 defined from v0 (v0 dies), all read at the end except v0
+    blocks = [[([0], []), ([1], []), ([2], [0]), ([], [1, 2])]]
+    p = synth.program_from_lists(blocks, [], 3, [2, 1, 2], 8)
+    op, lv = _oracle(oracle_mod, p)
+    occ = op.occupied(lv, H.row_from_table(p, [4, 6, 0]))
+    regs = [set(np.flatnonzero(r).tolist()) for r in occ]
+    assert regs[0] == set()                 # v0 is the instruction's own definition, nothing else is live
+    assert regs[1] == {4, 5}                # v0 live after the definition of v1
+    assert regs[2] == {6}                   # v0 dies at its read here; v1 stays; v2 is the own definition
+    assert regs[3] == set()                 # nothing is live after the last reads
+    # a vreg without a register yet (entry >= P) and a tuple sticking out of the file
+    occ = op.occupied(lv, H.row_from_table(p, [7, 0xFFFF, 0]))
+    regs = [set(np.flatnonzero(r).tolist()) for r in occ]
+    assert regs[1] == {7} and regs[2] == set()
+    op.set_constraints(reserved=[3])
+    occ = op.occupied(lv, H.row_from_table(p, [4, 6, 0]))
+    assert set(np.flatnonzero(occ[1]).tolist()) == {3, 4, 5} and set(np.flatnonzero(occ[3]).tolist()) == {3}
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_occupied_registers_from_path_liveness_and_the_safety_verdict(oracle_mod, seed):
+    """The mask is the union of the ranges of the vregs that the path definition of liveness finds
+    live after the instruction (own definitions left out); for instructions with one definition a
+    row is free of Safety violations iff no definition touches the mask of its instruction."""
+    rng = np.random.default_rng(5200 + seed)
+    p = H.random_program(9500 + seed, strict=True, reachable=True, max_instrs=40, max_vregs=14, P=24, widths=(1, 2, 4),
+                         multi_def=(seed % 2 == 1))
+    op, lv = _oracle(oracle_mod, p)
+    live_after, _, _ = H.path_liveness(p)
+    ins, _, _ = H.instr_lists(p)
+    single = all(len(d) <= 1 for d, _ in ins)
+    for _ in range(12):
+        T = rng.integers(0, 26, size=p.n_vregs)
+        row = H.row_from_table(p, T)
+        occ = op.occupied(lv, row)
+        clash = False
+        for i, (defs, _) in enumerate(ins):
+            want = set()
+            for u in live_after[i]:
+                if u not in defs:
+                    want |= {r for r in range(int(T[u]), int(T[u]) + int(p.vreg_width[u])) if r < p.P}
+            assert set(np.flatnonzero(occ[i]).tolist()) == want, f"instr {i}"
+            for v in defs:
+                clash = clash or any(r in want for r in range(int(T[v]), int(T[v]) + int(p.vreg_width[v])))
+        if single:
+            assert clash == bool(op.verify(lv, row)[0]["flags"] & INTERF)
+    assert single == (seed % 2 == 0)
