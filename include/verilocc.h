@@ -273,6 +273,19 @@ int vl_diagnose(vl_program *prog, const uint16_t *d_row, uint64_t cap, vl_confli
                 uint64_t *d_n_conflicts, uint8_t *d_kinds, uint64_t *d_bank_hist, void *cuda_stream);
 
 /*
+ * Registers the definitions of every instruction must keep off, for decoding that masks out occupied
+ * registers (Section 4.5, last paragraph).  For the row d_row (DEVICE, n_operands entries; a vreg that
+ * has no register yet carries any value >= P, e.g. 0xFFFF, and contributes nothing):
+ * d_masks[i * W + r / 32] bit (r & 31), W = ceil(P / 32), is set iff register r < P lies in the range of
+ * a vreg that is live after instruction i and is not defined by i, or is reserved
+ * (vl_program_set_constraints).  A definition of instruction i is safe iff its range touches no set bit
+ * and no other definition of i.  d_masks is DEVICE memory for n_instrs * W words.  Stream-ordered, no
+ * synchronisation; the first call allocates 8 * n_vregs + 8 bytes in the handle.
+ * Errors: INVALID_ARG, LIVENESS_NOT_RUN, CUDA.
+ */
+int vl_occupied_masks(vl_program *prog, const uint16_t *d_row, uint32_t *d_masks, void *cuda_stream);
+
+/*
  * Block-level liveness without any allocation.  (The paper has no counterpart; this exists for
  * hosts that cannot allocate device memory when they call in: a process that handed all of HBM to
  * its own pools at start-up, a plugin under a memory budget it does not control, or a loop that

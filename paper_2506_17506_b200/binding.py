@@ -29,7 +29,7 @@ VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERN
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
            "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static",
-           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints", "vl_diagnose"]
+           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints", "vl_diagnose", "vl_occupied_masks"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -92,6 +92,8 @@ class vl_constraints(C.Structure):
 
 _lib.vl_diagnose.restype = C.c_int
 _lib.vl_diagnose.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.vl_occupied_masks.restype = C.c_int
+_lib.vl_occupied_masks.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.vl_program_set_constraints.restype = C.c_int
 _lib.vl_program_set_constraints.argtypes = [C.c_void_p, C.c_void_p]
 SAMPLE_STATS_DTYPE = np.dtype([("first_pass", "<u8"), ("n_pass", "<u8")])
@@ -274,6 +276,19 @@ class Program:
         n = int(cnt.item())
         return (rec[: min(n, cap)].cpu().numpy().view(np.uint32), n, kinds[: self.n_instrs].cpu().numpy(),
                 hist.cpu().numpy().view(np.uint64))
+
+    def vl_occupied_masks(self, row, P: int, stream=None):
+        """uint8 numpy array [n_instrs, P]: registers the definitions of every instruction must keep off,
+        for one candidate (CUDA uint16 tensor; entries >= P mean "no register yet")."""
+        import torch
+        W = (P + 31) // 32
+        masks = torch.zeros((max(self.n_instrs, 1), W), dtype=torch.int32, device=row.device)
+        self._check(_lib.vl_occupied_masks(self._h, row.data_ptr(), masks.data_ptr(), _stream_ptr(stream)),
+                    "vl_occupied_masks")
+        torch.cuda.synchronize(row.device)
+        words = masks[: self.n_instrs].cpu().numpy().view(np.uint32)
+        bits = np.unpackbits(words.view(np.uint8).reshape(self.n_instrs, W * 4), axis=1, bitorder="little")
+        return bits[:, :P]
 
     def vl_verify_status(self, stream=None):
         self._check(_lib.vl_verify_status(self._h, _stream_ptr(stream)), "vl_verify_status")

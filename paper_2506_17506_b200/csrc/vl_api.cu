@@ -172,6 +172,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     if (p->h_rs) cudaFreeHost(p->h_rs);
     cudaFree(p->d_rs);
     cudaFree(p->d_diag_T);
+    cudaFree(p->d_diag_n);
     if (p->ev_live) cudaEventDestroy(p->ev_live);
     p->live_arena.release();
     p->tmp_arena.release();

@@ -1,4 +1,6 @@
-// Diagnostics of one candidate, for feedback to the sampler (Section 4.5 sorts failures into
+// Diagnostics of one candidate, for feedback to the sampler, and the registers occupied at every
+// definition point, for decoding that masks them out (Section 4.5, last paragraph).
+// Diagnostics (Section 4.5 sorts failures into
 // dataflow violations and hardware-constraint violations; Section 6 proposes the verifier's findings
 // as a training signal): every (instruction, defined vreg, other vreg) overlap, the violation kinds
 // raised at every instruction, and the extra read cycles per register bank.
@@ -103,7 +105,71 @@ __global__ void k_diag_instr(const DParams q)
     }
 }
 
+// Occupied registers per instruction: one warp per instruction ORs the ranges of the vregs live
+// after it (own definitions left out, reserved registers added) into a mask in shared memory and
+// writes the mask out.  W = words per mask.
+constexpr uint32_t OCC_WARPS = 4;
+__global__ void __launch_bounds__(OCC_WARPS * 32) k_occupied(const DParams q, uint32_t W, uint32_t *masks)
+{
+    extern __shared__ uint32_t s_mask[];
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t i = blockIdx.x * OCC_WARPS + warp;
+    if (i >= q.nI) return;
+    uint32_t *m = s_mask + warp * W;
+    for (uint32_t j = lane; j < W; j += 32) {  // reserved registers: bit r set iff the prefix count steps at r
+        uint32_t x = 0;
+        if (q.rs_prefix)
+            for (uint32_t b = 0; b < 32 && j * 32 + b < q.P; ++b)
+                x |= (uint32_t)(q.rs_prefix[j * 32 + b + 1] != q.rs_prefix[j * 32 + b]) << b;
+        m[j] = x;
+    }
+    __syncwarp();
+    const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
+    for (uint32_t e = q.lo_off[i] + lane; e < q.lo_off[i + 1]; e += 32) {
+        const uint32_t u = q.lo[e];
+        bool own = false;
+        for (uint32_t d = o0; d < o0 + nd; ++d) own = own || q.op_vreg[d] == u;
+        if (own) continue;
+        const uint32_t t = (uint32_t)(q.T64[u] & 0xFFFFu);
+        const uint32_t end = min(t + q.width[u], q.P);
+        for (uint32_t r = t; r < end;) {  // word by word
+            const uint32_t hi = min(end, (r | 31u) + 1u), n = hi - r;
+            atomicOr(&m[r >> 5], (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << (r & 31));
+            r = hi;
+        }
+    }
+    __syncwarp();
+    for (uint32_t j = lane; j < W; j += 32) masks[(size_t)i * W + j] = m[j];
+}
+
 }  // namespace
+
+extern "C" int vl_occupied_masks(vl_program *p, const uint16_t *d_row, uint32_t *d_masks, void *stream)
+{
+    if (!p || !d_row || !d_masks) return VL_ERR_INVALID_ARG;
+    if (((uintptr_t)d_row & 1) || ((uintptr_t)d_masks & 3)) return VL_ERR_INVALID_ARG;
+    if (p->live_pending) {
+        const int rc = vl_live_settle(p);
+        if (rc != VL_OK) return rc;
+    }
+    if (!p->live_ok) return VL_ERR_LIVENESS_NOT_RUN;
+    VL_CUDA(p, cudaSetDevice(p->device));
+    if (!p->d_diag_T) VL_CUDA(p, cudaMalloc(&p->d_diag_T, sizeof(unsigned long long) * (p->V ? p->V : 1)));
+    if (!p->d_diag_n) VL_CUDA(p, cudaMalloc(&p->d_diag_n, sizeof(unsigned long long)));
+    cudaStream_t st = (cudaStream_t)stream;
+    DParams q{};
+    q.nI = p->nI; q.nO = p->nO; q.V = p->V; q.P = p->P; q.B = p->B;
+    q.op_off = p->d_op_off; q.op_vreg = p->d_op_vreg; q.lo_off = p->d_lo_off; q.lo = p->d_lo;
+    q.ndefs = p->d_ndefs; q.width = p->d_width; q.rs_prefix = p->d_rs_prefix;
+    q.row = d_row; q.T64 = p->d_diag_T; q.n_conflicts = p->d_diag_n;
+    const uint32_t W = (p->P + 31) / 32;
+    k_diag_init<<<(p->V + 255) / 256 + 1, 256, 0, st>>>(q);
+    if (p->nO) k_diag_table<<<(p->nO + 255) / 256, 256, 0, st>>>(q);
+    if (p->nI) k_occupied<<<(p->nI + OCC_WARPS - 1) / OCC_WARPS, OCC_WARPS * 32, OCC_WARPS * W * sizeof(uint32_t), st>>>(q, W, d_masks);
+    g_vl_launches.fetch_add(1 + (p->nO ? 1 : 0) + (p->nI ? 1 : 0));
+    VL_CUDA(p, cudaGetLastError());
+    return VL_OK;
+}
 
 extern "C" int vl_diagnose(vl_program *p, const uint16_t *d_row, uint64_t cap, vl_conflict *d_conflicts,
                            uint64_t *d_n_conflicts, uint8_t *d_kinds, uint64_t *d_bank_hist, void *stream)

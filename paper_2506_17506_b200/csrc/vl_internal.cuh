@@ -172,6 +172,7 @@ struct vl_program {
     // one record for vl_verify_until_pass: device copy and its pinned landing place
     vl_sample_stats *d_rs = nullptr, *h_rs = nullptr;
     unsigned long long *d_diag_T = nullptr;  // [V] scratch of vl_diagnose: (first occurrence << 16) | value
+    unsigned long long *d_diag_n = nullptr;  // one counter: scratch of vl_occupied_masks
 };
 
 extern std::atomic<uint64_t> g_vl_launches;

@@ -86,3 +86,43 @@ def test_attention_workload_rows(B, oracle_mod):
     assert np.array_equal(kinds, op.violations(lv, zero))
     assert np.array_equal(hist, op.bank_histogram(lv, zero))
     gp.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_occupied_masks_random_small_programs(B, oracle_mod, seed):
+    rng = np.random.default_rng(6100 + seed)
+    p = H.random_program(9700 + seed, strict=True, reachable=(seed % 4 != 0), max_instrs=60, max_vregs=20,
+                         P=[8, 16, 33, 64, 100][seed % 5], widths=(1, 1, 2, 2, 4, 8) if seed % 2 else (1, 2, 3, 5))
+    gp = B.Program(p)
+    gp.vl_liveness()
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    if seed % 3 == 0:
+        reserved = sorted(set(rng.integers(0, p.P, size=3).tolist()))
+        op.set_constraints(reserved=reserved)
+        gp.set_constraints(P=p.P, reserved=reserved)
+    rows = _garbage_rows(p, 12, seed)
+    partial = H.row_from_table(p, np.where(rng.random(p.n_vregs) < 0.5, 0xFFFF, rng.integers(0, p.P, size=p.n_vregs)))
+    for row in list(rows) + [partial]:
+        got = gp.vl_occupied_masks(_to_dev(row[None, :])[0], p.P)
+        assert np.array_equal(got, op.occupied(lv, row))
+    gp.close()
+
+
+def test_occupied_masks_attention_workload(B, oracle_mod):
+    wl = synth.workload(2)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    rows, _ = synth.candidate_rows(p, 4, 0.0, wl.seeds[0])
+    gp = B.Program(p)
+    gp.vl_liveness()
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    rng = np.random.default_rng(5)
+    T = rows[1, np.array([int(np.flatnonzero(p.op_vreg == v)[0]) if (p.op_vreg == v).any() else 0 for v in range(p.n_vregs)])]
+    T = np.where(rng.random(p.n_vregs) < 0.3, 0xFFFF, T)            # a third of the vregs not assigned yet
+    for row in (rows[0], H.row_from_table(p, T)):
+        got = gp.vl_occupied_masks(_to_dev(row[None, :])[0], p.P)
+        want = op.occupied(lv, row)
+        assert np.array_equal(got, want)
+        assert want.sum() > 100_000                                  # hundreds of registers busy at most points
+    gp.close()

@@ -128,3 +128,7 @@ def test_resample_argument_checks(B):
     d.restype = C.c_int
     d.argtypes = [C.c_void_p] * 2 + [C.c_uint64] + [C.c_void_p] * 5
     assert d(None, None, 0, None, None, None, None, None) == B.VL_ERR_INVALID_ARG
+    m = lib.vl_occupied_masks
+    m.restype = C.c_int
+    m.argtypes = [C.c_void_p] * 4
+    assert m(None, None, None, None) == B.VL_ERR_INVALID_ARG
