@@ -12,7 +12,7 @@ and vl_verify_batch.  Also per workload: the time of one vl_resample_stats call 
 arrays (launch-latency bound: three or more small kernels), the statistics it returns (test cases
 solved, attempts summed and largest, Pass@1/10/100 counts), and the time of the early-exit loop
 vl_verify_until_pass in batches of 100 rows (it stops after the first batch with a passing row),
-and the time of vl_diagnose on one row.
+and the times of vl_diagnose and vl_occupied_masks on one row.
 """
 from __future__ import annotations
 
@@ -134,6 +134,22 @@ def main() -> int:
             diagnose()
         ed[1].record(stream)
         torch.cuda.synchronize()
+        Wm = (progs[0].P + 31) // 32
+        masks = torch.zeros((progs[0].n_instrs, Wm), dtype=torch.int32, device="cuda")
+
+        def occupied():
+            rc = vl._lib.vl_occupied_masks(gps[0].handle, cands[0].data_ptr(), masks.data_ptr(), sp)
+            assert rc == vl.VL_OK, rc
+
+        for _ in range(3):
+            occupied()
+        eo = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        eo[0].record(stream)
+        for _ in range(args.steps):
+            occupied()
+        eo[1].record(stream)
+        torch.cuda.synchronize()
+        occupied_us = eo[0].elapsed_time(eo[1]) / args.steps * 1e3
         diagnose_us = ed[0].elapsed_time(ed[1]) / args.steps * 1e3
         resample_us = er[0].elapsed_time(er[1]) / args.steps * 1e3
         until_ms = er[2].elapsed_time(er[3]) / args.steps
@@ -156,6 +172,7 @@ def main() -> int:
             "until_pass_batch100_ms": until_ms, "until_pass_rows_checked": rows_done,
             "until_pass_first_passing_row": first_pass,
             "diagnose_one_row_us": diagnose_us,
+            "occupied_masks_one_row_us": occupied_us,
         }), flush=True)
         for gp in gps:
             gp.close()
