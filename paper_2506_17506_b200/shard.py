@@ -2,7 +2,8 @@
 
 Candidates are independent (Section 3.4 checks each sampled allocation on its own), so the rows are
 split across ranks and no data-path collective is needed: the only exchanges are the reductions of
-the timing (max over ranks) and of the counts (sum over ranks) that a report needs.
+the timing (max over ranks), of the counts (sum over ranks) that a report needs, and of the first
+passing row of the re-sampling statistics (min over ranks).
 Nothing here computes any part of the check.
 """
 from __future__ import annotations
@@ -47,6 +48,24 @@ def job_totals(rows_local: int, ms_local: float, passing_local: int = 0,
     dist.all_reduce(s, op=dist.ReduceOp.SUM)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return int(s[0].item()), float(t[0].item()), int(s[1].item())
+
+
+def job_sample_stats(first_pass_local: int, n_pass_local: int, rows_local: int, row_offset: int, rows_total: int,
+                     device: Optional[torch.device] = None) -> Tuple[int, int]:
+    """(first passing row of the whole job, passing rows of the whole job) from every rank's record of
+    its own shard (as vl_resample_stats wrote it: first_pass_local == rows_local when the shard has no
+    passing row).  row_offset is the job row of the shard's row 0.  The job's first passing row is the
+    minimum over ranks of offset + local first (rows_total if no shard has one): one MIN and one SUM
+    all-reduce of a single number each.  Identity without a process group."""
+    first = row_offset + first_pass_local if first_pass_local < rows_local else rows_total
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return int(first), int(n_pass_local)
+    dev = device if device is not None else torch.device("cpu")
+    f = torch.tensor([first], dtype=torch.int64, device=dev)
+    n = torch.tensor([n_pass_local], dtype=torch.int64, device=dev)
+    dist.all_reduce(f, op=dist.ReduceOp.MIN)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return int(f.item()), int(n.item())
 
 
 def throughput(rows_total: int, ms: float) -> float:

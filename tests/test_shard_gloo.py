@@ -57,8 +57,14 @@ def _rank_main(rank, world, port, n_rows, tmpdir):
         np.save(os.path.join(tmpdir, f"v{rank}.npy"), v)
         passing = int((v["flags"] == 1).sum())
         total, ms, npass = shard.job_totals(hi - lo, 10.0 * (rank + 1), passing)
+        st = oracle.sample_stats(v)
+        first, n_all = shard.job_sample_stats(int(st["first_pass"]), int(st["n_pass"]), hi - lo, lo, n_rows)
+        # a job in which only the last rank has passing rows, and one in which nobody has
+        late = shard.job_sample_stats(3 if rank == world - 1 else hi - lo, 1 if rank == world - 1 else 0, hi - lo, lo, n_rows)
+        none = shard.job_sample_stats(hi - lo, 0, hi - lo, lo, n_rows)
         if rank == 0:
             np.save(os.path.join(tmpdir, "totals.npy"), np.array([total, ms, npass], dtype=np.float64))
+            np.save(os.path.join(tmpdir, "stats.npy"), np.array([first, n_all, *late, *none], dtype=np.int64))
     finally:
         dist.destroy_process_group()
 
@@ -76,3 +82,13 @@ def test_two_ranks_cover_the_job(tmp_path, oracle_mod):
     total, ms, npass = np.load(tmp_path / "totals.npy")
     assert total == n_rows and ms == 20.0 and npass == int((want["flags"] == 1).sum())
     assert 0 < npass < n_rows
+    first, n_all, late_first, late_n, none_first, none_n = np.load(tmp_path / "stats.npy")
+    st = oracle_mod.sample_stats(want)
+    assert (first, n_all) == (int(st["first_pass"]), int(st["n_pass"]))
+    last_lo = shard.row_range(world - 1, world, n_rows)[0]
+    assert (late_first, late_n) == (last_lo + 3, 1) and (none_first, none_n) == (n_rows, 0)
+
+
+def test_job_sample_stats_single_process():
+    assert shard.job_sample_stats(5, 2, 10, 100, 1000) == (105, 2)
+    assert shard.job_sample_stats(10, 0, 10, 100, 1000) == (1000, 0)
