@@ -126,3 +126,25 @@ def test_occupied_masks_attention_workload(B, oracle_mod):
         assert np.array_equal(got, want)
         assert want.sum() > 100_000                                  # hundreds of registers busy at most points
     gp.close()
+
+
+def test_stress_program_rows(B, oracle_mod):
+    """The largest program (32,000 instructions, 10,000 vregs, P = 512): a valid and a faulted row through
+    both calls, element by element against the oracle."""
+    wl = synth.workload(4)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    rows, faults = synth.candidate_rows(p, wl.K, 0.5, wl.seeds[0], 0, 8)
+    gp = B.Program(p)
+    gp.vl_liveness()
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    kinds_seen = set()
+    for k in range(8):
+        if int(faults[k, 0]) in kinds_seen:
+            continue
+        kinds_seen.add(int(faults[k, 0]))
+        _check_row(B, gp, op, lv, p, rows[k])
+        got = gp.vl_occupied_masks(_to_dev(rows[k][None, :])[0], p.P)
+        assert np.array_equal(got, op.occupied(lv, rows[k]))
+    assert len(kinds_seen) >= 2
+    gp.close()
