@@ -262,7 +262,7 @@ int vl_verify_until_pass(vl_program *prog, const uint16_t *d_cand, uint64_t K, u
  * equals the verdict's conflict_pairs); unless NULL, d_kinds[i] (DEVICE, n_instrs bytes) receives the OR
  * of the violation bits raised at instruction i (the lowest i with a bit is first_violation_instr) and
  * d_bank_hist[b] (DEVICE, B counters) the extra read cycles charged to bank b (their sum is
- * bank_conflicts).  Rules set with vl_program_set_constraints apply.  Not a hot path: one thread per
+ * bank_conflicts).  Rules set with vl_program_set_constraints apply.  Not a hot path: one warp per
  * instruction over the live-after lists.  Stream-ordered, no synchronisation; the first call allocates
  * 8 * n_vregs bytes in the handle.  Errors: INVALID_ARG, LIVENESS_NOT_RUN, CUDA.
  */

@@ -5,7 +5,7 @@
 // as a training signal): every (instruction, defined vreg, other vreg) overlap, the violation kinds
 // raised at every instruction, and the extra read cycles per register bank.
 //
-// This is not the hot path: one row, one thread per instruction, the per-instruction live-after
+// This is not the hot path: one row, one warp per instruction, the per-instruction live-after
 // lists of vl_liveness read as they are.  The numbers agree with the verdict of vl_verify for the
 // same row: the overlap count is conflict_pairs, the histogram sums to bank_conflicts, the lowest
 // instruction with a kind is first_violation_instr.
@@ -48,9 +48,12 @@ __device__ __forceinline__ bool overlap(uint32_t a, uint32_t wa, uint32_t b, uin
     return a < b + wb && b < a + wa;
 }
 
-__global__ void k_diag_instr(const DParams q)
+// one warp per instruction: the lanes share out the operands and the live-after list
+constexpr uint32_t DIAG_WARPS = 4;
+__global__ void __launch_bounds__(DIAG_WARPS * 32) k_diag_instr(const DParams q)
 {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t i = blockIdx.x * DIAG_WARPS + (threadIdx.x >> 5);
     if (i >= q.nI) return;
     const uint32_t o0 = q.op_off[i], o1 = q.op_off[i + 1], nd = q.ndefs[i];
     const uint32_t l0 = q.lo_off[i], l1 = q.lo_off[i + 1];
@@ -60,23 +63,25 @@ __global__ void k_diag_instr(const DParams q)
         if (k < q.cap) q.conflicts[k] = vl_conflict{i, v, u};
     };
     uint32_t kinds = 0;
-    for (uint32_t o = o0; o < o1; ++o)
+    for (uint32_t o = o0 + lane; o < o1; o += 32)
         if (q.row[o] != T(q.op_vreg[o])) kinds |= VL_INCONSISTENT;
     for (uint32_t d = o0; d < o0 + nd; ++d) {
         const uint32_t v = q.op_vreg[d], s = T(v), w = q.width[v];
-        bool unreal = s + w > q.P;
-        if (q.vcons) {
-            const uint4 vc = q.vcons[v];
-            const uint32_t clo = vc.x & 0xFFFFu, chi = vc.x >> 16, al = vc.y;
-            unreal = unreal || (al > 1 && s != __umulhi(s, vc.z) * al) || s < clo || s + w > chi;
-            if (q.rs_prefix) unreal = unreal || q.rs_prefix[min(s + w, q.P)] != q.rs_prefix[min(s, q.P)];
+        if (lane == 0) {
+            bool unreal = s + w > q.P;
+            if (q.vcons) {
+                const uint4 vc = q.vcons[v];
+                const uint32_t clo = vc.x & 0xFFFFu, chi = vc.x >> 16, al = vc.y;
+                unreal = unreal || (al > 1 && s != __umulhi(s, vc.z) * al) || s < clo || s + w > chi;
+                if (q.rs_prefix) unreal = unreal || q.rs_prefix[min(s + w, q.P)] != q.rs_prefix[min(s, q.P)];
+            }
+            if (unreal) kinds |= VL_OUT_OF_RANGE;
         }
-        if (unreal) kinds |= VL_OUT_OF_RANGE;
-        for (uint32_t e = l0; e < l1; ++e) {  // vregs live after the instruction
+        for (uint32_t e = l0 + lane; e < l1; e += 32) {  // vregs live after the instruction
             const uint32_t u = q.lo[e];
             if (u != v && overlap(s, w, T(u), q.width[u])) { emit(v, u); kinds |= VL_INTERFERENCE; }
         }
-        for (uint32_t d2 = o0; d2 < o0 + nd; ++d2) {  // vregs it also defines that are dead afterwards
+        for (uint32_t d2 = o0 + lane; d2 < o0 + nd; d2 += 32) {  // vregs it also defines that are dead afterwards
             const uint32_t u = q.op_vreg[d2];
             if (u == v) continue;
             uint32_t a = l0, b = l1;  // the list is ascending
@@ -88,11 +93,12 @@ __global__ void k_diag_instr(const DParams q)
             if (overlap(s, w, T(u), q.width[u])) { emit(v, u); kinds |= VL_INTERFERENCE; }
         }
     }
-    if (q.kinds) q.kinds[i] = (uint8_t)kinds;
+    kinds = __reduce_or_sync(0xffffffffu, kinds);
+    if (q.kinds && lane == 0) q.kinds[i] = (uint8_t)kinds;
     if (q.bank_hist) {
         // a read costs a cycle if an earlier read of this instruction uses another register of its bank
         // and no earlier read uses the same register
-        for (uint32_t a = o0 + nd; a < o1; ++a) {
+        for (uint32_t a = o0 + nd + lane; a < o1; a += 32) {
             const uint32_t ta = T(q.op_vreg[a]);
             bool dup = false, shared = false;
             for (uint32_t b = o0 + nd; b < a; ++b) {
@@ -196,7 +202,7 @@ extern "C" int vl_diagnose(vl_program *p, const uint16_t *d_row, uint64_t cap, v
     const uint32_t n0 = p->V > p->B ? p->V : p->B;
     k_diag_init<<<(n0 + 255) / 256 + 1, 256, 0, st>>>(q);
     if (p->nO) k_diag_table<<<(p->nO + 255) / 256, 256, 0, st>>>(q);
-    if (p->nI) k_diag_instr<<<(p->nI + 127) / 128, 128, 0, st>>>(q);
+    if (p->nI) k_diag_instr<<<(p->nI + DIAG_WARPS - 1) / DIAG_WARPS, DIAG_WARPS * 32, 0, st>>>(q);
     g_vl_launches.fetch_add(1 + (p->nO ? 1 : 0) + (p->nI ? 1 : 0));
     VL_CUDA(p, cudaGetLastError());
     return VL_OK;
