@@ -149,7 +149,7 @@ struct vl_program {
         uint32_t *work = nullptr;    // [1 + rows] count, then candidates that need the exact recount
         uint32_t *racc = nullptr;    // [rows][4] recount accumulators: pairs, lowest instruction, bank tally, slices done
         uint32_t *grp_done = nullptr;  // [rows / 32] walk thread blocks that have finished, per group of 32 candidates
-        uint64_t rows = 0, aw = 0, vregs = 0;
+        uint64_t rows = 0, aw = 0, vregs = 0, chunks = 0;
     } vs[VL_LANES + 2];              // one per lane, then one per staging buffer of vl_verify_host
     uint32_t sub_batch = 4096;       // candidates per pass of the verify kernels
     uint32_t lanes_opt = 3;          // lanes in use (1 = everything in order on the caller's stream)

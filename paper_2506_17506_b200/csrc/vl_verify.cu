@@ -1278,12 +1278,20 @@ cudaError_t launch_tables(const TParams &q, uint32_t grid, uint32_t smem, cudaSt
     return cudaGetLastError();
 }
 
+// Most work items one candidate can list for the recount: every chunk in RC_PARTS pieces, the bank
+// tally in RC_BANK_PARTS slices, one item per block whose through-set collided (through-sets are
+// used only by programs of at most 32 blocks).
+uint64_t rc_items_per_row(const vl_program *p)
+{
+    return (uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS + std::min<uint32_t>(p->nB, 32u);
+}
+
 int ensure_scratch(vl_program *p, int slot, uint64_t rows)
 {
     vl_program::VScratch &v = p->vs[slot];
     const uint64_t aw = std::max(1u, (p->nC + 31) / 32);
     const uint64_t groups = (rows + 31) / 32;
-    if (v.rows >= rows && v.aw == aw && v.vregs == p->V) return VL_OK;
+    if (v.rows >= rows && v.aw == aw && v.vregs == p->V && v.chunks == p->nC) return VL_OK;
     cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done);
     v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr; v.grp_done = nullptr;
     v.rows = 0;
@@ -1293,13 +1301,13 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.work,
-                          (2 + 2 * groups * 32 * ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * 32 * rc_items_per_row(p)) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.grp_done, (groups + 1) * sizeof(uint32_t)));
     v.rows = groups * 32;
     v.aw = aw;
     v.vregs = p->V;
+    v.chunks = p->nC;
     return VL_OK;
 }
 }  // namespace
@@ -1350,9 +1358,8 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     // the walk's table entries keep bit 15 for a mark: every in-file register number must be below 2^15
     // (the occupancy masks of a register file that large would not fit shared memory anyway)
     if (p->P + p->wmax > 32768u) return VL_ERR_UNSUPPORTED;
-    // the recount work list holds up to RC_PARTS items per chunk and candidate: keep it within 8 Mi items
-    const uint64_t sub_cap =
-        std::max<uint64_t>(32, ((8ull << 20) / ((uint64_t)RC_PARTS * p->nC + RC_BANK_PARTS)) / 32 * 32);
+    // the recount work list holds up to rc_items_per_row items per candidate: keep it within 8 Mi items
+    const uint64_t sub_cap = std::max<uint64_t>(32, ((8ull << 20) / rc_items_per_row(p)) / 32 * 32);
     pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
     // once per device: every verify kernel may use the whole shared memory of an SM
     static std::mutex attr_mutex;

@@ -217,27 +217,45 @@ def test_passes_over_lanes(B, oracle_mod, lanes, sub):
     gp.close()
 
 
+def _oracle_rows_threaded(oracle_mod, p, lv, rows):
+    """Oracle verdicts of every row, the rows split over the host's threads (the oracle itself stays
+    single-threaded; ctypes releases the interpreter lock during a call)."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    op = oracle_mod.OracleProgram(p)
+    threads = max(1, min(os.cpu_count() or 1, 32, len(rows)))
+    bounds = np.linspace(0, len(rows), threads + 1).astype(int)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        outs = list(ex.map(lambda j: op.verify(lv, rows[bounds[j]:bounds[j + 1]]), range(threads)))
+    return np.concatenate(outs)
+
+
 def test_batch_call(B, oracle_mod):
-    """Workload 4 (256 independent programs): a sample of members through vl_verify_batch."""
+    """Workload 4 in full: all 256 independent programs through vl_liveness_batch and vl_verify_batch,
+    every row of every program against the oracle."""
     import torch
     wl = synth.workload(3)
-    members = [0, 1, 2, 3, 100, 255]
+    members = list(range(len(wl.shapes)))
+    assert len(members) == 256
     progs, gps, cands, wants = [], [], [], []
     for j in members:
         p = synth.build_program(wl.shapes[j], wl.seeds[j])
-        gp, lv = _check_liveness(B, oracle_mod, p)
         rows, _ = synth.candidate_rows(p, wl.K, wl.fault_rate, wl.seeds[j])
-        progs.append(p); gps.append(gp); cands.append(_to_dev(rows))
+        lv = oracle_mod.OracleProgram(p).liveness()
+        progs.append(p); gps.append(B.Program(p)); cands.append(_to_dev(rows))
         wants.append(oracle_mod.OracleProgram(p).verify(lv, rows))
+    B.vl_liveness_batch(gps)
     outs = B.vl_verify_batch(gps, cands)
     torch.cuda.synchronize()
     for j, o, w in zip(members, outs, wants):
         _assert_same(B.verdicts_to_numpy(o), w, f"batch member {j}")
+    for gp, p in zip(gps, progs):
+        _check_liveness_result(B, oracle_mod, gp, p)
     # liveness of all members in one call, several times (the later runs are replayed recordings):
     # same liveness results, same verdicts
     for _ in range(4):
         B.vl_liveness_batch(gps)
-    for gp, p in zip(gps, progs):
+    for gp, p in zip(gps[::16], progs[::16]):
         _check_liveness_result(B, oracle_mod, gp, p)
     outs = B.vl_verify_batch(gps, cands)
     torch.cuda.synchronize()
@@ -247,12 +265,11 @@ def test_batch_call(B, oracle_mod):
         gp.close()
 
 
-def test_stress_workload_sampled(B, oracle_mod):
+def test_stress_workload_full(B, oracle_mod):
     """Workload 5 at full size, in the launch configuration the benchmark times (all 10,000 rows in
-    one call: three passes spread over the internal streams): liveness compared in full; verdicts
-    compared with the oracle on every faulted row and on every 40th row (each oracle row costs
-    ~10 ms), and on every row through what holds by construction (a row passes iff no fault was
-    injected; the host-buffer entry point gives the same records)."""
+    one call, its passes spread over the internal streams): liveness compared in full, every one of
+    the 10,000 verdicts compared with the oracle's, and besides that what holds by construction (a
+    row passes iff no fault was injected; the host-buffer entry point gives the same records)."""
     wl = synth.workload(4)
     p = synth.build_program(wl.shapes[0], wl.seeds[0])
     gp, lv = _check_liveness(B, oracle_mod, p)
@@ -260,15 +277,36 @@ def test_stress_workload_sampled(B, oracle_mod):
     rows = np.empty((K, p.pitch), dtype=np.uint16)
     _, faults = synth.candidate_rows(p, K, wl.fault_rate, wl.seeds[0], 0, K, out=rows, chunk=256)
     got = _gpu_verify(B, gp, rows)
+    want = _oracle_rows_threaded(oracle_mod, p, lv, rows)
+    _assert_same(got, want, "stress")
     assert np.array_equal(got["flags"] == B.VL_PASS, faults[:, 0] == 0)     # valid by construction / injected
     assert np.all(got["conflict_pairs"][faults[:, 0] == 0] == 0)
-    sample = sorted(set(np.nonzero(faults[:, 0] != 0)[0].tolist()) | set(range(0, K, 40)))
-    want = oracle_mod.OracleProgram(p).verify(lv, rows[sample])
-    _assert_same(got[sample], want, "stress")
     host = gp.vl_verify_host(rows[:1500])
     assert host.tobytes() == got[:1500].tobytes()
     garbage = _garbage_rows(p, 6, 9)
     _assert_same(_gpu_verify(B, gp, garbage), oracle_mod.OracleProgram(p).verify(lv, garbage), "stress garbage")
+    gp.close()
+
+
+def test_recount_work_list_full(B, oracle_mod):
+    """Passes in which every candidate collides in nearly every chunk and through-set: the work list
+    of the exact recount is as long as it gets (all-zero rows and uniform noise on the GEMM-shaped
+    program, which has through-sets; 32 rows per pass)."""
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    rng = np.random.default_rng(42)
+    rows = np.zeros((128, p.pitch), dtype=np.uint16)
+    rows[64:, : p.n_operands] = rng.integers(0, p.P, size=(64, p.n_operands))
+    for k in range(96, 128):                              # consistent random tables: every chunk collides
+        rows[k] = H.row_from_table(p, rng.integers(0, p.P, size=p.n_vregs))
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    for sub, chunk in ((32, 0), (64, 24), (32, 150)):
+        gp.set_option(B.VL_OPT_SUB_BATCH, sub)
+        if chunk:
+            gp.set_option(B.VL_OPT_CHUNK_INSTRS, chunk)
+            gp.vl_liveness()
+        _assert_same(_gpu_verify(B, gp, rows), want, f"sub {sub} chunk {chunk}")
     gp.close()
 
 
