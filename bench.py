@@ -181,6 +181,8 @@ def main():
     ap.add_argument("--lanes", type=int, default=0, help="internal streams of vl_verify (default: the library's)")
     ap.add_argument("--sub-batch", type=int, default=0, help="candidates per pass (default: the library's)")
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--threads", type=int, default=0, help="threads per block of the table kernel (default: the library's)")
+    ap.add_argument("--prefetch", type=int, default=-1, help="tiles the table kernel asks into L2 ahead (default: the library's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--fault-rate", type=float, default=-1.0, help="override the workload's faulted fraction")
     args = ap.parse_args()
@@ -208,6 +210,10 @@ def main():
         gp.set_option(vl.VL_OPT_LANES, args.lanes)
     if args.sub_batch:
         gp.set_option(vl.VL_OPT_SUB_BATCH, args.sub_batch)
+    if args.threads:
+        gp.set_option(vl.VL_OPT_THREADS, args.threads)
+    if args.prefetch >= 0:
+        gp.set_option(vl.VL_OPT_PREFETCH_TILES, args.prefetch)
     dev_rows = host.cuda().view(torch.uint16)
     out = torch.empty((K, 4), dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()

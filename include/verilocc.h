@@ -44,14 +44,20 @@ enum { VL_PASS = 1u, VL_INCONSISTENT = 2u, VL_OUT_OF_RANGE = 4u, VL_INTERFERENCE
 /* Tunables for vl_program_set_option (set before vl_liveness). */
 enum {
     VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 160; long blocks get a chunk count that is a multiple of 8) */
-    VL_OPT_GROUP = 2,        /* candidates per thread block: 0 = choose, else 1, 2 or 4 */
+    VL_OPT_GROUP = 2,        /* candidates per thread block of the table kernel: 0 = choose, else 1, 2, 4 or 8 */
     VL_OPT_THREADS = 3,      /* threads per thread block of the table kernel: 0 = choose, else 256 or 512 */
     VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
     VL_OPT_KERNEL_TIMING = 5,/* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
                                 set at any time; setting it discards the events recorded so far */
-    VL_OPT_LANES = 6         /* internal streams the passes of vl_verify are spread over, 1..8 (default 3);
+    VL_OPT_LANES = 6,        /* internal streams the passes of vl_verify are spread over, 1..8 (default 3);
                                 1 = every kernel in order on the caller's stream.  vl_verify_batch reads the
                                 option of its first program: 1 = in order, anything else = all 8 streams */
+    VL_OPT_PREFETCH_TILES = 8, /* tiles of the candidate rows that the table kernel (8 candidates per block) asks into
+                                L2 ahead of its copy ring, 0..64 (default 6; 0 = none) */
+    VL_OPT_TEST_WAIT = 7     /* test hook for the bounded device waits: 1 = the table kernel (8 candidates per
+                                block) waits for its first tile on a barrier that nothing completes, with a short
+                                poll limit, so that the wait runs out: the call still returns, its verdicts are
+                                garbage and vl_verify_status reports VL_ERR_DEVICE_WAIT.  0 = normal (default) */
 };
 
 /*

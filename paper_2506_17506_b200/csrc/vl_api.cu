@@ -94,6 +94,7 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
     p->P = d->P; p->B = d->B;
     p->Wv = std::max(1u, (p->V + 31) / 32);
     p->nOp8 = std::max(8u, (p->nO + 7) / 8 * 8);
+    p->nOpT = (p->nOp8 + 4095u) / 4096u * 4096u;
     p->wmax = 1;
     for (uint32_t v = 0; v < p->V; ++v) p->wmax = std::max<uint32_t>(p->wmax, d->vreg_width[v]);
     p->h_blk_off.assign(d->block_instr_off, d->block_instr_off + p->nB + 1);
@@ -150,7 +151,7 @@ void vl_free_liveness(vl_program *p)
     p->live_arena.reset();
     p->tmp_arena.reset();
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
-    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opflags = nullptr; p->d_iflags = nullptr;
+    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opoff = nullptr; p->d_first4 = nullptr; p->d_opflags = nullptr; p->d_iflags = nullptr;
     p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
@@ -208,7 +209,7 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
         p->live_ok = false;
         return VL_OK;
     case VL_OPT_GROUP:
-        if (value != 0 && value != 1 && value != 2 && value != 4) return VL_ERR_INVALID_ARG;
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return VL_ERR_INVALID_ARG;
         p->group_opt = value;
         return VL_OK;
     case VL_OPT_SUB_BATCH:
@@ -223,6 +224,14 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
     case VL_OPT_LANES:
         if (value < 1 || value > VL_LANES) return VL_ERR_INVALID_ARG;
         p->lanes_opt = value;
+        return VL_OK;
+    case VL_OPT_PREFETCH_TILES:
+        if (value > 64) return VL_ERR_INVALID_ARG;
+        p->prefetch_tiles = value;
+        return VL_OK;
+    case VL_OPT_TEST_WAIT:
+        if (value > 1) return VL_ERR_INVALID_ARG;
+        p->test_wait = value;
         return VL_OK;
     case VL_OPT_THREADS:
         if (value != 0 && value != 256 && value != 512) return VL_ERR_INVALID_ARG;

@@ -31,7 +31,7 @@ enum : uint32_t {
     ST_DEVICE_WAIT = 16u    // a bounded wait in a verify kernel ran out
 };
 
-#define VL_MAX_GROUP 4
+#define VL_MAX_GROUP 8
 #define VL_LANES 8  // internal streams that the passes of device-resident verify calls can be spread over
 
 // Device memory pool of a program handle: slabs are kept across calls, so that a repeated
@@ -72,6 +72,7 @@ struct vl_program {
     uint32_t nB = 0, nI = 0, V = 0, nO = 0, nE = 0, P = 0, B = 0;
     uint32_t Wv = 0;    // 32-bit words per vreg bitset
     uint32_t nOp8 = 0;  // n_operands rounded up to 8 (at least 8)
+    uint32_t nOpT = 0;  // n_operands rounded up to 4096 (whole tiles of the eight-candidate table kernel)
     uint32_t wmax = 1;  // widest vreg
     uint32_t chunk_instrs = 160;
     uint32_t group_opt = 0;
@@ -97,6 +98,8 @@ struct vl_program {
     // tables consumed by the verify kernels
     uint16_t *d_vreg16 = nullptr;           // [nOp8 + 8] vreg id per operand (padding operands: id V)
     uint64_t *d_slotmeta = nullptr;         // [nOp8 / 8] per 8 operands: first-occurrence bits, bank compare masks
+    uint4 *d_opoff = nullptr;               // [nOpT / 4] per 4 operands: byte offsets of their vregs' 16-byte table entries
+    uint8_t *d_first4 = nullptr;            // [nOpT / 4] per 4 operands: first-occurrence bits
     uint8_t *d_opflags = nullptr;           // [nO]
     uint8_t *d_iflags = nullptr;            // [nI] 1 if the instruction has a definition the walk skips
     uint32_t *d_first_def_instr = nullptr;  // [V] lowest instruction defining v, 0xFFFFFFFF if none
@@ -122,6 +125,8 @@ struct vl_program {
     uint2 *d_bank_list = nullptr;   // instructions with 2, 3, 4 distinct sources: their vreg ids, 16 bits each
     uint32_t bank_seg[4] = {0, 0, 0, 0};
     uint32_t threads_opt = 0;
+    uint32_t prefetch_tiles = 6;  // tiles the eight-candidate table kernel asks into L2 ahead of its copy ring
+    uint32_t test_wait = 0;  // test hook of the table kernel's bounded wait (VL_OPT_TEST_WAIT)
     int use_th = 0;
 
     VlArena live_arena, tmp_arena;  // liveness results and tables / liveness working sets

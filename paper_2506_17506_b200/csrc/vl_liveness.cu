@@ -560,6 +560,28 @@ __global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8
     slotmeta[s] = m;
 }
 
+// Operand metadata of the eight-candidate table kernel, per four operands: the byte offsets of the
+// vregs' 16-byte table entries and a nibble of first-occurrence bits.  Operands beyond n_operands
+// (the arrays are padded to whole tiles) name the spare entry V and are never a first occurrence.
+__global__ void k_meta8(uint32_t nO, uint32_t n_quads, uint32_t V, const uint16_t *__restrict__ vreg16,
+                        const uint64_t *__restrict__ slotmeta, uint4 *opoff, uint8_t *first4)
+{
+    const uint32_t qd = blockIdx.x * NT + threadIdx.x;
+    if (qd >= n_quads) return;
+    uint32_t off[4], f = 0;
+    for (uint32_t j = 0; j < 4; ++j) {
+        const uint32_t o = qd * 4 + j;
+        uint32_t v = V;
+        if (o < nO) {
+            v = vreg16[o];
+            if ((slotmeta[o >> 3] >> (o & 7)) & 1ull) f |= 1u << j;
+        }
+        off[j] = v * 16u;
+    }
+    opoff[qd] = make_uint4(off[0], off[1], off[2], off[3]);
+    first4[qd] = (uint8_t)f;
+}
+
 // Walk events are stored in groups of 8, 112 bytes per group, field by field so that the walk
 // fetches a group with 16-byte loads: off[8] (32 bit: byte offset of the vreg's row in a table of
 // 32 16-bit entries per vreg), toggle[8] (32 bit: the width-w mask (1<<w)-1, or 0), test[8]
@@ -777,6 +799,8 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     KEEP(&p->d_first_def_instr, (size_t)V);
     KEEP(&p->d_vreg16, (size_t)p->nOp8 + 8);
     KEEP(&p->d_slotmeta, (size_t)p->nOp8 / 8);
+    KEEP(&p->d_opoff, (size_t)p->nOpT / 4);
+    KEEP(&p->d_first4, (size_t)p->nOpT / 4);
     KEEP(&p->d_vinfo, (size_t)V);
     KEEP(&p->d_iflags, (size_t)nI);
     KEEP(&p->d_cev_off, (size_t)nC + 1);
@@ -874,10 +898,10 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
 
     KEEP(&p->d_lo, (size_t)p->lo_len);
     KEEP(&p->d_ls, (size_t)p->known_ls_len);
-    KEEP(&p->d_ev, (size_t)(steps / 8) * 7);
+    KEEP(&p->d_ev, (size_t)(steps / 8 + 2) * 7);  // two no-op groups behind the last chunk: the walk reads ahead
     KEEP(&p->d_th, (size_t)p->known_thn);
-    LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT), 0, st, p->d_ev, (size_t)(steps / 8),
-           V);  // every slot starts as a no-op event
+    LAUNCH(k_fill_noop, (uint32_t)std::min<uint64_t>(1024, (steps + NT - 1) / NT + 1), 0, st, p->d_ev,
+           (size_t)(steps / 8 + 2), V);  // every slot starts as a no-op event
 
     // The list fill, the operand tables and the walk events do not depend on each other: the latter
     // two run on side streams beside the fill (as parallel branches when the run is recorded).
@@ -900,6 +924,8 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_opflags, p->d_vreg16, opmeta, p->d_status);
     LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
+    LAUNCH(k_meta8, (p->nOpT / 4 + NT - 1) / NT, 0, sa, nO, p->nOpT / 4, V, p->d_vreg16, p->d_slotmeta, p->d_opoff,
+           p->d_first4);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     LAUNCH(k_fill_events, nC, 0, sb, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
            p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev, p->d_chunk_blk, p->d_el,

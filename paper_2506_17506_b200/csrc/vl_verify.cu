@@ -15,7 +15,10 @@
 //            candidates and lists the others for the recount.
 // k_recount  candidates with a collision are recounted exactly from the per-instruction live-after
 //            lists, one thread block per piece of a colliding chunk.
+#include <cuda.h>
+
 #include <algorithm>
+#include <cstring>
 #include <mutex>
 
 #include "vl_internal.cuh"
@@ -51,13 +54,28 @@ struct TParams {
     // the number of reserved registers below every register
     const uint4 *vcons;
     const uint16_t *rs_prefix;
+    // the eight-candidate kernel: per 4 operands the byte offsets of their vregs' table entries and
+    // their first-occurrence bits
+    const uint4 *opoff;
+    const uint8_t *first4;
+    uint32_t *grp_flag;   // per group of 32 candidates: some table entry carries the straddle mark
+    uint32_t test_wait;   // test hook: the wait for tile 0 polls a barrier nothing completes, with a short limit
+    uint32_t pf;          // tiles asked into L2 ahead of the copy ring
+    // the rows as a 3-D tensor [candidate][chunk of 256 operands][256]: nfull whole chunks per row; the
+    // operands from tail_start on (fewer than 256) come by plain bulk copies into a buffer of their own
+    uint32_t nfull, tail_start, tail_tile, off_tail;
 };
 
 struct TMisc {
     unsigned long long bar[MAX_STAGES];
+    unsigned long long bar_never;  // initialised, never completed: what the test hook waits on
+    unsigned long long bar_tail;   // the operands behind the last whole chunk of 256
+    unsigned long long empty[MAX_STAGES];  // k_tables8: every consumer warp has read the stage
+    unsigned long long stored[2];          // k_tables8: every consumer warp has stored its first occurrences of a tile (by tile parity)
     uint32_t flags[VL_MAX_GROUP], minop[VL_MAX_GROUP], minR[VL_MAX_GROUP], bank[VL_MAX_GROUP];
     uint32_t nout[VL_MAX_GROUP], out_v[VL_MAX_GROUP], out_raw[VL_MAX_GROUP];
     uint32_t abort_flag;
+    uint32_t marks;  // bit g: a table entry of candidate g carries the straddle mark
 };
 
 struct WParams {
@@ -68,6 +86,7 @@ struct WParams {
     const uint16_t *tg, *tg_zero;
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
+    uint32_t *grp_flag;  // per group: set by the table kernel when a walked candidate has a marked entry
     // hand-over to k_recount by the last thread block of each group of 32 candidates
     int list_all;
     const uint32_t *chunk_blk;
@@ -140,6 +159,25 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                      smem_u32(dst)),
                  "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Tiled copy of one box of a 3-D tensor (coordinates innermost first) into this block's shared memory,
+// completion counted on `bar` with the full size of the box (elements outside the tensor arrive as
+// zeros).  dst 128-byte aligned; the innermost coordinate times the element size a multiple of 16.
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tm, uint32_t x, uint32_t y, uint32_t z,
+                                            unsigned long long *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            smem_u32(dst)),
+        "l"(tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        : "memory");
+}
+// Asks for one box of the tensor to be brought into L2.
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *tm, uint32_t x, uint32_t y, uint32_t z)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
 
@@ -548,6 +586,476 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         cs[CS_WALK] = M->nout[g] >= 2 ? WALK_FULL : 0u;
         cs[CS_THCOL] = 0;
     }
+    // this kernel does not keep track of marked entries: its groups take the walk's checking path
+    if (tid == 0) atomicOr(&q.grp_flag[k0 >> 5], 1u);
+}
+
+// =========================================================================== k_tables8
+// The table kernel with eight candidates per thread block: a table entry is 16 bytes (the eight
+// candidates' registers of one vreg), so that one shared-memory load serves eight operand checks.
+// A thread takes 4 operands x 8 candidates per tile (one 8-byte load per row from the copy ring),
+// transposes them with byte permutes, stores first occurrences, and compares the occurrences of the
+// tile before (whose first occurrences a barrier has already ordered) while the current tile's loads
+// are in flight: one barrier per tile, no dependent wait behind it.
+__device__ __forceinline__ uint32_t pk8_get(const uint4 &x, int g)
+{
+    const uint32_t w = (g >> 1) == 0 ? x.x : ((g >> 1) == 1 ? x.y : ((g >> 1) == 2 ? x.z : x.w));
+    return (g & 1) ? (w >> 16) : (w & 0xFFFFu);
+}
+
+template <int NT>
+__device__ __noinline__ void rules_sweep8(const uint4 *vcons, const uint16_t *rs_prefix, const uint32_t *vinfo,
+                                          const uint32_t *first_def_instr, uint32_t V, uint32_t P, const uint4 *T,
+                                          TMisc *M)
+{
+    for (uint32_t v = threadIdx.x; v < V; v += NT) {
+        const uint32_t vi = vinfo[v];
+        if (!(vi & VINFO_DEFINED)) continue;
+        const uint4 vc = vcons[v];
+        const uint32_t clo = vc.x & 0xFFFFu, chi = vc.x >> 16, al = vc.y, recip = vc.z, w = vi & 0xFFu;
+        const uint4 tt = T[v];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const uint32_t tv = pk8_get(tt, g);
+            bool bad = (al > 1 && tv != __umulhi(tv, recip) * al) || tv < clo || tv + w > chi;
+            if (!bad && rs_prefix) bad = rs_prefix[min(tv + w, P)] != rs_prefix[min(tv, P)];
+            if (bad) {
+                atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
+                atomicMin(&M->minR[g], first_def_instr[v]);
+            }
+        }
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const __grid_constant__ CUtensorMap tm)
+{
+    constexpr int G = 8;
+    constexpr uint32_t TILE = NT * 4;  // operands per tile and candidate
+    constexpr uint32_t ROW_BYTES = TILE * 2, STAGE_BYTES = ROW_BYTES * G;
+    constexpr uint32_t CH = TILE / 256;      // chunks of 256 operands per tile
+    constexpr uint32_t TAIL_ROW_BYTES = 512;
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint4 *T = reinterpret_cast<uint4 *>(smem);  // [V + 1]
+    unsigned char *region = smem + q.off_region;
+    uint32_t *Hb = reinterpret_cast<uint32_t *>(region);  // [V] after the rows have been streamed: bank nibbles
+    unsigned char *tailbuf = smem + q.off_tail;           // [G][TAIL_ROW_BYTES]
+    TMisc *M = reinterpret_cast<TMisc *>(smem + q.off_misc);
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    const uint64_t k0 = (uint64_t)blockIdx.x * G;
+    const uint16_t *rows[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) rows[g] = q.cand + min(k0 + g, q.K - 1) * q.pitch;
+
+    if (tid < G) {
+        M->flags[tid] = 0; M->minop[tid] = 0xFFFFFFFFu; M->minR[tid] = 0xFFFFFFFFu; M->bank[tid] = 0;
+        M->nout[tid] = 0; M->out_v[tid] = 0; M->out_raw[tid] = 0;
+    }
+    if (tid == 0) {
+        M->abort_flag = 0;
+        M->marks = 0;
+        for (uint32_t s = 0; s < q.NS; ++s) { mbar_init(&M->bar[s], 1); mbar_init(&M->empty[s], NT / 32); }
+        mbar_init(&M->stored[0], NT / 32);
+        mbar_init(&M->stored[1], NT / 32);
+        mbar_init(&M->bar_never, 1);
+        mbar_init(&M->bar_tail, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        T[q.V] = make_uint4(0, 0, 0, 0);  // the spare entry: what padding operands are compared with
+    }
+    // state of this pass that the walk and the recount update with atomics starts at zero
+    for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
+    if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
+    if (tid == 0 && (k0 & 31) == 0) q.grp_done[k0 >> 5] = 0;
+    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
+    __syncthreads();
+
+    // A tile is one box of the row tensor: 8 candidates x CH chunks x 256 operands, one copy.  (Boxes
+    // that reach past the last whole chunk, or past the last candidate, are filled up with zeros.)
+    // Warp NT/32 is the producer: it refills a stage of the ring as soon as every consumer warp has
+    // read it.  The consumer warps are not held together by a block barrier per tile; what orders
+    // them is one counting barrier per tile parity, "the first occurrences of tile t are stored",
+    // on which a warp arrives after its stores and waits one tile later, before it compares tile t.
+    auto wait_bar = [&](unsigned long long *bar, uint32_t parity) {
+        // Bounded wait.  When it runs out the block raises the status bit and carries on with short
+        // waits (its results are garbage, every index still in bounds); the producer issues no
+        // further copies and, before the block returns, waits again for the copies it did issue.
+        uint32_t spins = 0;
+        const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 20);
+        while (!mbar_try_wait(bar, parity)) {
+            if (++spins > limit) {
+                M->abort_flag = 1;
+                atomicOr(q.status, ST_DEVICE_WAIT);
+                break;
+            }
+        }
+    };
+    if (tid >= NT) {  // ------------------------------------------------------------ producer warp
+        if (lane == 0) {
+            const uint32_t tail_bytes = (q.nOp8 - q.tail_start) * 2;
+            if (tail_bytes) {
+                mbar_expect_tx(&M->bar_tail, tail_bytes * G);
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    bulk_g2s(tailbuf + g * TAIL_ROW_BYTES, rows[g] + q.tail_start, tail_bytes, &M->bar_tail);
+            }
+            uint32_t issued = 0;  // tiles issued so far, in order
+            uint32_t stage = 0, parity = 0;
+            for (uint32_t t = 0; t < q.ntiles; ++t) {
+                if (t >= q.NS) {  // the stage still holds tile t - NS: wait until the 16 warps have read it
+                    wait_bar(&M->empty[stage], parity ^ 1u);
+                    if (*(volatile uint32_t *)&M->abort_flag) break;
+                }
+                issued = t + 1;
+                if (t * CH < q.nfull) {  // (a tile of nothing but tail operands has no box)
+                    mbar_expect_tx(&M->bar[stage], STAGE_BYTES);
+                    tma_load_3d(region + (size_t)stage * STAGE_BYTES, &tm, 0, t * CH, (uint32_t)k0, &M->bar[stage]);
+                }
+                // The ring holds too few bytes to cover the latency of HBM by itself: the tiles further
+                // ahead are asked into L2, so that the ring's copies come from there.
+                if (q.pf && (t + q.pf) * CH < q.nfull) tma_prefetch_3d(&tm, 0, (t + q.pf) * CH, (uint32_t)k0);
+                if (++stage == q.NS) { stage = 0; parity ^= 1; }
+            }
+            if (*(volatile uint32_t *)&M->abort_flag) {
+                // a wait ran out: give the copies that were issued their time before the block (and its
+                // shared memory) goes away
+                for (uint32_t s = 0; s < q.NS; ++s) {
+                    if (issued <= s) continue;
+                    uint32_t t_last = s + (issued - 1 - s) / q.NS * q.NS;  // the last tile issued into stage s
+                    if (t_last * CH >= q.nfull) {
+                        if (t_last < q.NS) continue;
+                        t_last -= q.NS;
+                    }
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&M->bar[s], (t_last / q.NS) & 1u) && ++spins < (1u << 20)) {}
+                }
+                if (tail_bytes) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&M->bar_tail, 0) && ++spins < (1u << 20)) {}
+                }
+            }
+        }
+    } else {  // ---------------------------------------------------------------------- consumer warps
+        const uint32_t spare_off = q.V * 16u;
+        const uint4 *opoff = q.opoff + tid;
+        const uint8_t *first4 = q.first4 + tid;
+        // every occurrence of a tile against the table (a first occurrence trivially matches; padding
+        // operands were zeroed and name the all-zero spare entry)
+        auto compare = [&](const uint4 (&pc)[4], const uint4 &off, uint32_t o_base) {
+            const uint32_t of[4] = {off.x, off.y, off.z, off.w};
+            uint4 x[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[j] = *reinterpret_cast<const uint4 *>(smem + of[j]);
+            uint32_t acc = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                acc |= (x[j].x ^ pc[j].x) | (x[j].y ^ pc[j].y) | (x[j].z ^ pc[j].z) | (x[j].w ^ pc[j].w);
+            if (acc) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t d[4] = {x[j].x ^ pc[j].x, x[j].y ^ pc[j].y, x[j].z ^ pc[j].z, x[j].w ^ pc[j].w};
+#pragma unroll
+                    for (int g = 0; g < G; ++g)
+                        if ((g & 1) ? (d[g >> 1] >> 16) : (d[g >> 1] & 0xFFFFu)) {
+                            atomicOr(&M->flags[g], (uint32_t)VL_INCONSISTENT);
+                            atomicMin(&M->minop[g], o_base + j);
+                        }
+                }
+            }
+        };
+        auto transpose = [&](const uint2 (&r)[G], uint4 (&pc)[4]) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;
+                uint32_t w[4];
+#pragma unroll
+                for (int m = 0; m < 4; ++m)
+                    w[m] = (j < 2) ? __byte_perm(r[2 * m].x, r[2 * m + 1].x, sel) : __byte_perm(r[2 * m].y, r[2 * m + 1].y, sel);
+                pc[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        };
+        auto store_first = [&](const uint4 (&pc)[4], const uint4 &off, uint32_t first) {
+            const uint32_t of[4] = {off.x, off.y, off.z, off.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if ((first >> j) & 1) *reinterpret_cast<uint4 *>(smem + of[j]) = pc[j];
+        };
+        // the warp has read its part of a stage / has stored its first occurrences of a tile
+        auto warp_arrive = [&](unsigned long long *bar) {
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+        };
+        uint32_t stage = 0, parity = 0;
+        uint4 off_n = opoff[0];
+        uint32_t first_n = first4[0];
+        // one whole tile (not the last): load and transpose, store first occurrences, compare the tile before
+        auto step = [&](uint32_t t, uint4 (&pc)[4], uint4 &off, const uint4 (&ppc)[4], const uint4 &poff) {
+            off = off_n;
+            const uint32_t first = first_n;
+            off_n = opoff[(size_t)(t + 1) * NT];  // (the arrays are padded to whole tiles)
+            first_n = first4[(size_t)(t + 1) * NT];
+            wait_bar(&M->bar[stage], parity);
+            uint2 r[G];
+            const unsigned char *src = region + (size_t)stage * STAGE_BYTES + tid * 8;
+#pragma unroll
+            for (int g = 0; g < G; ++g) r[g] = *reinterpret_cast<const uint2 *>(src + g * ROW_BYTES);
+            transpose(r, pc);
+            warp_arrive(&M->empty[stage]);
+            store_first(pc, off, first);
+            warp_arrive(&M->stored[t & 1]);
+            if (t) wait_bar(&M->stored[(t - 1) & 1], ((t - 1) >> 1) & 1u);
+            compare(ppc, poff, (t - 1) * TILE + tid * 4);
+            if (++stage == q.NS) { stage = 0; parity ^= 1; }
+        };
+        uint4 pcA[4], pcB[4], offA, offB;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pcB[j] = make_uint4(0, 0, 0, 0);
+        offB = make_uint4(spare_off, spare_off, spare_off, spare_off);  // "the tile before tile 0": zeros against the spare entry
+        if (q.test_wait) {  // test hook: this wait runs out
+            uint32_t spins = 0;
+            while (!mbar_try_wait(&M->bar_never, 0)) {
+                if (++spins > (1u << 16)) { M->abort_flag = 1; atomicOr(q.status, ST_DEVICE_WAIT); break; }
+            }
+        }
+        const uint32_t last = q.ntiles - 1;
+        uint32_t t = 0;
+        for (; t + 2 <= last; t += 2) {
+            step(t, pcA, offA, pcB, offB);
+            step(t + 1, pcB, offB, pcA, offA);
+        }
+        if (t < last) {  // an odd number of whole tiles before the last: keep "the tile before" in B
+            step(t, pcA, offA, pcB, offB);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) pcB[j] = pcA[j];
+            offB = offA;
+            ++t;
+        }
+        {   // the last tile: it may hold the row's tail (from its own buffer) and operands beyond the row
+            const uint32_t o_base = last * TILE + tid * 4;
+            offA = off_n;
+            const uint32_t first = first_n;
+            uint2 r[G];
+            if (o_base >= q.tail_start) {  // (a whole warp: the tail starts at a multiple of 256)
+                if (o_base < q.nOp8) {     // the tail buffer ends where the rows end; beyond it there is padding only
+                    wait_bar(&M->bar_tail, 0);
+                    const unsigned char *src = tailbuf + (o_base - q.tail_start) * 2;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) r[g] = *reinterpret_cast<const uint2 *>(src + g * TAIL_ROW_BYTES);
+                } else {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) r[g] = make_uint2(0, 0);
+                }
+            } else {
+                wait_bar(&M->bar[stage], parity);
+                const unsigned char *src = region + (size_t)stage * STAGE_BYTES + tid * 8;
+#pragma unroll
+                for (int g = 0; g < G; ++g) r[g] = *reinterpret_cast<const uint2 *>(src + g * ROW_BYTES);
+            }
+            transpose(r, pcA);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)  // operands beyond n_operands compare as zero against the spare entry
+                if (o_base + j >= q.nO) pcA[j] = make_uint4(0, 0, 0, 0);
+            store_first(pcA, offA, first);
+            warp_arrive(&M->stored[last & 1]);
+            if (last) wait_bar(&M->stored[(last - 1) & 1], ((last - 1) >> 1) & 1u);
+            compare(pcB, offB, (last - 1) * TILE + tid * 4);
+            wait_bar(&M->stored[last & 1], (last >> 1) & 1u);
+            compare(pcA, offA, o_base);
+        }
+    }
+    __syncthreads();
+
+    // ---- one sweep over the vregs: the table goes to global memory (32 candidates side by side per
+    // vreg; the spare entry V, looked up by no-op events, as 0), entries whose range reaches into the
+    // next 32-bit word of an occupancy mask get bit 15, the one-hot bank nibbles of the 8 candidates go
+    // to Hb, and [T, T+width) is checked against the register file (Realizability).
+    // (From here on the producer warp only keeps the block's barriers company.)
+    if (tid < NT) {
+        const uint64_t grp = k0 >> 5;
+        const uint32_t l0 = (uint32_t)(k0 & 31);
+        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        uint32_t mk = 0, mk2 = 0, mk3 = 0, mk4 = 0;
+        uint32_t vis_next[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) vis_next[u] = tid + u * NT < q.V ? q.vinfo[tid + u * NT] : 0u;
+        for (uint32_t v0 = tid; v0 <= q.V; v0 += 4 * NT) {
+            uint32_t vis[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                vis[u] = vis_next[u];
+                const uint32_t vn = v0 + 4 * NT + u * NT;
+                vis_next[u] = vn < q.V ? q.vinfo[vn] : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t v = v0 + u * NT, vi = vis[u];
+                if (v > q.V) break;
+                const uint4 tt = T[v];  // (the spare entry holds zeros)
+                const uint32_t x[4] = {tt.x, tt.y, tt.z, tt.w};
+                if (q.bank_fast && v < q.V) {
+                    uint32_t h = 0;
+#pragma unroll
+                    for (int m = 0; m < 4; ++m)
+                        h |= ((1u << (x[m] & q.Bmask)) << (8 * m)) | ((16u << ((x[m] >> 16) & q.Bmask)) << (8 * m));
+                    Hb[v] = h;
+                }
+                // bit 15 := ((register & 31) + width > 32), per 16-bit entry; 0x7FDF = 0x8000 - 33
+                const uint32_t wc = (vi & 0xFFu) * 0x10001u + 0x7FDF7FDFu;
+                uint32_t o[4];
+#pragma unroll
+                for (int m = 0; m < 4; ++m) o[m] = (x[m] & 0x7FFF7FFFu) | (((x[m] & 0x001F001Fu) + wc) & 0x80008000u);
+                *reinterpret_cast<uint4 *>(dst + (size_t)v * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (!(vi & VINFO_OCCURS)) continue;
+                mk |= o[0]; mk2 |= o[1]; mk3 |= o[2]; mk4 |= o[3];
+                // quick test for "all eight inside the file": with c = 0x7FFF - (P - width) added to an
+                // entry below 2^15, bit 15 of the sum is set iff entry + width > P; entries at or above
+                // 2^15 are outside any file this kernel accepts.  The exact test runs only if a bit shows.
+                const uint32_t w = vi & 0xFFu;
+                uint32_t f = 1;
+                if (w <= q.P) {
+                    const uint32_t c2 = (0x7FFFu - (q.P - w)) * 0x10001u;
+                    f = (((x[0] + c2) | x[0]) | ((x[1] + c2) | x[1]) | ((x[2] + c2) | x[2]) | ((x[3] + c2) | x[3])) & 0x80008000u;
+                }
+                if (f) {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const uint32_t tv = pk8_get(tt, g);
+                        if (tv + w > q.P) {
+                            if (vi & VINFO_DEFINED) {
+                                atomicOr(&M->flags[g], (uint32_t)VL_OUT_OF_RANGE);
+                                atomicMin(&M->minR[g], q.first_def_instr[v]);
+                            }
+                            if (atomicAdd(&M->nout[g], 1u) == 0) { M->out_v[g] = v; M->out_raw[g] = tv; }
+                        }
+                    }
+                }
+            }
+        }
+        const uint32_t mkw[4] = {mk, mk2, mk3, mk4};
+        uint32_t bits = 0;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) bits |= ((mkw[m] >> 15) & 1u) << (2 * m) | ((mkw[m] >> 31) & 1u) << (2 * m + 1);
+        bits = __reduce_or_sync(0xffffffffu, bits);
+        if (lane == 0 && bits) atomicOr(&M->marks, bits);
+    }
+    if (q.vcons && tid < NT) rules_sweep8<NT>(q.vcons, q.rs_prefix, q.vinfo, q.first_def_instr, q.V, q.P, T, M);
+    __syncthreads();
+
+    // ---- bank tally over the instructions with 2..4 distinct sources (see k_tables): the banks an
+    // instruction touches are the bits of the OR of its sources' nibbles, counted with carry-save adders
+    if (q.bank_fast && tid < NT) {
+        auto csa = [](uint32_t &h, uint32_t &l, uint32_t a, uint32_t b, uint32_t c) {
+            const uint32_t u = a ^ b;
+            h = (a & b) | (u & c);
+            l = u ^ c;
+        };
+        // population count of each of the 8 nibbles, as byte fields: even nibbles and odd nibbles
+        auto nib_even = [](uint32_t y) -> uint32_t { return y & 0x0F0F0F0Fu; };
+        auto nib_odd = [](uint32_t y) -> uint32_t { return (y >> 4) & 0x0F0F0F0Fu; };
+        auto nib_counts = [](uint32_t x) -> uint32_t {
+            const uint32_t y = x - ((x >> 1) & 0x55555555u);
+            return (y & 0x33333333u) + ((y >> 2) & 0x33333333u);
+        };
+        uint32_t ones = 0, twos = 0, fours = 0, acc_e = 0, acc_o = 0, rounds = 0;
+        uint32_t sum[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) sum[g] = 0;
+        auto flush = [&](uint32_t weight) {
+#pragma unroll
+            for (int g = 0; g < G; ++g) sum[g] += weight * ((((g & 1) ? acc_o : acc_e) >> (8 * (g >> 1))) & 0xFFu);
+            acc_e = 0; acc_o = 0;
+        };
+        const uint32_t n_ent = q.bank_seg[3];
+        uint2 ids_next[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) ids_next[u] = tid + u * NT < n_ent ? q.bank_list[tid + u * NT] : make_uint2(0, 0);
+        for (uint32_t e0 = tid; e0 < n_ent; e0 += 8 * NT) {
+            uint2 ids[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                ids[u] = ids_next[u];
+                const uint32_t en = e0 + 8 * NT + u * NT;
+                ids_next[u] = en < n_ent ? q.bank_list[en] : make_uint2(0, 0);
+            }
+            uint32_t x[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t o = Hb[ids[u].x & 0xFFFFu] | Hb[ids[u].x >> 16] | Hb[ids[u].y & 0xFFFFu] | Hb[ids[u].y >> 16];
+                x[u] = e0 + u * NT < n_ent ? o : 0u;
+            }
+            uint32_t ta, tb, fa, fb, eights;
+            csa(ta, ones, ones, x[0], x[1]);
+            csa(tb, ones, ones, x[2], x[3]);
+            csa(fa, twos, twos, ta, tb);
+            csa(ta, ones, ones, x[4], x[5]);
+            csa(tb, ones, ones, x[6], x[7]);
+            csa(fb, twos, twos, ta, tb);
+            csa(eights, fours, fours, fa, fb);
+            const uint32_t c8 = nib_counts(eights);
+            acc_e += nib_even(c8);
+            acc_o += nib_odd(c8);
+            if (++rounds == 32) {  // the byte fields hold at most 4 per round
+                flush(8u);
+                rounds = 0;
+            }
+        }
+        flush(8u);
+        uint32_t c = nib_counts(fours);
+        acc_e = nib_even(c); acc_o = nib_odd(c);
+        flush(4u);
+        c = nib_counts(twos);
+        acc_e = nib_even(c); acc_o = nib_odd(c);
+        flush(2u);
+        c = nib_counts(ones);
+        acc_e = nib_even(c); acc_o = nib_odd(c);
+        flush(1u);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const uint32_t x = __reduce_add_sync(0xffffffffu, sum[g]);
+            if (lane == 0 && x) atomicAdd(&M->bank[g], x);
+        }
+    }
+    __syncthreads();
+
+    // ------------------------------------------------- hand-over to the walk (see k_tables)
+#pragma unroll 1
+    for (int g = 0; g < G; ++g) {
+        if (M->nout[g] < 2 || tid >= NT) continue;
+        uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
+        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk8_get(T[v], g);
+    }
+    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
+        const uint32_t ov = M->out_v[tid];
+        const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
+        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)ov * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)(q.P | mark);
+        if (mark) atomicOr(&M->marks, 1u << tid);
+    }
+    __syncthreads();
+    if (tid < G && k0 + tid < q.K) {
+        const uint32_t g = tid;
+        uint32_t first = 0xFFFFFFFFu;
+        if (M->minop[g] != 0xFFFFFFFFu) {  // operand -> instruction: last i with op_off[i] <= operand
+            const uint32_t o = M->minop[g];
+            uint32_t lo_i = 0, hi_i = q.nI;  // invariant: op_off[lo_i] <= o < op_off[hi_i]
+            while (hi_i - lo_i > 1) {
+                const uint32_t mid = (lo_i + hi_i) >> 1;
+                if (q.op_off[mid] <= o) lo_i = mid; else hi_i = mid;
+            }
+            first = lo_i;
+        }
+        uint32_t *cs = q.cstate + (k0 + g) * 8;
+        cs[CS_FLAGS] = M->flags[g];
+        cs[CS_FIRST] = min(first, M->minR[g]);
+        cs[CS_BANK] = q.bank_fast ? q.bank_total - M->bank[g] : 0u;
+        cs[CS_NOUT] = M->nout[g];
+        cs[CS_OUTV] = M->out_v[g];
+        cs[CS_OUTRAW] = M->out_raw[g];
+        cs[CS_WALK] = M->nout[g] >= 2 ? WALK_FULL : 0u;
+        cs[CS_THCOL] = 0;
+        // a candidate that is walked and has a marked entry sends its group of 32 down the walk's
+        // checking path
+        if (M->nout[g] < 2 && ((M->marks >> g) & 1u)) atomicOr(&q.grp_flag[k0 >> 5], 1u);
+    }
 }
 
 __device__ __forceinline__ uint32_t lds32(uint32_t addr)
@@ -615,10 +1123,10 @@ __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tg
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
         // base + offset as one multiply-add: the integer ALU pipe is the walk's bottleneck, the
-        // multiply-add pipe has room
+        // multiply-add pipe has room.  The tables were written by the kernel before this one.
         unsigned long long addr;
         asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(addr) : "r"(off[u]), "l"(tgb));
-        t[u] = *reinterpret_cast<const uint16_t *>(addr);
+        asm("ld.global.nc.u16 %0, [%1];" : "=r"(t[u]) : "l"(addr));
     }
 }
 
@@ -628,12 +1136,16 @@ __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tg
 // anyway).  The common case, no range of the group reaching into the next 32-bit word for any
 // lane, is decided before anything is applied and takes one atomic per event: the table entries
 // carry that fact in bit 15 (very wide ranges are found from the event's width).
-template <bool WIDE>
+// With CHECK = false the caller vouches that no entry of any lane carries the mark and no range is
+// wider than 32 registers: nothing is decided, every event is the one-atomic form.
+template <bool WIDE, bool CHECK>
 __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, uint32_t *s_occ,
                                                 uint32_t lane)
 {
     bool slow;
-    if (!WIDE) {
+    if (!CHECK) {
+        slow = false;
+    } else if (!WIDE) {
         slow = ((t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & 0x8000u) != 0;
     } else {
         const uint4 w4 = lds128_at<96>(ga);
@@ -646,7 +1158,7 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
         }
     }
     uint32_t viol = 0;
-    if (!__any_sync(0xffffffffu, slow)) {
+    if (!CHECK || !__any_sync(0xffffffffu, slow)) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {  // the masks of four events at a time: fewer registers held
             const uint4 z4 = h ? lds128_at<48>(ga) : lds128_at<32>(ga), y4 = h ? lds128_at<80>(ga) : lds128_at<64>(ga);
@@ -691,6 +1203,33 @@ __device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)
     return viol;
 }
 
+// The ng event groups staged at shared address ev_addr (followed by two more staged groups, which
+// are fetched ahead but not applied), applied to this lane's occupancy mask.  Table entries are
+// fetched two groups ahead of the group that is applied; the loop body has no conditions.
+template <bool WIDE, bool CHECK>
+__device__ __forceinline__ uint32_t walk_piece(uint32_t ev_addr, uint32_t ng, const unsigned char *tgb, uint32_t occ_addr,
+                                               uint32_t *s_occ, uint32_t lane)
+{
+    uint32_t viol = 0;
+    uint32_t ta[8], tb[8], tc[8];
+    fetch_group(ev_addr, tgb, ta);
+    fetch_group(ev_addr + 112, tgb, tb);
+    uint32_t g = 0;
+    for (; g + 3 <= ng; g += 3) {
+        const uint32_t ga = ev_addr + g * 112;
+        fetch_group(ga + 224, tgb, tc);
+        viol |= apply_group<WIDE, CHECK>(ga, ta, occ_addr, s_occ, lane);
+        fetch_group(ga + 336, tgb, ta);
+        viol |= apply_group<WIDE, CHECK>(ga + 112, tb, occ_addr, s_occ, lane);
+        fetch_group(ga + 448, tgb, tb);
+        viol |= apply_group<WIDE, CHECK>(ga + 224, tc, occ_addr, s_occ, lane);
+    }
+    // up to two groups are left: ta holds group g, tb group g + 1
+    if (g < ng) viol |= apply_group<WIDE, CHECK>(ev_addr + g * 112, ta, occ_addr, s_occ, lane);
+    if (g + 1 < ng) viol |= apply_group<WIDE, CHECK>(ev_addr + (g + 1) * 112, tb, occ_addr, s_occ, lane);
+    return viol;
+}
+
 // =========================================================================== k_walk
 // grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
 // Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
@@ -700,7 +1239,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
     extern __shared__ __align__(16) uint32_t wsm[];
     uint32_t *s_th = wsm;  // [Wp][32]
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t per_warp = q.Wp * 32 + (q.ev_cap >> 3) * 28;  // words: 112 bytes per group of 8 events
+    const uint32_t per_warp = q.Wp * 32 + ((q.ev_cap >> 3) + 2) * 28;  // words: 112 bytes per group of 8 events
     uint32_t *s_occ = wsm + q.Wp * 32 + (size_t)warp * per_warp;  // [Wp][32]
     uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap / 8] groups of 7 x 16 bytes
     // with few candidates an item is cut into q.split parts, one thread block each
@@ -750,6 +1289,8 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
     }
 
     const uint32_t occ_addr = smem_u32(s_occ) + lane * 4, ev_addr = smem_u32(s_ev);
+    // no table entry of the group carries the straddle mark: the walk decides nothing per event
+    const bool check = __ldcg(q.grp_flag + grp) != 0;
     for (uint32_t c = c0 + warp; c < c1; c += WALK_WARPS) {
         for (uint32_t wd = 0; wd < q.Wp; ++wd) s_occ[wd * 32 + lane] = s_th[wd * 32 + lane];
         uint32_t viol = 0;
@@ -757,28 +1298,14 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
         for (uint32_t done = 0; done < n_ev; done += q.ev_cap) {
             const uint32_t n = min(q.ev_cap, n_ev - done), ng = n >> 3;
             __syncwarp();
-            {   // events of this piece, once: 7 x 16 bytes per group of 8
+            {   // events of this piece and of the two groups after it (the event array ends with two
+                // no-op groups), once: 7 x 16 bytes per group of 8
                 const uint4 *src = q.ev + (size_t)((s0 + done) >> 3) * 7;
-                for (uint32_t i = lane; i < ng * 7; i += 32) s_ev[i] = src[i];
+                for (uint32_t i = lane; i < (ng + 2) * 7; i += 32) s_ev[i] = src[i];
             }
             __syncwarp();
-            // table entries are fetched two groups ahead of the group that is applied
-            uint32_t ta[8], tb[8], tc[8];
-            fetch_group(ev_addr, tgb, ta);
-            if (ng > 1) fetch_group(ev_addr + 112, tgb, tb);
-            for (uint32_t g = 0; g < ng; g += 3) {
-                const uint32_t ga = ev_addr + g * 112;
-                if (g + 2 < ng) fetch_group(ga + 224, tgb, tc);
-                viol |= apply_group<WIDE>(ga, ta, occ_addr, s_occ, lane);
-                if (g + 1 < ng) {
-                    if (g + 3 < ng) fetch_group(ga + 336, tgb, ta);
-                    viol |= apply_group<WIDE>(ga + 112, tb, occ_addr, s_occ, lane);
-                }
-                if (g + 2 < ng) {
-                    if (g + 4 < ng) fetch_group(ga + 448, tgb, tb);
-                    viol |= apply_group<WIDE>(ga + 224, tc, occ_addr, s_occ, lane);
-                }
-            }
+            if (WIDE || check) viol |= walk_piece<WIDE, true>(ev_addr, ng, tgb, occ_addr, s_occ, lane);
+            else viol |= walk_piece<WIDE, false>(ev_addr, ng, tgb, occ_addr, s_occ, lane);
         }
         if (viol && walked) {
             atomicOr(&q.anom[k * q.AW + (c >> 5)], 1u << (c & 31));
@@ -794,6 +1321,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    if (threadIdx.x == 0) q.grp_flag[grp] = 0;  // every block of the group has read it: clear for the next pass
     for (uint32_t j = warp; j < 32; j += WALK_WARPS) {
         const uint64_t kk = (uint64_t)grp * 32 + j;
         if (kk < q.K) finish_candidate(kk, q.nC, q.AW, q.list_all, q.cstate, q.anom, q.chunk_blk, q.work, q.racc, q.out);
@@ -1248,7 +1776,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
 
 // --------------------------------------------------------------------------- host
 namespace {
-struct Plan { uint32_t G, NT, NS, smem, off_region, off_misc; bool ok; };
+struct Plan { uint32_t G, NT, NS, smem, off_region, off_misc, off_tail; bool ok; };  // G = 8: the eight-candidate kernel
 
 inline uint64_t align16(uint64_t x) { return (x + 15u) & ~15ull; }
 
@@ -1269,6 +1797,62 @@ Plan make_plan(const vl_program *p, uint32_t G, uint32_t NT, uint32_t budget)
     pl.smem = pl.off_misc + (uint32_t)misc;
     pl.ok = true;
     return pl;
+}
+
+// Shared memory of one k_tables8 block: [T, 16 bytes per vreg][copy ring][tail buffer][misc]; the
+// bank nibbles (4 bytes per vreg) reuse the copy ring.
+Plan make_plan8(const vl_program *p, uint32_t NT, uint32_t budget)
+{
+    Plan pl{};
+    pl.G = 8; pl.NT = NT;
+    const uint64_t stage = (uint64_t)NT * 4 * 2 * 8;
+    const uint64_t tbytes = ((uint64_t)(p->V + 1) * 16 + 127) & ~127ull;  // the ring is the target of tiled copies
+    const uint64_t tail = 8 * 512;
+    const uint64_t misc = align16(sizeof(TMisc));
+    const uint64_t hbytes = ((uint64_t)(p->V + 1) * 4 + 127) & ~127ull;
+    pl.ok = false;
+    if (tbytes + tail + misc + std::max(2 * stage, hbytes) > budget) return pl;
+    pl.NS = (uint32_t)std::min<uint64_t>(MAX_STAGES, (budget - tbytes - tail - misc) / stage);
+    pl.off_region = (uint32_t)tbytes;
+    pl.off_tail = (uint32_t)(tbytes + std::max(pl.NS * stage, hbytes));
+    pl.off_misc = pl.off_tail + (uint32_t)tail;
+    pl.smem = pl.off_misc + (uint32_t)misc;
+    pl.ok = true;
+    return pl;
+}
+
+// The candidate rows of one pass as a 3-D tensor for the tiled copies of k_tables8:
+// [n rows][nfull chunks][256 operands], a box = 8 rows x (tile / 256) chunks x 256 operands.
+int encode_row_tensor(vl_program *p, CUtensorMap *tm, const uint16_t *d_cand, uint64_t n, uint64_t pitch, uint32_t nfull,
+                      uint32_t chunks_per_tile)
+{
+    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static std::mutex mtx;
+    static encode_fn encode = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mtx);
+        if (!encode) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+            if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+                p->last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorUnknown);
+                return VL_ERR_CUDA;
+            }
+            encode = (encode_fn)fn;
+        }
+    }
+    const cuuint64_t dims[3] = {256, nfull, n};
+    const cuuint64_t strides[2] = {512, pitch * 2};
+    const cuuint32_t box[3] = {256, chunks_per_tile, 8};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, (void *)d_cand, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { p->last_cuda_error = (int)cudaErrorInvalidValue; return VL_ERR_CUDA; }
+    return VL_OK;
 }
 
 template <int G, int NT>
@@ -1303,7 +1887,9 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * 32 * rc_items_per_row(p)) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.grp_done, (groups + 1) * sizeof(uint32_t)));
+    // walk blocks finished per group, then the groups' straddle-mark flags (reset by the walk)
+    VL_CUDA(p, cudaMalloc((void **)&v.grp_done, 2 * (groups + 1) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMemset(v.grp_done, 0, 2 * (groups + 1) * sizeof(uint32_t)));
     v.rows = groups * 32;
     v.aw = aw;
     v.vregs = p->V;
@@ -1335,10 +1921,17 @@ struct PassPlan {
 int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
 {
     const uint32_t SM_BYTES = 227 * 1024;
-    // preference: the largest group that still lets two blocks share an SM, then anything that fits
+    // preference: eight candidates per block (two blocks of 256 threads per SM if the tables are small,
+    // else one block of 512 threads), then the largest group that still lets two blocks share an SM,
+    // then anything that fits
     Plan pl{};
     const uint32_t groups[3] = {4, 2, 1};
     const uint32_t NT = p->threads_opt ? p->threads_opt : 256;
+    if (p->group_opt == 0 || p->group_opt == 8) {
+        pl = make_plan8(p, p->threads_opt ? p->threads_opt : 256, SM_BYTES / 2 - 1024);
+        if (!pl.ok) pl = make_plan8(p, p->threads_opt ? p->threads_opt : 512, SM_BYTES);
+        if (!pl.ok && !p->threads_opt) pl = make_plan8(p, 256, SM_BYTES);
+    }
     for (int pass = 0; pass < 2 && !pl.ok; ++pass)
         for (uint32_t G : groups) {
             if (p->group_opt && G != p->group_opt) continue;
@@ -1349,7 +1942,7 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->pl = pl;
     pp->Wp = (p->P + p->wmax + 31) / 32;
     pp->ev_cap = 256;
-    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + (pp->ev_cap >> 3) * 28)) * 4;
+    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + ((pp->ev_cap >> 3) + 2) * 28)) * 4;
     if (pp->walk_smem > SM_BYTES - 1024) return VL_ERR_UNSUPPORTED;
     // the recount keeps one cache word per vreg in shared memory when that leaves room for several
     // thread blocks per SM, else it fetches from global memory every time
@@ -1379,6 +1972,8 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<4, 512>, at, sm);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<2, 512>, at, sm);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<1, 512>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables8<256>, at, sm);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables8<512>, at, sm);
             if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
             attr_done[p->device] = true;
         }
@@ -1412,9 +2007,28 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
     tq.vcons = p->d_vcons; tq.rs_prefix = p->d_rs_prefix;
+    tq.opoff = p->d_opoff; tq.first4 = p->d_first4;
+    tq.grp_flag = vs.grp_done + (vs.rows / 32 + 1);
+    tq.test_wait = p->test_wait;
+    tq.pf = p->prefetch_tiles;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
-    if (pl.NT == 256) {
+    if (pl.G == 8) {
+        tq.ntiles = (p->nOp8 + pl.NT * 4 - 1) / (pl.NT * 4);
+        tq.nfull = p->nOp8 / 256;
+        tq.tail_start = tq.nfull * 256;
+        tq.tail_tile = tq.tail_start / (pl.NT * 4);
+        tq.off_tail = pl.off_tail;
+        alignas(64) CUtensorMap tm;
+        memset(&tm, 0, sizeof(tm));
+        if (tq.nfull) {
+            rc = encode_row_tensor(p, &tm, d_cand, n, pitch, tq.nfull, pl.NT * 4 / 256);
+            if (rc != VL_OK) return rc;
+        }
+        if (pl.NT == 256) k_tables8<256><<<tgrid, 256 + 32, pl.smem, st>>>(tq, tm);
+        else k_tables8<512><<<tgrid, 512 + 32, pl.smem, st>>>(tq, tm);
+        e = cudaGetLastError();
+    } else if (pl.NT == 256) {
         if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
         else if (pl.G == 2) e = launch_tables<2, 256>(tq, tgrid, pl.smem, st);
         else e = launch_tables<1, 256>(tq, tgrid, pl.smem, st);
@@ -1435,6 +2049,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
         wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
         wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = pp.ev_cap;
         wq.cstate = vs.cstate; wq.anom = vs.anom;
+        wq.grp_flag = vs.grp_done + (vs.rows / 32 + 1);
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
         // few candidates: more, shorter thread blocks, so that the walk still fills the GPU

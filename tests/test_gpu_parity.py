@@ -82,7 +82,7 @@ def test_random_small_programs(B, oracle_mod, seed):
     gp, lv = _check_liveness(B, oracle_mod, p)
     rows = _garbage_rows(p, 48, seed)
     want = oracle_mod.OracleProgram(p).verify(lv, rows)
-    for G in (0, 1, 2, 4):
+    for G in (0, 1, 2, 4, 8):
         gp.set_option(B.VL_OPT_GROUP, G)
         _assert_same(_gpu_verify(B, gp, rows), want, f"seed {seed} G {G}")
     gp.close()
@@ -150,7 +150,8 @@ def test_workloads_full(B, oracle_mod, idx):
     gp.close()
 
 
-@pytest.mark.parametrize("chunk,G,threads", [(16, 4, 256), (64, 2, 512), (512, 1, 0), (4096, 0, 512), (128, 4, 512)])
+@pytest.mark.parametrize("chunk,G,threads", [(16, 4, 256), (64, 2, 512), (512, 1, 0), (4096, 0, 512), (128, 4, 512),
+                                              (48, 8, 256), (160, 8, 512)])
 def test_options_do_not_change_results(B, oracle_mod, chunk, G, threads):
     wl = synth.workload(1)
     p = synth.build_program(wl.shapes[0], wl.seeds[0])

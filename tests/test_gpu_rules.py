@@ -55,7 +55,7 @@ def test_random_small_programs_with_rules(B, oracle_mod, seed):
         gp.set_constraints(P=p.P, **rules)
         want = op.verify(lv, rows)
         seen_extra += int((want["flags"] != plain["flags"]).sum())
-        for G in (0, 1, 2, 4):
+        for G in (0, 1, 2, 4, 8):
             gp.set_option(B.VL_OPT_GROUP, G)
             _assert_same(_gpu_verify(B, gp, rows), want, f"seed {seed} trial {trial} G {G} rules {sorted(rules)}")
     # rules cleared: the plain check again
