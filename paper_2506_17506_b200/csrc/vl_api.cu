@@ -182,7 +182,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
     cudaFree(p->d_vcons); cudaFree(p->d_rs_prefix);
-    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); }
+    for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); cudaFree(v.thm); }
     for (int j = 0; j < 2; ++j) {
         cudaFree(p->d_stage[j]);
         cudaFree(p->d_stage_out[j]);

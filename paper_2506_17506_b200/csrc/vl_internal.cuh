@@ -148,12 +148,13 @@ struct vl_program {
 
     // per-call working memory of vl_verify (one set per internal stream slot), grown on demand
     struct VScratch {
-        uint16_t *tg = nullptr;      // [groups][V+1][32] tables, 32 candidates side by side
+        uint16_t *tg = nullptr;      // [groups][V+1][64] tables, 64 candidates side by side
         uint32_t *cstate = nullptr;  // [rows][8]
         uint32_t *anom = nullptr;    // [rows][AW] chunks whose walk collided
         uint32_t *work = nullptr;    // [1 + rows] count, then candidates that need the exact recount
         uint32_t *racc = nullptr;    // [rows][4] recount accumulators: pairs, lowest instruction, bank tally, slices done
-        uint32_t *grp_done = nullptr;  // [rows / 32] walk thread blocks that have finished, per group of 32 candidates
+        uint32_t *grp_done = nullptr;  // walk thread blocks that have finished, per group of 64 candidates; then the groups' mark flags
+        uint32_t *thm = nullptr;       // [groups][n_blocks][mask words][2][32] through-set masks
         uint64_t rows = 0, aw = 0, vregs = 0, chunks = 0;
     } vs[VL_LANES + 2];              // one per lane, then one per staging buffer of vl_verify_host
     uint32_t sub_batch = 4096;       // candidates per pass of the verify kernels

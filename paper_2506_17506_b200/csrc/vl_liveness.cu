@@ -507,7 +507,7 @@ __global__ void k_instr_flags(uint32_t nI, const uint32_t *__restrict__ op_off, 
 // Every event slot starts as a no-op (see put_event for the layout of a group of 8 events).
 __global__ void k_fill_noop(uint4 *dst, size_t n_groups, uint32_t spare_vreg)
 {
-    const uint32_t vv = spare_vreg * 64u, ww = 31u | (31u << 16);
+    const uint32_t vv = spare_vreg * 128u, ww = 31u | (31u << 16);
     for (size_t i = (size_t)blockIdx.x * NT + threadIdx.x; i < n_groups * 7; i += (size_t)gridDim.x * NT) {
         const uint32_t part = (uint32_t)(i % 7);
         dst[i] = part < 2 ? make_uint4(vv, vv, vv, vv) : (part == 6 ? make_uint4(ww, ww, ww, ww) : make_uint4(0, 0, 0, 0));
@@ -584,7 +584,7 @@ __global__ void k_meta8(uint32_t nO, uint32_t n_quads, uint32_t V, const uint16_
 
 // Walk events are stored in groups of 8, 112 bytes per group, field by field so that the walk
 // fetches a group with 16-byte loads: off[8] (32 bit: byte offset of the vreg's row in a table of
-// 32 16-bit entries per vreg), toggle[8] (32 bit: the width-w mask (1<<w)-1, or 0), test[8]
+// 64 16-bit entries per vreg), toggle[8] (32 bit: the width-w mask (1<<w)-1, or 0), test[8]
 // (likewise), wl[8] (16 bit: 32 - width; the range straddles a 32-bit word iff
 // (register & 31) > wl).  Ranges wider than 32 registers carry wl = 0x8000 | width and
 // toggle, test as 0/1 flags.  A no-op names the spare vreg V with empty masks.
@@ -593,7 +593,7 @@ __device__ __forceinline__ void put_event(uint4 *ev, size_t idx, uint32_t v, uin
     unsigned char *g = reinterpret_cast<unsigned char *>(ev) + (idx >> 3) * 112;
     const uint32_t slot = (uint32_t)(idx & 7);
     const uint32_t wm = w > 32 ? 1u : (w == 32 ? 0xFFFFFFFFu : ((1u << w) - 1u));
-    reinterpret_cast<uint32_t *>(g)[slot] = v * 64u;
+    reinterpret_cast<uint32_t *>(g)[slot] = v * 128u;
     reinterpret_cast<uint32_t *>(g + 32)[slot] = toggle ? wm : 0u;
     reinterpret_cast<uint32_t *>(g + 64)[slot] = test ? wm : 0u;
     reinterpret_cast<uint16_t *>(g + 96)[slot] = (uint16_t)(w > 32 ? (0x8000u | w) : (32u - w));

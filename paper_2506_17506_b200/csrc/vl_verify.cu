@@ -24,6 +24,7 @@
 #include "vl_internal.cuh"
 
 #define MAX_STAGES 4
+#define TGW 64  // candidates side by side per vreg in the tables handed from the table kernel to the walk
 #define WALK_WARPS 8
 #define RC_THREADS 256
 
@@ -79,11 +80,12 @@ struct TMisc {
 };
 
 struct WParams {
-    uint32_t V, P, nB, nC, Wp, AW, use_th, split;
+    uint32_t V, P, nB, nC, Wp, AW, use_th, wmax;
     uint64_t K;
-    const uint32_t *th_off, *th, *cev_off, *item_blk, *item_c0, *item_c1;
+    const uint32_t *th_off, *th, *cev_off;
+    uint32_t *thm;  // [groups][nB][Wp][2][32] through-set masks (k_through -> k_walk)
     const uint4 *ev;
-    const uint16_t *tg, *tg_zero;
+    const uint16_t *tg;
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
     uint32_t *grp_flag;  // per group: set by the table kernel when a walked candidate has a marked entry
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     // state of this pass that the walk and the recount update with atomics starts at zero
     for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
     if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
-    if (tid == 0 && (k0 & 31) == 0) q.grp_done[k0 >> 5] = 0;
+    if (tid == 0 && (k0 & (TGW - 1)) == 0) q.grp_done[k0 / TGW] = 0;
     if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
     __syncthreads();
 
@@ -417,9 +419,9 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     // vreg; the spare entry V, looked up by no-op events, as 0) and [T, T+width) is checked against the
     // register file (Realizability)
     {
-        const uint64_t grp = k0 >> 5;
-        const uint32_t l0 = (uint32_t)(k0 & 31);
-        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        const uint64_t grp = k0 / TGW;
+        const uint32_t l0 = (uint32_t)(k0 & (TGW - 1));
+        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * TGW + l0;
         uint32_t vis_next[8];  // the vreg descriptors of the next round are fetched during the current one
 #pragma unroll
         for (int u = 0; u < 8; ++u) vis_next[u] = tid + u * NT < q.V ? q.vinfo[tid + u * NT] : 0u;
@@ -451,11 +453,11 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
                     hi = (hi & 0x7FFF7FFFu) | (((hi & 0x001F001Fu) + wc) & 0x80008000u);
                 }
                 if constexpr (G == 4) {
-                    *reinterpret_cast<uint2 *>(dst + (size_t)v * 32) = make_uint2(lo, hi);
+                    *reinterpret_cast<uint2 *>(dst + (size_t)v * TGW) = make_uint2(lo, hi);
                 } else if constexpr (G == 2) {
-                    *reinterpret_cast<uint32_t *>(dst + (size_t)v * 32) = lo;
+                    *reinterpret_cast<uint32_t *>(dst + (size_t)v * TGW) = lo;
                 } else {
-                    dst[(size_t)v * 32] = (uint16_t)lo;
+                    dst[(size_t)v * TGW] = (uint16_t)lo;
                 }
                 if (!(vi & VINFO_OCCURS)) continue;
                 const uint32_t w = vi & 0xFFu;
@@ -556,13 +558,13 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         if (M->nout[g] < 2) continue;
-        uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
-        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk_get(t_load<G>(Tt, v), g);
+        uint16_t *col = q.tg + (k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (uint32_t)(k0 & (TGW - 1)) + g;
+        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * TGW] = (uint16_t)pk_get(t_load<G>(Tt, v), g);
     }
     if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
         const uint32_t ov = M->out_v[tid];
         const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
-        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)ov * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)(q.P | mark);
+        q.tg[(k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (size_t)ov * TGW + (uint32_t)(k0 & (TGW - 1)) + tid] = (uint16_t)(q.P | mark);
     }
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
@@ -587,7 +589,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
         cs[CS_THCOL] = 0;
     }
     // this kernel does not keep track of marked entries: its groups take the walk's checking path
-    if (tid == 0) atomicOr(&q.grp_flag[k0 >> 5], 1u);
+    if (tid == 0) atomicOr(&q.grp_flag[k0 / TGW], 1u);
 }
 
 // =========================================================================== k_tables8
@@ -666,7 +668,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     // state of this pass that the walk and the recount update with atomics starts at zero
     for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
     if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
-    if (tid == 0 && (k0 & 31) == 0) q.grp_done[k0 >> 5] = 0;
+    if (tid == 0 && (k0 & (TGW - 1)) == 0) q.grp_done[k0 / TGW] = 0;
     if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
     __syncthreads();
 
@@ -871,9 +873,9 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     // to Hb, and [T, T+width) is checked against the register file (Realizability).
     // (From here on the producer warp only keeps the block's barriers company.)
     if (tid < NT) {
-        const uint64_t grp = k0 >> 5;
-        const uint32_t l0 = (uint32_t)(k0 & 31);
-        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * 32 + l0;
+        const uint64_t grp = k0 / TGW;
+        const uint32_t l0 = (uint32_t)(k0 & (TGW - 1));
+        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * TGW + l0;
         uint32_t mk = 0, mk2 = 0, mk3 = 0, mk4 = 0;
         uint32_t vis_next[4];
 #pragma unroll
@@ -904,7 +906,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
                 uint32_t o[4];
 #pragma unroll
                 for (int m = 0; m < 4; ++m) o[m] = (x[m] & 0x7FFF7FFFu) | (((x[m] & 0x001F001Fu) + wc) & 0x80008000u);
-                *reinterpret_cast<uint4 *>(dst + (size_t)v * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(dst + (size_t)v * TGW) = make_uint4(o[0], o[1], o[2], o[3]);
                 if (!(vi & VINFO_OCCURS)) continue;
                 mk |= o[0]; mk2 |= o[1]; mk3 |= o[2]; mk4 |= o[3];
                 // quick test for "all eight inside the file": with c = 0x7FFF - (P - width) added to an
@@ -1021,13 +1023,13 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
 #pragma unroll 1
     for (int g = 0; g < G; ++g) {
         if (M->nout[g] < 2 || tid >= NT) continue;
-        uint16_t *col = q.tg + (k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (uint32_t)(k0 & 31) + g;
-        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * 32] = (uint16_t)pk8_get(T[v], g);
+        uint16_t *col = q.tg + (k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (uint32_t)(k0 & (TGW - 1)) + g;
+        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * TGW] = (uint16_t)pk8_get(T[v], g);
     }
     if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
         const uint32_t ov = M->out_v[tid];
         const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
-        q.tg[(k0 >> 5) * (uint64_t)(q.V + 1) * 32 + (size_t)ov * 32 + (uint32_t)(k0 & 31) + tid] = (uint16_t)(q.P | mark);
+        q.tg[(k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (size_t)ov * TGW + (uint32_t)(k0 & (TGW - 1)) + tid] = (uint16_t)(q.P | mark);
         if (mark) atomicOr(&M->marks, 1u << tid);
     }
     __syncthreads();
@@ -1054,7 +1056,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         cs[CS_THCOL] = 0;
         // a candidate that is walked and has a marked entry sends its group of 32 down the walk's
         // checking path
-        if (M->nout[g] < 2 && ((M->marks >> g) & 1u)) atomicOr(&q.grp_flag[k0 >> 5], 1u);
+        if (M->nout[g] < 2 && ((M->marks >> g) & 1u)) atomicOr(&q.grp_flag[k0 / TGW], 1u);
     }
 }
 
@@ -1080,24 +1082,6 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
-// A range wider than 32 registers (rare): word by word.
-__device__ __noinline__ uint32_t walk_very_wide(uint32_t *s_occ, uint32_t lane, uint32_t tv, uint32_t width,
-                                                uint32_t test, uint32_t toggle)
-{
-    uint32_t viol = 0, left = width, pos = tv;
-    while (left) {
-        const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
-        const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
-        uint32_t *a = s_occ + (pos >> 5) * 32 + lane;
-        const uint32_t o = *a;
-        if (test) viol |= o & m;
-        if (toggle) *a = o ^ m;
-        pos += nn;
-        left -= nn;
-    }
-    return viol;
-}
-
 __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_all, const uint32_t *cstate,
                                  const uint32_t *anom, const uint32_t *__restrict__ chunk_blk, uint32_t *work,
                                  uint32_t *racc, vl_verdict *out);
@@ -1115,7 +1099,11 @@ __device__ __forceinline__ uint4 lds128_at(uint32_t addr)
     return v;
 }
 
-// Table entries (this lane's candidate) of the 8 vregs of the event group at shared address ga.
+// A lane of the walk carries two candidates, 2 * lane and 2 * lane + 1 of its group of 64: their
+// table entries sit side by side (one 32-bit load per event), their occupancy masks in shared memory
+// at [word][slot 0 / 1][lane] (bank = lane for both).
+
+// Table entries (this lane's two candidates) of the 8 vregs of the event group at shared address ga.
 __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tgb, uint32_t (&t)[8])
 {
     const uint4 a = lds128_at<0>(ga), b = lds128_at<16>(ga);
@@ -1126,91 +1114,122 @@ __device__ __forceinline__ void fetch_group(uint32_t ga, const unsigned char *tg
         // multiply-add pipe has room.  The tables were written by the kernel before this one.
         unsigned long long addr;
         asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(addr) : "r"(off[u]), "l"(tgb));
-        asm("ld.global.nc.u16 %0, [%1];" : "=r"(t[u]) : "l"(addr));
+        asm("ld.global.nc.u32 %0, [%1];" : "=r"(t[u]) : "l"(addr));
     }
 }
 
-// Applies the 8 events of the group at shared address ga to this lane's occupancy mask; returns the
-// occupied bits that a test found.  Toggling returns the old word: occupied and released are both
-// a toggle as long as no collision has been seen (after one, the chunk is recounted exactly
-// anyway).  The common case, no range of the group reaching into the next 32-bit word for any
-// lane, is decided before anything is applied and takes one atomic per event: the table entries
-// carry that fact in bit 15 (very wide ranges are found from the event's width).
-// With CHECK = false the caller vouches that no entry of any lane carries the mark and no range is
-// wider than 32 registers: nothing is decided, every event is the one-atomic form.
-template <bool WIDE, bool CHECK>
-__device__ __forceinline__ uint32_t apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, uint32_t *s_occ,
-                                                uint32_t lane)
+// What a lane knows about one of its candidates: whether it is walked at all, and the address
+// arithmetic that keeps a candidate that is not walked (its table may hold anything) inside the mask.
+struct WalkSlot {
+    uint32_t alive;  // 1 if walked, else 0: shifted to the range's position it gives the bit masks, or nothing
+    uint32_t amask;  // slot 0: 0x7FE0 if walked else 0; slot 1: 2048 if walked else 0 (see apply_group)
+};
+
+// Applies the 8 events of the group at shared address ga to the occupancy masks of this lane's two
+// candidates; viol collects the occupied bits that a test found.  Toggling returns the old word:
+// occupied and released are both a toggle as long as no collision has been seen (after one, the
+// chunk is recounted exactly anyway).  The caller vouches that no range of the group reaches into
+// the next 32-bit word for any walked candidate and that none is wider than 32 registers: every
+// event is one atomic per candidate.  Masks and addresses are computed with multiply-adds where
+// possible, to spare the integer ALU pipe.
+__device__ __forceinline__ void apply_group(uint32_t ga, const uint32_t (&t)[8], uint32_t occ_addr, const WalkSlot &A,
+                                            const WalkSlot &B, uint32_t &violA, uint32_t &violB)
 {
-    bool slow;
-    if (!CHECK) {
-        slow = false;
-    } else if (!WIDE) {
-        slow = ((t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & 0x8000u) != 0;
-    } else {
-        const uint4 w4 = lds128_at<96>(ga);
-        const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
-        slow = false;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const uint32_t wl = (u & 1) ? (ew[u >> 1] >> 16) : (ew[u >> 1] & 0xFFFFu);
-            slow |= ((t[u] & 31u) > wl) || (WIDE && (wl & 0x8000u));
-        }
-    }
-    uint32_t viol = 0;
-    if (!CHECK || !__any_sync(0xffffffffu, slow)) {
+    for (int h = 0; h < 2; ++h) {  // the masks of four events at a time: fewer registers held
+        const uint4 z4 = h ? lds128_at<48>(ga) : lds128_at<32>(ga), y4 = h ? lds128_at<80>(ga) : lds128_at<64>(ga);
+        const uint32_t hz[4] = {z4.x, z4.y, z4.z, z4.w}, hy[4] = {y4.x, y4.y, y4.z, y4.w};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {  // the masks of four events at a time: fewer registers held
-            const uint4 z4 = h ? lds128_at<48>(ga) : lds128_at<32>(ga), y4 = h ? lds128_at<80>(ga) : lds128_at<64>(ga);
-            const uint32_t hz[4] = {z4.x, z4.y, z4.z, z4.w}, hy[4] = {y4.x, y4.y, y4.z, y4.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t tv = t[4 * h + u];
-                // word (tv / 32) of this lane's mask; the masks are moved to bit (tv & 31) by a
-                // multiplication with 1 << (tv & 31), again to spare the integer ALU pipe
-                uint32_t a, mz, my;
-                const uint32_t p2 = __funnelshift_l(0u, 1u, tv);
-                asm("mad.lo.u32 %0, %1, 4, %2;" : "=r"(a) : "r"(tv & 0x7FE0u), "r"(occ_addr));
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t t2 = t[4 * h + u];
+            uint32_t a, mz, my;
+            {   // slot 0: register = low half; its mask word (register / 32) is 256 bytes wide per word
+                const uint32_t p2 = __funnelshift_l(0u, A.alive, t2);
+                asm("mad.lo.u32 %0, %1, 8, %2;" : "=r"(a) : "r"(t2 & A.amask), "r"(occ_addr));
                 asm("mul.lo.u32 %0, %1, %2;" : "=r"(mz) : "r"(hz[u]), "r"(p2));
                 asm("mul.lo.u32 %0, %1, %2;" : "=r"(my) : "r"(hy[u]), "r"(p2));
                 const uint32_t o = atom_xor_shared(a, mz);
-                viol |= o & my;
+                violA |= o & my;
+            }
+            {   // slot 1: register = high half; register / 32 = bits 21.. of the pair = mulhi(pair, 2048)
+                const uint32_t tb = t2 >> 16;
+                const uint32_t p2 = __funnelshift_l(0u, B.alive, tb);
+                uint32_t wd;
+                asm("mul.hi.u32 %0, %1, %2;" : "=r"(wd) : "r"(t2), "r"(B.amask));
+                asm("mad.lo.u32 %0, %1, 256, %2;" : "=r"(a) : "r"(wd), "r"(occ_addr + 128u));
+                asm("mul.lo.u32 %0, %1, %2;" : "=r"(mz) : "r"(hz[u]), "r"(p2));
+                asm("mul.lo.u32 %0, %1, %2;" : "=r"(my) : "r"(hy[u]), "r"(p2));
+                const uint32_t o = atom_xor_shared(a, mz);
+                violB |= o & my;
             }
         }
-        return viol;
     }
-    const uint4 z0 = lds128_at<32>(ga), z1 = lds128_at<48>(ga), y0 = lds128_at<64>(ga), y1 = lds128_at<80>(ga);
-    const uint32_t ez[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
-    const uint32_t ey[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
-    const uint4 w4 = lds128_at<96>(ga);
-    const uint32_t ew[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        const uint32_t tv = t[u] & 0x7FFFu;
-        const uint32_t wl = (u & 1) ? (ew[u >> 1] >> 16) : (ew[u >> 1] & 0xFFFFu);
-        if (WIDE && (wl & 0x8000u)) {
-            viol |= walk_very_wide(s_occ, lane, tv, wl & 0xFFu, ey[u], ez[u]);
-            continue;
-        }
-        const uint32_t a = occ_addr + ((tv >> 5) << 7);
-        const uint32_t o = atom_xor_shared(a, __funnelshift_l(0u, ez[u], tv));
-        viol |= o & __funnelshift_l(0u, ey[u], tv);
-        if ((tv & 31u) > wl) {  // the range straddles into the next word
-            const uint32_t o2 = atom_xor_shared(a + 128, __funnelshift_l(ez[u], 0u, tv));
-            viol |= o2 & __funnelshift_l(ey[u], 0u, tv);
-        }
+}
+
+// One event applied to one candidate's mask word by word: any width, any position (occ = the
+// candidate's word 0; its words are 64 apart).
+__device__ __noinline__ uint32_t walk_event_general(uint32_t *occ, uint32_t tv, uint32_t width, bool test, bool toggle)
+{
+    uint32_t viol = 0, left = width, pos = tv;
+    while (left) {
+        const uint32_t s2 = pos & 31, nn = min(left, 32 - s2);
+        const uint32_t m = (nn == 32 ? 0xFFFFFFFFu : ((1u << nn) - 1u)) << s2;
+        uint32_t *a = occ + (pos >> 5) * 64;
+        const uint32_t o = *a;
+        if (test) viol |= o & m;
+        if (toggle) *a = o ^ m;
+        pos += nn;
+        left -= nn;
     }
     return viol;
 }
 
-// The ng event groups staged at shared address ev_addr (followed by two more staged groups, which
-// are fetched ahead but not applied), applied to this lane's occupancy mask.  Table entries are
-// fetched two groups ahead of the group that is applied; the loop body has no conditions.
-template <bool WIDE, bool CHECK>
-__device__ __forceinline__ uint32_t walk_piece(uint32_t ev_addr, uint32_t ng, const unsigned char *tgb, uint32_t occ_addr,
-                                               uint32_t *s_occ, uint32_t lane)
+// The 8 events of the group at shared address ga, event by event and word by word: for groups in
+// which a walked candidate has an entry with the straddle mark.
+__device__ __noinline__ uint2 apply_event_general(uint32_t ga, uint32_t u, uint32_t t2, uint32_t *occA, bool aliveA, bool aliveB)
 {
-    uint32_t viol = 0;
+    uint2 viol = make_uint2(0, 0);
+    const uint32_t toggle = lds32(ga + 32 + 4 * u), test = lds32(ga + 64 + 4 * u);
+    if (!(toggle | test)) return viol;
+    const uint32_t wl = (lds32(ga + 96 + 4 * (u >> 1)) >> (16 * (u & 1))) & 0xFFFFu;
+    const uint32_t width = (wl & 0x8000u) ? (wl & 0xFFu) : 32u - wl;
+    if (aliveA) viol.x = walk_event_general(occA, t2 & 0x7FFFu, width, test != 0, toggle != 0);
+    if (aliveB) viol.y = walk_event_general(occA + 32, (t2 >> 16) & 0x7FFFu, width, test != 0, toggle != 0);
+    return viol;
+}
+__device__ __forceinline__ void apply_group_general(uint32_t ga, const uint32_t (&t)[8], uint32_t *occA, bool aliveA, bool aliveB,
+                                                    uint32_t &violA, uint32_t &violB)
+{
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const uint2 v = apply_event_general(ga, u, t[u], occA, aliveA, aliveB);
+        violA |= v.x;
+        violB |= v.y;
+    }
+}
+
+// The ng event groups staged at shared address ev_addr (followed by two more staged groups, which
+// are fetched ahead but not applied), applied to the masks of this lane's two candidates.  Table
+// entries are fetched two groups ahead of the group that is applied.  With CHECK = false the
+// caller vouches that no walked candidate of the warp has a marked entry: the loop body has no
+// conditions.  With CHECK = true one vote per group decides between the one-atomic form and the
+// general one.
+template <bool CHECK>
+__device__ __forceinline__ void walk_piece(uint32_t ev_addr, uint32_t ng, const unsigned char *tgb, uint32_t occ_addr,
+                                           uint32_t *occA, const WalkSlot &A, const WalkSlot &B, uint32_t &violA,
+                                           uint32_t &violB)
+{
+    const uint32_t marks = (A.alive ? 0x8000u : 0u) | (B.alive ? 0x80000000u : 0u);
+    auto apply = [&](uint32_t ga, const uint32_t (&t)[8]) {
+        if (CHECK) {
+            const uint32_t any = (t[0] | t[1] | t[2] | t[3] | t[4] | t[5] | t[6] | t[7]) & marks;
+            if (__any_sync(0xffffffffu, any != 0)) {
+                apply_group_general(ga, t, occA, A.alive != 0, B.alive != 0, violA, violB);
+                return;
+            }
+        }
+        apply_group(ga, t, occ_addr, A, B, violA, violB);
+    };
     uint32_t ta[8], tb[8], tc[8];
     fetch_group(ev_addr, tgb, ta);
     fetch_group(ev_addr + 112, tgb, tb);
@@ -1218,82 +1237,117 @@ __device__ __forceinline__ uint32_t walk_piece(uint32_t ev_addr, uint32_t ng, co
     for (; g + 3 <= ng; g += 3) {
         const uint32_t ga = ev_addr + g * 112;
         fetch_group(ga + 224, tgb, tc);
-        viol |= apply_group<WIDE, CHECK>(ga, ta, occ_addr, s_occ, lane);
+        apply(ga, ta);
         fetch_group(ga + 336, tgb, ta);
-        viol |= apply_group<WIDE, CHECK>(ga + 112, tb, occ_addr, s_occ, lane);
+        apply(ga + 112, tb);
         fetch_group(ga + 448, tgb, tb);
-        viol |= apply_group<WIDE, CHECK>(ga + 224, tc, occ_addr, s_occ, lane);
+        apply(ga + 224, tc);
     }
     // up to two groups are left: ta holds group g, tb group g + 1
-    if (g < ng) viol |= apply_group<WIDE, CHECK>(ev_addr + g * 112, ta, occ_addr, s_occ, lane);
-    if (g + 1 < ng) viol |= apply_group<WIDE, CHECK>(ev_addr + (g + 1) * 112, tb, occ_addr, s_occ, lane);
-    return viol;
+    if (g < ng) apply(ev_addr + g * 112, ta);
+    if (g + 1 < ng) apply(ev_addr + (g + 1) * 112, tb);
 }
 
-// =========================================================================== k_walk
-// grid (items, groups of 32 candidates); WALK_WARPS warps per block; lane = candidate.
-// Shared memory: [through-set mask [Wp][32]] then per warp [occupancy [Wp][32]][events of the chunk].
-template <bool WIDE>
-__global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
+// The same for programs with vregs wider than a mask word (rare): event by event, word by word,
+// nothing fetched ahead.
+__device__ __noinline__ void walk_piece_general(const uint4 *s_ev, uint32_t ng, const unsigned char *tgb, uint32_t *occA,
+                                                bool aliveA, bool aliveB, uint32_t &violA, uint32_t &violB)
+{
+    for (uint32_t g = 0; g < ng; ++g) {
+        const uint32_t *grp_w = reinterpret_cast<const uint32_t *>(s_ev + (size_t)g * 7);
+        const uint16_t *grp_wl = reinterpret_cast<const uint16_t *>(grp_w + 24);
+        for (uint32_t u = 0; u < 8; ++u) {
+            const uint32_t off = grp_w[u], toggle = grp_w[8 + u], test = grp_w[16 + u], wl = grp_wl[u];
+            if (!(toggle | test)) continue;
+            const uint32_t width = (wl & 0x8000u) ? (wl & 0xFFu) : 32u - wl;
+            const uint32_t t2 = *reinterpret_cast<const uint32_t *>(tgb + off);
+            if (aliveA) violA |= walk_event_general(occA, t2 & 0x7FFFu, width, test != 0, toggle != 0);
+            if (aliveB) violB |= walk_event_general(occA + 32, (t2 >> 16) & 0x7FFFu, width, test != 0, toggle != 0);
+        }
+    }
+}
+
+// =========================================================================== k_through
+// grid (program blocks, groups of 64 candidates): the occupancy of the vregs that stay occupied
+// through the whole block (its through-set), for every candidate of the group, as masks in the
+// walk's layout [word][slot 0 / 1][lane]; a collision inside the through-set marks the block in the
+// candidate's state.  Every chunk walk of the block starts from these masks.
+__global__ void __launch_bounds__(256) k_through(const WParams q)
 {
     extern __shared__ __align__(16) uint32_t wsm[];
-    uint32_t *s_th = wsm;  // [Wp][32]
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t per_warp = q.Wp * 32 + ((q.ev_cap >> 3) + 2) * 28;  // words: 112 bytes per group of 8 events
-    uint32_t *s_occ = wsm + q.Wp * 32 + (size_t)warp * per_warp;  // [Wp][32]
-    uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 32);   // [ev_cap / 8] groups of 7 x 16 bytes
-    // with few candidates an item is cut into q.split parts, one thread block each
-    const uint32_t item = blockIdx.x / q.split, part = blockIdx.x % q.split, grp = blockIdx.y;
-    const uint32_t b = q.item_blk[item];
-    uint32_t c0 = q.item_c0[item], c1 = q.item_c1[item];
-    {
-        const uint32_t per = (c1 - c0 + q.split - 1) / q.split;
-        c0 = min(c1, c0 + part * per);
-        c1 = min(c1, c0 + per);
-    }
-    const uint64_t k = (uint64_t)grp * 32 + lane;
-    uint32_t *cs = q.cstate + k * 8;  // rows beyond K exist in the working buffers (whole groups)
-    // lanes without a candidate, and candidates that are recounted in full anyway (their table may
-    // hold anything), read an all-zero table instead
-    const bool walked = k < q.K && !(cs[CS_WALK] & WALK_FULL);
-    const uint16_t *tg = walked ? q.tg + (uint64_t)grp * (q.V + 1) * 32 + lane : q.tg_zero + lane;
-    const unsigned char *tgb = reinterpret_cast<const unsigned char *>(tg);
-
-    for (uint32_t i = threadIdx.x; i < q.Wp * 32; i += WALK_WARPS * 32) s_th[i] = 0;
+    uint32_t *s_th = wsm;  // [Wp][2][32]
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const uint32_t b = blockIdx.x, grp = blockIdx.y;
+    const uint64_t kA = (uint64_t)grp * TGW + 2 * lane, kB = kA + 1;
+    uint32_t *csA = q.cstate + kA * 8, *csB = csA + 8;  // rows beyond K exist in the working buffers (whole groups)
+    const bool walkedA = kA < q.K && !(csA[CS_WALK] & WALK_FULL), walkedB = kB < q.K && !(csB[CS_WALK] & WALK_FULL);
+    const unsigned char *tgb = reinterpret_cast<const unsigned char *>(q.tg + (uint64_t)grp * (q.V + 1) * TGW + 2 * lane);
+    for (uint32_t i = threadIdx.x; i < q.Wp * 64; i += blockDim.x) s_th[i] = 0;
     __syncthreads();
-    // mask of the vregs that stay occupied through the whole block
-    if (q.use_th) {
-        bool thcol = false;
-        const uint32_t e1 = q.th_off[b + 1];
-        for (uint32_t e0 = q.th_off[b] + warp * 8; e0 < e1; e0 += WALK_WARPS * 8) {
-            uint32_t x[8], t[8];
+    bool thcolA = false, thcolB = false;
+    const uint32_t e1 = q.th_off[b + 1];
+    for (uint32_t e0 = q.th_off[b] + warp * 8; e0 < e1; e0 += n_warps * 8) {
+        uint32_t x[8], t[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) x[u] = e0 + u < e1 ? q.th[e0 + u] : (q.V | (0u << 16));
+        for (int u = 0; u < 8; ++u) x[u] = e0 + u < e1 ? q.th[e0 + u] : (q.V | (0u << 16));
 #pragma unroll
-            for (int u = 0; u < 8; ++u) t[u] = tg[(size_t)(x[u] & 0xFFFFu) * 32];
+        for (int u = 0; u < 8; ++u) t[u] = *reinterpret_cast<const uint32_t *>(tgb + (size_t)(x[u] & 0xFFFFu) * (TGW * 2));
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                uint32_t pos = t[u] & 0x7FFFu, left = x[u] >> 16;
+        for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (!(h ? walkedB : walkedA)) continue;
+                uint32_t pos = (h ? (t[u] >> 16) : t[u]) & 0x7FFFu, left = x[u] >> 16;
                 while (left) {
                     const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
                     const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
-                    const uint32_t old = atomicOr(&s_th[(pos >> 5) * 32 + lane], m);
-                    thcol |= (old & m) != 0;
+                    const uint32_t old = atomicOr(&s_th[((pos >> 5) * 2 + h) * 32 + lane], m);
+                    if (h) thcolB |= (old & m) != 0; else thcolA |= (old & m) != 0;
                     pos += n;
                     left -= n;
                 }
             }
         }
-        if (thcol && walked) atomicOr(&cs[CS_THCOL], 1u << b);  // through-sets are used only if nB <= 32
-        __syncthreads();
     }
+    if (thcolA) atomicOr(&csA[CS_THCOL], 1u << b);  // through-sets are used only if nB <= 32
+    if (thcolB) atomicOr(&csB[CS_THCOL], 1u << b);
+    __syncthreads();
+    uint32_t *dst = q.thm + ((size_t)grp * q.nB + b) * q.Wp * 64;
+    for (uint32_t i = threadIdx.x; i < q.Wp * 64; i += blockDim.x) dst[i] = s_th[i];
+}
 
+// =========================================================================== k_walk
+// grid (octets of chunks, groups of 64 candidates); one warp per chunk; a lane carries two candidates.
+// Shared memory per warp: [occupancy [Wp][2][32]][events of the chunk].
+__global__ void __launch_bounds__(WALK_WARPS * 32, 3) k_walk(const WParams q)
+{
+    extern __shared__ __align__(16) uint32_t wsm[];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const uint32_t per_warp = q.Wp * 64 + ((q.ev_cap >> 3) + 2) * 28;  // words: 112 bytes per group of 8 events
+    uint32_t *s_occ = wsm + (size_t)warp * per_warp;             // [Wp][2][32]
+    uint4 *s_ev = reinterpret_cast<uint4 *>(s_occ + q.Wp * 64);  // [ev_cap / 8 + 2] groups of 7 x 16 bytes
+    const uint32_t grp = blockIdx.y, c = blockIdx.x * n_warps + warp;
+    const uint64_t kA = (uint64_t)grp * TGW + 2 * lane, kB = kA + 1;
+    uint32_t *csA = q.cstate + kA * 8, *csB = csA + 8;  // rows beyond K exist in the working buffers (whole groups)
+    // candidates beyond K, and candidates that are recounted in full anyway (their table may hold
+    // anything), are not walked
+    const bool walkedA = kA < q.K && !(csA[CS_WALK] & WALK_FULL), walkedB = kB < q.K && !(csB[CS_WALK] & WALK_FULL);
+    const unsigned char *tgb = reinterpret_cast<const unsigned char *>(q.tg + (uint64_t)grp * (q.V + 1) * TGW + 2 * lane);
     const uint32_t occ_addr = smem_u32(s_occ) + lane * 4, ev_addr = smem_u32(s_ev);
+    WalkSlot A, B;
+    A.alive = walkedA ? 1u : 0u; A.amask = walkedA ? 0x7FE0u : 0u;
+    B.alive = walkedB ? 1u : 0u; B.amask = walkedB ? 2048u : 0u;
     // no table entry of the group carries the straddle mark: the walk decides nothing per event
-    const bool check = __ldcg(q.grp_flag + grp) != 0;
-    for (uint32_t c = c0 + warp; c < c1; c += WALK_WARPS) {
-        for (uint32_t wd = 0; wd < q.Wp; ++wd) s_occ[wd * 32 + lane] = s_th[wd * 32 + lane];
-        uint32_t viol = 0;
+    const bool marked = __ldcg(q.grp_flag + grp) != 0;
+    if (c < q.nC) {
+        // the chunk starts from the through-set masks of its block
+        if (q.use_th) {
+            const uint32_t *src = q.thm + ((size_t)grp * q.nB + q.chunk_blk[c]) * q.Wp * 64;
+            for (uint32_t wd = 0; wd < q.Wp * 2; ++wd) s_occ[wd * 32 + lane] = src[wd * 32 + lane];
+        } else {
+            for (uint32_t wd = 0; wd < q.Wp * 2; ++wd) s_occ[wd * 32 + lane] = 0;
+        }
+        uint32_t violA = 0, violB = 0;
         const uint32_t s0 = q.cev_off[c], n_ev = q.cev_off[c + 1] - s0;  // a multiple of 8 events
         for (uint32_t done = 0; done < n_ev; done += q.ev_cap) {
             const uint32_t n = min(q.ev_cap, n_ev - done), ng = n >> 3;
@@ -1304,15 +1358,20 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
                 for (uint32_t i = lane; i < (ng + 2) * 7; i += 32) s_ev[i] = src[i];
             }
             __syncwarp();
-            if (WIDE || check) viol |= walk_piece<WIDE, true>(ev_addr, ng, tgb, occ_addr, s_occ, lane);
-            else viol |= walk_piece<WIDE, false>(ev_addr, ng, tgb, occ_addr, s_occ, lane);
+            if (q.wmax > 32) walk_piece_general(s_ev, ng, tgb, s_occ + lane, walkedA, walkedB, violA, violB);
+            else if (marked) walk_piece<true>(ev_addr, ng, tgb, occ_addr, s_occ + lane, A, B, violA, violB);
+            else walk_piece<false>(ev_addr, ng, tgb, occ_addr, s_occ + lane, A, B, violA, violB);
         }
-        if (viol && walked) {
-            atomicOr(&q.anom[k * q.AW + (c >> 5)], 1u << (c & 31));
-            atomicOr(&cs[CS_WALK], WALK_ANOM);
+        if (violA && walkedA) {
+            atomicOr(&q.anom[kA * q.AW + (c >> 5)], 1u << (c & 31));
+            atomicOr(&csA[CS_WALK], WALK_ANOM);
+        }
+        if (violB && walkedB) {
+            atomicOr(&q.anom[kB * q.AW + (c >> 5)], 1u << (c & 31));
+            atomicOr(&csB[CS_WALK], WALK_ANOM);
         }
     }
-    // the thread block that finishes a group's last item writes the verdicts of the group's clean
+    // the thread block that finishes a group's last chunk writes the verdicts of the group's clean
     // candidates and lists the others for the recount
     __shared__ uint32_t s_last;
     __threadfence();
@@ -1322,8 +1381,8 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 4) k_walk(const WParams q)
     if (!s_last) return;
     __threadfence();
     if (threadIdx.x == 0) q.grp_flag[grp] = 0;  // every block of the group has read it: clear for the next pass
-    for (uint32_t j = warp; j < 32; j += WALK_WARPS) {
-        const uint64_t kk = (uint64_t)grp * 32 + j;
+    for (uint32_t j = warp; j < TGW; j += n_warps) {
+        const uint64_t kk = (uint64_t)grp * TGW + j;
         if (kk < q.K) finish_candidate(kk, q.nC, q.AW, q.list_all, q.cstate, q.anom, q.chunk_blk, q.work, q.racc, q.out);
     }
 }
@@ -1458,7 +1517,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         const uint32_t code = q.work[3 + 2 * it];
         const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
         const uint32_t *cs = q.cstate + k * 8;
-        const uint16_t *tg = q.tg + (k >> 5) * (uint64_t)(q.V + 1) * 32 + (k & 31);
+        const uint16_t *tg = q.tg + (k / TGW) * (uint64_t)(q.V + 1) * TGW + (k & (TGW - 1));
         // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
         const uint32_t out_v = cs[CS_NOUT] == 1 ? cs[CS_OUTV] : 0xFFFFFFFFu, out_raw = cs[CS_OUTRAW];
         // a candidate with several out-of-file vregs was not walked and keeps its table unmarked
@@ -1471,7 +1530,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         RT(11);
         // register (low 16 bits) and width (bits 16..23) of vreg v for this candidate
         auto fetch = [&](uint32_t v) -> uint32_t {
-            const uint32_t r = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * 32] & tmask);
+            const uint32_t r = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * TGW] & tmask);
             return r | ((q.vinfo[v] & 0xFFu) << 16);
         };
         auto reg_w = [&](uint32_t v) -> uint32_t {
@@ -1874,23 +1933,24 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
 {
     vl_program::VScratch &v = p->vs[slot];
     const uint64_t aw = std::max(1u, (p->nC + 31) / 32);
-    const uint64_t groups = (rows + 31) / 32;
+    const uint64_t groups = (rows + TGW - 1) / TGW;
     if (v.rows >= rows && v.aw == aw && v.vregs == p->V && v.chunks == p->nC) return VL_OK;
-    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done);
-    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr; v.grp_done = nullptr;
+    cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); cudaFree(v.thm);
+    v.tg = nullptr; v.cstate = nullptr; v.anom = nullptr; v.work = nullptr; v.racc = nullptr; v.grp_done = nullptr; v.thm = nullptr;
     v.rows = 0;
-    // one more group than needed: it stays all zero, for lanes that have nothing to walk
-    VL_CUDA(p, cudaMalloc((void **)&v.tg, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
-    VL_CUDA(p, cudaMemset(v.tg, 0, (groups + 1) * (p->V + 1) * 32 * sizeof(uint16_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * 32 * 8 * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMemset(v.cstate, 0, groups * 32 * 8 * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * 32 * aw * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * 32 * rc_items_per_row(p)) * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * 32 * 4 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.tg, groups * (p->V + 1) * TGW * sizeof(uint16_t)));
+    VL_CUDA(p, cudaMemset(v.tg, 0, groups * (p->V + 1) * TGW * sizeof(uint16_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * TGW * 8 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMemset(v.cstate, 0, groups * TGW * 8 * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * TGW * aw * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * TGW * rc_items_per_row(p)) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * TGW * 4 * sizeof(uint32_t)));
     // walk blocks finished per group, then the groups' straddle-mark flags (reset by the walk)
     VL_CUDA(p, cudaMalloc((void **)&v.grp_done, 2 * (groups + 1) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMemset(v.grp_done, 0, 2 * (groups + 1) * sizeof(uint32_t)));
-    v.rows = groups * 32;
+    // through-set masks of every (group, program block), in the walk's layout
+    VL_CUDA(p, cudaMalloc((void **)&v.thm, std::max<uint64_t>(1, groups * p->nB * ((p->P + p->wmax + 31) / 32) * 64) * sizeof(uint32_t)));
+    v.rows = groups * TGW;
     v.aw = aw;
     v.vregs = p->V;
     v.chunks = p->nC;
@@ -1913,7 +1973,7 @@ static void kt_mark(vl_program *p, cudaStream_t st)
 namespace {
 struct PassPlan {
     Plan pl;
-    uint32_t Wp, ev_cap, walk_smem, rc_smem;
+    uint32_t Wp, ev_cap, walk_smem, walk_warps, rc_smem;
     uint64_t sub;
 };
 
@@ -1942,8 +2002,12 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     pp->pl = pl;
     pp->Wp = (p->P + p->wmax + 31) / 32;
     pp->ev_cap = 256;
-    pp->walk_smem = (pp->Wp * 32 + WALK_WARPS * (pp->Wp * 32 + ((pp->ev_cap >> 3) + 2) * 28)) * 4;
-    if (pp->walk_smem > SM_BYTES - 1024) return VL_ERR_UNSUPPORTED;
+    // the walk's warps each keep the occupancy masks of 64 candidates: fewer warps for large register files
+    for (pp->walk_warps = WALK_WARPS;; pp->walk_warps >>= 1) {
+        pp->walk_smem = pp->walk_warps * (pp->Wp * 64 + ((pp->ev_cap >> 3) + 2) * 28) * 4;
+        if (pp->walk_smem <= SM_BYTES - 1024) break;
+        if (pp->walk_warps == 1) return VL_ERR_UNSUPPORTED;
+    }
     // the recount keeps one cache word per vreg in shared memory when that leaves room for several
     // thread blocks per SM, else it fetches from global memory every time
     pp->rc_smem = (uint64_t)p->V * 4 <= 72 * 1024
@@ -1963,8 +2027,8 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
             const int sm = (int)SM_BYTES;
             const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
             // (the walk and the recount also have a few bytes of static shared memory)
-            cudaError_t e = cudaFuncSetAttribute(k_walk<true>, at, sm - 1024);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_walk<false>, at, sm - 1024);
+            cudaError_t e = cudaFuncSetAttribute(k_walk, at, sm - 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_through, at, sm - 1024);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_recount<true>, at, sm - 1024);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<4, 256>, at, sm);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tables<2, 256>, at, sm);
@@ -1990,7 +2054,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     if (rc != VL_OK) return rc;
     vl_program::VScratch &vs = p->vs[slot];
     cudaError_t e = cudaSuccess;
-    const uint32_t ngrp = (uint32_t)((n + 31) / 32);
+    const uint32_t ngrp = (uint32_t)((n + TGW - 1) / TGW);
 
     TParams tq{};
     tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
@@ -2008,7 +2072,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
     tq.vcons = p->d_vcons; tq.rs_prefix = p->d_rs_prefix;
     tq.opoff = p->d_opoff; tq.first4 = p->d_first4;
-    tq.grp_flag = vs.grp_done + (vs.rows / 32 + 1);
+    tq.grp_flag = vs.grp_done + (vs.rows / TGW + 1);
     tq.test_wait = p->test_wait;
     tq.pf = p->prefetch_tiles;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
@@ -2041,24 +2105,25 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     g_vl_launches.fetch_add(1);
 
     kt_mark(p, st);
-    if (p->nItems) {
+    if (p->nC) {
         WParams wq{};
         wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = pp.Wp; wq.AW = (uint32_t)vs.aw;
         wq.use_th = (uint32_t)p->use_th; wq.K = n;
         wq.th_off = p->d_th_off; wq.th = p->d_th; wq.cev_off = p->d_cev_off; wq.ev = p->d_ev;
-        wq.item_blk = p->d_item_blk; wq.item_c0 = p->d_item_c0; wq.item_c1 = p->d_item_c1;
-        wq.tg = vs.tg; wq.tg_zero = vs.tg + (vs.rows / 32) * (uint64_t)(p->V + 1) * 32; wq.ev_cap = pp.ev_cap;
+        wq.thm = vs.thm;
+        wq.tg = vs.tg; wq.ev_cap = pp.ev_cap; wq.wmax = p->wmax;
         wq.cstate = vs.cstate; wq.anom = vs.anom;
-        wq.grp_flag = vs.grp_done + (vs.rows / 32 + 1);
+        wq.grp_flag = vs.grp_done + (vs.rows / TGW + 1);
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
-        // few candidates: more, shorter thread blocks, so that the walk still fills the GPU
-        uint32_t split = 1;
-        while (split < 4 && (uint64_t)p->nItems * split * ngrp < 1184) split *= 2;
-        wq.split = split;
-        const dim3 wgrid(p->nItems * split, ngrp);
-        if (p->wmax > 32) k_walk<true><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
-        else k_walk<false><<<wgrid, WALK_WARPS * 32, pp.walk_smem, st>>>(wq);
+        if (p->use_th) {
+            k_through<<<dim3(p->nB, ngrp), 256, pp.Wp * 64 * 4, st>>>(wq);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
+            g_vl_launches.fetch_add(1);
+        }
+        const dim3 wgrid((p->nC + pp.walk_warps - 1) / pp.walk_warps, ngrp);
+        k_walk<<<wgrid, pp.walk_warps * 32, pp.walk_smem, st>>>(wq);
         e = cudaGetLastError();
         if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }
         g_vl_launches.fetch_add(1);
@@ -2067,7 +2132,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     // programs whose bank tally cannot take the fast path (banks not 1, 2 or 4, or an instruction
     // with more than 4 distinct sources) send every candidate through k_recount
     kt_mark(p, st);
-    if (!p->nItems) {  // nothing to walk: the verdict step runs on its own
+    if (!p->nC) {  // nothing to walk: the verdict step runs on its own
         k_finish<<<(uint32_t)((n * 32 + 127) / 128), 128, 0, st>>>(n, p->nC, (uint32_t)vs.aw, p->bank_fast ? 0 : 1,
                                                                   vs.cstate, vs.anom, p->d_chunk_blk, vs.work, vs.racc,
                                                                   d_out);
