@@ -10,6 +10,11 @@ internal streams, so its kernels overlap in the timed region; the per-kernel dur
 (VL_OPT_LANES = 1), where a kernel's duration is its own.  Prints one JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--rows R]
+
+With --gpus N > 1 and no launcher around it (WORLD_SIZE unset) the script starts the N ranks itself,
+by running itself under torch.distributed.run on 127.0.0.1; started by a launcher it reads
+RANK / LOCAL_RANK / WORLD_SIZE from the environment.  One process per GPU, rows sharded over the
+ranks, NCCL only for the barrier, the slowest rank's time and the row total.
 """
 from __future__ import annotations
 
@@ -163,10 +168,50 @@ def run_reference(args):
     return 0
 
 
-# DRAM bytes (read + write) per candidate of each kernel, from the profiler capture of a 4096-row launch
-# summarised under profiles/ (traffic grows in proportion to the rows of a launch); None = no capture of
-# the kernel as it stands.
-TRAFFIC_PER_CANDIDATE = {"k_tables": 891.05e6 / 4096, "k_walk": 86.28e6 / 4096}
+def spawn_ranks(n: int) -> int:
+    """Runs this script as n ranks on this node (one per GPU) and returns the launcher's exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_stub(args):
+    """What the several-rank path does around the GPU work, without a GPU: process group (gloo), barrier,
+    the reductions of the report, one JSON line from rank 0.  Used by the CPU test of `--gpus N`."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    rows_all, ms, _ = shard.job_totals(100 * args.steps, 1.0 + rank, 0, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"stub": True, "n_gpus": world, "gpus_arg": args.gpus, "rows_all": rows_all, "ms": ms}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def measured_traffic(kernel_names):
+    """DRAM bytes (read + write) per candidate of each verify kernel, from the profiler capture recorded in
+    `profiles/dram_traffic_stress.txt`, or None when the kernels' source has changed since (the record
+    carries a hash of vl_verify.cu): a figure must not outlive the kernel it was taken from."""
+    import hashlib
+    rec = os.path.join(ROOT, "profiles", "dram_traffic_stress.txt")
+    src = os.path.join(ROOT, "paper_2506_17506_b200", "csrc", "vl_verify.cu")
+    try:
+        fields = dict(line.split(":", 1) for line in open(rec).read().splitlines() if ":" in line and not line.startswith("#"))
+        if fields["vl_verify.cu sha256"].strip() != hashlib.sha256(open(src, "rb").read()).hexdigest():
+            return None
+        rows = float(fields["rows"])
+        return {n: float(fields[n + " dram bytes"]) / rows for n in kernel_names if n + " dram bytes" in fields}
+    except Exception:
+        return None
 
 
 def main():
@@ -188,6 +233,10 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus)
+    if os.environ.get("VL_BENCH_STUB") == "1":
+        return run_stub(args)
 
     import torch
     import torch.distributed as dist
@@ -198,6 +247,7 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")   # the communicator lines show the ranks that joined
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     wl, prog, K, host, arr = build_inputs(rank, args.rows, pinned=True, fault_rate=args.fault_rate)
@@ -305,7 +355,7 @@ def main():
         # algorithmic bytes: every candidate row is read once (2 bytes per operand column) and one 16-byte
         # verdict is written; the table kernel is the one that streams the rows
         bytes_per_step = 2.0 * prog.pitch * K + 16.0 * K
-        names = ["k_tables", "k_walk", "k_finish", "k_recount"]
+        names = ["k_tables", "k_walk", "k_finish", "k_recount"]   # (k_walk includes the through-set kernel before it)
         passes = max(1, kernel_passes)
         ksum = max(1e-9, sum(kernel_ms))
         kernels = {n: {"ms_per_launch": kernel_ms[j] / passes, "share": kernel_ms[j] / ksum} for j, n in enumerate(names)}
@@ -315,10 +365,10 @@ def main():
         dom = max(range(4), key=lambda j: kernel_ms[j])
         dom_ms = kernel_ms[dom] / passes
         bytes_per_launch = bytes_per_step * iso_steps / passes
-        achieved = bytes_per_launch / (dom_ms * 1e-3) / 1e9
+        dom_achieved = bytes_per_launch / (dom_ms * 1e-3) / 1e9
         path_achieved = bytes_per_step / (verify_ms * 1e-3) / 1e9
-        per_cand = TRAFFIC_PER_CANDIDATE.get(names[dom])
-        traffic = per_cand * K * iso_steps / passes if per_cand else None
+        per_cand = measured_traffic(names)
+        traffic = sum(per_cand.values()) * K if per_cand else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -329,14 +379,21 @@ def main():
                        "l2": "inputs (2 GB per step) larger than L2, no flush"},
             "operand_checks_per_sec": value * prog.n_operands,
             "verify_ms": verify_ms, "liveness_ms": live_ms,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "kernel": names[dom], "of": peak_kind,
-                         "launches": passes, "ms_per_launch": dom_ms, "bytes_per_launch": bytes_per_launch,
-                         "how": f"CUDA events around every launch, {iso_steps} vl_verify calls with their passes in order "
-                                "on one stream (VL_OPT_LANES=1), so that no other kernel runs beside the timed one",
-                         "path": {"what": "one vl_verify call as the timed region runs it (passes spread over the "
-                                          "library's internal streams, kernels overlapping)",
-                                  "achieved": path_achieved, "frac": path_achieved / peak, "ms": verify_ms},
+            # the figures of the whole vl_verify call as the timed region runs it (every verify kernel, passes
+            # spread over the library's internal streams); the dominant kernel alone is a sub-field
+            "roofline": {"bound": "hbm", "achieved": path_achieved, "peak": peak, "unit": "GB/s", "frac": path_achieved / peak,
+                         "traffic": traffic, "kernel": "vl_verify (k_tables8 + k_through + k_walk + k_recount)",
+                         "of": peak_kind, "launches": args.steps, "ms_per_launch": verify_ms,
+                         "bytes_per_launch": bytes_per_step,
+                         "how": "CUDA events on the caller's stream around each of the timed vl_verify calls; algorithmic "
+                                "bytes = rows read once + verdicts",
+                         "traffic_source": ("profiles/dram_traffic_stress.txt (ncu capture of one pass per kernel, scaled by rows)"
+                                            if traffic else None),
+                         "dominant_kernel": {"kernel": names[dom], "achieved": dom_achieved, "frac": dom_achieved / peak,
+                                             "launches": passes, "ms_per_launch": dom_ms, "bytes_per_launch": bytes_per_launch,
+                                             "how": f"CUDA events around every launch, {iso_steps} vl_verify calls with their "
+                                                    "passes in order on one stream (VL_OPT_LANES=1), so that no other "
+                                                    "kernel runs beside the timed one"},
                          "path_in_order": {"what": "one vl_verify call with VL_OPT_LANES=1", "ms": iso_verify_ms,
                                            "frac": bytes_per_step / (iso_verify_ms * 1e-3) / 1e9 / peak},
                          "kernels": kernels, "kernels_in_timed_region": overlapped},

@@ -53,7 +53,7 @@ enum {
                                 1 = every kernel in order on the caller's stream.  vl_verify_batch reads the
                                 option of its first program: 1 = in order, anything else = all 8 streams */
     VL_OPT_PREFETCH_TILES = 8, /* tiles of the candidate rows that the table kernel (8 candidates per block) asks into
-                                L2 ahead of its copy ring, 0..64 (default 6; 0 = none) */
+                                L2 ahead of its copy ring, 0..64 (default 3; 0 = none) */
     VL_OPT_TEST_WAIT = 7     /* test hook for the bounded device waits: 1 = the table kernel (8 candidates per
                                 block) waits for its first tile on a barrier that nothing completes, with a short
                                 poll limit, so that the wait runs out: the call still returns, its verdicts are
@@ -146,23 +146,31 @@ int vl_liveness_result(const vl_program *prog, const uint32_t **blk_live_in, con
  * Requirements: base 16-byte aligned, pitch_elems >= n_operands rounded up to 8,
  * pitch_elems % 8 == 0.  d_out is DEVICE memory for K records (4-byte aligned).
  * Buffers are borrowed for the call; the work is ordered after what `cuda_stream` holds at
- * the call, what is enqueued on `cuda_stream` later is ordered after the work, and the function
- * returns without synchronising.  K == 0 is a no-op.  A call with more than one pass
- * (VL_OPT_SUB_BATCH) spreads its passes over internal streams of the device (VL_OPT_LANES) that
- * fork from and join back into `cuda_stream`, so that kernels of different passes run side by
- * side; with VL_OPT_LANES = 1 every kernel is enqueued on `cuda_stream` itself.
+ * the call, and what is enqueued on `cuda_stream` later is ordered after the work.  K == 0 is a no-op.
+ * A call with more than one pass (VL_OPT_SUB_BATCH; the passes of a call are made equally long)
+ * spreads its passes over internal streams of the device (VL_OPT_LANES) that fork from and join
+ * back into `cuda_stream`, so that kernels of different passes run side by side; with
+ * VL_OPT_LANES = 1 every kernel is enqueued on `cuda_stream` itself.
+ * Host work of a call: the handle is modified (it owns the working memory of its calls).  The first
+ * call on a handle, and a later one that needs larger working sets (more rows per pass, another
+ * chunk size, more internal streams in use), allocates them with cudaMalloc and clears them, which
+ * waits for the device: make one call of the intended size before timing or capturing.  A call that
+ * fits the working sets allocates nothing and does not wait for the device, with one exception: the
+ * first vl_verify* after a vl_liveness that returned early (see there) waits for that run's status
+ * word, after its own kernels have been enqueued.  Each pass encodes one tensor-map descriptor for
+ * the tiled copies on the host (no device work).
  *
  * Per candidate (Section 3.4): T[v] = register at the first occurrence of v;
  * Consistency: every occurrence equals T[v]; Realizability: at every definition
  * [T[v], T[v]+width) lies inside [0, P); Safety: at every definition of v the range of
  * v is disjoint from the range of every other vreg live after that instruction or
  * defined by it.  Bank tally per Section 2 with B banks.
- * UNSUPPORTED: the occupancy masks of the walk, (P + widest vreg) / 32 + 1 words for each of 32
- * candidates and 9 copies, do not fit the shared memory of an SM (P up to about 6,000 fits), or the
- * packed table of one candidate, 2 (n_vregs + 1) bytes, does not.
+ * UNSUPPORTED: P + widest vreg > 32768; the occupancy masks of one warp of the walk,
+ * (P + widest vreg + 31) / 32 words for each of 64 candidates, do not fit the shared memory of an SM
+ * (P up to about 28,000 fits); or the table of one candidate, 2 (n_vregs + 1) bytes, does not.
  * Errors: INVALID_ARG, LIVENESS_NOT_RUN, UNSUPPORTED, CUDA.
  */
-int vl_verify(const vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pitch_elems,
+int vl_verify(vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pitch_elems,
               vl_verdict *d_out, void *cuda_stream);
 
 /*
@@ -170,7 +178,7 @@ int vl_verify(const vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64
  * first program): program j checks K[j] rows of d_cand[j] into d_out[j].  The arrays of
  * pointers and sizes are HOST memory.  Stream-ordered, no synchronisation.
  */
-int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
+int vl_verify_batch(uint32_t n, vl_program *const *progs, const uint16_t *const *d_cand,
                     const uint64_t *K, const uint64_t *pitch_elems, vl_verdict *const *d_out,
                     void *cuda_stream);
 
@@ -299,9 +307,11 @@ int vl_occupied_masks(vl_program *prog, const uint16_t *d_row, uint32_t *d_masks
  *
  * Computes the same live-in / live-out block bitsets as vl_liveness + vl_liveness_result, from a
  * program whose CSR arrays are already in DEVICE memory (same meaning and layout as the fields of
- * vl_program_desc; the program is not validated), into the caller's DEVICE buffers d_live_in and
- * d_live_out, each [n_blocks][max(1, ceil(n_vregs/32))] 32-bit words.  Nothing is checked for
- * strictness here.
+ * vl_program_desc; the program is not validated on the host, but an operand that names no vreg of
+ * the program, or a successor that names no block, is skipped on the device and the call returns
+ * VL_ERR_MALFORMED_PROGRAM), into the caller's DEVICE buffers d_live_in and d_live_out, each
+ * [n_blocks][max(1, ceil(n_vregs/32))] 32-bit words.  d_succ may be NULL only for a program without
+ * edges.  Nothing is checked for strictness here.
  *
  * The per-block read and write sets are kept in one fixed array inside the library,
  * VL_STATIC_SCRATCH_WORDS words (1 MiB) on every GPU that loads it, for the life of the process.
@@ -314,7 +324,7 @@ int vl_occupied_masks(vl_program *prog, const uint16_t *d_row, uint32_t *d_masks
  * first call outside any stream capture.  The call launches on `cuda_stream`, then waits for it,
  * because the convergence status is read back.  It calls no cudaMalloc, cudaFree or other
  * allocating routine.
- * Errors: INVALID_ARG, UNSUPPORTED, NO_CONVERGE, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED, MALFORMED_PROGRAM, NO_CONVERGE, CUDA.
  */
 #define VL_STATIC_SCRATCH_WORDS (1u << 18)
 int vl_block_liveness_static(int device, uint32_t n_blocks, uint32_t n_vregs, const uint32_t *d_block_instr_off,

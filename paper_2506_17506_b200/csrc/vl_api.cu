@@ -94,7 +94,7 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
     p->P = d->P; p->B = d->B;
     p->Wv = std::max(1u, (p->V + 31) / 32);
     p->nOp8 = std::max(8u, (p->nO + 7) / 8 * 8);
-    p->nOpT = (p->nOp8 + 4095u) / 4096u * 4096u;
+    p->nOpT = (p->nOp8 + 4095u) / 4096u * 4096u + 4096u;  // (the table kernel reads its metadata up to two tiles ahead)
     p->wmax = 1;
     for (uint32_t v = 0; v < p->V; ++v) p->wmax = std::max<uint32_t>(p->wmax, d->vreg_width[v]);
     p->h_blk_off.assign(d->block_instr_off, d->block_instr_off + p->nB + 1);
@@ -196,6 +196,23 @@ extern "C" void vl_program_destroy(vl_program *p)
     for (cudaEvent_t ev : p->ev_join)
         if (ev) cudaEventDestroy(ev);
     delete p;
+}
+
+// Multiprocessors of a device, asked once per device and process.
+int vl_device_sm_count(int device)
+{
+    static std::atomic<int> cached[64];
+    if (device >= 0 && device < 64 && cached[device].load() > 0) return cached[device].load();
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 1;
+    if (device >= 0 && device < 64) cached[device].store(n);
+    return n;
+}
+
+int vl_sm_count(vl_program *p)
+{
+    if (p->sm_count <= 0) p->sm_count = vl_device_sm_count(p->device);
+    return p->sm_count;
 }
 
 extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
@@ -352,7 +369,7 @@ static int check_verify_args(const vl_program *p, const void *cand, uint64_t K, 
     return VL_OK;
 }
 
-extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+extern "C" int vl_verify(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
                          void *stream)
 {
     int rc = check_verify_args(p, d_cand, K, pitch, d_out);
@@ -362,11 +379,11 @@ extern "C" int vl_verify(const vl_program *p, const uint16_t *d_cand, uint64_t K
     rc = vl_verify_lanes(1, &p, &d_cand, &K, &pitch, &d_out, (cudaStream_t)stream);
     // a repeated liveness run may still be in flight: the kernels above are ordered behind it on the
     // stream; its outcome is checked here, after they have been enqueued
-    const int rl = vl_live_settle(const_cast<vl_program *>(p));
+    const int rl = vl_live_settle(p);
     return rc != VL_OK ? rc : rl;
 }
 
-extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const uint16_t *const *d_cand,
+extern "C" int vl_verify_batch(uint32_t n, vl_program *const *progs, const uint16_t *const *d_cand,
                                const uint64_t *K, const uint64_t *pitch, vl_verdict *const *d_out, void *stream)
 {
     if (n == 0) return VL_OK;
@@ -383,7 +400,7 @@ extern "C" int vl_verify_batch(uint32_t n, const vl_program *const *progs, const
     int rc = vl_verify_lanes(n - first, progs + first, d_cand + first, K + first, pitch + first, d_out + first,
                              (cudaStream_t)stream);
     for (uint32_t j = 0; j < n; ++j) {
-        const int rl = vl_live_settle(const_cast<vl_program *>(progs[j]));
+        const int rl = vl_live_settle(progs[j]);
         if (rc == VL_OK) rc = rl;
     }
     return rc;
@@ -454,19 +471,6 @@ extern "C" int vl_verify_status(vl_program *p, void *stream)
     VL_CUDA(p, cudaStreamSynchronize((cudaStream_t)stream));
     return (st & ST_DEVICE_WAIT) ? VL_ERR_DEVICE_WAIT : VL_OK;
 }
-
-#ifdef VL_PHASE_TIMERS
-// Profiling builds only: copies the 16 device status words (phase cycle counters from word 2 of the
-// verify status on) to the host and clears them.
-extern "C" int vl_debug_read_status(vl_program *p, uint32_t *out16)
-{
-    if (!p || !out16) return VL_ERR_INVALID_ARG;
-    VL_CUDA(p, cudaDeviceSynchronize());
-    VL_CUDA(p, cudaMemcpy(out16, p->d_status, 64, cudaMemcpyDeviceToHost));
-    VL_CUDA(p, cudaMemset(p->d_status + 1, 0, 60));
-    return VL_OK;
-}
-#endif
 
 extern "C" uint64_t vl_kernel_launches(void) { return g_vl_launches.load(); }
 

@@ -72,7 +72,7 @@ struct vl_program {
     uint32_t nB = 0, nI = 0, V = 0, nO = 0, nE = 0, P = 0, B = 0;
     uint32_t Wv = 0;    // 32-bit words per vreg bitset
     uint32_t nOp8 = 0;  // n_operands rounded up to 8 (at least 8)
-    uint32_t nOpT = 0;  // n_operands rounded up to 4096 (whole tiles of the eight-candidate table kernel)
+    uint32_t nOpT = 0;  // n_operands rounded up to 4096 (whole tiles of the eight-candidate table kernel), plus 4096
     uint32_t wmax = 1;  // widest vreg
     uint32_t chunk_instrs = 160;
     uint32_t group_opt = 0;
@@ -125,7 +125,8 @@ struct vl_program {
     uint2 *d_bank_list = nullptr;   // instructions with 2, 3, 4 distinct sources: their vreg ids, 16 bits each
     uint32_t bank_seg[4] = {0, 0, 0, 0};
     uint32_t threads_opt = 0;
-    uint32_t prefetch_tiles = 6;  // tiles the eight-candidate table kernel asks into L2 ahead of its copy ring
+    uint32_t prefetch_tiles = 3;
+    int sm_count = 0;             // multiprocessors of the device (asked once)  // tiles the eight-candidate table kernel asks into L2 ahead of its copy ring
     uint32_t test_wait = 0;  // test hook of the table kernel's bounded wait (VL_OPT_TEST_WAIT)
     int use_th = 0;
 
@@ -193,9 +194,9 @@ extern std::atomic<uint64_t> g_vl_launches;
     } while (0)
 
 int vl_liveness_impl(vl_program *p, cudaStream_t st);
-int vl_verify_impl(const vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
                    cudaStream_t st, int slot);
-int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
+int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
                     const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st);
 // The lane streams of the handle's device (created once per device; two side streams for liveness
 // follow the VL_LANES lanes in the array) and the handle's fork / join events.
@@ -203,4 +204,7 @@ int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);
 // Waits for a liveness run that is still in flight and checks its outcome; VL_OK if none is pending.
 int vl_live_settle(vl_program *p);
+// Multiprocessors of a device / of the handle's device (asked once).
+int vl_device_sm_count(int device);
+int vl_sm_count(vl_program *p);
 void vl_drop_live_graph(vl_program *p);

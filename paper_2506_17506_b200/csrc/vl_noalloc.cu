@@ -15,7 +15,8 @@
 // Fixed scratch: VL_STATIC_SCRATCH_WORDS 32-bit words (1 MiB) plus a small header, per GPU that loads
 // the library, held until exit.
 #define NA_SCRATCH_WORDS (VL_STATIC_SCRATCH_WORDS + 16u)
-#define NA_HEADER_WORDS 16u  // word 0: status bits of the last call
+#define NA_HEADER_WORDS 16u  // words 0, 1: status bits of the last call (cleared by the call itself)
+#define ST_BAD_INDEX 32u     // an operand names no vreg of the program, or a successor no block
 
 static __device__ __align__(256) uint32_t g_na_scratch[NA_SCRATCH_WORDS];
 
@@ -30,26 +31,31 @@ uint32_t *g_na_ptr[64] = {nullptr};  // device address of g_na_scratch, per devi
 // earlier call survives.
 __global__ void k_na_block_sets(const uint32_t *__restrict__ blk_off, const uint32_t *__restrict__ op_off,
                                 const uint8_t *__restrict__ ndefs, const uint32_t *__restrict__ op_vreg, uint32_t Wv,
-                                uint32_t *blk_use, uint32_t *blk_def, uint32_t *status)
+                                uint32_t n_vregs, uint32_t *blk_use, uint32_t *blk_def, uint32_t *status)
 {
     extern __shared__ uint32_t sm[];
     uint32_t *s_use = sm, *s_def = sm + Wv;
     const uint32_t b = blockIdx.x;
-    if (b == 0 && threadIdx.x == 0) *status = 0;
+
     for (uint32_t w = threadIdx.x; w < 2 * Wv; w += NA_THREADS) sm[w] = 0;
     __syncthreads();
     if (threadIdx.x == 0) {
+        bool bad = false;
         for (uint32_t i = blk_off[b]; i < blk_off[b + 1]; ++i) {
             const uint32_t o0 = op_off[i], o1 = op_off[i + 1], nd = ndefs[i];
+            // (the program is not validated on the host: an id outside the program is skipped and reported)
             for (uint32_t o = o0 + nd; o < o1; ++o) {
                 const uint32_t v = op_vreg[o];
+                if (v >= n_vregs) { bad = true; continue; }
                 if (!((s_def[v >> 5] >> (v & 31)) & 1u)) s_use[v >> 5] |= 1u << (v & 31);
             }
-            for (uint32_t o = o0; o < o0 + nd; ++o) {
+            for (uint32_t o = o0; o < o0 + nd && o < o1; ++o) {
                 const uint32_t v = op_vreg[o];
+                if (v >= n_vregs) { bad = true; continue; }
                 s_def[v >> 5] |= 1u << (v & 31);
             }
         }
+        if (bad) atomicOr(status + 1, ST_BAD_INDEX);
     }
     __syncthreads();
     for (uint32_t w = threadIdx.x; w < Wv; w += NA_THREADS) {
@@ -71,13 +77,17 @@ __global__ void k_na_fixed_point(uint32_t nB, uint32_t Wv, const uint32_t *__res
         live_in[(size_t)b * Wv + w] = 0;
         live_out[(size_t)b * Wv + w] = 0;
     }
-    bool changed = true;
+    bool changed = true, bad = false;
     for (uint32_t sweep = 0; sweep < nB + 2 && changed; ++sweep) {
         changed = false;
         for (uint32_t n = 0; n < nB; ++n) {
             const uint32_t b = nB - 1 - n;
             uint32_t o = 0;
-            for (uint32_t e = succ_off[b]; e < succ_off[b + 1]; ++e) o |= live_in[(size_t)succ[e] * Wv + w];
+            for (uint32_t e = succ_off[b]; e < succ_off[b + 1]; ++e) {
+                const uint32_t sb = succ ? succ[e] : nB;
+                if (sb >= nB) { bad = true; continue; }  // not a block of the program: skipped and reported
+                o |= live_in[(size_t)sb * Wv + w];
+            }
             const uint32_t in = blk_use[(size_t)b * Wv + w] | (o & ~blk_def[(size_t)b * Wv + w]);
             if (o != live_out[(size_t)b * Wv + w] || in != live_in[(size_t)b * Wv + w]) changed = true;
             live_out[(size_t)b * Wv + w] = o;
@@ -85,6 +95,7 @@ __global__ void k_na_fixed_point(uint32_t nB, uint32_t Wv, const uint32_t *__res
         }
     }
     if (changed) atomicOr(status, ST_NO_CONVERGE);
+    if (bad) atomicOr(status + 1, ST_BAD_INDEX);
 }
 
 extern "C" int vl_block_liveness_static(int device, uint32_t n_blocks, uint32_t n_vregs,
@@ -94,7 +105,8 @@ extern "C" int vl_block_liveness_static(int device, uint32_t n_blocks, uint32_t 
                                         uint32_t *d_live_in, uint32_t *d_live_out, void *cuda_stream)
 {
     if (device < 0 || device >= 64 || n_blocks == 0) return VL_ERR_INVALID_ARG;
-    if (!d_block_instr_off || !d_succ_off || !d_instr_op_off || !d_live_in || !d_live_out) return VL_ERR_INVALID_ARG;
+    if (!d_block_instr_off || !d_succ_off || !d_instr_op_off || !d_instr_n_defs || !d_op_vreg || !d_live_in || !d_live_out)
+        return VL_ERR_INVALID_ARG;
     if (n_vregs > 65535) return VL_ERR_UNSUPPORTED;
     const uint32_t Wv = n_vregs ? (n_vregs + 31) / 32 : 1;
     // two bitset rows per basic block must fit the fixed array
@@ -116,15 +128,17 @@ extern "C" int vl_block_liveness_static(int device, uint32_t n_blocks, uint32_t 
     uint32_t *blk_use = scratch + NA_HEADER_WORDS;
     uint32_t *blk_def = blk_use + (size_t)n_blocks * Wv;
 
+    if (cudaMemsetAsync(status, 0, 2 * sizeof(uint32_t), st) != cudaSuccess) return VL_ERR_CUDA;
     k_na_block_sets<<<n_blocks, NA_THREADS, 2 * Wv * sizeof(uint32_t), st>>>(d_block_instr_off, d_instr_op_off,
-                                                                             d_instr_n_defs, d_op_vreg, Wv, blk_use,
+                                                                             d_instr_n_defs, d_op_vreg, Wv, n_vregs, blk_use,
                                                                              blk_def, status);
     k_na_fixed_point<<<(Wv + NA_THREADS - 1) / NA_THREADS, NA_THREADS, 0, st>>>(n_blocks, Wv, d_succ_off, d_succ, blk_use,
                                                                                blk_def, d_live_in, d_live_out, status);
     g_vl_launches.fetch_add(2);
     if (cudaGetLastError() != cudaSuccess) return VL_ERR_CUDA;
-    uint32_t h_status = 0;
-    if (cudaMemcpyAsync(&h_status, status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VL_ERR_CUDA;
+    uint32_t h_status[2] = {0, 0};
+    if (cudaMemcpyAsync(h_status, status, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return VL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return VL_ERR_CUDA;
-    return (h_status & ST_NO_CONVERGE) ? VL_ERR_NO_CONVERGE : VL_OK;
+    if (h_status[1] & ST_BAD_INDEX) return VL_ERR_MALFORMED_PROGRAM;
+    return (h_status[0] & ST_NO_CONVERGE) ? VL_ERR_NO_CONVERGE : VL_OK;
 }

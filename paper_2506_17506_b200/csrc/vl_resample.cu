@@ -13,7 +13,6 @@ namespace {
 constexpr uint32_t RS_CASES = 96;     // test cases per launch (their pointers travel as kernel arguments)
 constexpr uint32_t RS_THREADS = 512;
 constexpr uint32_t RS_ROWS_PER_BLOCK = RS_THREADS * 16;  // a block takes about this many rows
-constexpr uint32_t RS_MAX_PARTS = 592;                    // 4 blocks on each of 148 SMs
 
 struct RsParams {
     const uint4 *out[RS_CASES];  // verdict arrays
@@ -112,7 +111,7 @@ __global__ void __launch_bounds__(256) k_resample_summary(const RsSumParams q)
 
 // records of cases [c0, c0 + m) into d_stats + c0
 cudaError_t launch_stats(uint32_t m, const vl_verdict *const *d_out, const uint64_t *K, vl_sample_stats *d_stats,
-                         cudaStream_t st)
+                         cudaStream_t st, uint32_t max_parts)
 {
     RsParams q;
     uint64_t kmax = 0;
@@ -127,7 +126,7 @@ cudaError_t launch_stats(uint32_t m, const vl_verdict *const *d_out, const uint6
     g_vl_launches.fetch_add(1);
     if (kmax) {
         uint64_t parts = (kmax + RS_ROWS_PER_BLOCK - 1) / RS_ROWS_PER_BLOCK;
-        if (parts > RS_MAX_PARTS) parts = RS_MAX_PARTS;
+        if (parts > max_parts) parts = max_parts;
         k_sample_stats<<<dim3((uint32_t)parts, m), RS_THREADS, 0, st>>>(q);
         g_vl_launches.fetch_add(1);
     }
@@ -150,7 +149,9 @@ extern "C" int vl_resample_stats(int device, uint32_t n, const vl_verdict *const
     cudaStream_t st = (cudaStream_t)stream;
     for (uint32_t c0 = 0; c0 < n; c0 += RS_CASES) {
         const uint32_t m = n - c0 < RS_CASES ? n - c0 : RS_CASES;
-        if (launch_stats(m, d_out + c0, K + c0, d_stats + c0, st) != cudaSuccess) return VL_ERR_CUDA;
+        // at most 4 thread blocks per multiprocessor work on one verdict array
+        if (launch_stats(m, d_out + c0, K + c0, d_stats + c0, st, 4u * (uint32_t)vl_device_sm_count(device)) != cudaSuccess)
+            return VL_ERR_CUDA;
     }
     if (d_summary) {
         RsSumParams s;
@@ -182,7 +183,7 @@ extern "C" int vl_verify_until_pass(vl_program *p, const uint16_t *d_cand, uint6
         const int rc = vl_verify(p, d_cand + b0 * pitch, nb, pitch, d_out + b0, stream);
         if (rc != VL_OK) return rc;
         const vl_verdict *outs = d_out + b0;
-        VL_CUDA(p, launch_stats(1, &outs, &nb, p->d_rs, st));
+        VL_CUDA(p, launch_stats(1, &outs, &nb, p->d_rs, st, 4u * (uint32_t)vl_sm_count(p)));
         VL_CUDA(p, cudaMemcpyAsync(p->h_rs, p->d_rs, sizeof(vl_sample_stats), cudaMemcpyDeviceToHost, st));
         VL_CUDA(p, cudaStreamSynchronize(st));
         *rows_checked = b0 + nb;

@@ -116,23 +116,6 @@ struct RParams {
     uint32_t R;                            // registers covered by the recount's through-set counters
 };
 
-// Optional per-phase cycle counters (thread 0 of every k_tables block adds its elapsed clocks to
-// status[2 + phase]); compiled in only with -DVL_PHASE_TIMERS, for profiling builds.
-#ifdef VL_PHASE_TIMERS
-#define PT_INIT() long long pt_last = clock64()
-#define PT(idx)                                                                \
-    do {                                                                       \
-        if (threadIdx.x == 0) {                                                \
-            long long now = clock64();                                         \
-            atomicAdd(q.status + 2 + (idx), (uint32_t)((now - pt_last) >> 6)); \
-            pt_last = now;                                                     \
-        }                                                                      \
-    } while (0)
-#else
-#define PT_INIT()
-#define PT(idx)
-#endif
-
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -300,7 +283,6 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     };
     if (tid == 0)
         for (uint32_t t = 0; t < q.NS && t < q.ntiles; ++t) issue_tile(t, t);
-    PT_INIT();
 
     // Per tile: load it from the ring and store its first occurrences to the table, barrier, compare
     // every occurrence with the table.  The compare of tile t may overlap the stores of tile t+1 by
@@ -414,7 +396,6 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     __syncthreads();
 
-    PT(0);
     // ---- one sweep over the vregs: the table goes to global memory (32 candidates side by side per
     // vreg; the spare entry V, looked up by no-op events, as 0) and [T, T+width) is checked against the
     // register file (Realizability)
@@ -475,11 +456,9 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
             }
         }
     }
-    PT(1);
     if (q.vcons) rules_sweep<G, NT>(q.vcons, q.rs_prefix, q.vinfo, q.first_def_instr, q.V, q.P, Tt, M);
 
     __syncthreads();
-    PT(2);
     // ------------------------------- bank tally: instructions with 2..4 distinct sources.
     // Distinct vregs read by one instruction are live together, so a candidate whose walk sees no
     // collision has them on distinct registers, and its tally for one instruction is the number of
@@ -550,7 +529,6 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     __syncthreads();
 
-    PT(3);
     // ------------------------------------------------- hand-over to the walk
     // One vreg sticking out of the file cannot overlap another one out there: the walk sees it
     // parked at P (bits beyond P are padding).  Two or more: the candidate is recounted in full.
@@ -682,6 +660,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         // Bounded wait.  When it runs out the block raises the status bit and carries on with short
         // waits (its results are garbage, every index still in bounds); the producer issues no
         // further copies and, before the block returns, waits again for the copies it did issue.
+        if (mbar_try_wait(bar, parity)) return;
         uint32_t spins = 0;
         const uint32_t limit = *(volatile uint32_t *)&M->abort_flag ? 64u : (1u << 20);
         while (!mbar_try_wait(bar, parity)) {
@@ -713,9 +692,6 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
                     mbar_expect_tx(&M->bar[stage], STAGE_BYTES);
                     tma_load_3d(region + (size_t)stage * STAGE_BYTES, &tm, 0, t * CH, (uint32_t)k0, &M->bar[stage]);
                 }
-                // The ring holds too few bytes to cover the latency of HBM by itself: the tiles further
-                // ahead are asked into L2, so that the ring's copies come from there.
-                if (q.pf && (t + q.pf) * CH < q.nfull) tma_prefetch_3d(&tm, 0, (t + q.pf) * CH, (uint32_t)k0);
                 if (++stage == q.NS) { stage = 0; parity ^= 1; }
             }
             if (*(volatile uint32_t *)&M->abort_flag) {
@@ -788,14 +764,28 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
         };
         uint32_t stage = 0, parity = 0;
-        uint4 off_n = opoff[0];
-        uint32_t first_n = first4[0];
+        const uint32_t last = q.ntiles - 1;
+        // thread i asks for line i % (ROW_BYTES / 128) of row i / (ROW_BYTES / 128) of a tile
+        const unsigned char *pf_ptr = nullptr;
+        if (q.pf && tid < G * (ROW_BYTES / 128))
+            pf_ptr = reinterpret_cast<const unsigned char *>(q.cand + min(k0 + tid / (ROW_BYTES / 128), q.K - 1) * q.pitch) +
+                     (tid % (ROW_BYTES / 128)) * 128;
+        // operand metadata is fetched two tiles ahead (the arrays are padded to whole tiles, and one
+        // tile more is readable behind them)
+        uint4 off_n = opoff[0], off_n2 = opoff[NT];
+        uint32_t first_n = first4[0], first_n2 = first4[NT];
         // one whole tile (not the last): load and transpose, store first occurrences, compare the tile before
         auto step = [&](uint32_t t, uint4 (&pc)[4], uint4 &off, const uint4 (&ppc)[4], const uint4 &poff) {
             off = off_n;
             const uint32_t first = first_n;
-            off_n = opoff[(size_t)(t + 1) * NT];  // (the arrays are padded to whole tiles)
-            first_n = first4[(size_t)(t + 1) * NT];
+            off_n = off_n2;
+            first_n = first_n2;
+            off_n2 = opoff[(size_t)(t + 2) * NT];
+            first_n2 = first4[(size_t)(t + 2) * NT];
+            // The ring holds too few bytes to cover the latency of HBM by itself: the lines of a tile
+            // further ahead are asked into L2 (one 128-byte line per thread), so that the ring's
+            // copies come from there.
+            if (pf_ptr && t + q.pf < last) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf_ptr + (size_t)(t + q.pf) * ROW_BYTES));
             wait_bar(&M->bar[stage], parity);
             uint2 r[G];
             const unsigned char *src = region + (size_t)stage * STAGE_BYTES + tid * 8;
@@ -819,7 +809,6 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
                 if (++spins > (1u << 16)) { M->abort_flag = 1; atomicOr(q.status, ST_DEVICE_WAIT); break; }
             }
         }
-        const uint32_t last = q.ntiles - 1;
         uint32_t t = 0;
         for (; t + 2 <= last; t += 2) {
             step(t, pcA, offA, pcB, offB);
@@ -1495,10 +1484,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr uint32_t NW = RC_THREADS / 32;
     const uint32_t nitems = q.work[0];
-#ifdef VL_PHASE_TIMERS
-    const long long rc_t0 = clock64();
-    if (tid == 0 && blockIdx.x == 0) atomicAdd(q.status + 8, nitems);
-#endif
     __shared__ uint32_t s_item;
     for (;;) {
         // the items differ a lot in length: thread blocks take the next one from a shared cursor
@@ -1507,12 +1492,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         __syncthreads();
         const uint32_t it = s_item;
         if (it >= nitems) break;
-#ifdef VL_PHASE_TIMERS
-        long long rt = clock64();
-#define RT(idx) do { if (tid == 0) { long long n_ = clock64(); atomicAdd(q.status + (idx), (uint32_t)((n_ - rt) >> 4)); rt = n_; } } while (0)
-#else
-#define RT(idx)
-#endif
         const uint64_t k = q.work[2 + 2 * it];
         const uint32_t code = q.work[3 + 2 * it];
         const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
@@ -1527,7 +1506,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             for (uint32_t v = tid; v < q.V; v += RC_THREADS) Cv[v] = 0;
         if (tid == 0) { s_pairs = 0; s_mind = 0xFFFFFFFFu; s_bank = 0; }
         __syncthreads();
-        RT(11);
         // register (low 16 bits) and width (bits 16..23) of vreg v for this candidate
         auto fetch = [&](uint32_t v) -> uint32_t {
             const uint32_t r = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * TGW] & tmask);
@@ -1665,7 +1643,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 }
                 __syncthreads();
             }
-            RT(12);
             // this warp's instructions: i_lo + warp, i_lo + warp + NW, ...; 32 of them per round
             for (uint32_t ib = i_lo + warp; ib < i_hi; ib += 32 * NW) {
                 const uint32_t my_i = ib + lane * NW;
@@ -1800,7 +1777,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             if (lane == 0 && bt) atomicAdd(&s_bank, bt);
         }
         __syncthreads();
-        RT(kind == RC_KIND_BANK ? 6 : (kind == RC_KIND_THROUGH ? 7 : 13));
         if (tid == 0) {
             uint32_t *acc = q.racc + k * 4;
             if (s_pairs) atomicAdd(&acc[0], s_pairs);
@@ -1822,15 +1798,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 q.out[k] = vd;
             }
         }
-        RT(14);
     }
-#ifdef VL_PHASE_TIMERS
-    if (tid == 0) {
-        const uint32_t dt = (uint32_t)((clock64() - rc_t0) >> 6);
-        atomicAdd(q.status + 9, dt);
-        atomicMax(q.status + 10, dt);
-    }
-#endif
 }
 
 // --------------------------------------------------------------------------- host
@@ -2018,6 +1986,12 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
     // the recount work list holds up to rc_items_per_row items per candidate: keep it within 8 Mi items
     const uint64_t sub_cap = std::max<uint64_t>(32, ((8ull << 20) / rc_items_per_row(p)) / 32 * 32);
     pp->sub = std::min<uint64_t>(K, std::min<uint64_t>(p->sub_batch, sub_cap));
+    // passes of equal size (whole groups of the tables) rather than full ones and a short last one
+    if (K > pp->sub) {
+        const uint64_t n_pass = (K + pp->sub - 1) / pp->sub;
+        const uint64_t even = ((K + n_pass - 1) / n_pass + TGW - 1) / TGW * TGW;
+        pp->sub = std::min(pp->sub, even);
+    }
     // once per device: every verify kernel may use the whole shared memory of an SM
     static std::mutex attr_mutex;
     static bool attr_done[64];
@@ -2151,7 +2125,7 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     rq.tg = vs.tg; rq.cstate = vs.cstate; rq.anom = vs.anom; rq.work = vs.work; rq.out = d_out;
     rq.bank_list = p->d_bank_list;
     for (int j = 0; j < 4; ++j) rq.bank_seg[j] = p->bank_seg[j];
-    const uint32_t rgrid = 148 * 6;
+    const uint32_t rgrid = (uint32_t)vl_sm_count(p) * 6;  // thread blocks of the recount: they take items from a shared cursor
     kt_mark(p, st);
     if (pp.rc_smem) k_recount<true><<<rgrid, RC_THREADS, pp.rc_smem, st>>>(rq);
     else k_recount<false><<<rgrid, RC_THREADS, 0, st>>>(rq);
@@ -2164,10 +2138,9 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
 }  // namespace
 
 // All passes in order on one stream, with one working set.
-int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
                    cudaStream_t st, int slot)
 {
-    vl_program *p = const_cast<vl_program *>(cp);  // the handle owns the working memory of its calls
     PassPlan pp{};
     int rc = plan_passes(p, K, &pp);
     if (rc != VL_OK) return rc;
@@ -2182,10 +2155,10 @@ int vl_verify_impl(const vl_program *cp, const uint16_t *d_cand, uint64_t K, uin
 // the table kernel of one pass (bound by the row stream) runs beside the walk of another (bound by
 // instruction issue).  Pass j of a program uses working set j mod lanes and runs on lane
 // (first_lane + j) mod lanes: two passes that share a working set are ordered by their stream.
-int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
+int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
                     const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st)
 {
-    vl_program *p0 = const_cast<vl_program *>(progs[0]);
+    vl_program *p0 = progs[0];
     cudaStream_t *lane = nullptr;
     int rc = vl_lane_streams(p0, &lane);
     if (rc != VL_OK) return rc;
@@ -2206,7 +2179,7 @@ int vl_verify_lanes(uint32_t nprog, const vl_program *const *progs, const uint16
     uint64_t job = 0;
     for (uint32_t j = 0; j < nprog && rc == VL_OK; ++j) {
         if (K[j] == 0) continue;
-        vl_program *p = const_cast<vl_program *>(progs[j]);
+        vl_program *p = progs[j];
         PassPlan pp{};
         rc = plan_passes(p, K[j], &pp);
         if (rc != VL_OK) break;

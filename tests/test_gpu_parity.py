@@ -311,6 +311,31 @@ def test_recount_work_list_full(B, oracle_mod):
     gp.close()
 
 
+def test_bounded_device_wait_runs_out(B, oracle_mod):
+    """The waits of the table kernel on its copy ring are bounded.  With the test hook switched on
+    the kernel waits on a barrier that nothing completes, with a short poll limit: the wait gives up,
+    the call still returns (nothing traps, nothing keeps spinning), vl_verify_status reports
+    VL_ERR_DEVICE_WAIT, and the next call without the hook is bit-exact again."""
+    import torch
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    rows, _ = synth.candidate_rows(p, 40, 0.3, 21)
+    want = oracle_mod.OracleProgram(p).verify(lv, rows)
+    _assert_same(_gpu_verify(B, gp, rows), want, "before")
+    gp.set_option(B.VL_OPT_GROUP, 8)                      # the hook sits in the eight-candidate table kernel
+    gp.set_option(B.VL_OPT_TEST_WAIT, 1)
+    gp.vl_verify(_to_dev(rows))
+    torch.cuda.synchronize()                              # the kernels end by themselves
+    with pytest.raises(B.VlError) as e:
+        gp.vl_verify_status()
+    assert e.value.code == B.VL_ERR_DEVICE_WAIT
+    gp.set_option(B.VL_OPT_TEST_WAIT, 0)
+    for _ in range(2):
+        _assert_same(_gpu_verify(B, gp, rows), want, "after the wait ran out")
+    gp.close()
+
+
 def test_repeated_liveness_runs(B, oracle_mod):
     """Later liveness runs of a handle return without waiting for the GPU and are replayed from a
     recording: the results stay those of the first run, a changed chunk size starts over, and the

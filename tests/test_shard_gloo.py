@@ -92,3 +92,21 @@ def test_two_ranks_cover_the_job(tmp_path, oracle_mod):
 def test_job_sample_stats_single_process():
     assert shard.job_sample_stats(5, 2, 10, 100, 1000) == (105, 2)
     assert shard.job_sample_stats(10, 0, 10, 100, 1000) == (1000, 0)
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a launcher around it starts two ranks (here with the stub step, which
+    does everything around the GPU work on CPU: process group, barrier, reductions, one JSON line)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    env["VL_BENCH_STUB"] = "1"
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "3"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(ln) for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    assert lines[0]["n_gpus"] == 2 and lines[0]["gpus_arg"] == 2
+    assert lines[0]["rows_all"] == 2 * 300 and lines[0]["ms"] == 2.0      # sum of rows, slowest rank's time
