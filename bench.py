@@ -140,6 +140,13 @@ def oracle_rate(prog, arr, n_rows: int, threads: int):
     return n_rows / dt, dt, t_live, np.concatenate(outs), lv
 
 
+def config_of(prog, wl, K, world):
+    """The `config` object of the JSON line: the workload both arms are quoted on."""
+    return {"workload": "stress", "n_blocks": prog.n_blocks, "n_instrs": prog.n_instrs, "n_vregs": prog.n_vregs,
+            "n_operands": prog.n_operands, "P": prog.P, "B": prog.B, "K_per_gpu": K, "fault_rate": wl.fault_rate,
+            "parallelism": f"rows sharded over {world} GPU(s)", "l2": "inputs (2 GB per step) larger than L2, no flush"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -157,10 +164,10 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * sample / value, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u16", "data": "synthetic",
-        "config": {"workload": "stress", "n_instrs": prog.n_instrs, "n_vregs": prog.n_vregs,
-                   "n_operands": prog.n_operands, "P": prog.P, "K": sample},
+        # the workload is the GPU arm's; a step of this arm checks a bounded sample of its rows
+        "config": config_of(prog, wl, wl.K, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": f"{sample} rows of the stress workload per step, {threads} host threads"},
+                         "sample": f"the first {sample} of the workload's {wl.K} rows per step, {threads} host threads"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -373,10 +380,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u16", "data": "synthetic",
-            "config": {"workload": "stress", "n_blocks": prog.n_blocks, "n_instrs": prog.n_instrs,
-                       "n_vregs": prog.n_vregs, "n_operands": prog.n_operands, "P": prog.P, "B": prog.B,
-                       "K_per_gpu": K, "fault_rate": wl.fault_rate, "parallelism": f"rows sharded over {world} GPU(s)",
-                       "l2": "inputs (2 GB per step) larger than L2, no flush"},
+            "config": config_of(prog, wl, K, world),
             "operand_checks_per_sec": value * prog.n_operands,
             "verify_ms": verify_ms, "liveness_ms": live_ms,
             # the figures of the whole vl_verify call as the timed region runs it (every verify kernel, passes

@@ -1,6 +1,6 @@
 """Throughput of vl_liveness + vl_verify on the five synthetic workloads, one line per workload.
 
-    python -m paper_2506_17506_b200.workloads_report [--steps N]
+    python workloads_report.py [--steps N]
 
 For every workload: candidate verifications per second and operand checks per second with the rows
 resident in device memory (CUDA events around `steps` repetitions of liveness + verify, after
@@ -23,11 +23,14 @@ import sys
 
 import numpy as np
 
-from . import synth
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2506_17506_b200 import synth  # noqa: E402
 
 
 def peak_gbs() -> float:
-    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"])
@@ -41,7 +44,7 @@ def main() -> int:
     ap.add_argument("--workloads", default="1,2,3,4,5")
     args = ap.parse_args()
     import torch
-    from . import binding as vl
+    from paper_2506_17506_b200 import binding as vl
 
     peak = peak_gbs()
     stream = torch.cuda.current_stream()
