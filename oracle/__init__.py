@@ -64,6 +64,10 @@ def _load():
         lib.vlo_bank_histogram.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.vlo_occupied.restype = None
         lib.vlo_occupied.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.vlo_dict_layout.restype = C.c_uint32
+        lib.vlo_dict_layout.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.vlo_verify_dict_rows.restype = None
+        lib.vlo_verify_dict_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
         lib.vlo_sample_stats_of.restype = None
         lib.vlo_sample_stats_of.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         lib.vlo_resample_summary.restype = None
@@ -161,6 +165,29 @@ class OracleProgram:
         out = np.zeros(K, dtype=VERDICT_DTYPE)
         lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
         lib.vlo_verify_rows(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(rows), K, pitch, _ptr(out))
+        return out
+
+    def dict_layout(self):
+        """(dict_off [n_blocks+1], dict_vreg [n_entries], entry_instr [n_entries]) of the per-basic-block
+        dictionary form of a candidate: blocks in order, a block's vregs in order of first occurrence."""
+        lib = _load()
+        n_ops = int(self.src.n_operands)
+        off = np.zeros(self.n_blocks + 1, dtype=np.uint32)
+        vreg = np.zeros(n_ops + 1, dtype=np.uint32)
+        instr = np.zeros(n_ops + 1, dtype=np.uint32)
+        n = int(lib.vlo_dict_layout(C.byref(self.c), _ptr(off), _ptr(vreg), _ptr(instr)))
+        return off, vreg[:n].copy(), instr[:n].copy()
+
+    def verify_dict(self, live: Liveness, rows: np.ndarray) -> np.ndarray:
+        """Verdict record for every row of a uint16 [K, pitch] matrix of dictionary candidates."""
+        lib = _load()
+        rows = np.ascontiguousarray(rows, dtype=np.uint16)
+        if rows.ndim == 1:
+            rows = rows[None, :]
+        K, pitch = rows.shape
+        out = np.zeros(K, dtype=VERDICT_DTYPE)
+        lo = live.lo if len(live.lo) else np.zeros(1, np.uint32)
+        lib.vlo_verify_dict_rows(C.byref(self.c), _ptr(live.lo_off), _ptr(lo), _ptr(rows), K, pitch, _ptr(out))
         return out
 
     def violations(self, live: Liveness, row: np.ndarray) -> np.ndarray:

@@ -354,6 +354,74 @@ void vlo_occupied(const vlo_program *p, const uint64_t *lo_off, const uint32_t *
     free(T);
 }
 
+/* ------------------------------------------------- dictionary candidates */
+
+/*
+ * The model of the paper does not emit one register per operand occurrence: it emits, for every
+ * basic block, a dictionary from the block's virtual registers to physical registers (Section 3.1:
+ * the assignment is generated "per basic block" along the control-flow graph, as a JSON-style
+ * dictionary; Section 3.2: registers are renumbered per block, so the same virtual register shows
+ * up in the dictionaries of several blocks).  A candidate in that form is one 16-bit value per
+ * (block, virtual register occurring in the block).
+ *
+ * Layout of such a row (a reading: the paper fixes no order inside a dictionary): blocks in program
+ * order; inside a block its virtual registers in the order of their first occurrence in the block
+ * (definitions of an instruction before its reads).  vlo_dict_layout writes dict_off[n_blocks+1],
+ * and, per entry, the vreg and the first instruction of the block in which it occurs; it returns the
+ * number of entries (the arrays must hold n_operands entries at most).
+ *
+ * Meaning: every occurrence of v inside block b carries the register of entry (b, v).  The check is
+ * then the check of that per-occurrence assignment: Consistency compares the entries of one vreg
+ * across blocks (the entry of the lowest block that uses it is the table value; a differing entry is
+ * a violation reported at the first instruction of its block that touches the vreg), everything
+ * else follows from the table as before.
+ */
+uint32_t vlo_dict_layout(const vlo_program *p, uint32_t *dict_off, uint32_t *dict_vreg, uint32_t *entry_instr)
+{
+    uint32_t n = 0;
+    uint8_t *seen = malloc((size_t)p->n_vregs + 1);
+    for (uint32_t b = 0; b < p->n_blocks; ++b) {
+        dict_off[b] = n;
+        memset(seen, 0, (size_t)p->n_vregs + 1);
+        for (uint32_t i = p->block_instr_off[b]; i < p->block_instr_off[b + 1]; ++i)
+            for (uint32_t o = p->instr_op_off[i]; o < p->instr_op_off[i + 1]; ++o) {
+                uint32_t v = p->op_vreg[o];
+                if (seen[v]) continue;
+                seen[v] = 1;
+                dict_vreg[n] = v;
+                entry_instr[n] = i;
+                ++n;
+            }
+    }
+    dict_off[p->n_blocks] = n;
+    free(seen);
+    return n;
+}
+
+/* rows of dictionary candidates, pitch entries apart, checked one by one */
+void vlo_verify_dict_rows(const vlo_program *p, const uint64_t *lo_off, const uint32_t *lo,
+                          const uint16_t *rows, uint64_t K, uint64_t pitch, vlo_verdict *out)
+{
+    uint32_t *dict_off = malloc(((size_t)p->n_blocks + 1) * sizeof(uint32_t));
+    uint32_t *dict_vreg = malloc(((size_t)p->n_operands + 1) * sizeof(uint32_t));
+    uint32_t *entry_instr = malloc(((size_t)p->n_operands + 1) * sizeof(uint32_t));
+    uint16_t *occ = malloc(((size_t)p->n_operands + 1) * sizeof(uint16_t));
+    uint32_t *entry_of = malloc(((size_t)p->n_vregs + 1) * sizeof(uint32_t));
+    vlo_dict_layout(p, dict_off, dict_vreg, entry_instr);
+    for (uint64_t k = 0; k < K; ++k) {
+        const uint16_t *row = rows + k * pitch;
+        /* the per-occurrence assignment the dictionaries stand for */
+        for (uint32_t b = 0; b < p->n_blocks; ++b) {
+            for (uint32_t e = dict_off[b]; e < dict_off[b + 1]; ++e) entry_of[dict_vreg[e]] = e;
+            for (uint32_t i = p->block_instr_off[b]; i < p->block_instr_off[b + 1]; ++i)
+                for (uint32_t o = p->instr_op_off[i]; o < p->instr_op_off[i + 1]; ++o)
+                    occ[o] = row[entry_of[p->op_vreg[o]]];
+        }
+        walk(p, lo_off, lo, occ, out + k, NULL, NULL, 0, NULL, NULL);
+    }
+    free(entry_of); free(occ); free(entry_instr); free(dict_vreg); free(dict_off);
+}
+
 /* ------------------------------------------------- re-sampling statistics */
 
 /*

@@ -506,6 +506,45 @@ def candidate_rows(prog: Program, K: int, fault_rate: float, seed: int,
     return out, faults
 
 
+# ---------------------------------------------------- dictionary form of a candidate
+def dict_layout(prog: Program):
+    """The per-basic-block dictionary form of a candidate row (the form the paper's model emits: one
+    vreg -> register dictionary per basic block): one entry per (block, vreg occurring in the block),
+    blocks in program order, a block's vregs in the order of their first occurrence in the block.
+    Returns (dict_off u32 [n_blocks+1], dict_vreg u32 [n_entries], first_op i64 [n_entries]) where
+    first_op is the operand column of the entry's first occurrence in its block.  Input format only:
+    nothing of the check is computed here."""
+    opv = prog.op_vreg.astype(np.int64)
+    iop = prog.instr_op_off.astype(np.int64)
+    offs, vregs, firsts = [0], [], []
+    for b in range(prog.n_blocks):
+        o0, o1 = int(iop[int(prog.block_instr_off[b])]), int(iop[int(prog.block_instr_off[b + 1])])
+        seg = opv[o0:o1]
+        _, idx = np.unique(seg, return_index=True)
+        idx = np.sort(idx)
+        vregs.append(seg[idx])
+        firsts.append(idx + o0)
+        offs.append(offs[-1] + len(idx))
+    cat = (lambda xs, dt: np.concatenate(xs).astype(dt) if xs and sum(len(x) for x in xs) else np.zeros(0, dtype=dt))
+    return np.asarray(offs, dtype=np.uint32), cat(vregs, np.uint32), cat(firsts, np.int64)
+
+
+def dict_pitch(n_entries: int) -> int:
+    """Row pitch of dictionary rows in elements: the entry count rounded up to 8 (16-byte rows)."""
+    return max(8, (n_entries + 7) // 8 * 8)
+
+
+def dict_rows(prog: Program, rows: np.ndarray, layout=None) -> np.ndarray:
+    """Dictionary rows (uint16 [K, dict_pitch]) standing for per-occurrence rows: every entry takes
+    the register its vreg has at its first occurrence in the block.  (A per-occurrence row that is
+    inconsistent inside one block has no dictionary form; the entry then keeps the first value.)"""
+    _, vregs, first_op = layout if layout is not None else dict_layout(prog)
+    rows = np.atleast_2d(rows)
+    out = np.zeros((rows.shape[0], dict_pitch(len(vregs))), dtype=np.uint16)
+    out[:, : len(vregs)] = rows[:, first_op]
+    return out
+
+
 def _inject(prog: Program, seed: int, k: int, row: np.ndarray, tab: np.ndarray, rec: np.ndarray) -> None:
     g = prog.gen
     P = prog.P

@@ -40,6 +40,13 @@ MUTANTS = [
      "if (s < p->class_lo[c] || s + w > p->class_hi[c] + 1) unreal = 1;"),
     ("class lower bound dropped", "if (s < p->class_lo[c] || s + w > p->class_hi[c]) unreal = 1;",
      "if (s + w > p->class_hi[c]) unreal = 1;"),
+    ("dictionary entry reported at the first instruction of its block", "entry_instr[n] = i;",
+     "entry_instr[n] = p->block_instr_off[b];"),
+    ("every occurrence takes the entry of the last block that uses the vreg",
+     "for (uint32_t e = dict_off[b]; e < dict_off[b + 1]; ++e) entry_of[dict_vreg[e]] = e;",
+     "for (uint32_t e = 0; e < dict_off[p->n_blocks]; ++e) entry_of[dict_vreg[e]] = e;"),
+    ("a vreg gets a dictionary entry only in the first block that uses it", "memset(seen, 0, (size_t)p->n_vregs + 1);\n        for",
+     "if (b == 0) memset(seen, 0, (size_t)p->n_vregs + 1);\n        for"),
     ("reserved check leaves out the last register of a tuple", "for (uint32_t r = s; r < s + w && r < p->P; ++r)",
      "for (uint32_t r = s; r + 1 < s + w && r < p->P; ++r)"),
 ]

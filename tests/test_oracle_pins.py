@@ -586,3 +586,111 @@ def test_occupied_registers_from_path_liveness_and_the_safety_verdict(oracle_mod
         if single:
             assert clash == bool(op.verify(lv, row)[0]["flags"] & INTERF)
     assert single == (seed % 2 == 0)
+
+
+# ---------------------------------------------------------------- dictionary candidates
+def _expand_dict_row(p, drow):
+    """Per-occurrence row that a dictionary row stands for, by plain loops (independent of the oracle's
+    own expansion): every occurrence of v in block b takes the entry of (b, v); entries are laid out
+    block by block, a block's vregs in the order they first occur."""
+    row = np.zeros(p.pitch, dtype=np.uint16)
+    e = 0
+    for b in range(p.n_blocks):
+        slot = {}
+        i0, i1 = int(p.block_instr_off[b]), int(p.block_instr_off[b + 1])
+        for o in range(int(p.instr_op_off[i0]), int(p.instr_op_off[i1])):
+            v = int(p.op_vreg[o])
+            if v not in slot:
+                slot[v] = e
+                e += 1
+            row[o] = drow[slot[v]]
+    return row, e
+
+
+def test_dictionary_layout_hand_case(oracle_mod):
+    # block 0: v0 =; v1 = v0 ; block 1: v2 = v1, v0 ; v0 = v2 ; block 2: use v1
+    p = synth.program_from_lists([[([0], []), ([1], [0])], [([2], [1, 0]), ([0], [2])], [([], [1])]],
+                                 [(0, 1), (1, 1), (1, 2)], 3, [1, 1, 1], 8)
+    off, vreg, instr = oracle_mod.OracleProgram(p).dict_layout()
+    assert off.tolist() == [0, 2, 5, 6]
+    assert vreg.tolist() == [0, 1, 2, 1, 0, 1]          # block 1: the definition (v2) before the reads (v1, v0)
+    assert instr.tolist() == [0, 1, 2, 2, 2, 4]
+    soff, svreg, sfirst = synth.dict_layout(p)
+    assert soff.tolist() == off.tolist() and svreg.tolist() == vreg.tolist()
+    assert sfirst.tolist() == [0, 1, 3, 4, 5, 8]
+
+
+def test_dictionary_disagreement_between_blocks_hand_case(oracle_mod):
+    p = synth.program_from_lists([[([0], []), ([1], [0])], [([2], [1, 0]), ([0], [2])], [([], [1])]],
+                                 [(0, 1), (1, 1), (1, 2)], 3, [1, 1, 1], 8)
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    good = np.zeros(8, dtype=np.uint16)
+    good[:6] = [0, 1, 2, 1, 0, 1]                        # v0 -> 0, v1 -> 1, v2 -> 2 in every block
+    v = op.verify_dict(lv, good)[0]
+    assert (v["flags"], v["first_violation_instr"], v["conflict_pairs"]) == (PASS, -1, 0)
+    bad = good.copy()
+    bad[5] = 5                                           # block 2 says v1 -> 5: the table keeps block 0's value
+    w = op.verify_dict(lv, bad)[0]
+    assert w["flags"] == INCONS and w["first_violation_instr"] == 4
+    assert (w["conflict_pairs"], w["bank_conflicts"]) == (v["conflict_pairs"], v["bank_conflicts"])
+    bad2 = good.copy()
+    bad2[4] = 2                                          # block 1 says v0 -> 2 (= v2's register): still only inconsistent,
+    w2 = op.verify_dict(lv, bad2)[0]                     # because every later check uses the table value 0
+    assert w2["flags"] == INCONS and w2["first_violation_instr"] == 2
+    first = good.copy()
+    first[0] = 1                                         # block 0 (the table value) puts v0 on v1's register
+    w3 = op.verify_dict(lv, first)[0]
+    assert w3["flags"] & INCONS and w3["flags"] & INTERF
+    assert w3["first_violation_instr"] == 1              # v1 is written at instruction 1 while v0 (register 1) is live
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_dictionary_rows_equal_their_per_occurrence_expansion(oracle_mod, seed):
+    """A dictionary row means: every occurrence of v in block b has the register of entry (b, v).  Its
+    verdict must be that of the expanded per-occurrence row (expansion written out here by plain loops),
+    for consistent tables, for tables that disagree between blocks, and for garbage."""
+    p = H.random_program(7000 + seed, strict=True, reachable=(seed % 3 != 0), max_instrs=50, max_vregs=14,
+                         P=[8, 16, 32][seed % 3], widths=(1, 1, 2, 4), B=[4, 2, 3][seed % 3])
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    off, vreg, instr = op.dict_layout()
+    n = len(vreg)
+    soff, svreg, sfirst = synth.dict_layout(p)
+    assert np.array_equal(soff, off) and np.array_equal(svreg, vreg)
+    assert np.array_equal(np.searchsorted(p.instr_op_off, sfirst, side="right") - 1, instr)
+    rng = np.random.default_rng(seed)
+    rows = np.zeros((24, synth.dict_pitch(n)), dtype=np.uint16)
+    for k in range(24):
+        T = rng.integers(0, p.P + (4 if k % 4 == 3 else 0), size=p.n_vregs)
+        rows[k, :n] = T[vreg]                                           # every block agrees
+        if k % 3 == 1 and n:
+            rows[k, rng.integers(0, n, size=2)] = rng.integers(0, p.P, size=2)   # some blocks disagree
+        if k % 8 == 7:
+            rows[k, :n] = rng.integers(0, 65536, size=n)
+    got = op.verify_dict(lv, rows)
+    for k in range(24):
+        exp, used = _expand_dict_row(p, rows[k])
+        assert used == n
+        want = op.verify(lv, exp)[0]
+        assert got[k].tobytes() == want.tobytes(), (seed, k)
+        if k % 3 == 0 and k % 8 != 7:                                    # a consistent table: the row of that table
+            T = {int(v): int(rows[k, e]) for e, v in enumerate(vreg)}
+            tab = [T.get(v, 0) for v in range(p.n_vregs)]
+            assert got[k].tobytes() == op.verify(lv, H.row_from_table(p, tab))[0].tobytes()
+
+
+def test_dictionary_form_of_generator_rows(oracle_mod):
+    """Generator rows in dictionary form: valid rows pass; a row with a vreg moved (interference or
+    out-of-file fault: every occurrence moved, so every block's entry moved) keeps its verdict."""
+    wl = synth.workload(1)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    op = oracle_mod.OracleProgram(p)
+    lv = op.liveness()
+    rows, faults = synth.candidate_rows(p, 120, 0.4, 9)
+    per_occ = op.verify(lv, rows)
+    got = op.verify_dict(lv, synth.dict_rows(p, rows))
+    keep = faults[:, 0] != synth.FAULT_INCONSISTENT
+    assert keep.sum() > 60 and (~keep).sum() > 5
+    assert got[keep].tobytes() == per_occ[keep].tobytes()
+    assert np.all(got["flags"][faults[:, 0] == synth.FAULT_NONE] == PASS)
