@@ -174,6 +174,32 @@ int vl_verify(vl_program *prog, const uint16_t *d_cand, uint64_t K, uint64_t pit
               vl_verdict *d_out, void *cuda_stream);
 
 /*
+ * Candidates in the form the paper's model emits them (Section 3.1: the allocation is generated per
+ * basic block, as a dictionary from the block's virtual registers to physical registers; Section 3.2:
+ * registers are renumbered per basic block, so one virtual register appears in the dictionaries of
+ * every block that uses it).  A dictionary row holds one uint16 per (block, vreg occurring in the
+ * block): blocks in program order, the vregs of a block in the order of their first occurrence in it
+ * (definitions of an instruction before its reads; the paper fixes no order, this is the library's).
+ * vl_dict_layout gives the layout: *n_entries columns, dict_off[n_blocks + 1] (first column of every
+ * block) and dict_vreg[n_entries]; the arrays are HOST memory owned by the handle, valid until
+ * vl_program_destroy.  Any out pointer may be NULL.
+ */
+int vl_dict_layout(const vl_program *prog, uint32_t *n_entries, const uint32_t **dict_off, const uint32_t **dict_vreg);
+
+/*
+ * vl_verify for K dictionary rows: d_dict[k * pitch_elems + e] is the register row k gives to
+ * column e of the layout above (DEVICE memory, base 16-byte aligned, pitch_elems % 8 == 0 and at
+ * least n_entries rounded up to 8).  Meaning: every occurrence of v inside block b carries the
+ * register of column (b, v), and the row is checked as that per-occurrence assignment.  The table
+ * value T[v] is the entry of the lowest block that uses v; Consistency (Section 3.4) compares the
+ * entries of one vreg across blocks, and a differing entry is reported at the first instruction of
+ * its block that touches the vreg; Realizability, Safety and the bank tally follow from T as in
+ * vl_verify.  Same stream ordering, host work, limits and errors as vl_verify.
+ */
+int vl_verify_dict(vl_program *prog, const uint16_t *d_dict, uint64_t K, uint64_t pitch_elems, vl_verdict *d_out,
+                   void *cuda_stream);
+
+/*
  * The same check for n independent programs in one call (all on the device of the
  * first program): program j checks K[j] rows of d_cand[j] into d_out[j].  The arrays of
  * pointers and sizes are HOST memory.  Stream-ordered, no synchronisation.

@@ -31,7 +31,8 @@ VL_OPT_PREFETCH_TILES = 8
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",
            "vl_kernel_launches", "vl_kernel_times", "vl_last_cuda_error", "vl_strerror", "vl_block_liveness_static",
-           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints", "vl_diagnose", "vl_occupied_masks"]
+           "vl_resample_stats", "vl_verify_until_pass", "vl_program_set_constraints", "vl_diagnose", "vl_occupied_masks",
+           "vl_dict_layout", "vl_verify_dict"]
 
 VERDICT_DTYPE = np.dtype([("flags", "<u4"), ("first_violation_instr", "<i4"),
                           ("conflict_pairs", "<u4"), ("bank_conflicts", "<u4")])
@@ -58,6 +59,10 @@ _lib.vl_liveness_batch.restype = C.c_int
 _lib.vl_liveness_batch.argtypes = [C.c_uint32, C.c_void_p, C.c_void_p]
 _lib.vl_liveness_result.restype = C.c_int
 _lib.vl_liveness_result.argtypes = [C.c_void_p] + [C.POINTER(C.c_void_p)] * 4 + [C.POINTER(C.c_uint64)]
+_lib.vl_verify_dict.restype = C.c_int
+_lib.vl_verify_dict.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+_lib.vl_dict_layout.restype = C.c_int
+_lib.vl_dict_layout.argtypes = [C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]
 _lib.vl_verify.restype = C.c_int
 _lib.vl_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
 _lib.vl_verify_batch.restype = C.c_int
@@ -233,6 +238,27 @@ class Program:
         if out is None:
             out = torch.empty((K, 4), dtype=torch.int32, device=cand.device)
         self._check(_lib.vl_verify(self._h, cand.data_ptr(), K, pitch, out.data_ptr(), _stream_ptr(stream)), "vl_verify")
+        return out
+
+    def vl_dict_layout(self):
+        """(dict_off [n_blocks+1], dict_vreg [n_entries]) of rows in dictionary form, as numpy copies."""
+        n = C.c_uint32(0)
+        off, vreg = C.c_void_p(), C.c_void_p()
+        self._check(_lib.vl_dict_layout(self._h, C.byref(n), C.byref(off), C.byref(vreg)), "vl_dict_layout")
+        d_off = np.ctypeslib.as_array(C.cast(off, C.POINTER(C.c_uint32)), shape=(self.n_blocks + 1,)).copy()
+        d_vreg = (np.ctypeslib.as_array(C.cast(vreg, C.POINTER(C.c_uint32)), shape=(n.value,)).copy()
+                  if n.value else np.zeros(0, dtype=np.uint32))
+        return d_off, d_vreg
+
+    def vl_verify_dict(self, rows, out=None, stream=None):
+        """rows: CUDA uint16 tensor [K, pitch] of dictionary rows; returns a CUDA int32 tensor [K, 4]."""
+        import torch
+        assert rows.is_cuda and rows.dtype in (torch.uint16, torch.int16) and rows.dim() == 2 and rows.is_contiguous()
+        K, pitch = rows.shape
+        if out is None:
+            out = torch.empty((K, 4), dtype=torch.int32, device=rows.device)
+        self._check(_lib.vl_verify_dict(self._h, rows.data_ptr(), K, pitch, out.data_ptr(), _stream_ptr(stream)),
+                    "vl_verify_dict")
         return out
 
     def vl_verify_host(self, cand: "np.ndarray | object", out: np.ndarray | None = None, stream=None):

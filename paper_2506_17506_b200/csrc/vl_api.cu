@@ -134,6 +134,54 @@ extern "C" int vl_program_create(const vl_program_desc *d, int device, vl_progra
         }
         if (e == cudaSuccess) e = upload(&p->d_bank_list, all.data(), all.size());
     }
+    {   // The dictionary form of a candidate row (Section 3.1: one vreg -> register dictionary per basic
+        // block): one entry per (block, vreg occurring in the block), blocks in order, a block's vregs
+        // in order of first occurrence.  The operand tables of the table kernels, for rows in that
+        // form: vreg of every entry, first-entry bits (the entry of the lowest block that uses the
+        // vreg gives the table value), and the instruction a differing entry is reported at.
+        std::vector<uint32_t> dict_instr;
+        std::vector<uint32_t> stamp(p->V ? p->V : 1, 0xFFFFFFFFu);
+        std::vector<uint8_t> has_entry(p->V ? p->V : 1, 0);
+        std::vector<uint8_t> is_first;
+        p->h_dict_off.assign(1, 0u);
+        for (uint32_t b = 0; b < p->nB; ++b) {
+            for (uint32_t i = d->block_instr_off[b]; i < d->block_instr_off[b + 1]; ++i)
+                for (uint32_t o = d->instr_op_off[i]; o < d->instr_op_off[i + 1]; ++o) {
+                    const uint32_t v = d->op_vreg[o];
+                    if (stamp[v] == b) continue;
+                    stamp[v] = b;
+                    p->h_dict_vreg.push_back(v);
+                    dict_instr.push_back(i);
+                    is_first.push_back(has_entry[v] ? 0 : 1);
+                    has_entry[v] = 1;
+                }
+            p->h_dict_off.push_back((uint32_t)p->h_dict_vreg.size());
+        }
+        p->nD = (uint32_t)p->h_dict_vreg.size();
+        p->nD8 = std::max(8u, (p->nD + 7) / 8 * 8);
+        p->nDT = (p->nD8 + 4095u) / 4096u * 4096u + 4096u;
+        std::vector<uint16_t> v16((size_t)p->nD8 + 8, (uint16_t)p->V);
+        std::vector<uint64_t> slot((size_t)p->nD8 / 8, 0);
+        std::vector<uint4> off((size_t)p->nDT / 4, make_uint4(p->V * 16u, p->V * 16u, p->V * 16u, p->V * 16u));
+        std::vector<uint8_t> f4((size_t)p->nDT / 4, 0);
+        dict_instr.resize(p->nD8, 0);
+        for (uint32_t e2 = 0; e2 < p->nD8; ++e2) {
+            if (e2 < p->nD) {
+                const uint32_t v = p->h_dict_vreg[e2];
+                v16[e2] = (uint16_t)v;
+                uint32_t *w = &off[e2 / 4].x;
+                w[e2 % 4] = v * 16u;
+                if (is_first[e2]) { slot[e2 / 8] |= 1ull << (e2 % 8); f4[e2 / 4] |= (uint8_t)(1u << (e2 % 4)); }
+            } else {
+                slot[e2 / 8] |= 1ull << (e2 % 8);  // padding column: writes the spare table entry, never compared
+            }
+        }
+        if (e == cudaSuccess) e = upload(&p->d_dict_vreg16, v16.data(), v16.size());
+        if (e == cudaSuccess) e = upload(&p->d_dict_slotmeta, slot.data(), slot.size());
+        if (e == cudaSuccess) e = upload(&p->d_dict_opoff, off.data(), off.size());
+        if (e == cudaSuccess) e = upload(&p->d_dict_first4, f4.data(), f4.size());
+        if (e == cudaSuccess) e = upload(&p->d_dict_instr, dict_instr.data(), dict_instr.size());
+    }
     if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_status, 64);
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 64);
     if (e != cudaSuccess) {
@@ -181,6 +229,8 @@ extern "C" void vl_program_destroy(vl_program *p)
     cudaFree(p->d_blk_off); cudaFree(p->d_succ_off); cudaFree(p->d_succ); cudaFree(p->d_op_off);
     cudaFree(p->d_ndefs); cudaFree(p->d_op_vreg); cudaFree(p->d_width); cudaFree(p->d_status);
     cudaFree(p->d_bank_list);
+    cudaFree(p->d_dict_vreg16); cudaFree(p->d_dict_slotmeta); cudaFree(p->d_dict_opoff); cudaFree(p->d_dict_first4);
+    cudaFree(p->d_dict_instr);
     cudaFree(p->d_vcons); cudaFree(p->d_rs_prefix);
     for (auto &v : p->vs) { cudaFree(v.tg); cudaFree(v.cstate); cudaFree(v.anom); cudaFree(v.work); cudaFree(v.racc); cudaFree(v.grp_done); cudaFree(v.thm); }
     for (int j = 0; j < 2; ++j) {
@@ -379,6 +429,29 @@ extern "C" int vl_verify(vl_program *p, const uint16_t *d_cand, uint64_t K, uint
     rc = vl_verify_lanes(1, &p, &d_cand, &K, &pitch, &d_out, (cudaStream_t)stream);
     // a repeated liveness run may still be in flight: the kernels above are ordered behind it on the
     // stream; its outcome is checked here, after they have been enqueued
+    const int rl = vl_live_settle(p);
+    return rc != VL_OK ? rc : rl;
+}
+
+extern "C" int vl_dict_layout(const vl_program *p, uint32_t *n_entries, const uint32_t **dict_off, const uint32_t **dict_vreg)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    if (n_entries) *n_entries = p->nD;
+    if (dict_off) *dict_off = p->h_dict_off.data();
+    if (dict_vreg) *dict_vreg = p->h_dict_vreg.data();
+    return VL_OK;
+}
+
+extern "C" int vl_verify_dict(vl_program *p, const uint16_t *d_dict, uint64_t K, uint64_t pitch, vl_verdict *d_out,
+                              void *stream)
+{
+    if (!p) return VL_ERR_INVALID_ARG;
+    if (!p->live_ok) return VL_ERR_LIVENESS_NOT_RUN;
+    if (K == 0) return VL_OK;
+    if (!d_dict || !d_out || ((uintptr_t)d_dict & 15) || ((uintptr_t)d_out & 3)) return VL_ERR_INVALID_ARG;
+    if (pitch % 8 != 0 || pitch < p->nD8 || K > 0x7FFFFFFFull) return VL_ERR_INVALID_ARG;
+    if (cudaSetDevice(p->device) != cudaSuccess) return VL_ERR_CUDA;
+    int rc = vl_verify_lanes(1, &p, &d_dict, &K, &pitch, &d_out, (cudaStream_t)stream, true);
     const int rl = vl_live_settle(p);
     return rc != VL_OK ? rc : rl;
 }

@@ -98,6 +98,15 @@ struct vl_program {
     // tables consumed by the verify kernels
     uint16_t *d_vreg16 = nullptr;           // [nOp8 + 8] vreg id per operand (padding operands: id V)
     uint64_t *d_slotmeta = nullptr;         // [nOp8 / 8] per 8 operands: first-occurrence bits, bank compare masks
+    // the same tables for rows in dictionary form (one column per (block, vreg of the block)); made once,
+    // when the handle is created
+    uint32_t nD = 0, nD8 = 0, nDT = 0;  // entries; rounded up to 8 (at least 8); to whole tiles plus one
+    std::vector<uint32_t> h_dict_off, h_dict_vreg;
+    uint16_t *d_dict_vreg16 = nullptr;
+    uint64_t *d_dict_slotmeta = nullptr;
+    uint4 *d_dict_opoff = nullptr;
+    uint8_t *d_dict_first4 = nullptr;
+    uint32_t *d_dict_instr = nullptr;     // [nD8] first instruction of the entry's block that touches its vreg
     uint4 *d_opoff = nullptr;               // [nOpT / 4] per 4 operands: byte offsets of their vregs' 16-byte table entries
     uint8_t *d_first4 = nullptr;            // [nOpT / 4] per 4 operands: first-occurrence bits
     uint8_t *d_opflags = nullptr;           // [nO]
@@ -195,9 +204,9 @@ extern std::atomic<uint64_t> g_vl_launches;
 
 int vl_liveness_impl(vl_program *p, cudaStream_t st);
 int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
-                   cudaStream_t st, int slot);
+                   cudaStream_t st, int slot, bool dict = false);
 int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
-                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st);
+                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st, bool dict = false);
 // The lane streams of the handle's device (created once per device; two side streams for liveness
 // follow the VL_LANES lanes in the array) and the handle's fork / join events.
 int vl_lane_streams(vl_program *p, cudaStream_t **lanes);

@@ -59,6 +59,9 @@ struct TParams {
     // their first-occurrence bits
     const uint4 *opoff;
     const uint8_t *first4;
+    // dictionary rows: the instruction a Consistency violation of entry e is reported at (null: the rows
+    // hold one column per operand, and the instruction is the one the operand belongs to)
+    const uint32_t *entry_instr;
     uint32_t *grp_flag;   // per group of 32 candidates: some table entry carries the straddle mark
     uint32_t test_wait;   // test hook: the wait for tile 0 polls a barrier nothing completes, with a short limit
     uint32_t pf;          // tiles asked into L2 ahead of the copy ring
@@ -547,7 +550,11 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
-        if (M->minop[g] != 0xFFFFFFFFu) {  // operand -> instruction: last i with op_off[i] <= operand
+        if (M->minop[g] != 0xFFFFFFFFu && q.entry_instr) {
+            // dictionary rows: entries are in block order and, inside a block, in order of first
+            // occurrence, so the lowest violating entry is also the lowest violating instruction
+            first = q.entry_instr[M->minop[g]];
+        } else if (M->minop[g] != 0xFFFFFFFFu) {  // operand -> instruction: last i with op_off[i] <= operand
             const uint32_t o = M->minop[g];
             uint32_t lo_i = 0, hi_i = q.nI;  // invariant: op_off[lo_i] <= o < op_off[hi_i]
             while (hi_i - lo_i > 1) {
@@ -1025,7 +1032,11 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
-        if (M->minop[g] != 0xFFFFFFFFu) {  // operand -> instruction: last i with op_off[i] <= operand
+        if (M->minop[g] != 0xFFFFFFFFu && q.entry_instr) {
+            // dictionary rows: entries are in block order and, inside a block, in order of first
+            // occurrence, so the lowest violating entry is also the lowest violating instruction
+            first = q.entry_instr[M->minop[g]];
+        } else if (M->minop[g] != 0xFFFFFFFFu) {  // operand -> instruction: last i with op_off[i] <= operand
             const uint32_t o = M->minop[g];
             uint32_t lo_i = 0, hi_i = q.nI;  // invariant: op_off[lo_i] <= o < op_off[hi_i]
             while (hi_i - lo_i > 1) {
@@ -2021,8 +2032,10 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
 
 // One pass: the four kernels over n <= sub candidates, in order on `st`, with working set `slot`.
 int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t n, uint64_t pitch, vl_verdict *d_out,
-             cudaStream_t st, int slot)
+             cudaStream_t st, int slot, bool dict)
 {
+    // what the rows hold: one column per operand occurrence, or one per dictionary entry
+    const uint32_t nO = dict ? p->nD : p->nO, nOp8 = dict ? p->nD8 : p->nOp8;
     const Plan &pl = pp.pl;
     int rc = ensure_scratch(p, slot, pp.sub);
     if (rc != VL_OK) return rc;
@@ -2031,10 +2044,12 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     const uint32_t ngrp = (uint32_t)((n + TGW - 1) / TGW);
 
     TParams tq{};
-    tq.nI = p->nI; tq.V = p->V; tq.nO = p->nO; tq.nOp8 = p->nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
-    tq.ntiles = (p->nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
+    tq.nI = p->nI; tq.V = p->V; tq.nO = nO; tq.nOp8 = nOp8; tq.P = p->P; tq.Bmask = p->B - 1;
+    tq.ntiles = (nOp8 + pl.NT * 8 - 1) / (pl.NT * 8);
     tq.bank_fast = p->bank_fast;
-    tq.vreg16 = p->d_vreg16; tq.slotmeta = p->d_slotmeta; tq.vinfo = p->d_vinfo;
+    tq.vreg16 = dict ? p->d_dict_vreg16 : p->d_vreg16; tq.slotmeta = dict ? p->d_dict_slotmeta : p->d_slotmeta;
+    tq.vinfo = p->d_vinfo;
+    tq.entry_instr = dict ? p->d_dict_instr : nullptr;
     tq.first_def_instr = p->d_first_def_instr; tq.op_off = p->d_op_off;
     tq.bank_list = p->d_bank_list;
     for (int j = 0; j < 4; ++j) tq.bank_seg[j] = p->bank_seg[j];
@@ -2045,15 +2060,15 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.NS = pl.NS; tq.off_region = pl.off_region; tq.off_misc = pl.off_misc;
     tq.AW = (uint32_t)vs.aw; tq.anom = vs.anom; tq.racc = vs.racc; tq.grp_done = vs.grp_done; tq.work = vs.work;
     tq.vcons = p->d_vcons; tq.rs_prefix = p->d_rs_prefix;
-    tq.opoff = p->d_opoff; tq.first4 = p->d_first4;
+    tq.opoff = dict ? p->d_dict_opoff : p->d_opoff; tq.first4 = dict ? p->d_dict_first4 : p->d_first4;
     tq.grp_flag = vs.grp_done + (vs.rows / TGW + 1);
     tq.test_wait = p->test_wait;
     tq.pf = p->prefetch_tiles;
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
     if (pl.G == 8) {
-        tq.ntiles = (p->nOp8 + pl.NT * 4 - 1) / (pl.NT * 4);
-        tq.nfull = p->nOp8 / 256;
+        tq.ntiles = (nOp8 + pl.NT * 4 - 1) / (pl.NT * 4);
+        tq.nfull = nOp8 / 256;
         tq.tail_start = tq.nfull * 256;
         tq.tail_tile = tq.tail_start / (pl.NT * 4);
         tq.off_tail = pl.off_tail;
@@ -2139,13 +2154,13 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
 
 // All passes in order on one stream, with one working set.
 int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t pitch, vl_verdict *d_out,
-                   cudaStream_t st, int slot)
+                   cudaStream_t st, int slot, bool dict)
 {
     PassPlan pp{};
     int rc = plan_passes(p, K, &pp);
     if (rc != VL_OK) return rc;
     for (uint64_t kb = 0; kb < K; kb += pp.sub) {
-        rc = run_pass(p, pp, d_cand + kb * pitch, std::min(pp.sub, K - kb), pitch, d_out + kb, st, slot);
+        rc = run_pass(p, pp, d_cand + kb * pitch, std::min(pp.sub, K - kb), pitch, d_out + kb, st, slot, dict);
         if (rc != VL_OK) return rc;
     }
     return VL_OK;
@@ -2156,7 +2171,7 @@ int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t p
 // instruction issue).  Pass j of a program uses working set j mod lanes and runs on lane
 // (first_lane + j) mod lanes: two passes that share a working set are ordered by their stream.
 int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *const *d_cand, const uint64_t *K,
-                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st)
+                    const uint64_t *pitch, vl_verdict *const *d_out, cudaStream_t st, bool dict)
 {
     vl_program *p0 = progs[0];
     cudaStream_t *lane = nullptr;
@@ -2169,7 +2184,7 @@ int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *co
     if (L == 1 || jobs <= 1) {
         for (uint32_t j = 0; j < nprog; ++j) {
             if (K[j] == 0) continue;
-            rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], st, 0);
+            rc = vl_verify_impl(progs[j], d_cand[j], K[j], pitch[j], d_out[j], st, 0, dict);
             if (rc != VL_OK) return rc;
         }
         return VL_OK;
@@ -2188,7 +2203,7 @@ int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *co
         uint64_t s = 0;
         for (uint64_t kb = 0; kb < K[j] && rc == VL_OK; kb += pp.sub, ++s, ++job)
             rc = run_pass(p, pp, d_cand[j] + kb * pitch[j], std::min(pp.sub, K[j] - kb), pitch[j], d_out[j] + kb,
-                          lane[(base + s) % L], (int)(s % L));
+                          lane[(base + s) % L], (int)(s % L), dict);
     }
     // join even after an error, so that the caller's stream stays ordered after what was launched
     for (uint32_t l = 0; l < L; ++l) {
