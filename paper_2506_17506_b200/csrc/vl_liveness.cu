@@ -538,48 +538,40 @@ __global__ void k_operand_meta(uint32_t nI, const uint32_t *__restrict__ op_off,
 
 // Per 8 operands: bits 0..7 first occurrence; for d = 1..3 a 16-bit field at 8 + 16 (d-1) with
 // bit 2 j set when operand j compares its bank with the operand d places before it.
-__global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t V, const uint8_t *__restrict__ opmeta,
-                             uint16_t *vreg16, uint64_t *slotmeta)
+// Also the operand metadata of the eight-candidate table kernel, per four operands: the byte offsets
+// of the vregs' 16-byte table entries and a nibble of first-occurrence bits; there, operands beyond
+// n_operands (the arrays are padded to whole tiles) name the spare entry V and are never a first
+// occurrence.  One thread per 8 operands of the padded arrays.
+__global__ void k_pack_slots(uint32_t nO, uint32_t nOp8, uint32_t n_slots_padded, uint32_t V,
+                             const uint8_t *__restrict__ opmeta, uint16_t *vreg16, uint64_t *slotmeta, uint4 *opoff,
+                             uint8_t *first4)
 {
     const uint32_t s = blockIdx.x * NT + threadIdx.x;
-    if (s >= nOp8 / 8) return;
+    if (s >= n_slots_padded) return;
     uint64_t m = 0;
+    uint32_t off[8], f = 0;
     for (uint32_t j = 0; j < 8; ++j) {
         const uint32_t o = s * 8 + j;
+        off[j] = V * 16u;
         if (o >= nO) {
-            vreg16[o] = (uint16_t)V;  // padding operand: writes the spare table entry, never compared
-            m |= 1ull << j;
+            if (o < nOp8) {
+                vreg16[o] = (uint16_t)V;  // padding operand: writes the spare table entry, never compared
+                m |= 1ull << j;
+            }
             continue;
         }
+        off[j] = (uint32_t)vreg16[o] * 16u;
         const uint8_t x = opmeta[o];
-        if (x & 1) m |= 1ull << j;
+        if (x & 1) { m |= 1ull << j; f |= 1u << j; }
         if (x & 2) m |= 1ull << (8 + 2 * j);
         if (x & 4) m |= 1ull << (24 + 2 * j);
         if (x & 8) m |= 1ull << (40 + 2 * j);
     }
-    slotmeta[s] = m;
-}
-
-// Operand metadata of the eight-candidate table kernel, per four operands: the byte offsets of the
-// vregs' 16-byte table entries and a nibble of first-occurrence bits.  Operands beyond n_operands
-// (the arrays are padded to whole tiles) name the spare entry V and are never a first occurrence.
-__global__ void k_meta8(uint32_t nO, uint32_t n_quads, uint32_t V, const uint16_t *__restrict__ vreg16,
-                        const uint64_t *__restrict__ slotmeta, uint4 *opoff, uint8_t *first4)
-{
-    const uint32_t qd = blockIdx.x * NT + threadIdx.x;
-    if (qd >= n_quads) return;
-    uint32_t off[4], f = 0;
-    for (uint32_t j = 0; j < 4; ++j) {
-        const uint32_t o = qd * 4 + j;
-        uint32_t v = V;
-        if (o < nO) {
-            v = vreg16[o];
-            if ((slotmeta[o >> 3] >> (o & 7)) & 1ull) f |= 1u << j;
-        }
-        off[j] = v * 16u;
-    }
-    opoff[qd] = make_uint4(off[0], off[1], off[2], off[3]);
-    first4[qd] = (uint8_t)f;
+    if (s < nOp8 / 8) slotmeta[s] = m;
+    opoff[2 * s] = make_uint4(off[0], off[1], off[2], off[3]);
+    opoff[2 * s + 1] = make_uint4(off[4], off[5], off[6], off[7]);
+    first4[2 * s] = (uint8_t)(f & 15u);
+    first4[2 * s + 1] = (uint8_t)(f >> 4);
 }
 
 // Walk events are stored in groups of 8, 112 bytes per group, field by field so that the walk
@@ -923,9 +915,8 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, sa, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
     LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
            p->d_opflags, p->d_vreg16, opmeta, p->d_status);
-    LAUNCH(k_pack_slots, (p->nOp8 / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, V, opmeta, p->d_vreg16, p->d_slotmeta);
-    LAUNCH(k_meta8, (p->nOpT / 4 + NT - 1) / NT, 0, sa, nO, p->nOpT / 4, V, p->d_vreg16, p->d_slotmeta, p->d_opoff,
-           p->d_first4);
+    LAUNCH(k_pack_slots, (p->nOpT / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, p->nOpT / 8, V, opmeta, p->d_vreg16, p->d_slotmeta,
+           p->d_opoff, p->d_first4);
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     LAUNCH(k_fill_events, nC, 0, sb, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
            p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev, p->d_chunk_blk, p->d_el,

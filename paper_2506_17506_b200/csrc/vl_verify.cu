@@ -1340,12 +1340,45 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 3) k_walk(const WParams q)
     // no table entry of the group carries the straddle mark: the walk decides nothing per event
     const bool marked = __ldcg(q.grp_flag + grp) != 0;
     if (c < q.nC) {
-        // the chunk starts from the through-set masks of its block
-        if (q.use_th) {
+        // the chunk starts from the through-set masks of its block: made by k_through, or (small jobs,
+        // where one launch more costs more than the repeated work) by this warp on the spot
+        if (q.use_th && q.thm) {
             const uint32_t *src = q.thm + ((size_t)grp * q.nB + q.chunk_blk[c]) * q.Wp * 64;
             for (uint32_t wd = 0; wd < q.Wp * 2; ++wd) s_occ[wd * 32 + lane] = src[wd * 32 + lane];
         } else {
             for (uint32_t wd = 0; wd < q.Wp * 2; ++wd) s_occ[wd * 32 + lane] = 0;
+        }
+        if (q.use_th && !q.thm) {
+            const uint32_t b = q.chunk_blk[c];
+            bool thcolA = false, thcolB = false;
+            const uint32_t e1 = q.th_off[b + 1];
+            for (uint32_t e0 = q.th_off[b]; e0 < e1; e0 += 8) {  // the table entries of 8 members in flight together
+                uint32_t x[8], t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) x[u] = e0 + u < e1 ? q.th[e0 + u] : (q.V | (0u << 16));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t[u] = *reinterpret_cast<const uint32_t *>(tgb + (size_t)(x[u] & 0xFFFFu) * (TGW * 2));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (!(h ? walkedB : walkedA)) continue;
+                        uint32_t pos = (h ? (t[u] >> 16) : t[u]) & 0x7FFFu, left = x[u] >> 16;
+                        while (left) {
+                            const uint32_t s2 = pos & 31, n = min(left, 32 - s2);
+                            const uint32_t m = (n == 32 ? 0xFFFFFFFFu : ((1u << n) - 1u)) << s2;
+                            uint32_t *a = &s_occ[((pos >> 5) * 2 + h) * 32 + lane];
+                            const uint32_t old = *a;
+                            *a = old | m;
+                            if (h) thcolB |= (old & m) != 0; else thcolA |= (old & m) != 0;
+                            pos += n;
+                            left -= n;
+                        }
+                    }
+                }
+            }
+            if (thcolA) atomicOr(&csA[CS_THCOL], 1u << b);  // through-sets are used only if nB <= 32
+            if (thcolB) atomicOr(&csB[CS_THCOL], 1u << b);
         }
         uint32_t violA = 0, violB = 0;
         const uint32_t s0 = q.cev_off[c], n_ev = q.cev_off[c + 1] - s0;  // a multiple of 8 events
@@ -2099,13 +2132,15 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
         wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = pp.Wp; wq.AW = (uint32_t)vs.aw;
         wq.use_th = (uint32_t)p->use_th; wq.K = n;
         wq.th_off = p->d_th_off; wq.th = p->d_th; wq.cev_off = p->d_cev_off; wq.ev = p->d_ev;
-        wq.thm = vs.thm;
+        // the through-set masks come from a kernel of their own, except for small jobs
+        const bool own_through = p->use_th && n >= 512;
+        wq.thm = own_through ? vs.thm : nullptr;
         wq.tg = vs.tg; wq.ev_cap = pp.ev_cap; wq.wmax = p->wmax;
         wq.cstate = vs.cstate; wq.anom = vs.anom;
         wq.grp_flag = vs.grp_done + (vs.rows / TGW + 1);
         wq.list_all = p->bank_fast ? 0 : 1; wq.chunk_blk = p->d_chunk_blk;
         wq.grp_done = vs.grp_done; wq.work = vs.work; wq.racc = vs.racc; wq.out = d_out;
-        if (p->use_th) {
+        if (own_through) {
             k_through<<<dim3(p->nB, ngrp), 256, pp.Wp * 64 * 4, st>>>(wq);
             e = cudaGetLastError();
             if (e != cudaSuccess) { p->last_cuda_error = (int)e; return VL_ERR_CUDA; }

@@ -12,7 +12,8 @@ and vl_verify_batch.  Also per workload: the time of one vl_resample_stats call 
 arrays (launch-latency bound: three or more small kernels), the statistics it returns (test cases
 solved, attempts summed and largest, Pass@1/10/100 counts), and the time of the early-exit loop
 vl_verify_until_pass in batches of 100 rows (it stops after the first batch with a passing row),
-and the times of vl_diagnose and vl_occupied_masks on one row.
+and the times of vl_diagnose and vl_occupied_masks on one row, and vl_verify_dict over the rows of the
+first program in dictionary form (its algorithmic bytes are 2 bytes per dictionary column + the verdict).
 """
 from __future__ import annotations
 
@@ -152,6 +153,21 @@ def main() -> int:
             occupied()
         eo[1].record(stream)
         torch.cuda.synchronize()
+        # the same candidates in dictionary form (one column per (block, vreg of the block)): first program
+        layout = synth.dict_layout(progs[0])
+        d_host = synth.dict_rows(progs[0], cands[0].cpu().numpy().view(np.uint16), layout)
+        d_rows = torch.from_numpy(d_host.view(np.int16)).cuda().view(torch.uint16)
+        d_out = torch.empty((wl.K, 4), dtype=torch.int32, device="cuda")
+        for _ in range(3):
+            gps[0].vl_verify_dict(d_rows, d_out, stream)
+        edd = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        edd[0].record(stream)
+        for _ in range(args.steps):
+            gps[0].vl_verify_dict(d_rows, d_out, stream)
+        edd[1].record(stream)
+        torch.cuda.synchronize()
+        dict_ms = edd[0].elapsed_time(edd[1]) / args.steps
+        dict_bytes = (2 * d_host.shape[1] + 16) * wl.K
         occupied_us = eo[0].elapsed_time(eo[1]) / args.steps * 1e3
         diagnose_us = ed[0].elapsed_time(ed[1]) / args.steps * 1e3
         resample_us = er[0].elapsed_time(er[1]) / args.steps * 1e3
@@ -176,6 +192,10 @@ def main() -> int:
             "until_pass_first_passing_row": first_pass,
             "diagnose_one_row_us": diagnose_us,
             "occupied_masks_one_row_us": occupied_us,
+            "dict_form_first_program": {"columns": int(len(layout[1])), "verify_dict_ms": dict_ms,
+                                        "verifications_per_sec": wl.K / (dict_ms * 1e-3),
+                                        "gb_per_sec": dict_bytes / (dict_ms * 1e-3) / 1e9,
+                                        "frac_of_measured_copy_peak": dict_bytes / (dict_ms * 1e-3) / 1e9 / peak},
         }), flush=True)
         for gp in gps:
             gp.close()
