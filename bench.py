@@ -233,6 +233,7 @@ def main():
     ap.add_argument("--lanes", type=int, default=0, help="internal streams of vl_verify (default: the library's)")
     ap.add_argument("--sub-batch", type=int, default=0, help="candidates per pass (default: the library's)")
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--stagger", type=int, default=-1, help="start offset (us) between the classes of the first wave of the table kernel")
     ap.add_argument("--threads", type=int, default=0, help="threads per block of the table kernel (default: the library's)")
     ap.add_argument("--prefetch", type=int, default=-1, help="tiles the table kernel asks into L2 ahead (default: the library's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -269,6 +270,8 @@ def main():
         gp.set_option(vl.VL_OPT_SUB_BATCH, args.sub_batch)
     if args.threads:
         gp.set_option(vl.VL_OPT_THREADS, args.threads)
+    if args.stagger >= 0:
+        gp.set_option(vl.VL_OPT_STAGGER_US, args.stagger)
     if args.prefetch >= 0:
         gp.set_option(vl.VL_OPT_PREFETCH_TILES, args.prefetch)
     dev_rows = host.cuda().view(torch.uint16)

@@ -54,6 +54,9 @@ enum {
                                 option of its first program: 1 = in order, anything else = all 8 streams */
     VL_OPT_PREFETCH_TILES = 8, /* tiles of the candidate rows that the table kernel (8 candidates per block) asks into
                                 L2 ahead of its copy ring, 0..64 (default 3; 0 = none) */
+    VL_OPT_STAGGER_US = 9,     /* the first wave of thread blocks of a call's first table kernel starts in four classes this
+                                many microseconds apart (0..200, default 12), so that not all of them stream, then all of them
+                                sweep, in step; only for calls of at least two waves */
     VL_OPT_TEST_WAIT = 7     /* test hook for the bounded device waits: 1 = the table kernel (8 candidates per
                                 block) waits for its first tile on a barrier that nothing completes, with a short
                                 poll limit, so that the wait runs out: the call still returns, its verdicts are

@@ -27,6 +27,7 @@ VL_PASS, VL_INCONSISTENT, VL_OUT_OF_RANGE, VL_INTERFERENCE = 1, 2, 4, 8
 VL_OPT_CHUNK_INSTRS, VL_OPT_GROUP, VL_OPT_THREADS, VL_OPT_SUB_BATCH, VL_OPT_KERNEL_TIMING, VL_OPT_LANES = 1, 2, 3, 4, 5, 6
 VL_OPT_TEST_WAIT = 7
 VL_OPT_PREFETCH_TILES = 8
+VL_OPT_STAGGER_US = 9
 
 EXPORTS = ["vl_program_create", "vl_program_destroy", "vl_program_set_option", "vl_liveness", "vl_liveness_batch",
            "vl_liveness_result", "vl_verify", "vl_verify_batch", "vl_verify_host", "vl_verify_status",

@@ -296,6 +296,10 @@ extern "C" int vl_program_set_option(vl_program *p, int option, uint32_t value)
         if (value > 64) return VL_ERR_INVALID_ARG;
         p->prefetch_tiles = value;
         return VL_OK;
+    case VL_OPT_STAGGER_US:
+        if (value > 200) return VL_ERR_INVALID_ARG;
+        p->stagger_us = value;
+        return VL_OK;
     case VL_OPT_TEST_WAIT:
         if (value > 1) return VL_ERR_INVALID_ARG;
         p->test_wait = value;

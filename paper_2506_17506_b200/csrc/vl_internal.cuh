@@ -135,6 +135,7 @@ struct vl_program {
     uint32_t bank_seg[4] = {0, 0, 0, 0};
     uint32_t threads_opt = 0;
     uint32_t prefetch_tiles = 3;
+    uint32_t stagger_us = 12;     // start offset between the classes of the first wave of the table kernel (0 = none)
     int sm_count = 0;             // multiprocessors of the device (asked once)  // tiles the eight-candidate table kernel asks into L2 ahead of its copy ring
     uint32_t test_wait = 0;  // test hook of the table kernel's bounded wait (VL_OPT_TEST_WAIT)
     int use_th = 0;

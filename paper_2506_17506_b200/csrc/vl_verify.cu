@@ -65,6 +65,7 @@ struct TParams {
     uint32_t *grp_flag;   // per group of 32 candidates: some table entry carries the straddle mark
     uint32_t test_wait;   // test hook: the wait for tile 0 polls a barrier nothing completes, with a short limit
     uint32_t pf;          // tiles asked into L2 ahead of the copy ring
+    uint32_t stagger_ns, stagger_blocks;  // k_tables8: start offset between the four classes of the first wave's blocks
     // the rows as a 3-D tensor [candidate][chunk of 256 operands][256]: nfull whole chunks per row; the
     // operands from tail_start on (fewer than 256) come by plain bulk copies into a buffer of their own
     uint32_t nfull, tail_start, tail_tile, off_tail;
@@ -631,6 +632,21 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
 
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     const uint64_t k0 = (uint64_t)blockIdx.x * G;
+    // The thread blocks of a wave would otherwise run in step: all of them stream (HBM saturated) and
+    // then all of them sweep (HBM idle).  The first wave of a call starts in four classes a quarter of a
+    // block's time apart; later blocks start when earlier ones end, so the offsets persist.
+    if (q.stagger_ns && blockIdx.x < q.stagger_blocks && (blockIdx.x & 3u)) {
+        if (tid == 0) {
+            unsigned long long t0, t1;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+            const unsigned long long until = t0 + (unsigned long long)(blockIdx.x & 3u) * q.stagger_ns;
+            do {
+                __nanosleep(2000);
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            } while (t1 < until && t1 - t0 < 1000000ull);  // (never longer than a millisecond)
+        }
+        __syncthreads();
+    }
     const uint16_t *rows[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) rows[g] = q.cand + min(k0 + g, q.K - 1) * q.pitch;
@@ -2065,7 +2081,7 @@ int plan_passes(vl_program *p, uint64_t K, PassPlan *pp)
 
 // One pass: the four kernels over n <= sub candidates, in order on `st`, with working set `slot`.
 int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t n, uint64_t pitch, vl_verdict *d_out,
-             cudaStream_t st, int slot, bool dict)
+             cudaStream_t st, int slot, bool dict, bool stagger)
 {
     // what the rows hold: one column per operand occurrence, or one per dictionary entry
     const uint32_t nO = dict ? p->nD : p->nO, nOp8 = dict ? p->nD8 : p->nOp8;
@@ -2097,6 +2113,8 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     tq.grp_flag = vs.grp_done + (vs.rows / TGW + 1);
     tq.test_wait = p->test_wait;
     tq.pf = p->prefetch_tiles;
+    tq.stagger_ns = stagger ? p->stagger_us * 1000u : 0u;
+    tq.stagger_blocks = (uint32_t)vl_sm_count(p);
     const uint32_t tgrid = (uint32_t)((n + pl.G - 1) / pl.G);
     kt_mark(p, st);
     if (pl.G == 8) {
@@ -2195,7 +2213,8 @@ int vl_verify_impl(vl_program *p, const uint16_t *d_cand, uint64_t K, uint64_t p
     int rc = plan_passes(p, K, &pp);
     if (rc != VL_OK) return rc;
     for (uint64_t kb = 0; kb < K; kb += pp.sub) {
-        rc = run_pass(p, pp, d_cand + kb * pitch, std::min(pp.sub, K - kb), pitch, d_out + kb, st, slot, dict);
+        rc = run_pass(p, pp, d_cand + kb * pitch, std::min(pp.sub, K - kb), pitch, d_out + kb, st, slot, dict,
+                      kb == 0 && K >= 8ull * 2 * (uint64_t)vl_sm_count(p));
         if (rc != VL_OK) return rc;
     }
     return VL_OK;
@@ -2238,7 +2257,7 @@ int vl_verify_lanes(uint32_t nprog, vl_program *const *progs, const uint16_t *co
         uint64_t s = 0;
         for (uint64_t kb = 0; kb < K[j] && rc == VL_OK; kb += pp.sub, ++s, ++job)
             rc = run_pass(p, pp, d_cand[j] + kb * pitch[j], std::min(pp.sub, K[j] - kb), pitch[j], d_out[j] + kb,
-                          lane[(base + s) % L], (int)(s % L), dict);
+                          lane[(base + s) % L], (int)(s % L), dict, job == 0 && K[j] >= 8ull * 2 * (uint64_t)vl_sm_count(p));
     }
     // join even after an error, so that the caller's stream stays ordered after what was launched
     for (uint32_t l = 0; l < L; ++l) {
