@@ -365,7 +365,9 @@ def main():
         # algorithmic bytes: every candidate row is read once (2 bytes per operand column) and one 16-byte
         # verdict is written; the table kernel is the one that streams the rows
         bytes_per_step = 2.0 * prog.pitch * K + 16.0 * K
-        names = ["k_tables", "k_walk", "k_finish", "k_recount"]   # (k_walk includes the through-set kernel before it)
+        # the four timing slots of a pass (the table kernel; the through-set kernel and the walk; the stand-alone
+        # verdict step of programs without instructions; the recount)
+        names = ["k_tables8", "k_through+k_walk", "k_finish", "k_recount"]
         passes = max(1, kernel_passes)
         ksum = max(1e-9, sum(kernel_ms))
         kernels = {n: {"ms_per_launch": kernel_ms[j] / passes, "share": kernel_ms[j] / ksum} for j, n in enumerate(names)}
