@@ -155,13 +155,21 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
 // completion counted on `bar` with the full size of the box (elements outside the tensor arrive as
 // zeros).  dst 128-byte aligned; the innermost coordinate times the element size a multiple of 16.
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tm, uint32_t x, uint32_t y, uint32_t z,
-                                            unsigned long long *bar)
+                                            unsigned long long *bar, unsigned long long policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(
             smem_u32(dst)),
-        "l"(tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        "l"(tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
+}
+// L2 policy for data that is read once: first in line for eviction, so that it does not push out what
+// other kernels are about to read again.
+__device__ __forceinline__ unsigned long long l2_policy_evict_first()
+{
+    unsigned long long policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
 }
 // Asks for one box of the tensor to be brought into L2.
 __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *tm, uint32_t x, uint32_t y, uint32_t z)
@@ -705,6 +713,8 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
             }
             uint32_t issued = 0;  // tiles issued so far, in order
             uint32_t stage = 0, parity = 0;
+            // the rows are read once: they should not push the tables written for the walk out of L2
+            const unsigned long long stream_once = l2_policy_evict_first();
             for (uint32_t t = 0; t < q.ntiles; ++t) {
                 if (t >= q.NS) {  // the stage still holds tile t - NS: wait until the 16 warps have read it
                     wait_bar(&M->empty[stage], parity ^ 1u);
@@ -713,7 +723,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
                 issued = t + 1;
                 if (t * CH < q.nfull) {  // (a tile of nothing but tail operands has no box)
                     mbar_expect_tx(&M->bar[stage], STAGE_BYTES);
-                    tma_load_3d(region + (size_t)stage * STAGE_BYTES, &tm, 0, t * CH, (uint32_t)k0, &M->bar[stage]);
+                    tma_load_3d(region + (size_t)stage * STAGE_BYTES, &tm, 0, t * CH, (uint32_t)k0, &M->bar[stage], stream_once);
                 }
                 if (++stage == q.NS) { stage = 0; parity ^= 1; }
             }
