@@ -114,29 +114,38 @@ int vl_program_set_option(vl_program *prog, int option, uint32_t value);
  * Liveness (what "overlapping life cycles" in Section 2 and "Safety" in Section 3.4
  * rest on): per-block read/write bitsets, backward dataflow to the least fixed point,
  * then the set of vregs live after every instruction as CSR lists (ascending ids),
- * plus the per-program tables vl_verify consumes.  Runs on `cuda_stream`
- * (a cudaStream_t, may be NULL).  The first run of a handle (and the first after the chunk
- * size changed) synchronises the stream before returning, because list lengths and the
- * status word are read back; it is the run that reports NOT_STRICT or NO_CONVERGE.  Later
- * runs recompute everything on the device but allocate from the remembered lengths and
- * return without waiting: their outcome is checked by the next call that uses the results
- * (vl_verify*, vl_liveness_result, vl_liveness), which may then return the error.  From the
- * third such run on the sequence of kernels is replayed as a CUDA graph.
+ * plus the tables vl_verify consumes.  Stream order: the run is enqueued on an internal stream
+ * of the device, behind everything `cuda_stream` (a cudaStream_t, may be NULL) holds at the call;
+ * `cuda_stream` itself is NOT made to wait for it.  Every call of this library that reads the
+ * results waits for the run where it needs them: vl_verify* on the device (its table kernel, which
+ * reads the candidates and the program's operand tables only, runs beside the liveness kernels;
+ * the kernels after it wait), vl_liveness_result, vl_verify_host, vl_diagnose and
+ * vl_occupied_masks on the host.  A caller whose own kernels read the result arrays calls
+ * vl_liveness_result after every run (it returns when the run has finished).
+ * The first run of a handle (and the first after the chunk size changed) waits for the device
+ * before returning, because list lengths and the status word are read back; it is the run that
+ * reports NOT_STRICT or NO_CONVERGE, and the one that makes the operand tables (they depend on
+ * the program alone and are kept).  Later runs recompute the liveness results on the device but
+ * allocate from the remembered lengths and return without waiting: their outcome is checked by
+ * the next call that uses the results, which may then return the error.  From the third such run
+ * on the sequence of kernels is replayed as a CUDA graph.
  * Errors: NOT_STRICT, NO_CONVERGE, UNSUPPORTED, CUDA.
  */
 int vl_liveness(vl_program *prog, void *cuda_stream);
 
 /*
  * vl_liveness for n independent programs (all on the device of the first) in one call: the
- * runs are spread over internal streams that fork from and join back into `cuda_stream`, so
- * that the short kernels of different programs run side by side.  `progs` is HOST memory.
+ * runs are spread over internal streams that fork from and join back into `cuda_stream` (unlike
+ * a single vl_liveness, `cuda_stream` waits for them), so that the short kernels of different
+ * programs run side by side.  `progs` is HOST memory.
  * Stops at the first error and returns it.  Errors: as vl_liveness, INVALID_ARG.
  */
 int vl_liveness_batch(uint32_t n, vl_program *const *progs, void *cuda_stream);
 
 /*
  * Device pointers to the liveness results; owned by the handle, valid until
- * vl_program_destroy or the next vl_liveness.  Any out pointer may be NULL.
+ * vl_program_destroy or the next vl_liveness.  Any out pointer may be NULL.  Waits on the host
+ * until the last liveness run of the handle has finished and returns its outcome.
  *   blk_live_in / blk_live_out : [n_blocks][ceil(n_vregs/32)] little-endian bitsets
  *   lo_off [n_instrs+1], lo [lo_len] : vregs live after each instruction, ascending
  */

@@ -211,6 +211,11 @@ class Program:
     def vl_liveness(self, stream=None):
         self._check(_lib.vl_liveness(self._h, _stream_ptr(stream)), "vl_liveness")
 
+    def vl_liveness_wait(self):
+        """Blocks the host until the last vl_liveness run has finished and reports its outcome
+        (vl_liveness_result with no output pointers)."""
+        self._check(_lib.vl_liveness_result(self._h, None, None, None, None, None), "vl_liveness_result")
+
     def vl_liveness_result(self):
         """Copies of the liveness results as numpy arrays:
         (blk_live_in [nB, W] u32, blk_live_out [nB, W] u32, lo_off [nI+1] u32, lo [len] u32)."""

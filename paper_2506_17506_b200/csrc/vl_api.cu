@@ -11,7 +11,7 @@ std::atomic<uint64_t> g_vl_launches{0};
 // Lane streams are per device and shared by every handle on it; they live until the process exits.
 #define VL_MAX_DEVICES 64
 static std::mutex g_lane_mutex;
-static cudaStream_t g_lanes[VL_MAX_DEVICES][VL_LANES + 2];  // the lanes, then two side streams for liveness
+static cudaStream_t g_lanes[VL_MAX_DEVICES][VL_STREAMS];  // the lanes, two side streams of a liveness run, the liveness stream
 static bool g_lanes_made[VL_MAX_DEVICES];
 
 int vl_lane_streams(vl_program *p, cudaStream_t **lanes)
@@ -22,10 +22,15 @@ int vl_lane_streams(vl_program *p, cudaStream_t **lanes)
         if (!g_lanes_made[p->device]) {
             for (int l = 0; l < VL_LANES + 2; ++l)
                 VL_CUDA(p, cudaStreamCreateWithFlags(&g_lanes[p->device][l], cudaStreamNonBlocking));
+            // the liveness stream: its small kernels go first wherever a multiprocessor has room
+            int least = 0, greatest = 0;
+            VL_CUDA(p, cudaDeviceGetStreamPriorityRange(&least, &greatest));
+            VL_CUDA(p, cudaStreamCreateWithPriority(&g_lanes[p->device][VL_LIVE_STREAM], cudaStreamNonBlocking, greatest));
             g_lanes_made[p->device] = true;
         }
     }
     if (!p->ev_fork) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+    if (!p->ev_pre) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_pre, cudaEventDisableTiming));
     for (int l = 0; l < 3; ++l)
         if (!p->ev_side[l]) VL_CUDA(p, cudaEventCreateWithFlags(&p->ev_side[l], cudaEventDisableTiming));
     for (int l = 0; l < VL_LANES; ++l)
@@ -199,8 +204,7 @@ void vl_free_liveness(vl_program *p)
     p->live_arena.reset();
     p->tmp_arena.reset();
     p->d_blk_in = p->d_blk_out = p->d_lo_off = p->d_lo = nullptr;
-    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opoff = nullptr; p->d_first4 = nullptr; p->d_opflags = nullptr; p->d_iflags = nullptr;
-    p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
+    p->d_opflags = nullptr; p->d_iflags = nullptr;  // (the operand tables live in the layout arena)
     p->d_th_off = p->d_th = p->d_cev_off = nullptr;
     p->d_ev = nullptr;
     p->d_el = nullptr; p->d_el_count = nullptr;
@@ -241,6 +245,7 @@ extern "C" void vl_program_destroy(vl_program *p)
     }
     for (cudaEvent_t ev : p->kt_ev) cudaEventDestroy(ev);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->ev_pre) cudaEventDestroy(p->ev_pre);
     for (cudaEvent_t ev : p->ev_side)
         if (ev) cudaEventDestroy(ev);
     for (cudaEvent_t ev : p->ev_join)
@@ -366,7 +371,24 @@ extern "C" int vl_liveness(vl_program *p, void *stream)
 {
     if (!p) return VL_ERR_INVALID_ARG;
     VL_CUDA(p, cudaSetDevice(p->device));
-    return vl_liveness_impl(p, (cudaStream_t)stream);
+    // The run goes to an internal stream, behind everything the caller's stream holds now.  The
+    // caller's stream does not wait for it: the calls that read the results do (vl_live_join), and
+    // the table kernel of a following vl_verify, which needs none of them, runs beside it.
+    cudaStream_t *lanes = nullptr;
+    int rc = vl_lane_streams(p, &lanes);
+    if (rc != VL_OK) return rc;
+    cudaStream_t ls = lanes[VL_LIVE_STREAM];
+    VL_CUDA(p, cudaEventRecord(p->ev_pre, (cudaStream_t)stream));
+    VL_CUDA(p, cudaStreamWaitEvent(ls, p->ev_pre, 0));
+    rc = vl_liveness_impl(p, ls);
+    p->live_deferred = true;
+    return rc;
+}
+
+int vl_live_join(vl_program *p, cudaStream_t st)
+{
+    if (p->live_deferred && p->ev_live) VL_CUDA(p, cudaStreamWaitEvent(st, p->ev_live, 0));
+    return VL_OK;
 }
 
 extern "C" int vl_liveness_batch(uint32_t n, vl_program *const *progs, void *stream)
@@ -381,6 +403,11 @@ extern "C" int vl_liveness_batch(uint32_t n, vl_program *const *progs, void *str
     cudaStream_t *lane = nullptr;
     int rc = vl_lane_streams(p0, &lane);
     if (rc != VL_OK) return rc;
+    for (uint32_t j = 0; j < n; ++j) {
+        // an earlier single run of one of these programs may still sit on the liveness stream
+        if ((rc = vl_live_join(progs[j], st)) != VL_OK) return rc;
+        progs[j]->live_deferred = false;
+    }
     if (n == 1) return vl_liveness_impl(p0, st);
     VL_CUDA(p0, cudaEventRecord(p0->ev_fork, st));
     for (uint32_t l = 0; l < VL_LANES; ++l) VL_CUDA(p0, cudaStreamWaitEvent(lane[l], p0->ev_fork, 0));

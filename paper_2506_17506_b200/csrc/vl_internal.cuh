@@ -33,6 +33,8 @@ enum : uint32_t {
 
 #define VL_MAX_GROUP 8
 #define VL_LANES 8  // internal streams that the passes of device-resident verify calls can be spread over
+#define VL_LIVE_STREAM (VL_LANES + 2)  // index of the internal stream a single vl_liveness call runs on
+#define VL_STREAMS (VL_LANES + 3)      // the lanes, two side streams of a liveness run, the liveness stream
 
 // Device memory pool of a program handle: slabs are kept across calls, so that a repeated
 // vl_liveness on the same handle allocates nothing.
@@ -151,6 +153,16 @@ struct vl_program {
     uint32_t *h_live = nullptr;      // pinned: [0] status, [2..9] four 64-bit totals
     cudaEvent_t ev_live = nullptr;
     bool live_pending = false;
+    // vl_liveness runs on an internal stream behind what the caller's stream held when it was called;
+    // the caller's stream is not made to wait.  Calls that read the results make their stream wait
+    // for ev_live (vl_live_join); the table kernel, which reads the program's operand tables only,
+    // runs beside the liveness kernels.
+    bool live_deferred = false;
+    cudaEvent_t ev_pre = nullptr;
+    // The operand tables of the verify kernels (vreg per operand, first-occurrence bits, table
+    // offsets, vreg descriptors, first definitions) depend on the program alone: they are made by the
+    // first liveness run and kept (layout arena).
+    bool tables_built = false;
     // the recorded form of a liveness run with settled layout and lengths (see vl_liveness_impl)
     cudaGraphExec_t live_graph = nullptr;
     uint64_t live_graph_launches = 0;
@@ -214,6 +226,7 @@ int vl_lane_streams(vl_program *p, cudaStream_t **lanes);
 void vl_free_liveness(vl_program *p);
 // Waits for a liveness run that is still in flight and checks its outcome; VL_OK if none is pending.
 int vl_live_settle(vl_program *p);
+int vl_live_join(vl_program *p, cudaStream_t st);  // st waits for the liveness run in flight, if any
 // Multiprocessors of a device / of the handle's device (asked once).
 int vl_device_sm_count(int device);
 int vl_sm_count(vl_program *p);

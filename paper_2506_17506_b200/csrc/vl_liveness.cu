@@ -719,8 +719,11 @@ static int vl_layout(vl_program *p, cudaStream_t st)
     const uint32_t nB = p->nB;
     p->layout_chunk_instrs = 0;
     p->sizes_known = false;
-    VL_CUDA(p, cudaStreamSynchronize(st));  // earlier work on the stream may still read the old layout
+    VL_CUDA(p, cudaDeviceSynchronize());  // earlier work (on any stream) may still read the old layout
     p->layout_arena.reset();
+    p->tables_built = false;
+    p->d_vreg16 = nullptr; p->d_slotmeta = nullptr; p->d_opoff = nullptr; p->d_first4 = nullptr;
+    p->d_first_def_instr = nullptr; p->d_vinfo = nullptr;
     std::vector<uint32_t> c_i0, c_i1, c_blk, blk_c_off(nB + 1, 0), p_i0, p_i1, p_chunk, c_p_off;
     for (uint32_t b = 0; b < nB; ++b) {
         const uint64_t s = p->h_blk_off[b], n = p->h_blk_off[b + 1] - s;
@@ -788,12 +791,16 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     p->d_blk_out = p->d_blk_in + (size_t)nB * Wv;
     KEEP(&p->d_lo_off, (size_t)nI + 1);
     KEEP(&p->d_opflags, (size_t)nO);
-    KEEP(&p->d_first_def_instr, (size_t)V);
-    KEEP(&p->d_vreg16, (size_t)p->nOp8 + 8);
-    KEEP(&p->d_slotmeta, (size_t)p->nOp8 / 8);
-    KEEP(&p->d_opoff, (size_t)p->nOpT / 4);
-    KEEP(&p->d_first4, (size_t)p->nOpT / 4);
-    KEEP(&p->d_vinfo, (size_t)V);
+    // the operand tables of the verify kernels depend on the program alone: made by the first run, kept
+    const bool make_tables = !p->tables_built;
+    if (!p->d_opoff) {
+        LAYOUT(&p->d_first_def_instr, (size_t)V);
+        LAYOUT(&p->d_vreg16, (size_t)p->nOp8 + 8);
+        LAYOUT(&p->d_slotmeta, (size_t)p->nOp8 / 8);
+        LAYOUT(&p->d_first4, (size_t)p->nOpT / 4);
+        LAYOUT(&p->d_vinfo, (size_t)V);
+        LAYOUT(&p->d_opoff, (size_t)p->nOpT / 4);
+    }
     KEEP(&p->d_iflags, (size_t)nI);
     KEEP(&p->d_cev_off, (size_t)nC + 1);
     KEEP(&p->d_th_off, (size_t)nB + 1);
@@ -822,8 +829,12 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     TMP(&ev_off, (size_t)nI + 1);
     TMP(&centry_cnt, (size_t)nC);
     TMP(&cev, (size_t)nC);
-    TMP(&first_occ, (size_t)V);
-    TMP(&opmeta, (size_t)nO);
+    first_occ = nullptr;
+    opmeta = nullptr;
+    if (make_tables) {
+        TMP(&first_occ, (size_t)V);
+        TMP(&opmeta, (size_t)nO);
+    }
     TMP(&chunk_touch, (size_t)nC * Wv + 16);  // followed by the totals: one memset clears both
     totals = reinterpret_cast<unsigned long long *>(chunk_touch + (((size_t)nC * Wv + 1) & ~(size_t)1));
     // what has to start from a known value: the fixed point's sets, the touch sets (updated with
@@ -832,8 +843,10 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     VL_CUDA(p, cudaMemsetAsync(chunk_touch, 0, ((size_t)nC * Wv + 16) * 4, st));
     VL_CUDA(p, cudaMemsetAsync(p->d_status, 0, 4, st));
     VL_CUDA(p, cudaMemsetAsync(p->d_el_count, 0, 4, st));
-    VL_CUDA(p, cudaMemsetAsync(first_occ, 0xFF, std::max<size_t>(V, 1) * 4, st));
-    VL_CUDA(p, cudaMemsetAsync(p->d_first_def_instr, 0xFF, std::max<size_t>(V, 1) * 4, st));
+    if (make_tables) {
+        VL_CUDA(p, cudaMemsetAsync(first_occ, 0xFF, std::max<size_t>(V, 1) * 4, st));
+        VL_CUDA(p, cudaMemsetAsync(p->d_first_def_instr, 0xFF, std::max<size_t>(V, 1) * 4, st));
+    }
 
     LAUNCH(k_chunk_sets, nP, smem2, st, p->d_piece_i0, p->d_piece_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, Wv,
            piece_use, piece_def);
@@ -910,13 +923,15 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
            (const uint32_t *)p->d_chunk_blk, (const uint32_t *)blk_th, (const uint32_t *)p->d_ls_adj,
            (const uint32_t *)th_cnt, p->d_ls);
     if (nP) g_vl_launches.fetch_add(1);
-    LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
-           p->d_first_def_instr);
-    LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, sa, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
-    LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
-           p->d_opflags, p->d_vreg16, opmeta, p->d_status);
-    LAUNCH(k_pack_slots, (p->nOpT / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, p->nOpT / 8, V, opmeta, p->d_vreg16, p->d_slotmeta,
-           p->d_opoff, p->d_first4);
+    if (make_tables) {
+        LAUNCH(k_first_occ, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+               p->d_first_def_instr);
+        LAUNCH(k_vreg_info, (V + NT - 1) / NT, 0, sa, V, p->d_width, first_occ, p->d_first_def_instr, p->d_vinfo);
+        LAUNCH(k_operand_meta, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_op_vreg, first_occ,
+               p->d_opflags, p->d_vreg16, opmeta, p->d_status);
+        LAUNCH(k_pack_slots, (p->nOpT / 8 + NT - 1) / NT, 0, sa, nO, p->nOp8, p->nOpT / 8, V, opmeta, p->d_vreg16, p->d_slotmeta,
+               p->d_opoff, p->d_first4);
+    }
     LAUNCH(k_instr_flags, (nI + NT - 1) / NT, 0, sa, nI, p->d_op_off, p->d_ndefs, p->d_opflags, p->d_iflags);
     LAUNCH(k_fill_events, nC, 0, sb, p->d_chunk_i0, p->d_chunk_i1, p->d_op_off, p->d_ndefs, p->d_op_vreg, p->d_width,
            p->d_opflags, Wv, chunk_entry, centry_cnt, ev_off, p->d_cev_off, p->d_ev, p->d_chunk_blk, p->d_el,
@@ -929,6 +944,7 @@ static int live_enqueue(vl_program *p, cudaStream_t st)
     p->bank_fast = ((p->B == 1 || p->B == 2 || p->B == 4) && !p->bank_many) ? 1 : 0;
     VL_CUDA(p, cudaMemcpyAsync(p->h_live, p->d_status, 4, cudaMemcpyDeviceToHost, st));
     VL_CUDA(p, cudaMemcpyAsync(p->h_live + 2, totals, 40, cudaMemcpyDeviceToHost, st));
+    p->tables_built = true;
     return rc;
 }
 

@@ -2155,6 +2155,10 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
     g_vl_launches.fetch_add(1);
 
     kt_mark(p, st);
+    // Everything from here on reads what vl_liveness computes (through-sets, walk events, live-after
+    // lists); the table kernel above reads the program's operand tables only and may run beside a
+    // liveness run that is still in flight.
+    if ((rc = vl_live_join(p, st)) != VL_OK) return rc;
     if (p->nC) {
         WParams wq{};
         wq.V = p->V; wq.P = p->P; wq.nB = p->nB; wq.nC = p->nC; wq.Wp = pp.Wp; wq.AW = (uint32_t)vs.aw;
