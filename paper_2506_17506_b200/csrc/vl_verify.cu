@@ -1494,18 +1494,19 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
     uint32_t n_chunks = 0;
     for (uint32_t c0 = 0; c0 < nC; c0 += 32) n_chunks += __popc(__ballot_sync(0xffffffffu, all_defs(c0 + lane)));
     const uint32_t n_blocks = full ? 0u : __popc(thcol);
-    const uint32_t n = RC_BANK_PARTS + RC_PARTS * n_chunks + n_blocks;
+    const uint32_t n_bank = RC_BANK_PARTS;
+    const uint32_t n = n_bank + RC_PARTS * n_chunks + n_blocks;
     uint32_t at = 0;
     if (lane == 0) {
         racc[k * 4 + 3] = n;
         at = atomicAdd(work, n);
     }
     at = __shfl_sync(0xffffffffu, at, 0);
-    if (lane < RC_BANK_PARTS) {
+    if (lane < n_bank) {
         work[2 + 2 * (at + lane)] = (uint32_t)k;
         work[3 + 2 * (at + lane)] = rc_code(RC_KIND_BANK, lane, 0);
     }
-    at += RC_BANK_PARTS;
+    at += n_bank;
     if (!full && ((thcol >> lane) & 1u)) {  // through-sets are used only if the program has at most 32 blocks
         const uint32_t slot = at + __popc(thcol & ((1u << lane) - 1u));
         work[2 + 2 * slot] = (uint32_t)k;
@@ -1713,8 +1714,62 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 }
                 __syncthreads();
             }
-            // this warp's instructions: i_lo + warp, i_lo + warp + NW, ...; 32 of them per round
-            for (uint32_t ib = i_lo + warp; ib < i_hi; ib += 32 * NW) {
+            if (use_short) {
+                // Short lists (the through-set is counted from the arrays): four lanes per instruction, 64
+                // instructions per round, so that the loads of a whole round (bookkeeping, then defined vregs
+                // and list entries) are in flight together instead of instruction after instruction.
+                const uint32_t sub = lane & 3u, slot = tid >> 2;
+                for (uint32_t ib = i_lo; ib < i_hi; ib += RC_THREADS / 4) {
+                    const uint32_t i = ib + slot;
+                    uint32_t cnt_i = 0;
+                    if (i < i_hi) {
+                        const uint32_t o0 = q.op_off[i], nd = q.ndefs[i];
+                        const uint32_t f0 = q.lo_off[i], f1 = q.lo_off[i + 1];
+                        const uint32_t l0 = list_lo(i, f0), l1 = l0 + list_n(f0, f1);
+                        for (uint32_t d = o0; d < o0 + nd; ++d) {
+                            const uint32_t v = q.op_vreg[d];
+                            const uint32_t sw = reg_w(v);
+                            const uint32_t s = sw & 0xFFFFu, w = (sw >> 16) & 0xFFu;
+                            uint32_t cnt = 0;
+                            if (s < q.R) {  // the through-set members that overlap [s, s+w), v itself excepted
+                                if (sub == 0) cnt = cover[s] - ((sw >> 30) & 1u);
+                                for (uint32_t r = s + 1 + sub; r < min(s + w, q.R); r += 4) cnt += start[r];
+                            }
+                            for (uint32_t e0 = l0 + sub; e0 < l1; e0 += 32) {  // 8 list entries per lane in flight
+                                uint32_t us[8], xs[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) {
+                                    const uint32_t e = e0 + u * 4;
+                                    us[u] = e < l1 ? lst[e] : v;
+                                }
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) xs[u] = reg_w(us[u]);
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    if (us[u] != v && ranges_overlap(s, w, xs[u] & 0xFFFFu, (xs[u] >> 16) & 0xFFu)) ++cnt;
+                            }
+                            // co-defined vregs that are not live after the instruction
+                            if (nd > 1)
+                                for (uint32_t d2 = o0 + sub; d2 < o0 + nd; d2 += 4) {
+                                    if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
+                                    const uint32_t x = reg_w(q.op_vreg[d2]);
+                                    if (ranges_overlap(s, w, x & 0xFFFFu, (x >> 16) & 0xFFu)) ++cnt;
+                                }
+                            cnt_i += cnt;
+                        }
+                    }
+                    cnt_i += __shfl_xor_sync(0xffffffffu, cnt_i, 1);
+                    cnt_i += __shfl_xor_sync(0xffffffffu, cnt_i, 2);
+                    if (cnt_i && sub == 0) { pairs += cnt_i; mind = min(mind, i); }
+                }
+#pragma unroll
+                for (int dd = 16; dd; dd >>= 1) {  // (lane 0 reports for the warp)
+                    pairs += __shfl_xor_sync(0xffffffffu, pairs, dd);
+                    mind = min(mind, __shfl_xor_sync(0xffffffffu, mind, dd));
+                }
+            }
+            // full lists: this warp's instructions are i_lo + warp, i_lo + warp + NW, ...; 32 of them per round
+            for (uint32_t ib = i_lo + warp; !use_short && ib < i_hi; ib += 32 * NW) {
                 const uint32_t my_i = ib + lane * NW;
                 uint32_t m_o0 = 0, m_nd = 0, m_l0 = 0, m_l1 = 0;
                 if (my_i < i_hi) {
@@ -1794,17 +1849,32 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         } else {
             // a source counts when its register is new among the instruction's sources and its bank is not
             uint32_t bt = 0;
+            if (CACHE) {
+                // a slice of the list touches most vregs: the candidate's table column is fetched in one go
+                // (every load in flight at once) instead of entry by entry as the list asks for it
+#pragma unroll 8
+                for (uint32_t v = tid; v < q.V; v += RC_THREADS) Cv[v] = fetch(v) | 0x80000000u;
+                __syncthreads();
+            }
             if (q.bank_fast) {
                 const uint32_t n_all = q.bank_seg[3];
                 const uint32_t e_lo = (uint32_t)((uint64_t)n_all * part / RC_BANK_PARTS);
                 const uint32_t e_hi = (uint32_t)((uint64_t)n_all * (part + 1) / RC_BANK_PARTS);
-                for (uint32_t e0 = e_lo + tid; e0 < e_hi; e0 += 4 * RC_THREADS) {
-                    uint2 idv[4];
+                // 8 list entries per thread and round; the entries of the next round are fetched meanwhile
+                uint2 id_next[8];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        idv[u] = e0 + u * RC_THREADS < e_hi ? q.bank_list[e0 + u * RC_THREADS] : make_uint2(0, 0);
+                for (int u = 0; u < 8; ++u)
+                    id_next[u] = e_lo + tid + u * RC_THREADS < e_hi ? q.bank_list[e_lo + tid + u * RC_THREADS] : make_uint2(0, 0);
+                for (uint32_t e0 = e_lo + tid; e0 < e_hi; e0 += 8 * RC_THREADS) {
+                    uint2 idv[8];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 8; ++u) {
+                        idv[u] = id_next[u];
+                        const uint32_t en = e0 + (8 + u) * RC_THREADS;
+                        id_next[u] = en < e_hi ? q.bank_list[en] : make_uint2(0, 0);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
                         const uint32_t e = e0 + u * RC_THREADS;
                         if (e >= e_hi) break;
                         const uint2 ids = idv[u];
