@@ -1494,7 +1494,9 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
     uint32_t n_chunks = 0;
     for (uint32_t c0 = 0; c0 < nC; c0 += 32) n_chunks += __popc(__ballot_sync(0xffffffffu, all_defs(c0 + lane)));
     const uint32_t n_blocks = full ? 0u : __popc(thcol);
-    const uint32_t n_bank = RC_BANK_PARTS;
+    // the fast-path tally is one item per candidate (its table column is fetched once); the general tally
+    // of the other programs, which every candidate takes, is sliced
+    const uint32_t n_bank = list_all ? (uint32_t)RC_BANK_PARTS : 1u;
     const uint32_t n = n_bank + RC_PARTS * n_chunks + n_blocks;
     uint32_t at = 0;
     if (lane == 0) {
@@ -1715,11 +1717,11 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                 __syncthreads();
             }
             if (use_short) {
-                // Short lists (the through-set is counted from the arrays): four lanes per instruction, 64
+                // Short lists (the through-set is counted from the arrays): two lanes per instruction, 128
                 // instructions per round, so that the loads of a whole round (bookkeeping, then defined vregs
                 // and list entries) are in flight together instead of instruction after instruction.
-                const uint32_t sub = lane & 3u, slot = tid >> 2;
-                for (uint32_t ib = i_lo; ib < i_hi; ib += RC_THREADS / 4) {
+                const uint32_t sub = lane & 1u, slot = tid >> 1;
+                for (uint32_t ib = i_lo; ib < i_hi; ib += RC_THREADS / 2) {
                     const uint32_t i = ib + slot;
                     uint32_t cnt_i = 0;
                     if (i < i_hi) {
@@ -1733,13 +1735,13 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                             uint32_t cnt = 0;
                             if (s < q.R) {  // the through-set members that overlap [s, s+w), v itself excepted
                                 if (sub == 0) cnt = cover[s] - ((sw >> 30) & 1u);
-                                for (uint32_t r = s + 1 + sub; r < min(s + w, q.R); r += 4) cnt += start[r];
+                                for (uint32_t r = s + 1 + sub; r < min(s + w, q.R); r += 2) cnt += start[r];
                             }
-                            for (uint32_t e0 = l0 + sub; e0 < l1; e0 += 32) {  // 8 list entries per lane in flight
+                            for (uint32_t e0 = l0 + sub; e0 < l1; e0 += 16) {  // 8 list entries per lane in flight
                                 uint32_t us[8], xs[8];
 #pragma unroll
                                 for (int u = 0; u < 8; ++u) {
-                                    const uint32_t e = e0 + u * 4;
+                                    const uint32_t e = e0 + u * 2;
                                     us[u] = e < l1 ? lst[e] : v;
                                 }
 #pragma unroll
@@ -1750,7 +1752,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                             }
                             // co-defined vregs that are not live after the instruction
                             if (nd > 1)
-                                for (uint32_t d2 = o0 + sub; d2 < o0 + nd; d2 += 4) {
+                                for (uint32_t d2 = o0 + sub; d2 < o0 + nd; d2 += 2) {
                                     if (d2 == d || !(q.opflags[d2] & OPF_DEAD)) continue;
                                     const uint32_t x = reg_w(q.op_vreg[d2]);
                                     if (ranges_overlap(s, w, x & 0xFFFFu, (x >> 16) & 0xFFu)) ++cnt;
@@ -1759,7 +1761,6 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
                         }
                     }
                     cnt_i += __shfl_xor_sync(0xffffffffu, cnt_i, 1);
-                    cnt_i += __shfl_xor_sync(0xffffffffu, cnt_i, 2);
                     if (cnt_i && sub == 0) { pairs += cnt_i; mind = min(mind, i); }
                 }
 #pragma unroll
@@ -1858,8 +1859,7 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
             }
             if (q.bank_fast) {
                 const uint32_t n_all = q.bank_seg[3];
-                const uint32_t e_lo = (uint32_t)((uint64_t)n_all * part / RC_BANK_PARTS);
-                const uint32_t e_hi = (uint32_t)((uint64_t)n_all * (part + 1) / RC_BANK_PARTS);
+                const uint32_t e_lo = 0, e_hi = n_all;  // (one item per candidate: part is 0)
                 // 8 list entries per thread and round; the entries of the next round are fetched meanwhile
                 uint2 id_next[8];
 #pragma unroll
