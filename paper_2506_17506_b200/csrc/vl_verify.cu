@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
     if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
     if (tid == 0 && (k0 & (TGW - 1)) == 0) q.grp_done[k0 / TGW] = 0;
-    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
+    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; q.work[2] = 0; }  // item count and the recount's two cursors
     __syncthreads();
 
     // The ring stage and the barrier phase of the current tile are kept as running counters (stage
@@ -678,7 +678,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     for (uint32_t j = tid; j < G * q.AW; j += NT) q.anom[k0 * q.AW + j] = 0;
     if (tid < G * 4) q.racc[k0 * 4 + tid] = 0;
     if (tid == 0 && (k0 & (TGW - 1)) == 0) q.grp_done[k0 / TGW] = 0;
-    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; }  // item count and the recount's cursor
+    if (tid == 0 && blockIdx.x == 0) { q.work[0] = 0; q.work[1] = 0; q.work[2] = 0; }  // item count and the recount's two cursors
     __syncthreads();
 
     // A tile is one box of the row tensor: 8 candidates x CH chunks x 256 operands, one copy.  (Boxes
@@ -1453,6 +1453,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32, 3) k_walk(const WParams q)
 // definitions the walk skipped in its other chunks; racc[k][3] counts the items pending.  An item
 // is (candidate, code) with code = kind << 30 | piece << 24 | chunk (or block).
 #define RC_PARTS 2
+#define RC_HDR 4  // words in front of the work items: item count, cursor of the first round, cursor of the second
 #define RC_BANK_PARTS 4
 #define RC_KIND_ALL 0u     // every definition of the piece
 #define RC_KIND_THROUGH 1u // a block whose through-set collided: the definitions the walk skipped, chunk = block
@@ -1505,14 +1506,14 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
     }
     at = __shfl_sync(0xffffffffu, at, 0);
     if (lane < n_bank) {
-        work[2 + 2 * (at + lane)] = (uint32_t)k;
-        work[3 + 2 * (at + lane)] = rc_code(RC_KIND_BANK, lane, 0);
+        work[RC_HDR + 2 * (at + lane)] = (uint32_t)k;
+        work[RC_HDR + 1 + 2 * (at + lane)] = rc_code(RC_KIND_BANK, lane, 0);
     }
     at += n_bank;
     if (!full && ((thcol >> lane) & 1u)) {  // through-sets are used only if the program has at most 32 blocks
         const uint32_t slot = at + __popc(thcol & ((1u << lane) - 1u));
-        work[2 + 2 * slot] = (uint32_t)k;
-        work[3 + 2 * slot] = rc_code(RC_KIND_THROUGH, 0, lane);
+        work[RC_HDR + 2 * slot] = (uint32_t)k;
+        work[RC_HDR + 1 + 2 * slot] = rc_code(RC_KIND_THROUGH, 0, lane);
     }
     at += n_blocks;
     for (uint32_t c0 = 0; c0 < nC; c0 += 32) {
@@ -1522,8 +1523,8 @@ __device__ void finish_candidate(uint64_t k, uint32_t nC, uint32_t AW, int list_
             const uint32_t slot = at + RC_PARTS * __popc(m & ((1u << lane) - 1u));
 #pragma unroll
             for (uint32_t part = 0; part < RC_PARTS; ++part) {
-                work[2 + 2 * (slot + part)] = (uint32_t)k;
-                work[3 + 2 * (slot + part)] = rc_code(RC_KIND_ALL, part, c0 + lane);
+                work[RC_HDR + 2 * (slot + part)] = (uint32_t)k;
+                work[RC_HDR + 1 + 2 * (slot + part)] = rc_code(RC_KIND_ALL, part, c0 + lane);
             }
         }
         at += RC_PARTS * __popc(m);
@@ -1537,6 +1538,44 @@ __global__ void k_finish(uint64_t K, uint32_t nC, uint32_t AW, int list_all, con
 {
     const uint64_t k = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (k < K) finish_candidate(k, nC, AW, list_all, cstate, anom, chunk_blk, work, racc, out);
+}
+
+// Bank list entries [e_lo, e_hi) with N distinct source vregs each: how many sources hold the register
+// of an earlier source of the same entry.  regs[v] = register of vreg v (shared memory).  8 entries per
+// thread and round; the entries of the next round are fetched meanwhile.
+template <int N>
+__device__ __forceinline__ uint32_t bank_duplicates(const uint2 *__restrict__ list, uint32_t e_lo, uint32_t e_hi,
+                                                    const uint32_t *regs, uint32_t tid)
+{
+    uint32_t dups = 0;
+    uint2 id_next[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        id_next[u] = e_lo + tid + u * RC_THREADS < e_hi ? list[e_lo + tid + u * RC_THREADS] : make_uint2(0, 0);
+    for (uint32_t e0 = e_lo + tid; e0 < e_hi; e0 += 8 * RC_THREADS) {
+        uint2 idv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            idv[u] = id_next[u];
+            const uint32_t en = e0 + (8 + u) * RC_THREADS;
+            id_next[u] = en < e_hi ? list[en] : make_uint2(0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (e0 + u * RC_THREADS >= e_hi) break;
+            const uint32_t x0 = regs[idv[u].x & 0xFFFFu], x1 = regs[idv[u].x >> 16];
+            dups += (x1 == x0);
+            if (N >= 3) {
+                const uint32_t x2 = regs[idv[u].y & 0xFFFFu];
+                dups += (x2 == x0) | (x2 == x1);
+                if (N >= 4) {
+                    const uint32_t x3 = regs[idv[u].y >> 16];
+                    dups += (x3 == x0) | (x3 == x1) | (x3 == x2);
+                }
+            }
+        }
+    }
+    return dups;
 }
 
 // =========================================================================== k_recount
@@ -1558,16 +1597,19 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
     constexpr uint32_t NW = RC_THREADS / 32;
     const uint32_t nitems = q.work[0];
     __shared__ uint32_t s_item;
-    for (;;) {
-        // the items differ a lot in length: thread blocks take the next one from a shared cursor
+    // The items differ a lot in length: thread blocks take the next one from a shared cursor.  Two rounds
+    // over the list: the long items first (a bank tally sweeps the whole program, a through-set item is
+    // quadratic in the set), then the chunk pieces, so that no long item starts when the others end.
+    for (uint32_t round = 0; round < 2;) {
         __syncthreads();
-        if (tid == 0) s_item = atomicAdd(q.work + 1, 1u);
+        if (tid == 0) s_item = atomicAdd(q.work + 1 + round, 1u);
         __syncthreads();
         const uint32_t it = s_item;
-        if (it >= nitems) break;
-        const uint64_t k = q.work[2 + 2 * it];
-        const uint32_t code = q.work[3 + 2 * it];
+        if (it >= nitems) { ++round; continue; }
+        const uint64_t k = q.work[RC_HDR + 2 * it];
+        const uint32_t code = q.work[RC_HDR + 1 + 2 * it];
         const uint32_t kind = code >> 30, part = (code >> 24) & 63u, c = code & 0xFFFFFFu;
+        if ((kind == RC_KIND_ALL) != (round == 1)) continue;
         const uint32_t *cs = q.cstate + k * 8;
         const uint16_t *tg = q.tg + (k / TGW) * (uint64_t)(q.V + 1) * TGW + (k & (TGW - 1));
         // a single out-of-file vreg sits parked in the table: its true register is in the candidate's state
@@ -1850,13 +1892,21 @@ __global__ void __launch_bounds__(RC_THREADS) k_recount(const RParams q)
         } else {
             // a source counts when its register is new among the instruction's sources and its bank is not
             uint32_t bt = 0;
-            if (CACHE) {
-                // a slice of the list touches most vregs: the candidate's table column is fetched in one go
-                // (every load in flight at once) instead of entry by entry as the list asks for it
+            if (CACHE && q.bank_fast) {
+                // The table kernel's tally (sources minus banks touched, per instruction) counts a register
+                // that two source vregs share twice: the exact tally is that figure minus the number of such
+                // duplicates.  The candidate's registers are fetched in one go (every load in flight at once),
+                // then the list is swept from shared memory, one segment per source count.
 #pragma unroll 8
-                for (uint32_t v = tid; v < q.V; v += RC_THREADS) Cv[v] = fetch(v) | 0x80000000u;
+                for (uint32_t v = tid; v < q.V; v += RC_THREADS)
+                    Cv[v] = v == out_v ? out_raw : ((uint32_t)tg[(size_t)v * TGW] & tmask);
                 __syncthreads();
-            }
+                const uint32_t dups = bank_duplicates<2>(q.bank_list, q.bank_seg[0], q.bank_seg[1], Cv, tid) +
+                                      bank_duplicates<3>(q.bank_list, q.bank_seg[1], q.bank_seg[2], Cv, tid) +
+                                      bank_duplicates<4>(q.bank_list, q.bank_seg[2], q.bank_seg[3], Cv, tid);
+                if (tid == 0) atomicAdd(&s_bank, cs[CS_BANK]);
+                if (dups) atomicSub(&s_bank, dups);
+            } else
             if (q.bank_fast) {
                 const uint32_t n_all = q.bank_seg[3];
                 const uint32_t e_lo = 0, e_hi = n_all;  // (one item per candidate: part is 0)
@@ -2051,7 +2101,7 @@ int ensure_scratch(vl_program *p, int slot, uint64_t rows)
     VL_CUDA(p, cudaMalloc((void **)&v.cstate, groups * TGW * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMemset(v.cstate, 0, groups * TGW * 8 * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.anom, groups * TGW * aw * sizeof(uint32_t)));
-    VL_CUDA(p, cudaMalloc((void **)&v.work, (2 + 2 * groups * TGW * rc_items_per_row(p)) * sizeof(uint32_t)));
+    VL_CUDA(p, cudaMalloc((void **)&v.work, (RC_HDR + 2 * groups * TGW * rc_items_per_row(p)) * sizeof(uint32_t)));
     VL_CUDA(p, cudaMalloc((void **)&v.racc, groups * TGW * 4 * sizeof(uint32_t)));
     // walk blocks finished per group, then the groups' straddle-mark flags (reset by the walk)
     VL_CUDA(p, cudaMalloc((void **)&v.grp_done, 2 * (groups + 1) * sizeof(uint32_t)));
