@@ -46,7 +46,7 @@ enum {
     VL_OPT_CHUNK_INSTRS = 1, /* instructions per walk chunk (default 160; long blocks get a chunk count that is a multiple of 8) */
     VL_OPT_GROUP = 2,        /* candidates per thread block of the table kernel: 0 = choose, else 1, 2, 4 or 8 */
     VL_OPT_THREADS = 3,      /* threads per thread block of the table kernel: 0 = choose, else 256 or 512 */
-    VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 4096) */
+    VL_OPT_SUB_BATCH = 4,    /* candidates per pass of the verify kernels (multiple of 32, default 5120) */
     VL_OPT_KERNEL_TIMING = 5,/* 1: vl_verify records CUDA events around its kernels (see vl_kernel_times); may be
                                 set at any time; setting it discards the events recorded so far */
     VL_OPT_LANES = 6,        /* internal streams the passes of vl_verify are spread over, 1..8 (default 3);

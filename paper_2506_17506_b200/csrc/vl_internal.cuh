@@ -180,7 +180,7 @@ struct vl_program {
         uint32_t *thm = nullptr;       // [groups][n_blocks][mask words][2][32] through-set masks
         uint64_t rows = 0, aw = 0, vregs = 0, chunks = 0;
     } vs[VL_LANES + 2];              // one per lane, then one per staging buffer of vl_verify_host
-    uint32_t sub_batch = 4096;       // candidates per pass of the verify kernels
+    uint32_t sub_batch = 5120;       // candidates per pass of the verify kernels
     uint32_t lanes_opt = 3;          // lanes in use (1 = everything in order on the caller's stream)
     cudaEvent_t ev_fork = nullptr, ev_join[VL_LANES] = {};
     cudaEvent_t ev_side[3] = {};     // fork and two joins of the side streams of a liveness run
