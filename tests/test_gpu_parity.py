@@ -368,3 +368,31 @@ def test_determinism(B):
     b = _gpu_verify(B, gp, rows)
     assert a.tobytes() == b.tobytes()
     gp.close()
+
+
+def test_liveness_and_verify_on_different_streams(B, oracle_mod):
+    """vl_liveness runs on an internal stream and holds no caller stream; vl_verify waits for it on the
+    device where it reads its results.  Liveness on one stream, verify on another, no synchronisation
+    in between, new rows every step, several passes per call: every verdict must be right."""
+    import torch
+    wl = synth.workload(2)
+    p = synth.build_program(wl.shapes[0], wl.seeds[0])
+    gp, lv = _check_liveness(B, oracle_mod, p)
+    gp.set_option(B.VL_OPT_SUB_BATCH, 128)
+    orc = oracle_mod.OracleProgram(p)
+    s_live, s_ver = torch.cuda.Stream(), torch.cuda.Stream()
+    outs, wants = [], []
+    for step in range(6):
+        rows, _ = synth.candidate_rows(p, 600, 0.3, 100 + step)
+        dev = _to_dev(rows)                      # (copied on the default stream; make s_ver wait for it)
+        s_ver.wait_stream(torch.cuda.current_stream())
+        s_live.wait_stream(s_ver)                # (the run rewrites what the previous step's verify still reads)
+        gp.vl_liveness(s_live)
+        outs.append((gp.vl_verify(dev, None, s_ver), dev))
+        wants.append(orc.verify(lv, rows))
+    torch.cuda.synchronize()
+    gp.vl_verify_status()
+    for step, ((out, _), want) in enumerate(zip(outs, wants)):
+        _assert_same(B.verdicts_to_numpy(out), want, f"step {step}")
+    _check_liveness_result(B, oracle_mod, gp, p)
+    gp.close()
