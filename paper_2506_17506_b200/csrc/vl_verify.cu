@@ -1,20 +1,23 @@
-// The verify path: three kernels per pass over at most `sub_batch` candidates.
+// The verify path: four kernels per pass over at most `sub_batch` candidates.
 //
-// k_tables   one thread block per G candidates, packed side by side.  Streams the G rows (bulk
-//            async copies into a shared-memory ring, completion on mbarriers), builds the
-//            vreg -> preg tables T (G 16-bit entries per vreg, shared memory) from first
-//            occurrences, compares every other occurrence with T (Consistency), sweeps the vregs for
-//            [T, T+width) inside the register file (Realizability), tallies bank conflicts from T
-//            over the instructions with 2..4 distinct sources, and writes T to global memory with 32
-//            candidates side by side per vreg.
-// k_walk     one lane per candidate, one warp per chunk of instructions: the program's precompiled
-//            event stream is the same for all 32 lanes, the occupancy bitmask of each lane sits in
-//            shared memory at [word][lane] (Safety).  A chunk whose walk sees no collision provably
-//            has no overlap.
-//            The thread block that ends a group of 32 candidates writes the verdicts of its clean
-//            candidates and lists the others for the recount.
+// k_tables8  one thread block per 8 candidates, packed side by side (16 bytes per vreg).  A producer warp
+//            streams the 8 rows with tiled bulk copies into a shared-memory ring (completion on
+//            mbarriers); 16 consumer warps build the vreg -> register table T in shared memory from first
+//            occurrences and compare every other occurrence with T (Consistency).  Then the block sweeps
+//            the vregs ([T, T+width) inside the register file: Realizability; T to global memory, 64
+//            candidates side by side per vreg) and tallies bank conflicts over the instructions with
+//            2..4 distinct sources.  k_tables<G,NT> (G = 4, 2, 1 candidates per block, block barrier per
+//            tile) serves programs whose 16-byte tables do not fit an SM.
+// k_through  the occupancy masks of every block's through-set (vregs occupied through the whole block),
+//            per candidate, in the walk's layout.
+// k_walk     two candidates per lane, one warp per chunk of instructions: the program's precompiled
+//            event stream is the same for all lanes, the occupancy bitmasks of a lane sit in shared
+//            memory at [word][slot][lane] (Safety).  A chunk whose walk sees no collision provably
+//            has no overlap.  The thread block that ends a group of 64 candidates writes the verdicts
+//            of its clean candidates and lists the others for the recount.
 // k_recount  candidates with a collision are recounted exactly from the per-instruction live-after
-//            lists, one thread block per piece of a colliding chunk.
+//            lists: work items (a piece of a colliding chunk, a block whose through-set collided, the
+//            bank tally of a candidate) taken from a shared cursor, long items first.
 #include <cuda.h>
 
 #include <algorithm>
@@ -62,7 +65,7 @@ struct TParams {
     // dictionary rows: the instruction a Consistency violation of entry e is reported at (null: the rows
     // hold one column per operand, and the instruction is the one the operand belongs to)
     const uint32_t *entry_instr;
-    uint32_t *grp_flag;   // per group of 32 candidates: some table entry carries the straddle mark
+    uint32_t *grp_flag;   // per group of 64 candidates: some table entry carries the straddle mark
     uint32_t test_wait;   // test hook: the wait for tile 0 polls a barrier nothing completes, with a short limit
     uint32_t pf;          // tiles asked into L2 ahead of the copy ring
     uint32_t stagger_ns, stagger_blocks;  // k_tables8: start offset between the four classes of the first wave's blocks
@@ -93,7 +96,7 @@ struct WParams {
     uint32_t ev_cap;  // events a warp stages at a time (multiple of 8)
     uint32_t *cstate, *anom;
     uint32_t *grp_flag;  // per group: set by the table kernel when a walked candidate has a marked entry
-    // hand-over to k_recount by the last thread block of each group of 32 candidates
+    // hand-over to k_recount by the last thread block of each group of 64 candidates
     int list_all;
     const uint32_t *chunk_blk;
     uint32_t *grp_done, *work, *racc;
@@ -408,7 +411,7 @@ __global__ void __launch_bounds__(NT) k_tables(const TParams q)
     }
     __syncthreads();
 
-    // ---- one sweep over the vregs: the table goes to global memory (32 candidates side by side per
+    // ---- one sweep over the vregs: the table goes to global memory (64 candidates side by side per
     // vreg; the spare entry V, looked up by no-op events, as 0) and [T, T+width) is checked against the
     // register file (Realizability)
     {
@@ -889,7 +892,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     }
     __syncthreads();
 
-    // ---- one sweep over the vregs: the table goes to global memory (32 candidates side by side per
+    // ---- one sweep over the vregs: the table goes to global memory (64 candidates side by side per
     // vreg; the spare entry V, looked up by no-op events, as 0), entries whose range reaches into the
     // next 32-bit word of an occupancy mask get bit 15, the one-hot bank nibbles of the 8 candidates go
     // to Hb, and [T, T+width) is checked against the register file (Realizability).
@@ -1080,7 +1083,7 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         cs[CS_OUTRAW] = M->out_raw[g];
         cs[CS_WALK] = M->nout[g] >= 2 ? WALK_FULL : 0u;
         cs[CS_THCOL] = 0;
-        // a candidate that is walked and has a marked entry sends its group of 32 down the walk's
+        // a candidate that is walked and has a marked entry sends its group of 64 down the walk's
         // checking path
         if (M->nout[g] < 2 && ((M->marks >> g) & 1u)) atomicOr(&q.grp_flag[k0 / TGW], 1u);
     }
