@@ -128,7 +128,8 @@ int vl_program_set_option(vl_program *prog, int option, uint32_t value);
  * the program alone and are kept).  Later runs recompute the liveness results on the device but
  * allocate from the remembered lengths and return without waiting: their outcome is checked by
  * the next call that uses the results, which may then return the error.  From the third such run
- * on the sequence of kernels is replayed as a CUDA graph.
+ * on the sequence of kernels is replayed as a CUDA graph (a recording of the library's own: do not
+ * call vl_liveness while `cuda_stream` is itself being captured).
  * Errors: NOT_STRICT, NO_CONVERGE, UNSUPPORTED, CUDA.
  */
 int vl_liveness(vl_program *prog, void *cuda_stream);
