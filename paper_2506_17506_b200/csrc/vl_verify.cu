@@ -65,6 +65,7 @@ struct TParams {
     // dictionary rows: the instruction a Consistency violation of entry e is reported at (null: the rows
     // hold one column per operand, and the instruction is the one the operand belongs to)
     const uint32_t *entry_instr;
+    uint32_t tg_rows;     // k_tables8: vregs per bulk store of the table (rows of the box of the tg tensor)
     uint32_t *grp_flag;   // per group of 64 candidates: some table entry carries the straddle mark
     uint32_t test_wait;   // test hook: the wait for tile 0 polls a barrier nothing completes, with a short limit
     uint32_t pf;          // tiles asked into L2 ahead of the copy ring
@@ -168,6 +169,15 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tm, ui
 }
 // L2 policy for data that is read once: first in line for eviction, so that it does not push out what
 // other kernels are about to read again.
+// Tiled bulk store of one box from shared memory (elements outside the tensor are not written); completion is
+// tracked by the issuing thread's bulk async-groups.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, uint32_t x, uint32_t y, uint32_t z, const void *src)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(src))
+                 : "memory");
+}
+
 __device__ __forceinline__ unsigned long long l2_policy_evict_first()
 {
     unsigned long long policy;
@@ -627,7 +637,8 @@ __device__ __noinline__ void rules_sweep8(const uint4 *vcons, const uint16_t *rs
 }
 
 template <int NT>
-__global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const __grid_constant__ CUtensorMap tm)
+__global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const __grid_constant__ CUtensorMap tm,
+                                                          const __grid_constant__ CUtensorMap tmg)
 {
     constexpr int G = 8;
     constexpr uint32_t TILE = NT * 4;  // operands per tile and candidate
@@ -892,20 +903,14 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     }
     __syncthreads();
 
-    // ---- one sweep over the vregs: the table goes to global memory (64 candidates side by side per
-    // vreg; the spare entry V, looked up by no-op events, as 0), entries whose range reaches into the
-    // next 32-bit word of an occupancy mask get bit 15, the one-hot bank nibbles of the 8 candidates go
-    // to Hb, and [T, T+width) is checked against the register file (Realizability).
+    // ---- first sweep over the vregs: the one-hot bank nibbles of the 8 candidates go to Hb, and
+    // [T, T+width) is checked against the register file (Realizability).
     // (From here on the producer warp only keeps the block's barriers company.)
     if (tid < NT) {
-        const uint64_t grp = k0 / TGW;
-        const uint32_t l0 = (uint32_t)(k0 & (TGW - 1));
-        uint16_t *dst = q.tg + grp * (uint64_t)(q.V + 1) * TGW + l0;
-        uint32_t mk = 0, mk2 = 0, mk3 = 0, mk4 = 0;
         uint32_t vis_next[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) vis_next[u] = tid + u * NT < q.V ? q.vinfo[tid + u * NT] : 0u;
-        for (uint32_t v0 = tid; v0 <= q.V; v0 += 4 * NT) {
+        for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NT) {
             uint32_t vis[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -916,24 +921,17 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const uint32_t v = v0 + u * NT, vi = vis[u];
-                if (v > q.V) break;
-                const uint4 tt = T[v];  // (the spare entry holds zeros)
+                if (v >= q.V) break;
+                const uint4 tt = T[v];
                 const uint32_t x[4] = {tt.x, tt.y, tt.z, tt.w};
-                if (q.bank_fast && v < q.V) {
+                if (q.bank_fast) {
                     uint32_t h = 0;
 #pragma unroll
                     for (int m = 0; m < 4; ++m)
                         h |= ((1u << (x[m] & q.Bmask)) << (8 * m)) | ((16u << ((x[m] >> 16) & q.Bmask)) << (8 * m));
                     Hb[v] = h;
                 }
-                // bit 15 := ((register & 31) + width > 32), per 16-bit entry; 0x7FDF = 0x8000 - 33
-                const uint32_t wc = (vi & 0xFFu) * 0x10001u + 0x7FDF7FDFu;
-                uint32_t o[4];
-#pragma unroll
-                for (int m = 0; m < 4; ++m) o[m] = (x[m] & 0x7FFF7FFFu) | (((x[m] & 0x001F001Fu) + wc) & 0x80008000u);
-                *reinterpret_cast<uint4 *>(dst + (size_t)v * TGW) = make_uint4(o[0], o[1], o[2], o[3]);
                 if (!(vi & VINFO_OCCURS)) continue;
-                mk |= o[0]; mk2 |= o[1]; mk3 |= o[2]; mk4 |= o[3];
                 // quick test for "all eight inside the file": with c = 0x7FFF - (P - width) added to an
                 // entry below 2^15, bit 15 of the sum is set iff entry + width > P; entries at or above
                 // 2^15 are outside any file this kernel accepts.  The exact test runs only if a bit shows.
@@ -958,6 +956,50 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
                 }
             }
         }
+    }
+    if (q.vcons && tid < NT) rules_sweep8<NT>(q.vcons, q.rs_prefix, q.vinfo, q.first_def_instr, q.V, q.P, T, M);
+    __syncthreads();
+
+    // ---- second sweep, in place: entries whose range reaches into the next 32-bit word of an occupancy
+    // mask get bit 15.  The entries of a candidate with two or more vregs outside the register file stay as
+    // they are (it is not walked; the full recount reads them as plain numbers).
+    if (tid < NT) {
+        uint32_t keep[4];  // 16-bit fields of the candidates whose entries stay as they are
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+            keep[m] = (M->nout[2 * m] >= 2 ? 0xFFFFu : 0u) | (M->nout[2 * m + 1] >= 2 ? 0xFFFF0000u : 0u);
+        uint32_t mk = 0, mk2 = 0, mk3 = 0, mk4 = 0;
+        uint32_t vis_next[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) vis_next[u] = tid + u * NT < q.V ? q.vinfo[tid + u * NT] : 0u;
+        for (uint32_t v0 = tid; v0 < q.V; v0 += 4 * NT) {
+            uint32_t vis[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                vis[u] = vis_next[u];
+                const uint32_t vn = v0 + 4 * NT + u * NT;
+                vis_next[u] = vn < q.V ? q.vinfo[vn] : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t v = v0 + u * NT, vi = vis[u];
+                if (v >= q.V) break;
+                if (!(vi & VINFO_OCCURS)) continue;  // (never looked up)
+                const uint4 tt = T[v];
+                const uint32_t x[4] = {tt.x, tt.y, tt.z, tt.w};
+                // bit 15 := ((register & 31) + width > 32), per 16-bit entry; 0x7FDF = 0x8000 - 33
+                const uint32_t wc = (vi & 0xFFu) * 0x10001u + 0x7FDF7FDFu;
+                uint32_t o[4], diff = 0;
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    const uint32_t marked = (x[m] & 0x7FFF7FFFu) | (((x[m] & 0x001F001Fu) + wc) & 0x80008000u);
+                    o[m] = (marked & ~keep[m]) | (x[m] & keep[m]);
+                    diff |= o[m] ^ x[m];
+                }
+                if (diff) T[v] = make_uint4(o[0], o[1], o[2], o[3]);
+                mk |= o[0] & ~keep[0]; mk2 |= o[1] & ~keep[1]; mk3 |= o[2] & ~keep[2]; mk4 |= o[3] & ~keep[3];
+            }
+        }
         const uint32_t mkw[4] = {mk, mk2, mk3, mk4};
         uint32_t bits = 0;
 #pragma unroll
@@ -965,8 +1007,28 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         bits = __reduce_or_sync(0xffffffffu, bits);
         if (lane == 0 && bits) atomicOr(&M->marks, bits);
     }
-    if (q.vcons && tid < NT) rules_sweep8<NT>(q.vcons, q.rs_prefix, q.vinfo, q.first_def_instr, q.V, q.P, T, M);
     __syncthreads();
+    // a single out-of-file vreg is parked at register P (the walk's masks have spare bits there)
+    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
+        const uint32_t ov = M->out_v[tid];
+        const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
+        reinterpret_cast<uint16_t *>(T + ov)[tid] = (uint16_t)(q.P | mark);
+        if (mark) atomicOr(&M->marks, 1u << tid);
+    }
+    __syncthreads();
+    // The table goes to global memory, 64 candidates side by side per vreg (this block's 8 are 16 bytes of
+    // every 128): tiled bulk stores of up to 256 vregs each, carried out by the copy
+    // engine while the block tallies bank conflicts.  (Rows past the spare entry V are clipped by the tensor.)
+    // (Issuing a store holds its thread for thousands of cycles: the lanes of the producer warp, idle since
+    // the last tile, issue them.)
+    bool stored = false;  // this thread has bulk stores under way
+    if (tid >= NT && lane * q.tg_rows <= q.V) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const uint32_t x0 = (uint32_t)(k0 & (TGW - 1)), z0 = (uint32_t)(k0 / TGW);
+        for (uint32_t v0 = lane * q.tg_rows; v0 <= q.V; v0 += 32 * q.tg_rows) tma_store_3d(&tmg, x0, v0, z0, T + v0);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        stored = true;
+    }
 
     // ---- bank tally over the instructions with 2..4 distinct sources (see k_tables): the banks an
     // instruction touches are the bits of the OR of its sources' nibbles, counted with carry-save adders
@@ -1045,19 +1107,6 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
     __syncthreads();
 
     // ------------------------------------------------- hand-over to the walk (see k_tables)
-#pragma unroll 1
-    for (int g = 0; g < G; ++g) {
-        if (M->nout[g] < 2 || tid >= NT) continue;
-        uint16_t *col = q.tg + (k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (uint32_t)(k0 & (TGW - 1)) + g;
-        for (uint32_t v = tid; v < q.V; v += NT) col[(size_t)v * TGW] = (uint16_t)pk8_get(T[v], g);
-    }
-    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
-        const uint32_t ov = M->out_v[tid];
-        const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
-        q.tg[(k0 / TGW) * (uint64_t)(q.V + 1) * TGW + (size_t)ov * TGW + (uint32_t)(k0 & (TGW - 1)) + tid] = (uint16_t)(q.P | mark);
-        if (mark) atomicOr(&M->marks, 1u << tid);
-    }
-    __syncthreads();
     if (tid < G && k0 + tid < q.K) {
         const uint32_t g = tid;
         uint32_t first = 0xFFFFFFFFu;
@@ -1087,6 +1136,8 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         // checking path
         if (M->nout[g] < 2 && ((M->marks >> g) & 1u)) atomicOr(&q.grp_flag[k0 / TGW], 1u);
     }
+    // the bulk stores read the table from shared memory: the block stays until they are done
+    if (stored) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 __device__ __forceinline__ uint32_t lds32(uint32_t addr)
@@ -2043,32 +2094,59 @@ Plan make_plan8(const vl_program *p, uint32_t NT, uint32_t budget)
 
 // The candidate rows of one pass as a 3-D tensor for the tiled copies of k_tables8:
 // [n rows][nfull chunks][256 operands], a box = 8 rows x (tile / 256) chunks x 256 operands.
+typedef CUresult (*tm_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled, asked from the runtime once per process.
+int tensor_encoder(vl_program *p, tm_encode_fn *out)
+{
+    static std::mutex mtx;
+    static tm_encode_fn encode = nullptr;
+    std::lock_guard<std::mutex> lock(mtx);
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+            p->last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorUnknown);
+            return VL_ERR_CUDA;
+        }
+        encode = (tm_encode_fn)fn;
+    }
+    *out = encode;
+    return VL_OK;
+}
+
 int encode_row_tensor(vl_program *p, CUtensorMap *tm, const uint16_t *d_cand, uint64_t n, uint64_t pitch, uint32_t nfull,
                       uint32_t chunks_per_tile)
 {
-    typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-    static std::mutex mtx;
-    static encode_fn encode = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(mtx);
-        if (!encode) {
-            void *fn = nullptr;
-            cudaDriverEntryPointQueryResult qres;
-            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-            if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
-                p->last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorUnknown);
-                return VL_ERR_CUDA;
-            }
-            encode = (encode_fn)fn;
-        }
-    }
+    tm_encode_fn encode = nullptr;
+    int rc = tensor_encoder(p, &encode);
+    if (rc != VL_OK) return rc;
     const cuuint64_t dims[3] = {256, nfull, n};
     const cuuint64_t strides[2] = {512, pitch * 2};
     const cuuint32_t box[3] = {256, chunks_per_tile, 8};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, (void *)d_cand, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { p->last_cuda_error = (int)cudaErrorInvalidValue; return VL_ERR_CUDA; }
+    return VL_OK;
+}
+
+// The tables of one pass as a 3-D tensor for the tiled stores of k_tables8: [groups][V + 1 vregs][64 candidates],
+// a box = 8 candidates (16 bytes) x `rows` vregs of one group.
+int encode_tg_tensor(vl_program *p, CUtensorMap *tm, uint16_t *tg, uint32_t groups, uint32_t rows)
+{
+    tm_encode_fn encode = nullptr;
+    int rc = tensor_encoder(p, &encode);
+    if (rc != VL_OK) return rc;
+    const cuuint64_t dims[3] = {TGW, (cuuint64_t)p->V + 1, groups};
+    const cuuint64_t strides[2] = {TGW * 2, ((cuuint64_t)p->V + 1) * TGW * 2};
+    const cuuint32_t box[3] = {8, rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, (void *)tg, dims, strides, box, estr,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { p->last_cuda_error = (int)cudaErrorInvalidValue; return VL_ERR_CUDA; }
@@ -2262,8 +2340,12 @@ int run_pass(vl_program *p, const PassPlan &pp, const uint16_t *d_cand, uint64_t
             rc = encode_row_tensor(p, &tm, d_cand, n, pitch, tq.nfull, pl.NT * 4 / 256);
             if (rc != VL_OK) return rc;
         }
-        if (pl.NT == 256) k_tables8<256><<<tgrid, 256 + 32, pl.smem, st>>>(tq, tm);
-        else k_tables8<512><<<tgrid, 512 + 32, pl.smem, st>>>(tq, tm);
+        alignas(64) CUtensorMap tmg;
+        tq.tg_rows = std::min<uint32_t>(256u, p->V + 1);
+        rc = encode_tg_tensor(p, &tmg, vs.tg, ngrp, tq.tg_rows);
+        if (rc != VL_OK) return rc;
+        if (pl.NT == 256) k_tables8<256><<<tgrid, 256 + 32, pl.smem, st>>>(tq, tm, tmg);
+        else k_tables8<512><<<tgrid, 512 + 32, pl.smem, st>>>(tq, tm, tmg);
         e = cudaGetLastError();
     } else if (pl.NT == 256) {
         if (pl.G == 4) e = launch_tables<4, 256>(tq, tgrid, pl.smem, st);
