@@ -1006,28 +1006,31 @@ __global__ void __launch_bounds__(NT + 32, 1) k_tables8(const TParams q, const _
         for (int m = 0; m < 4; ++m) bits |= ((mkw[m] >> 15) & 1u) << (2 * m) | ((mkw[m] >> 31) & 1u) << (2 * m + 1);
         bits = __reduce_or_sync(0xffffffffu, bits);
         if (lane == 0 && bits) atomicOr(&M->marks, bits);
+        // the consumers go on to the bank tally (it reads Hb only); the producer warp waits for all of them here
+        asm volatile("bar.arrive 1, %0;" ::"r"(NT + 32) : "memory");
     }
-    __syncthreads();
-    // a single out-of-file vreg is parked at register P (the walk's masks have spare bits there)
-    if (tid < G && M->nout[tid] == 1 && M->out_raw[tid] >= q.P) {
-        const uint32_t ov = M->out_v[tid];
-        const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
-        reinterpret_cast<uint16_t *>(T + ov)[tid] = (uint16_t)(q.P | mark);
-        if (mark) atomicOr(&M->marks, 1u << tid);
-    }
-    __syncthreads();
     // The table goes to global memory, 64 candidates side by side per vreg (this block's 8 are 16 bytes of
-    // every 128): tiled bulk stores of up to 256 vregs each, carried out by the copy
-    // engine while the block tallies bank conflicts.  (Rows past the spare entry V are clipped by the tensor.)
-    // (Issuing a store holds its thread for thousands of cycles: the lanes of the producer warp, idle since
-    // the last tile, issue them.)
+    // every 128): tiled bulk stores of up to 256 vregs each, carried out by the copy engine while the block
+    // tallies bank conflicts.  (Rows past the spare entry V are clipped by the tensor.)  Issuing a store holds
+    // its thread for thousands of cycles: the lanes of the producer warp, idle since the last tile, issue them.
     bool stored = false;  // this thread has bulk stores under way
-    if (tid >= NT && lane * q.tg_rows <= q.V) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        const uint32_t x0 = (uint32_t)(k0 & (TGW - 1)), z0 = (uint32_t)(k0 / TGW);
-        for (uint32_t v0 = lane * q.tg_rows; v0 <= q.V; v0 += 32 * q.tg_rows) tma_store_3d(&tmg, x0, v0, z0, T + v0);
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        stored = true;
+    if (tid >= NT) {
+        asm volatile("bar.sync 1, %0;" ::"r"(NT + 32) : "memory");
+        // a single out-of-file vreg is parked at register P (the walk's masks have spare bits there)
+        if (lane < G && M->nout[lane] == 1 && M->out_raw[lane] >= q.P) {
+            const uint32_t ov = M->out_v[lane];
+            const uint32_t mark = ((q.P & 31u) + (q.vinfo[ov] & 0xFFu) > 32u) ? 0x8000u : 0u;
+            reinterpret_cast<uint16_t *>(T + ov)[lane] = (uint16_t)(q.P | mark);
+            if (mark) atomicOr(&M->marks, 1u << lane);
+        }
+        __syncwarp();
+        if (lane * q.tg_rows <= q.V) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const uint32_t x0 = (uint32_t)(k0 & (TGW - 1)), z0 = (uint32_t)(k0 / TGW);
+            for (uint32_t v0 = lane * q.tg_rows; v0 <= q.V; v0 += 32 * q.tg_rows) tma_store_3d(&tmg, x0, v0, z0, T + v0);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            stored = true;
+        }
     }
 
     // ---- bank tally over the instructions with 2..4 distinct sources (see k_tables): the banks an
